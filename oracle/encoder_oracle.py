@@ -1,0 +1,220 @@
+"""CPU fp64 oracle for the Encode stage  V_m = E(I_m)  (Section 3.1 "Encode Stage", Eq. 1).
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition the CUDA path is
+checked against.  Only the tests, the smoke check and the benchmark's CPU-baseline leg
+may import it; the product never does, and it shares no code with the CUDA path.
+
+The paper fixes the stage's contract -- multimodal items in, one [n, d] feature matrix
+per item out, consumed by Prefill (Eq. 1; the printed E->P tensors of the prefetching
+table in Section 4) -- and says E is a Vision Transformer whose attention cost grows
+quadratically with the visual sequence length (Section 1).  It gives no layer-level
+formulae, so the encoder evaluated here is the standard pre-norm ViT the benchmark
+configurations name, written out step by step in float64 with no blocking, fusion or
+intermediate rounding:
+
+  O0  packing: image i has grid (t, h, w); its tokens are raster-ordered (frame, row, col)
+      and occupy rows cu[i]..cu[i+1] of every activation matrix; every frame reuses the
+      image's (row, col) positions.
+  O1  X = patches @ W_pe^T + b_pe
+  per layer:
+  O2  A = rmsnorm(X; g1)
+  O3  [q|k|v] = A @ W_qkv^T + b_qkv, heads are consecutive head_dim-wide column groups
+  O4  2-D rotary embedding on q and k: first half of each head rotates by the row index,
+      second half by the column index, rotate-half pairing inside each half
+  O5  per image, per head: softmax(q k^T / sqrt(head_dim)) v over ALL tokens of that image
+      (bidirectional, block-diagonal across images)
+  O6  X += O @ W_o^T + b_o
+  O7  X += gelu(rmsnorm(X; g2) @ W_1^T + b_1) @ W_2^T + b_2
+  O8  Y = rmsnorm(X; g_final)
+  O9  2x2 spatial merge: merged token (f, R, C) concatenates Y at (2R+dy, 2C+dx) for
+      (dy,dx) = (0,0),(0,1),(1,0),(1,1)
+  O10 projector: linear, or linear-GELU-linear, producing the [n, d] hand-off features.
+
+Parity pins (tests/test_oracle_*.py): pure-Python brute force on tiny inputs, PyTorch CPU
+float64 library routines for each step, closed forms and invariants, and the merged-row
+counts the paper prints.  The numerical values of the features themselves are
+"parity unpinned" by the paper (it prints none); they are pinned only by that chain.
+"""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+from scipy.special import erf as _erf
+
+ACT_GELU_TANH = 0
+ACT_GELU_ERF = 1
+
+
+# ----------------------------------------------------------------------------- O0 / O9 integers
+
+def bookkeeping(grid_thw: Sequence[Sequence[int]], merge: int = 2) -> Dict[str, np.ndarray]:
+    """Integer layout of a packed batch (step O0 and the index side of step O9).
+
+    Returns int32 arrays: cu_seqlens [n+1], pos_row [T], pos_col [T], cu_out [n+1] and
+    merge_idx [Tm, merge*merge] with merge_idx[o, 2*dy+dx] = source token of merged row o.
+    The contract is Eq. 1's V_m in R^{n x d}: rows cu_out[i]..cu_out[i+1] are image i's n rows.
+    """
+    n = len(grid_thw)
+    cu = np.zeros(n + 1, dtype=np.int64)
+    cu_out = np.zeros(n + 1, dtype=np.int64)
+    pos_row: List[np.ndarray] = []
+    pos_col: List[np.ndarray] = []
+    idx: List[np.ndarray] = []
+    for i, (t, h, w) in enumerate(grid_thw):
+        t, h, w = int(t), int(h), int(w)
+        if t < 1 or h < 1 or w < 1 or h % merge or w % merge:
+            raise ValueError(f"bad grid {(t, h, w)}")
+        cu[i + 1] = cu[i] + t * h * w
+        cu_out[i + 1] = cu_out[i] + t * (h // merge) * (w // merge)
+        r = np.repeat(np.arange(h), w)
+        c = np.tile(np.arange(w), h)
+        pos_row.append(np.tile(r, t))
+        pos_col.append(np.tile(c, t))
+        f, R, C = np.meshgrid(np.arange(t), np.arange(h // merge), np.arange(w // merge), indexing="ij")
+        cols = []
+        for dy in range(merge):
+            for dx in range(merge):
+                cols.append(cu[i] + f * h * w + (merge * R + dy) * w + (merge * C + dx))
+        idx.append(np.stack([c_.reshape(-1) for c_ in cols], axis=1))
+    cat = lambda xs, width=None: (np.concatenate(xs) if xs else np.zeros((0,) if width is None else (0, width)))
+    return {
+        "cu_seqlens": cu.astype(np.int32),
+        "cu_out": cu_out.astype(np.int32),
+        "pos_row": cat(pos_row).astype(np.int32),
+        "pos_col": cat(pos_col).astype(np.int32),
+        "merge_idx": cat(idx, merge * merge).astype(np.int32).reshape(-1, merge * merge),
+    }
+
+
+# ----------------------------------------------------------------------------- elementwise pieces
+
+def rmsnorm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
+    """Step O2/O8: x / sqrt(mean(x^2) + eps) * g, row-wise."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * g
+
+
+def gelu(x: np.ndarray, act: int) -> np.ndarray:
+    if act == ACT_GELU_TANH:
+        return 0.5 * x * (1.0 + np.tanh(np.sqrt(2.0 / np.pi) * (x + 0.044715 * x ** 3)))
+    if act == ACT_GELU_ERF:
+        return 0.5 * x * (1.0 + _erf(x / np.sqrt(2.0)))
+    raise ValueError("unknown activation")
+
+
+def linear(x: np.ndarray, w: np.ndarray, b: Optional[np.ndarray]) -> np.ndarray:
+    """y = x @ w^T + b with w stored [out, in]."""
+    y = x @ w.T
+    if b is not None:
+        y = y + b
+    return y
+
+
+def rope_2d(x: np.ndarray, pos_row: np.ndarray, pos_col: np.ndarray, theta: float) -> np.ndarray:
+    """Step O4 on x [T, heads, head_dim].
+
+    With d2 = head_dim/2 and nf = head_dim/4, frequency f has omega_f = theta^(-2f/d2).
+    Dims [0, d2) use p = row, dims [d2, head_dim) use p = col.  Inside a half, dims f and
+    f+nf form a pair:  x'_f = x_f cos(p w_f) - x_{f+nf} sin(p w_f),
+                       x'_{f+nf} = x_{f+nf} cos(p w_f) + x_f sin(p w_f).
+    """
+    T, nH, dh = x.shape
+    assert dh % 4 == 0
+    d2, nf = dh // 2, dh // 4
+    omega = theta ** (-2.0 * np.arange(nf, dtype=np.float64) / d2)
+    out = np.empty_like(x)
+    for half, pos in ((0, pos_row), (1, pos_col)):
+        ang = pos.astype(np.float64)[:, None] * omega[None, :]          # [T, nf]
+        c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+        a = x[:, :, half * d2: half * d2 + nf]
+        b = x[:, :, half * d2 + nf: (half + 1) * d2]
+        out[:, :, half * d2: half * d2 + nf] = a * c - b * s
+        out[:, :, half * d2 + nf: (half + 1) * d2] = b * c + a * s
+    return out
+
+
+def attention_block_diagonal(q: np.ndarray, k: np.ndarray, v: np.ndarray, cu_seqlens: np.ndarray,
+                             return_probs: bool = False):
+    """Step O5 on q, k, v [T, heads, head_dim]: per image and head, softmax(q k^T / sqrt(dh)) v."""
+    T, nH, dh = q.shape
+    o = np.zeros_like(q)
+    probs = []
+    for i in range(len(cu_seqlens) - 1):
+        a, b = int(cu_seqlens[i]), int(cu_seqlens[i + 1])
+        for hd in range(nH):
+            s = (q[a:b, hd, :] @ k[a:b, hd, :].T) / np.sqrt(float(dh))
+            s = s - s.max(axis=1, keepdims=True)
+            p = np.exp(s)
+            p = p / p.sum(axis=1, keepdims=True)
+            o[a:b, hd, :] = p @ v[a:b, hd, :]
+            if return_probs:
+                probs.append(p)
+    return (o, probs) if return_probs else o
+
+
+def merge_2x2(y: np.ndarray, merge_idx: np.ndarray) -> np.ndarray:
+    """Step O9: M[o, q*h:(q+1)*h] = Y[merge_idx[o, q], :]."""
+    Tm, nq = merge_idx.shape
+    return y[merge_idx.reshape(-1)].reshape(Tm, nq * y.shape[1])
+
+
+# ----------------------------------------------------------------------------- blocks / whole stage
+
+def _f64(a):
+    return None if a is None else np.asarray(a, dtype=np.float64)
+
+
+def attention_sublayer(cfg, lw: Dict, x: np.ndarray, bk: Dict) -> np.ndarray:
+    """Steps O2-O6: returns x + out_proj(attn(rope(qkv(rmsnorm(x)))))."""
+    T = x.shape[0]
+    h, nH, dh = cfg.hidden, cfg.heads, cfg.head_dim
+    a = rmsnorm(x, _f64(lw["norm1_w"]), cfg.eps)
+    qkv = linear(a, _f64(lw["qkv_w"]), _f64(lw["qkv_b"]))
+    q = qkv[:, 0:h].reshape(T, nH, dh)
+    k = qkv[:, h:2 * h].reshape(T, nH, dh)
+    v = qkv[:, 2 * h:3 * h].reshape(T, nH, dh)
+    if cfg.rope_theta > 0:
+        q = rope_2d(q, bk["pos_row"], bk["pos_col"], cfg.rope_theta)
+        k = rope_2d(k, bk["pos_row"], bk["pos_col"], cfg.rope_theta)
+    o = attention_block_diagonal(q, k, v, bk["cu_seqlens"]).reshape(T, h)
+    return x + linear(o, _f64(lw["out_w"]), _f64(lw["out_b"]))
+
+
+def mlp_sublayer(cfg, lw: Dict, x: np.ndarray) -> np.ndarray:
+    """Step O7."""
+    b = rmsnorm(x, _f64(lw["norm2_w"]), cfg.eps)
+    u = gelu(linear(b, _f64(lw["fc1_w"]), _f64(lw["fc1_b"])), cfg.act)
+    return x + linear(u, _f64(lw["fc2_w"]), _f64(lw["fc2_b"]))
+
+
+def block(cfg, lw: Dict, x: np.ndarray, bk: Dict) -> np.ndarray:
+    """One encoder block (O2-O7) applied to a given block input x [T, hidden]."""
+    return mlp_sublayer(cfg, lw, attention_sublayer(cfg, lw, _f64(x), bk))
+
+
+def head(cfg, weights: Dict, x: np.ndarray, bk: Dict) -> np.ndarray:
+    """Steps O8-O10 on the residual stream after the last block."""
+    y = rmsnorm(_f64(x), _f64(weights["final_norm_w"]), cfg.eps) if cfg.final_norm else _f64(x)
+    m = merge_2x2(y, bk["merge_idx"])
+    f = linear(m, _f64(weights["proj_w1"]), _f64(weights["proj_b1"]))
+    if weights.get("proj_w2") is not None:
+        f = linear(gelu(f, cfg.act), _f64(weights["proj_w2"]), _f64(weights["proj_b2"]))
+    return f
+
+
+def encode(cfg, weights: Dict, patches: np.ndarray, grid_thw: Sequence[Sequence[int]],
+           return_taps: bool = False):
+    """The whole stage (Eq. 1): packed patches [T, K] -> features [Tm, out_dim] in float64.
+
+    With return_taps, also returns the residual stream entering block 0, 1, ..., L-1 and
+    leaving the last block (L+1 arrays [T, hidden]).
+    """
+    bk = bookkeeping(grid_thw, cfg.merge)
+    x = linear(_f64(patches), _f64(weights["patch_w"]), _f64(weights["patch_b"]))
+    taps = [x]
+    for l in range(cfg.layers):
+        x = block(cfg, weights["layers"][l], x, bk)
+        taps.append(x)
+    f = head(cfg, weights, x, bk)
+    return (f, taps) if return_taps else f
