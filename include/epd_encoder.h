@@ -1,0 +1,249 @@
+/*
+ * epd_encoder.h -- C ABI of the Encode stage  V_m = E(I_m)  (Section 3.1 "Encode Stage", Eq. 1).
+ *
+ * E is a Vision Transformer: a packed batch of images / video clips, given as pixel patches
+ * plus one (t, h, w) patch grid per item, is turned into one contiguous [n, d] feature
+ * matrix per item -- the tensor that crosses the Encode -> Prefill boundary (Section 3.1
+ * "Cross-Stage Transmission"; the [n, 3584] tensors of the E-P prefetching table, Section 4).
+ * The call is stateless per request, so the fault-tolerant recomputation of Section 3.2 is
+ * simply calling it again.
+ *
+ * Conventions
+ *   - Every function returns an epd_status_t (0 = OK, < 0 = error); nothing throws, aborts or
+ *     prints.  epd_strerror() names a code.
+ *   - "device" pointers are CUDA global-memory addresses on the current device, "HOST"
+ *     pointers are ordinary process memory.  All matrices are row-major.  Weight matrices
+ *     are [out_features, in_features] (the contraction dimension is contiguous).
+ *   - dtype EPD_DTYPE_F32: activations, weights and features are float.
+ *     dtype EPD_DTYPE_BF16: weights, patches and features are bfloat16, all contractions
+ *     accumulate in float and the residual stream is kept in float.
+ *   - All work is enqueued on the given cudaStream_t and the call returns without
+ *     synchronising, unless stated otherwise.  The library never allocates device memory
+ *     after epd_encoder_create(): activations live in the caller-provided workspace.
+ *   - One encode may be in flight per encoder object (the workspace is per encoder).
+ *   - The CUDA device current at create time must be current for every later call.
+ */
+#ifndef EPD_ENCODER_H_
+#define EPD_ENCODER_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct epd_encoder epd_encoder_t;
+
+typedef enum {
+  EPD_OK = 0,
+  EPD_EINVAL = -1,       /* NULL / misaligned pointer, bad size, inconsistent configuration */
+  EPD_ENOMEM = -2,       /* workspace too small, host allocation failed */
+  EPD_ECUDA = -3,        /* a CUDA runtime / driver call failed */
+  EPD_ECAPACITY = -4,    /* batch exceeds max_tokens / max_images / the feature buffer */
+  EPD_EUNSUPPORTED = -5, /* shape the kernels do not cover */
+  EPD_ETIMEOUT = -6      /* a bounded device-side wait expired (reported by epd_encoder_last_status) */
+} epd_status_t;
+
+enum { EPD_DTYPE_F32 = 0, EPD_DTYPE_BF16 = 1 };
+enum { EPD_ACT_GELU_TANH = 0, EPD_ACT_GELU_ERF = 1 };
+enum { EPD_PROJ_LINEAR = 0, EPD_PROJ_MLP = 1 };
+
+/* Static description of the encoder E of Eq. 1. */
+typedef struct {
+  int32_t dtype;          /* EPD_DTYPE_* */
+  int32_t in_channels;    /* C */
+  int32_t patch;          /* P: patch side in pixels */
+  int32_t temporal_patch; /* Tp: frames folded into one patch; patch vector length K = C*Tp*P*P */
+  int32_t hidden;         /* h */
+  int32_t layers;         /* L */
+  int32_t heads;          /* heads * head_dim == hidden */
+  int32_t head_dim;       /* multiple of 4 (2-D rotary pairs), <= 128 */
+  int32_t mlp;            /* MLP width m */
+  int32_t act;            /* EPD_ACT_* (MLP and projector) */
+  float eps;              /* RMSNorm epsilon (inside the square root) */
+  float rope_theta;       /* rotary base; <= 0 disables the rotary embedding */
+  int32_t merge;          /* spatial merge factor; must be 2 */
+  int32_t final_norm;     /* 1: RMSNorm before the merge */
+  int32_t proj_kind;      /* EPD_PROJ_* */
+  int32_t proj_hidden;    /* width of the projector's hidden layer (EPD_PROJ_MLP) */
+  int32_t out_dim;        /* d of Eq. 1 */
+  int64_t max_tokens;     /* capacity: largest packed token count T of one call */
+  int32_t max_images;     /* capacity: largest number of items of one call */
+  int32_t max_grid;       /* capacity: largest h or w of any grid (rotary table rows) */
+} epd_config_t;
+
+/*
+ * Encoder parameters: device pointers, borrowed for the lifetime of the encoder (the caller
+ * keeps them alive and unchanged).  Per-layer entries are HOST arrays of `layers` device
+ * pointers.  Any bias pointer may be NULL (no bias).  Matrix rows are contiguous
+ * (leading dimension == in_features) except patch_w, whose leading dimension is patch_w_ld.
+ * In EPD_DTYPE_BF16 every leading dimension must be a multiple of 8 elements.
+ */
+typedef struct {
+  const void* patch_w;      /* [hidden, patch_w_ld], first K columns used */
+  int64_t patch_w_ld;       /* >= K */
+  const void* patch_b;      /* [hidden] */
+  const void* const* norm1_w; /* [L] -> [hidden] gains */
+  const void* const* qkv_w;   /* [L] -> [3*hidden, hidden]; rows 0..h-1 = q, h..2h-1 = k, 2h..3h-1 = v */
+  const void* const* qkv_b;   /* [L] -> [3*hidden] */
+  const void* const* out_w;   /* [L] -> [hidden, hidden] */
+  const void* const* out_b;   /* [L] -> [hidden] */
+  const void* const* norm2_w; /* [L] -> [hidden] */
+  const void* const* fc1_w;   /* [L] -> [mlp, hidden] */
+  const void* const* fc1_b;   /* [L] -> [mlp] */
+  const void* const* fc2_w;   /* [L] -> [hidden, mlp] */
+  const void* const* fc2_b;   /* [L] -> [hidden] */
+  const void* final_norm_w;   /* [hidden]; ignored when final_norm == 0 */
+  const void* proj_w1;        /* LINEAR: [out_dim, 4*hidden]; MLP: [proj_hidden, 4*hidden] */
+  const void* proj_b1;
+  const void* proj_w2;        /* MLP: [out_dim, proj_hidden]; LINEAR: NULL */
+  const void* proj_b2;
+} epd_weights_t;
+
+/* ------------------------------------------------------------------------------------------
+ * Encoder object
+ * ---------------------------------------------------------------------------------------- */
+
+/* Bytes of device workspace epd_encoder_create() needs for this configuration (0 on a bad config). */
+size_t epd_encoder_workspace_bytes(const epd_config_t* cfg);
+
+/*
+ * Build an encoder.  `workspace` is device memory of at least epd_encoder_workspace_bytes(cfg)
+ * bytes, 256-byte aligned, owned by the caller and reserved for this encoder until destroy.
+ * Synchronous: builds the rotary table on the device and returns after it is ready.
+ * Errors: EPD_EINVAL (bad config / NULL / alignment), EPD_ENOMEM (workspace too small),
+ * EPD_EUNSUPPORTED, EPD_ECUDA.
+ */
+int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, void* workspace,
+                       size_t workspace_bytes, epd_encoder_t** out);
+
+/*
+ * The Encode stage (Eq. 1) for one packed batch.
+ *   patches      device [T, patches_ld], element type per dtype; row j is the patch vector of
+ *                token j, element order inside a patch (channel, temporal, y, x).  Tokens of
+ *                item i occupy rows cu[i]..cu[i+1], raster order (frame, row, col).
+ *                16-byte aligned; in bf16 patches_ld must be a multiple of 8.
+ *   grid_thw     HOST [n_images, 3] = (t, h, w) of each item in patch units; t,h,w >= 1 and
+ *                h, w even.  An item with t > 1 is a clip: attention spans all its frames.
+ *   features     device [features_capacity_rows, out_dim], caller-owned E->P buffer.  Item i's
+ *                feature matrix V_m is rows out_cu_rows[i]..out_cu_rows[i+1], merged tokens in
+ *                (frame, row/2, col/2) raster order, each row = projector(concat of the 2x2
+ *                neighbours (dy,dx) = (0,0),(0,1),(1,0),(1,1)).
+ *   out_rows     HOST, optional: total feature rows written (T/4).
+ *   out_cu_rows  HOST [n_images+1], optional: prefix sums of per-item feature rows.
+ *   stream       cudaStream_t (NULL = legacy default stream).
+ * Validation happens on the host before anything is launched; host outputs are filled
+ * synchronously (they depend on grid_thw only).  n_images == 0 is valid and launches nothing.
+ * Errors: EPD_EINVAL, EPD_ECAPACITY, EPD_ECUDA.
+ */
+int epd_encode(epd_encoder_t* enc, const void* patches, int64_t patches_ld, const int32_t* grid_thw,
+               int32_t n_images, void* features, int64_t features_capacity_rows, int64_t* out_rows,
+               int32_t* out_cu_rows, void* stream);
+
+/*
+ * Same stage with HOST patches and a HOST feature buffer (both should be page-locked for the
+ * copies to be asynchronous): copies patches to a staging area inside the workspace, encodes,
+ * copies the features back, all on `stream`.  Returns without synchronising; the features are
+ * valid after the stream is synchronised.  patches_ld == K here.
+ */
+int epd_encode_host(epd_encoder_t* enc, const void* host_patches, const int32_t* grid_thw,
+                    int32_t n_images, void* host_features, int64_t features_capacity_rows,
+                    int64_t* out_rows, int32_t* out_cu_rows, void* stream);
+
+/* Reads the encoder's device status word (synchronises the device): EPD_OK or the first
+ * device-side error (EPD_ETIMEOUT), then clears it. */
+int epd_encoder_last_status(epd_encoder_t* enc);
+
+/* Number of kernels the last epd_encode() call launched. */
+int64_t epd_encoder_last_launch_count(const epd_encoder_t* enc);
+
+/* 1 if the encoder runs its contractions on the tcgen05 tensor-core kernels, 0 if on the
+ * plain-FMA kernels (EPD_DTYPE_F32 always does). */
+int epd_encoder_uses_tensor_cores(const epd_encoder_t* enc);
+
+int epd_encoder_destroy(epd_encoder_t* enc);
+
+const char* epd_strerror(int status);
+
+/* ------------------------------------------------------------------------------------------
+ * Test hooks on an encoder
+ * ---------------------------------------------------------------------------------------- */
+
+/* Copies the integer layout of the LAST encoded batch back to HOST arrays (synchronises):
+ * cu_seqlens [n+1], pos_row [T], pos_col [T], merge_idx [T/4, 4] (source token of each merged
+ * slot).  Any pointer may be NULL. */
+int epd_debug_bookkeeping(epd_encoder_t* enc, int32_t* cu_seqlens, int32_t* pos_row, int32_t* pos_col,
+                          int32_t* merge_idx);
+
+/* `taps` is a HOST array of layers+1 device pointers (or NULL to clear).  During later encodes,
+ * a non-NULL taps[l] receives the float residual stream [T, hidden] entering block l
+ * (l == layers: leaving the last block). */
+int epd_debug_set_taps(epd_encoder_t* enc, void* const* taps);
+
+/* Runs only block `layer` (steps RMSNorm..MLP of one layer) on a caller-supplied residual
+ * stream x (device float [T, hidden], updated in place) for the given grids. */
+int epd_debug_run_block(epd_encoder_t* enc, int32_t layer, void* x, const int32_t* grid_thw,
+                        int32_t n_images, void* stream);
+
+/* Per-step timing of the next encodes: with enable != 0 every launch of epd_encode() is bracketed
+ * by CUDA events on the launching stream (this costs a few microseconds per launch, so it is
+ * meant for a separate measuring pass).  epd_debug_profile_read() synchronises on the last event
+ * and fills ms[c] / launches[c] (HOST arrays of epd_debug_profile_classes() entries) with the
+ * device time and launch count of step class c of the most recent encode;
+ * epd_debug_profile_class_name(c) names the class ("qkv_linear", "attention", ...). */
+int epd_debug_profile(epd_encoder_t* enc, int32_t enable);
+int32_t epd_debug_profile_classes(void);
+const char* epd_debug_profile_class_name(int32_t cls);
+int epd_debug_profile_read(epd_encoder_t* enc, float* ms, int64_t* launches);
+
+/* ------------------------------------------------------------------------------------------
+ * Single steps of the path (each is what the encoder itself launches)
+ * ---------------------------------------------------------------------------------------- */
+
+enum {
+  EPD_LINEAR_GELU_TANH = 1,  /* apply tanh-GELU after the bias */
+  EPD_LINEAR_GELU_ERF = 2,   /* apply erf-GELU after the bias */
+  EPD_LINEAR_ACCUMULATE = 4, /* out (float) += result: the residual update */
+  EPD_LINEAR_OUT_F32 = 8,    /* out is float even when dtype is bf16 */
+  EPD_LINEAR_FORCE_FMA = 16  /* use the plain-FMA kernel even where the tensor-core kernel applies */
+};
+
+/* out[M,N] = act(x[M,K] . w[N,K]^T + bias[N]) (optionally accumulated into a float out).
+ * x, w: element type per dtype, leading dimensions ldx, ldw (elements); out: leading dimension
+ * ldo.  All device pointers, 16-byte aligned. */
+int epd_op_linear(int32_t dtype, const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias,
+                  void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t flags, void* stream);
+
+/* out[j,:] = x[j,:] / sqrt(mean(x[j,:]^2) + eps) * gain, x float [T, hidden], out per dtype.
+ * If dst_row != NULL (device int32 [T]) row j is written at element offset dst_row[j]*hidden
+ * instead of j*hidden (used to fuse the 2x2 merge into the final norm). */
+int epd_op_rmsnorm(int32_t dtype, const void* x, const void* gain, void* out, const int32_t* dst_row,
+                   int64_t T, int32_t hidden, float eps, void* stream);
+
+/* Rotary embedding + head split.  qkv [T, 3*hidden] per dtype -> q, k, v each
+ * [heads, T, head_dim_padded] per dtype (head_dim_padded = epd_padded_head_dim(head_dim), pad
+ * columns zero).  q and k are rotated by (pos_row, pos_col) (device int32 [T]); q is also
+ * multiplied by q_scale.  theta <= 0 skips the rotation. */
+int epd_op_rope_split(int32_t dtype, const void* qkv, const int32_t* pos_row, const int32_t* pos_col,
+                      void* q, void* k, void* v, int64_t T, int32_t heads, int32_t head_dim, float theta,
+                      float q_scale, void* stream);
+
+int32_t epd_padded_head_dim(int32_t head_dim);
+
+/* Block-diagonal bidirectional attention.  q, k, v [heads, T, head_dim_padded] per dtype with q
+ * already multiplied by log2(e)/sqrt(head_dim); cu_seqlens device int32 [n_seg+1] and the same
+ * values in HOST memory (host_cu_seqlens) for the launch geometry.  out [T, heads*head_dim] per
+ * dtype: for each segment and head softmax over all keys of the segment. */
+int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                     const int32_t* host_cu_seqlens, int32_t n_seg, void* out, int64_t T, int32_t heads,
+                     int32_t head_dim, int32_t flags, void* stream);
+
+/* out[o, q*hidden:(q+1)*hidden] = y[merge_idx[o*4+q], :], y [T, hidden], out [T/4, 4*hidden] per dtype. */
+int epd_op_merge(int32_t dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm,
+                 int32_t hidden, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EPD_ENCODER_H_ */

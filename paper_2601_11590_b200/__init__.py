@@ -1,0 +1,377 @@
+"""Python binding of the Encode-stage C library (libepd_encoder.so).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+PyTorch supplies device memory and streams.  There is no CPU fallback: importing works
+without a GPU (so the exported symbols can be inspected), but creating an encoder or calling
+an op requires the compiled library and a CUDA device.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libepd_encoder.so")
+
+EPD_OK, EPD_EINVAL, EPD_ENOMEM, EPD_ECUDA, EPD_ECAPACITY, EPD_EUNSUPPORTED, EPD_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+DTYPE_F32, DTYPE_BF16 = 0, 1
+LINEAR_GELU_TANH, LINEAR_GELU_ERF, LINEAR_ACCUMULATE, LINEAR_OUT_F32, LINEAR_FORCE_FMA = 1, 2, 4, 8, 16
+
+EXPORTED_SYMBOLS = [
+    "epd_encoder_workspace_bytes", "epd_encoder_create", "epd_encode", "epd_encode_host",
+    "epd_encoder_last_status", "epd_encoder_last_launch_count", "epd_encoder_uses_tensor_cores",
+    "epd_encoder_destroy", "epd_strerror", "epd_debug_bookkeeping", "epd_debug_set_taps",
+    "epd_debug_run_block", "epd_debug_profile", "epd_debug_profile_classes",
+    "epd_debug_profile_class_name", "epd_debug_profile_read", "epd_op_linear", "epd_op_rmsnorm", "epd_op_rope_split",
+    "epd_padded_head_dim", "epd_op_attention", "epd_op_merge",
+]
+
+
+class EpdError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {strerror(status)} ({status})")
+
+
+class ConfigStruct(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("dtype", "in_channels", "patch", "temporal_patch", "hidden", "layers", "heads",
+                 "head_dim", "mlp", "act")] + \
+               [("eps", ctypes.c_float), ("rope_theta", ctypes.c_float)] + \
+               [(n, ctypes.c_int32) for n in ("merge", "final_norm", "proj_kind", "proj_hidden", "out_dim")] + \
+               [("max_tokens", ctypes.c_int64), ("max_images", ctypes.c_int32), ("max_grid", ctypes.c_int32)]
+
+
+_PP = ctypes.POINTER(ctypes.c_void_p)
+
+
+class WeightsStruct(ctypes.Structure):
+    _fields_ = [("patch_w", ctypes.c_void_p), ("patch_w_ld", ctypes.c_int64), ("patch_b", ctypes.c_void_p)] + \
+               [(n, _PP) for n in ("norm1_w", "qkv_w", "qkv_b", "out_w", "out_b", "norm2_w",
+                                   "fc1_w", "fc1_b", "fc2_w", "fc2_b")] + \
+               [(n, ctypes.c_void_p) for n in ("final_norm_w", "proj_w1", "proj_b1", "proj_w2", "proj_b2")]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen the compiled library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2601_11590_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64, f32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_float
+    i32p, i64p = ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int64)
+    lib.epd_encoder_workspace_bytes.restype = ctypes.c_size_t
+    lib.epd_encoder_workspace_bytes.argtypes = [ctypes.POINTER(ConfigStruct)]
+    lib.epd_encoder_create.restype = ctypes.c_int
+    lib.epd_encoder_create.argtypes = [ctypes.POINTER(ConfigStruct), ctypes.POINTER(WeightsStruct), vp,
+                                       ctypes.c_size_t, ctypes.POINTER(vp)]
+    lib.epd_encode.restype = ctypes.c_int
+    lib.epd_encode.argtypes = [vp, vp, i64, i32p, i32, vp, i64, i64p, i32p, vp]
+    lib.epd_encode_host.restype = ctypes.c_int
+    lib.epd_encode_host.argtypes = [vp, vp, i32p, i32, vp, i64, i64p, i32p, vp]
+    lib.epd_encoder_last_status.restype = ctypes.c_int
+    lib.epd_encoder_last_status.argtypes = [vp]
+    lib.epd_encoder_last_launch_count.restype = ctypes.c_int64
+    lib.epd_encoder_last_launch_count.argtypes = [vp]
+    lib.epd_encoder_uses_tensor_cores.restype = ctypes.c_int
+    lib.epd_encoder_uses_tensor_cores.argtypes = [vp]
+    lib.epd_encoder_destroy.restype = ctypes.c_int
+    lib.epd_encoder_destroy.argtypes = [vp]
+    lib.epd_strerror.restype = ctypes.c_char_p
+    lib.epd_strerror.argtypes = [ctypes.c_int]
+    lib.epd_debug_bookkeeping.restype = ctypes.c_int
+    lib.epd_debug_bookkeeping.argtypes = [vp, i32p, i32p, i32p, i32p]
+    lib.epd_debug_set_taps.restype = ctypes.c_int
+    lib.epd_debug_set_taps.argtypes = [vp, _PP]
+    lib.epd_debug_run_block.restype = ctypes.c_int
+    lib.epd_debug_run_block.argtypes = [vp, i32, vp, i32p, i32, vp]
+    lib.epd_debug_profile.restype = ctypes.c_int
+    lib.epd_debug_profile.argtypes = [vp, i32]
+    lib.epd_debug_profile_classes.restype = i32
+    lib.epd_debug_profile_classes.argtypes = []
+    lib.epd_debug_profile_class_name.restype = ctypes.c_char_p
+    lib.epd_debug_profile_class_name.argtypes = [i32]
+    lib.epd_debug_profile_read.restype = ctypes.c_int
+    lib.epd_debug_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_float), i64p]
+    lib.epd_op_linear.restype = ctypes.c_int
+    lib.epd_op_linear.argtypes = [i32, vp, i64, vp, i64, vp, vp, i64, i64, i64, i64, i32, vp]
+    lib.epd_op_rmsnorm.restype = ctypes.c_int
+    lib.epd_op_rmsnorm.argtypes = [i32, vp, vp, vp, vp, i64, i32, f32, vp]
+    lib.epd_op_rope_split.restype = ctypes.c_int
+    lib.epd_op_rope_split.argtypes = [i32, vp, vp, vp, vp, vp, vp, i64, i32, i32, f32, f32, vp]
+    lib.epd_padded_head_dim.restype = i32
+    lib.epd_padded_head_dim.argtypes = [i32]
+    lib.epd_op_attention.restype = ctypes.c_int
+    lib.epd_op_attention.argtypes = [i32, vp, vp, vp, vp, i32p, i32, vp, i64, i32, i32, i32, vp]
+    lib.epd_op_merge.restype = ctypes.c_int
+    lib.epd_op_merge.argtypes = [i32, vp, vp, vp, i64, i32, vp]
+    _lib = lib
+    return lib
+
+
+def strerror(status: int) -> str:
+    return load_library().epd_strerror(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != EPD_OK:
+        raise EpdError(status, what)
+
+
+def _torch():
+    import torch
+    if not torch.cuda.is_available():
+        raise RuntimeError("the Encode-stage library needs a CUDA device; there is no CPU path")
+    return torch
+
+
+def _stream_ptr(stream) -> int:
+    torch = _torch()
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else int(t.data_ptr())
+
+
+def _i32_array(values: Sequence[int]):
+    arr = np.ascontiguousarray(np.asarray(values, dtype=np.int32).reshape(-1))
+    return arr, arr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+
+
+def torch_dtype(dtype: int):
+    torch = _torch()
+    return torch.float32 if dtype == DTYPE_F32 else torch.bfloat16
+
+
+def to_device(arr: Optional[np.ndarray], dtype: int, device="cuda"):
+    """float32 numpy values -> device tensor of the configuration's element type (exact for
+    values already representable in it)."""
+    if arr is None:
+        return None
+    torch = _torch()
+    return torch.from_numpy(np.ascontiguousarray(arr, dtype=np.float32)).to(device=device, dtype=torch_dtype(dtype))
+
+
+def make_config(cfg, max_tokens: int, max_images: int, max_grid: int) -> ConfigStruct:
+    """cfg: any object with the fields of epd_config_t (e.g. synth.EncoderConfig)."""
+    c = ConfigStruct()
+    for name in ("dtype", "in_channels", "patch", "temporal_patch", "hidden", "layers", "heads", "head_dim",
+                 "mlp", "act", "merge", "final_norm", "proj_kind", "proj_hidden", "out_dim"):
+        setattr(c, name, int(getattr(cfg, name)))
+    c.eps = float(cfg.eps)
+    c.rope_theta = float(cfg.rope_theta)
+    c.max_tokens, c.max_images, c.max_grid = int(max_tokens), int(max_images), int(max_grid)
+    return c
+
+
+class Encoder:
+    """Owns one epd_encoder_t, its device weights (torch tensors) and its workspace."""
+
+    def __init__(self, cfg, weights: Dict, max_tokens: int, max_images: int = 64, max_grid: int = 128,
+                 device="cuda", patch_w_ld: Optional[int] = None):
+        """weights: dict of float32 numpy arrays or device tensors laid out as synth.make_weights()."""
+        torch = _torch()
+        self.lib = load_library()
+        self.cfg = cfg
+        self.dtype = int(cfg.dtype)
+        self.device = torch.device(device)
+        self.max_tokens = int(max_tokens)
+        self._c = make_config(cfg, max_tokens, max_images, max_grid)
+        K = cfg.in_channels * cfg.temporal_patch * cfg.patch * cfg.patch
+        self.patch_dim = K
+        if patch_w_ld is None:
+            patch_w_ld = K if self.dtype == DTYPE_F32 else (K + 7) // 8 * 8
+        self.patch_w_ld = patch_w_ld
+
+        def dev(a):
+            if a is None:
+                return None
+            if isinstance(a, np.ndarray):
+                return to_device(a, self.dtype, self.device)
+            return a.to(device=self.device, dtype=torch_dtype(self.dtype)).contiguous()
+
+        pw = dev(weights["patch_w"])
+        if patch_w_ld != K:
+            padded = torch.zeros((cfg.hidden, patch_w_ld), dtype=pw.dtype, device=self.device)
+            padded[:, :K] = pw
+            pw = padded
+        self._keep = {"patch_w": pw, "patch_b": dev(weights["patch_b"]),
+                      "final_norm_w": dev(weights.get("final_norm_w")),
+                      "proj_w1": dev(weights["proj_w1"]), "proj_b1": dev(weights.get("proj_b1")),
+                      "proj_w2": dev(weights.get("proj_w2")), "proj_b2": dev(weights.get("proj_b2"))}
+        names = ("norm1_w", "qkv_w", "qkv_b", "out_w", "out_b", "norm2_w", "fc1_w", "fc1_b", "fc2_w", "fc2_b")
+        self._layers: List[Dict] = [{n: dev(lw.get(n)) for n in names} for lw in weights["layers"]]
+        assert len(self._layers) == cfg.layers
+        w = WeightsStruct()
+        w.patch_w, w.patch_w_ld, w.patch_b = _ptr(pw), patch_w_ld, _ptr(self._keep["patch_b"])
+        self._arrays = {}
+        for n in names:
+            arr = (ctypes.c_void_p * max(1, cfg.layers))(*[_ptr(lw[n]) for lw in self._layers])
+            self._arrays[n] = arr
+            setattr(w, n, ctypes.cast(arr, _PP))
+        for n in ("final_norm_w", "proj_w1", "proj_b1", "proj_w2", "proj_b2"):
+            setattr(w, n, _ptr(self._keep[n]))
+        nbytes = self.lib.epd_encoder_workspace_bytes(ctypes.byref(self._c))
+        if nbytes == 0:
+            raise EpdError(EPD_EINVAL, "epd_encoder_workspace_bytes")
+        self.workspace_bytes = int(nbytes)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        handle = ctypes.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(self.lib.epd_encoder_create(ctypes.byref(self._c), ctypes.byref(w), base, nbytes,
+                                               ctypes.byref(handle)), "epd_encoder_create")
+        self._h = handle
+        self._taps = None
+
+    # ---- the stage -------------------------------------------------------------------------
+    def encode(self, patches, grid_thw, features=None, stream=None):
+        """patches: device tensor [T, ld]; returns (features tensor [rows, out_dim], cu_rows ndarray)."""
+        torch = _torch()
+        g, gp = _i32_array(grid_thw)
+        n = g.size // 3
+        T = int(sum(int(g[3 * i]) * int(g[3 * i + 1]) * int(g[3 * i + 2]) for i in range(n)))
+        if features is None:
+            features = torch.empty((max(T // 4, 1), self.cfg.out_dim), dtype=torch_dtype(self.dtype),
+                                   device=self.device)
+        rows = ctypes.c_int64(0)
+        cu_rows = np.zeros(n + 1, dtype=np.int32)
+        ld = int(patches.stride(0)) if (patches is not None and patches.dim() == 2 and patches.shape[0] > 0) \
+            else self.patch_dim
+        _check(self.lib.epd_encode(self._h, _ptr(patches), ld, gp, n, _ptr(features), int(features.shape[0]),
+                                   ctypes.byref(rows), cu_rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                   _stream_ptr(stream)), "epd_encode")
+        return features[: rows.value], cu_rows
+
+    def encode_host(self, host_patches, grid_thw, host_features, stream=None):
+        """host_patches / host_features: CPU tensors (pinned for asynchronous copies)."""
+        g, gp = _i32_array(grid_thw)
+        n = g.size // 3
+        rows = ctypes.c_int64(0)
+        cu_rows = np.zeros(n + 1, dtype=np.int32)
+        _check(self.lib.epd_encode_host(self._h, _ptr(host_patches), gp, n, _ptr(host_features),
+                                        int(host_features.shape[0]), ctypes.byref(rows),
+                                        cu_rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                        _stream_ptr(stream)), "epd_encode_host")
+        return rows.value, cu_rows
+
+    def last_status(self) -> int:
+        return int(self.lib.epd_encoder_last_status(self._h))
+
+    def last_launch_count(self) -> int:
+        return int(self.lib.epd_encoder_last_launch_count(self._h))
+
+    def uses_tensor_cores(self) -> bool:
+        return bool(self.lib.epd_encoder_uses_tensor_cores(self._h))
+
+    # ---- test hooks ------------------------------------------------------------------------
+    def debug_bookkeeping(self, n_images: int, T: int):
+        cu = np.zeros(n_images + 1, np.int32)
+        pr, pc, mi = np.zeros(T, np.int32), np.zeros(T, np.int32), np.zeros(T, np.int32)
+        p = lambda a: a.ctypes.data_as(ctypes.POINTER(ctypes.c_int32))
+        _check(self.lib.epd_debug_bookkeeping(self._h, p(cu), p(pr), p(pc), p(mi)), "epd_debug_bookkeeping")
+        return {"cu_seqlens": cu, "pos_row": pr, "pos_col": pc, "merge_idx": mi.reshape(-1, 4)}
+
+    def set_taps(self, taps):
+        """taps: list of layers+1 float32 device tensors or None entries; None clears."""
+        if taps is None:
+            self._taps = None
+            _check(self.lib.epd_debug_set_taps(self._h, None), "epd_debug_set_taps")
+            return
+        assert len(taps) == self.cfg.layers + 1
+        self._taps = list(taps)
+        arr = (ctypes.c_void_p * len(taps))(*[_ptr(t) for t in taps])
+        _check(self.lib.epd_debug_set_taps(self._h, ctypes.cast(arr, _PP)), "epd_debug_set_taps")
+
+    def run_block(self, layer: int, x, grid_thw, stream=None):
+        g, gp = _i32_array(grid_thw)
+        _check(self.lib.epd_debug_run_block(self._h, int(layer), _ptr(x), gp, g.size // 3, _stream_ptr(stream)),
+               "epd_debug_run_block")
+        return x
+
+    def profile(self, enable: bool):
+        _check(self.lib.epd_debug_profile(self._h, 1 if enable else 0), "epd_debug_profile")
+
+    def profile_read(self) -> Dict[str, Dict]:
+        """Device time (ms) and launch count per step class of the most recent profiled encode."""
+        n = int(self.lib.epd_debug_profile_classes())
+        ms = (ctypes.c_float * n)()
+        cnt = (ctypes.c_int64 * n)()
+        _check(self.lib.epd_debug_profile_read(self._h, ms, cnt), "epd_debug_profile_read")
+        return {self.lib.epd_debug_profile_class_name(i).decode(): {"ms": float(ms[i]), "launches": int(cnt[i])}
+                for i in range(n)}
+
+    def close(self):
+        if getattr(self, "_h", None) is not None and self._h.value:
+            self.lib.epd_encoder_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+# ---- single steps ------------------------------------------------------------------------------
+
+def op_linear(dtype, x, w, bias, out, M, N, K, flags=0, ldx=None, ldw=None, ldo=None, stream=None):
+    lib = load_library()
+    _check(lib.epd_op_linear(dtype, _ptr(x), ldx if ldx is not None else x.stride(0), _ptr(w),
+                             ldw if ldw is not None else w.stride(0), _ptr(bias), _ptr(out),
+                             ldo if ldo is not None else out.stride(0), M, N, K, flags, _stream_ptr(stream)),
+           "epd_op_linear")
+    return out
+
+
+def op_rmsnorm(dtype, x, gain, out, eps, dst_row=None, stream=None):
+    lib = load_library()
+    _check(lib.epd_op_rmsnorm(dtype, _ptr(x), _ptr(gain), _ptr(out), _ptr(dst_row), x.shape[0], x.shape[1],
+                              eps, _stream_ptr(stream)), "epd_op_rmsnorm")
+    return out
+
+
+def padded_head_dim(head_dim: int) -> int:
+    return int(load_library().epd_padded_head_dim(head_dim))
+
+
+def op_rope_split(dtype, qkv, pos_row, pos_col, heads, head_dim, theta, q_scale, stream=None):
+    torch = _torch()
+    lib = load_library()
+    T = qkv.shape[0]
+    dhp = padded_head_dim(head_dim)
+    q, k, v = (torch.empty((heads, T, dhp), dtype=qkv.dtype, device=qkv.device) for _ in range(3))
+    _check(lib.epd_op_rope_split(dtype, _ptr(qkv), _ptr(pos_row), _ptr(pos_col), _ptr(q), _ptr(k), _ptr(v), T,
+                                 heads, head_dim, theta, q_scale, _stream_ptr(stream)), "epd_op_rope_split")
+    return q, k, v
+
+
+def op_attention(dtype, q, k, v, cu_seqlens_dev, cu_seqlens_host, head_dim, flags=0, stream=None):
+    torch = _torch()
+    lib = load_library()
+    heads, T, _ = q.shape
+    out = torch.empty((T, heads * head_dim), dtype=q.dtype, device=q.device)
+    hcu, hp = _i32_array(cu_seqlens_host)
+    _check(lib.epd_op_attention(dtype, _ptr(q), _ptr(k), _ptr(v), _ptr(cu_seqlens_dev), hp, hcu.size - 1,
+                                _ptr(out), T, heads, head_dim, flags, _stream_ptr(stream)), "epd_op_attention")
+    return out
+
+
+def op_merge(dtype, y, merge_idx, stream=None):
+    torch = _torch()
+    lib = load_library()
+    T, h = y.shape
+    out = torch.empty((T // 4, 4 * h), dtype=y.dtype, device=y.device)
+    _check(lib.epd_op_merge(dtype, _ptr(y), _ptr(merge_idx), _ptr(out), T // 4, h, _stream_ptr(stream)),
+           "epd_op_merge")
+    return out

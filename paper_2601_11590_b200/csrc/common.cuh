@@ -1,0 +1,53 @@
+// Internal declarations shared by the kernels of the Encode-stage library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "epd_encoder.h"
+
+namespace epd {
+
+// Device status word values written by kernels whose bounded waits expire.
+constexpr int kStatusTimeout = EPD_ETIMEOUT;
+
+// Largest head_dim the attention kernels cover.
+constexpr int kMaxHeadDim = 128;
+
+// Padded head width of the head-major q/k/v buffers: a multiple of 16 elements so that every
+// row starts on a 32-byte boundary and the contraction over head_dim splits into 16-wide steps.
+__host__ __device__ inline int padded_head_dim(int dh) { return (dh + 15) / 16 * 16; }
+
+template <typename T> __device__ __forceinline__ float to_float(T v);
+template <> __device__ __forceinline__ float to_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_float(float v);
+template <> __device__ __forceinline__ float from_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float gelu_tanh_f(float x) {
+  const float c = 0.7978845608028654f;  // sqrt(2/pi)
+  return 0.5f * x * (1.0f + tanhf(c * (x + 0.044715f * x * x * x)));
+}
+__device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f)); }
+
+// ---- plain-FMA kernels (kernels_fma.cu) -----------------------------------------------------
+cudaError_t linear_fma(int dtype, const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias,
+                       void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, cudaStream_t s);
+cudaError_t rmsnorm(int dtype, const void* x, const void* gain, void* out, const int32_t* dst_row, int64_t T,
+                    int hidden, float eps, cudaStream_t s);
+cudaError_t rope_split(int dtype, const void* qkv, const int32_t* pos_row, const int32_t* pos_col,
+                       const float2* table, int table_rows, void* q, void* k, void* v, int64_t T, int heads,
+                       int head_dim, float theta, float q_scale, cudaStream_t s);
+cudaError_t rope_table(float2* table, int rows, int head_dim, float theta, cudaStream_t s);
+cudaError_t attention_fma(int dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                          int n_seg, void* out, int64_t T, int heads, int head_dim, cudaStream_t s);
+cudaError_t merge_gather(int dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm, int hidden,
+                         cudaStream_t s);
+cudaError_t token_layout(const int32_t* grid_thw, const int32_t* cu_seqlens, const int32_t* cu_out, int n_images,
+                         int64_t T, int32_t* pos_row, int32_t* pos_col, int32_t* merge_slot, int32_t* merge_idx,
+                         cudaStream_t s);
+
+}  // namespace epd

@@ -1,0 +1,584 @@
+// C ABI of the Encode stage: the encoder object, host-side validation and integer layout,
+// and the launch sequence of one forward pass.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace epd;
+
+namespace {
+
+// Step classes reported by epd_debug_profile_read().
+enum { KC_LAYOUT = 0, KC_PATCH, KC_RMSNORM, KC_QKV, KC_ROPE, KC_ATTENTION, KC_OUT, KC_FC1, KC_FC2, KC_MERGE, KC_PROJ,
+       KC_END, KC_COUNT = KC_END };
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Offsets of every activation buffer inside the caller's workspace.
+struct Layout {
+  size_t x, a, qkv, qh, kh, vh, u, merged, proj_hidden, stage_patches, stage_features;
+  size_t grid, cu, cu_out, pos_row, pos_col, merge_slot, merge_idx, rope, status, aux, total;
+};
+
+bool config_ok(const epd_config_t* c) {
+  if (!c) return false;
+  if (c->dtype != EPD_DTYPE_F32 && c->dtype != EPD_DTYPE_BF16) return false;
+  if (c->in_channels < 1 || c->patch < 1 || c->temporal_patch < 1) return false;
+  if (c->hidden < 1 || c->layers < 0 || c->heads < 1 || c->head_dim < 4) return false;
+  if (c->heads * c->head_dim != c->hidden || c->head_dim % 4 || c->head_dim > kMaxHeadDim) return false;
+  if (c->mlp < 1 || (c->act != EPD_ACT_GELU_TANH && c->act != EPD_ACT_GELU_ERF)) return false;
+  if (c->merge != 2 || !(c->eps >= 0.0f)) return false;
+  if (c->proj_kind != EPD_PROJ_LINEAR && c->proj_kind != EPD_PROJ_MLP) return false;
+  if (c->proj_kind == EPD_PROJ_MLP && c->proj_hidden < 1) return false;
+  if (c->out_dim < 1 || c->max_tokens < 4 || c->max_tokens > (1 << 30) || c->max_images < 1 || c->max_grid < 2)
+    return false;
+  if (c->dtype == EPD_DTYPE_BF16 && (c->hidden % 8 || c->mlp % 8 || c->out_dim % 8 || c->proj_hidden % 8))
+    return false;
+  return true;
+}
+
+Layout make_layout(const epd_config_t& c) {
+  Layout L{};
+  const size_t es = c.dtype == EPD_DTYPE_F32 ? 4 : 2;
+  const size_t T = (size_t)c.max_tokens, Tm = T / 4, h = c.hidden;
+  const size_t dhp = padded_head_dim(c.head_dim);
+  const size_t K = (size_t)c.in_channels * c.temporal_patch * c.patch * c.patch;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  L.x = take(T * h * 4);
+  L.a = take(T * h * es);
+  L.qkv = take(T * 3 * h * es);
+  L.qh = take((size_t)c.heads * T * dhp * es);
+  L.kh = take((size_t)c.heads * T * dhp * es);
+  L.vh = take((size_t)c.heads * T * dhp * es);
+  L.u = take(T * (size_t)c.mlp * es);
+  L.merged = take(Tm * 4 * h * es);
+  L.proj_hidden = take(c.proj_kind == EPD_PROJ_MLP ? Tm * (size_t)c.proj_hidden * es : 0);
+  L.stage_patches = take(T * K * es);
+  L.stage_features = take(Tm * (size_t)c.out_dim * es);
+  L.grid = take((size_t)c.max_images * 3 * 4);
+  L.cu = take(((size_t)c.max_images + 1) * 4);
+  L.cu_out = take(((size_t)c.max_images + 1) * 4);
+  L.pos_row = take(T * 4);
+  L.pos_col = take(T * 4);
+  L.merge_slot = take(T * 4);
+  L.merge_idx = take(T * 4);
+  L.rope = take((size_t)c.max_grid * (c.head_dim / 4) * sizeof(float2));
+  L.status = take(256);
+  L.aux = take(0);
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+
+struct epd_encoder {
+  epd_config_t cfg;
+  epd_weights_t w;
+  std::vector<const void*> norm1_w, qkv_w, qkv_b, out_w, out_b, norm2_w, fc1_w, fc1_b, fc2_w, fc2_b;
+  Layout lay;
+  uint8_t* ws = nullptr;
+  int32_t* pinned = nullptr;       // [3*max_images | max_images+1 | max_images+1]
+  cudaEvent_t staged = nullptr;    // recorded after the layout copy of the last batch
+  bool staged_valid = false;
+  std::vector<int32_t> last_grid;  // grids of the batch whose layout is on the device
+  std::vector<int32_t> host_cu;
+  int64_t last_T = -1;
+  std::vector<void*> taps;
+  int64_t launches = 0;
+  int64_t patch_dim = 0;
+  // optional per-step timing: one event before every launch, one after the last
+  bool profile = false;
+  std::vector<cudaEvent_t> prof_events;
+  std::vector<int> prof_class;
+  size_t prof_used = 0;
+  bool use_tc = false;
+
+  template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+namespace {
+
+#define EPD_CUDA(expr)                        \
+  do {                                        \
+    cudaError_t e__ = (expr);                 \
+    if (e__ != cudaSuccess) return EPD_ECUDA; \
+  } while (0)
+
+// Counts a launch of step class `cls` and, in profiling mode, records an event before it.
+int mark(epd_encoder* enc, int cls, cudaStream_t s) {
+  enc->launches++;
+  if (!enc->profile) return EPD_OK;
+  if (enc->prof_used == enc->prof_events.size()) {
+    cudaEvent_t ev;
+    EPD_CUDA(cudaEventCreate(&ev));
+    enc->prof_events.push_back(ev);
+  }
+  EPD_CUDA(cudaEventRecord(enc->prof_events[enc->prof_used], s));
+  if (enc->prof_class.size() <= enc->prof_used) enc->prof_class.resize(enc->prof_used + 1);
+  enc->prof_class[enc->prof_used] = cls;
+  enc->prof_used++;
+  return EPD_OK;
+}
+#define EPD_MARK(cls)                              \
+  do {                                             \
+    int rc__ = mark(enc, (cls), s);                \
+    if (rc__) return rc__;                         \
+  } while (0)
+
+int linear_dispatch(epd_encoder* enc, int dtype, const void* x, int64_t ldx, const void* w, int64_t ldw,
+                    const void* bias, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int flags,
+                    cudaStream_t s) {
+  (void)enc;
+  EPD_CUDA(linear_fma(dtype, x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, s));
+  return EPD_OK;
+}
+
+// Validates the grids, fills host outputs and (if the batch differs from the last one) stages
+// the integer layout on the device.
+int prepare_batch(epd_encoder* enc, const int32_t* grid_thw, int32_t n, int64_t capacity_rows, int64_t* out_rows,
+                  int32_t* out_cu_rows, int64_t* T_out, cudaStream_t s) {
+  const epd_config_t& c = enc->cfg;
+  if (n < 0 || (n > 0 && !grid_thw)) return EPD_EINVAL;
+  if (n > c.max_images) return EPD_ECAPACITY;
+  int64_t T = 0, Tm = 0;
+  std::vector<int32_t> cu(n + 1, 0), cuo(n + 1, 0);
+  for (int i = 0; i < n; ++i) {
+    const int64_t t = grid_thw[3 * i], h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
+    if (t < 1 || h < 1 || w < 1 || (h & 1) || (w & 1)) return EPD_EINVAL;
+    if (h > c.max_grid || w > c.max_grid) return EPD_ECAPACITY;
+    if (t > c.max_tokens || t * h > c.max_tokens || t * h * w > c.max_tokens) return EPD_ECAPACITY;
+    T += t * h * w;
+    Tm += t * (h / 2) * (w / 2);
+    if (T > c.max_tokens) return EPD_ECAPACITY;
+    cu[i + 1] = (int32_t)T;
+    cuo[i + 1] = (int32_t)Tm;
+  }
+  if (capacity_rows >= 0 && Tm > capacity_rows) return EPD_ECAPACITY;
+  if (out_rows) *out_rows = Tm;
+  if (out_cu_rows) std::memcpy(out_cu_rows, cuo.data(), (n + 1) * sizeof(int32_t));
+  *T_out = T;
+  if (n == 0) return EPD_OK;
+
+  const bool same = enc->last_T == T && (int)enc->last_grid.size() == 3 * n &&
+                    std::memcmp(enc->last_grid.data(), grid_thw, 3 * n * sizeof(int32_t)) == 0;
+  if (same) return EPD_OK;
+  // The pinned staging buffer may still be the source of the previous batch's copy.
+  if (enc->staged_valid) EPD_CUDA(cudaEventSynchronize(enc->staged));
+  int32_t* pg = enc->pinned;
+  int32_t* pcu = pg + 3 * (size_t)c.max_images;
+  int32_t* pcuo = pcu + c.max_images + 1;
+  std::memcpy(pg, grid_thw, 3 * n * sizeof(int32_t));
+  std::memcpy(pcu, cu.data(), (n + 1) * sizeof(int32_t));
+  std::memcpy(pcuo, cuo.data(), (n + 1) * sizeof(int32_t));
+  EPD_CUDA(cudaMemcpyAsync(enc->at<int32_t>(enc->lay.grid), pg, 3 * n * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+  EPD_CUDA(cudaMemcpyAsync(enc->at<int32_t>(enc->lay.cu), pcu, (n + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, s));
+  EPD_CUDA(cudaMemcpyAsync(enc->at<int32_t>(enc->lay.cu_out), pcuo, (n + 1) * sizeof(int32_t),
+                           cudaMemcpyHostToDevice, s));
+  EPD_CUDA(cudaEventRecord(enc->staged, s));
+  enc->staged_valid = true;
+  EPD_MARK(KC_LAYOUT);
+  EPD_CUDA(token_layout(enc->at<int32_t>(enc->lay.grid), enc->at<int32_t>(enc->lay.cu),
+                        enc->at<int32_t>(enc->lay.cu_out), n, T, enc->at<int32_t>(enc->lay.pos_row),
+                        enc->at<int32_t>(enc->lay.pos_col), enc->at<int32_t>(enc->lay.merge_slot),
+                        enc->at<int32_t>(enc->lay.merge_idx), s));
+  enc->last_grid.assign(grid_thw, grid_thw + 3 * n);
+  enc->host_cu = cu;
+  enc->last_T = T;
+  return EPD_OK;
+}
+
+int attention_dispatch(epd_encoder* enc, int64_t T, int n_seg, cudaStream_t s) {
+  const epd_config_t& c = enc->cfg;
+  EPD_MARK(KC_ATTENTION);
+  EPD_CUDA(attention_fma(c.dtype, enc->at<void>(enc->lay.qh), enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh),
+                         enc->at<int32_t>(enc->lay.cu), n_seg, enc->at<void>(enc->lay.a), T, c.heads, c.head_dim, s));
+  return EPD_OK;
+}
+
+// Steps RMSNorm .. MLP of block l on the float residual stream x.
+int run_block(epd_encoder* enc, int l, float* x, int64_t T, int n_seg, cudaStream_t s) {
+  const epd_config_t& c = enc->cfg;
+  const int h = c.hidden, m = c.mlp;
+  const int dt = c.dtype;
+  void* a = enc->at<void>(enc->lay.a);
+  void* qkv = enc->at<void>(enc->lay.qkv);
+  void* u = enc->at<void>(enc->lay.u);
+  const int gelu = c.act == EPD_ACT_GELU_TANH ? EPD_LINEAR_GELU_TANH : EPD_LINEAR_GELU_ERF;
+  int rc;
+  EPD_MARK(KC_RMSNORM);
+  EPD_CUDA(rmsnorm(dt, x, enc->norm1_w[l], a, nullptr, T, h, c.eps, s));
+  EPD_MARK(KC_QKV);
+  if ((rc = linear_dispatch(enc, dt, a, h, enc->qkv_w[l], h, enc->qkv_b[l], qkv, 3 * h, T, 3 * h, h, 0, s))) return rc;
+  const float q_scale = 1.4426950408889634f / sqrtf((float)c.head_dim);
+  EPD_MARK(KC_ROPE);
+  EPD_CUDA(rope_split(dt, qkv, enc->at<int32_t>(enc->lay.pos_row), enc->at<int32_t>(enc->lay.pos_col),
+                      enc->at<float2>(enc->lay.rope), c.max_grid, enc->at<void>(enc->lay.qh),
+                      enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh), T, c.heads, c.head_dim, c.rope_theta,
+                      q_scale, s));
+  if ((rc = attention_dispatch(enc, T, n_seg, s))) return rc;
+  EPD_MARK(KC_OUT);
+  if ((rc = linear_dispatch(enc, dt, a, h, enc->out_w[l], h, enc->out_b[l], x, h, T, h, h, EPD_LINEAR_ACCUMULATE, s)))
+    return rc;
+  EPD_MARK(KC_RMSNORM);
+  EPD_CUDA(rmsnorm(dt, x, enc->norm2_w[l], a, nullptr, T, h, c.eps, s));
+  EPD_MARK(KC_FC1);
+  if ((rc = linear_dispatch(enc, dt, a, h, enc->fc1_w[l], h, enc->fc1_b[l], u, m, T, m, h, gelu, s))) return rc;
+  EPD_MARK(KC_FC2);
+  if ((rc = linear_dispatch(enc, dt, u, m, enc->fc2_w[l], m, enc->fc2_b[l], x, h, T, h, m, EPD_LINEAR_ACCUMULATE, s)))
+    return rc;
+  return EPD_OK;
+}
+
+// Closes the event list of a profiled pass.
+int finish_profile(epd_encoder* enc, cudaStream_t s) {
+  if (!enc->profile) return EPD_OK;
+  enc->launches--;  // the closing event is not a launch
+  return mark(enc, KC_END, s);
+}
+
+int encode_device(epd_encoder* enc, const void* patches, int64_t patches_ld, const int32_t* grid_thw, int32_t n,
+                  void* features, int64_t cap_rows, int64_t* out_rows, int32_t* out_cu_rows, cudaStream_t s) {
+  const epd_config_t& c = enc->cfg;
+  const int dt = c.dtype;
+  const int h = c.hidden;
+  if (cap_rows < 0) return EPD_EINVAL;
+  enc->launches = 0;
+  enc->prof_used = 0;
+  int64_t T = 0;
+  int rc = prepare_batch(enc, grid_thw, n, cap_rows, out_rows, out_cu_rows, &T, s);
+  if (rc) return rc;
+  if (T == 0) return EPD_OK;
+  if (!patches || !features) return EPD_EINVAL;
+  if (((uintptr_t)patches & 15) || ((uintptr_t)features & 15)) return EPD_EINVAL;
+  if (patches_ld < enc->patch_dim) return EPD_EINVAL;
+  if (dt == EPD_DTYPE_BF16 && (patches_ld % 8)) return EPD_EINVAL;
+  const int64_t Tm = T / 4;
+  float* x = enc->at<float>(enc->lay.x);
+
+  // patch embedding -> float residual stream
+  EPD_MARK(KC_PATCH);
+  if ((rc = linear_dispatch(enc, dt, patches, patches_ld, enc->w.patch_w, enc->w.patch_w_ld, enc->w.patch_b, x, h, T,
+                            h, enc->patch_dim, EPD_LINEAR_OUT_F32, s)))
+    return rc;
+  for (int l = 0; l < c.layers; ++l) {
+    if (!enc->taps.empty() && enc->taps[l])
+      EPD_CUDA(cudaMemcpyAsync(enc->taps[l], x, (size_t)T * h * 4, cudaMemcpyDeviceToDevice, s));
+    if ((rc = run_block(enc, l, x, T, n, s))) return rc;
+  }
+  if (!enc->taps.empty() && enc->taps[c.layers])
+    EPD_CUDA(cudaMemcpyAsync(enc->taps[c.layers], x, (size_t)T * h * 4, cudaMemcpyDeviceToDevice, s));
+
+  // final norm fused with the 2x2 merge: token j is written to slot merge_slot[j] of [4*Tm, h]
+  void* merged = enc->at<void>(enc->lay.merged);
+  if (c.final_norm) {
+    EPD_MARK(KC_RMSNORM);
+    EPD_CUDA(rmsnorm(dt, x, enc->w.final_norm_w, merged, enc->at<int32_t>(enc->lay.merge_slot), T, h, c.eps, s));
+  } else if (dt == EPD_DTYPE_F32) {
+    EPD_MARK(KC_MERGE);
+    EPD_CUDA(merge_gather(dt, x, enc->at<int32_t>(enc->lay.merge_idx), merged, Tm, h, s));
+  } else {
+    return EPD_EUNSUPPORTED;  // bf16 without a final norm: the float stream has no bf16 copy to gather
+  }
+  if (c.proj_kind == EPD_PROJ_LINEAR) {
+    EPD_MARK(KC_PROJ);
+    if ((rc = linear_dispatch(enc, dt, merged, 4 * h, enc->w.proj_w1, 4 * h, enc->w.proj_b1, features, c.out_dim, Tm,
+                              c.out_dim, 4 * h, 0, s)))
+      return rc;
+  } else {
+    void* ph = enc->at<void>(enc->lay.proj_hidden);
+    const int gelu = c.act == EPD_ACT_GELU_TANH ? EPD_LINEAR_GELU_TANH : EPD_LINEAR_GELU_ERF;
+    EPD_MARK(KC_PROJ);
+    if ((rc = linear_dispatch(enc, dt, merged, 4 * h, enc->w.proj_w1, 4 * h, enc->w.proj_b1, ph, c.proj_hidden, Tm,
+                              c.proj_hidden, 4 * h, gelu, s)))
+      return rc;
+    EPD_MARK(KC_PROJ);
+    if ((rc = linear_dispatch(enc, dt, ph, c.proj_hidden, enc->w.proj_w2, c.proj_hidden, enc->w.proj_b2, features,
+                              c.out_dim, Tm, c.out_dim, c.proj_hidden, 0, s)))
+      return rc;
+  }
+  return finish_profile(enc, s);
+}
+
+}  // namespace
+
+// =============================================================================================
+// exported functions
+// =============================================================================================
+extern "C" {
+
+size_t epd_encoder_workspace_bytes(const epd_config_t* cfg) {
+  if (!config_ok(cfg)) return 0;
+  return make_layout(*cfg).total;
+}
+
+int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, void* workspace,
+                       size_t workspace_bytes, epd_encoder_t** out) {
+  if (!out) return EPD_EINVAL;
+  *out = nullptr;
+  if (!config_ok(cfg) || !weights || !workspace) return EPD_EINVAL;
+  if ((uintptr_t)workspace & 255) return EPD_EINVAL;
+  const Layout lay = make_layout(*cfg);
+  if (workspace_bytes < lay.total) return EPD_ENOMEM;
+  const int L = cfg->layers;
+  const int64_t K = (int64_t)cfg->in_channels * cfg->temporal_patch * cfg->patch * cfg->patch;
+  if (!weights->patch_w || weights->patch_w_ld < K || !weights->proj_w1) return EPD_EINVAL;
+  if (cfg->final_norm && !weights->final_norm_w) return EPD_EINVAL;
+  if (cfg->proj_kind == EPD_PROJ_MLP && !weights->proj_w2) return EPD_EINVAL;
+  if (L > 0 && (!weights->norm1_w || !weights->qkv_w || !weights->out_w || !weights->norm2_w || !weights->fc1_w ||
+                !weights->fc2_w))
+    return EPD_EINVAL;
+  if (cfg->dtype == EPD_DTYPE_BF16 && (weights->patch_w_ld % 8)) return EPD_EINVAL;
+
+  epd_encoder* e = new (std::nothrow) epd_encoder();
+  if (!e) return EPD_ENOMEM;
+  e->cfg = *cfg;
+  e->w = *weights;
+  e->lay = lay;
+  e->ws = static_cast<uint8_t*>(workspace);
+  e->patch_dim = K;
+  auto copy_list = [&](std::vector<const void*>& dst, const void* const* src, bool required) -> bool {
+    dst.assign(L, nullptr);
+    if (!src) return !required || L == 0;
+    for (int l = 0; l < L; ++l) {
+      dst[l] = src[l];
+      if (required && !src[l]) return false;
+    }
+    return true;
+  };
+  bool ok = copy_list(e->norm1_w, weights->norm1_w, true) && copy_list(e->qkv_w, weights->qkv_w, true) &&
+            copy_list(e->qkv_b, weights->qkv_b, false) && copy_list(e->out_w, weights->out_w, true) &&
+            copy_list(e->out_b, weights->out_b, false) && copy_list(e->norm2_w, weights->norm2_w, true) &&
+            copy_list(e->fc1_w, weights->fc1_w, true) && copy_list(e->fc1_b, weights->fc1_b, false) &&
+            copy_list(e->fc2_w, weights->fc2_w, true) && copy_list(e->fc2_b, weights->fc2_b, false);
+  if (!ok) { delete e; return EPD_EINVAL; }
+  // the struct's per-layer arrays belong to the caller: keep only our copies
+  e->w.norm1_w = e->w.qkv_w = e->w.qkv_b = e->w.out_w = e->w.out_b = e->w.norm2_w = nullptr;
+  e->w.fc1_w = e->w.fc1_b = e->w.fc2_w = e->w.fc2_b = nullptr;
+
+  const size_t pinned_ints = 3 * (size_t)cfg->max_images + 2 * ((size_t)cfg->max_images + 1);
+  if (cudaMallocHost(reinterpret_cast<void**>(&e->pinned), pinned_ints * sizeof(int32_t)) != cudaSuccess) {
+    delete e;
+    return EPD_ECUDA;
+  }
+  if (cudaEventCreateWithFlags(&e->staged, cudaEventDisableTiming) != cudaSuccess) {
+    cudaFreeHost(e->pinned);
+    delete e;
+    return EPD_ECUDA;
+  }
+  cudaError_t err = cudaMemset(e->ws + lay.status, 0, 256);
+  if (err == cudaSuccess && cfg->rope_theta > 0.0f)
+    err = rope_table(e->at<float2>(lay.rope), cfg->max_grid, cfg->head_dim, cfg->rope_theta, 0);
+  if (err == cudaSuccess) err = cudaDeviceSynchronize();
+  if (err != cudaSuccess) {
+    cudaEventDestroy(e->staged);
+    cudaFreeHost(e->pinned);
+    delete e;
+    return EPD_ECUDA;
+  }
+  *out = e;
+  return EPD_OK;
+}
+
+int epd_encode(epd_encoder_t* enc, const void* patches, int64_t patches_ld, const int32_t* grid_thw,
+               int32_t n_images, void* features, int64_t features_capacity_rows, int64_t* out_rows,
+               int32_t* out_cu_rows, void* stream) {
+  if (!enc) return EPD_EINVAL;
+  return encode_device(enc, patches, patches_ld, grid_thw, n_images, features, features_capacity_rows, out_rows,
+                       out_cu_rows, static_cast<cudaStream_t>(stream));
+}
+
+int epd_encode_host(epd_encoder_t* enc, const void* host_patches, const int32_t* grid_thw, int32_t n_images,
+                    void* host_features, int64_t features_capacity_rows, int64_t* out_rows, int32_t* out_cu_rows,
+                    void* stream) {
+  if (!enc) return EPD_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const epd_config_t& c = enc->cfg;
+  const size_t es = c.dtype == EPD_DTYPE_F32 ? 4 : 2;
+  if (n_images < 0 || (n_images > 0 && !grid_thw)) return EPD_EINVAL;
+  int64_t T = 0;
+  for (int i = 0; i < n_images; ++i) {
+    const int64_t t = grid_thw[3 * i], h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
+    if (t < 1 || h < 1 || w < 1) return EPD_EINVAL;
+    if (t > c.max_tokens || t * h > c.max_tokens || t * h * w > c.max_tokens) return EPD_ECAPACITY;
+    T += t * h * w;
+    if (T > c.max_tokens) return EPD_ECAPACITY;
+  }
+  if (T > 0 && (!host_patches || !host_features)) return EPD_EINVAL;
+  void* dp = enc->at<void>(enc->lay.stage_patches);
+  void* df = enc->at<void>(enc->lay.stage_features);
+  if (T > 0)
+    EPD_CUDA(cudaMemcpyAsync(dp, host_patches, (size_t)T * enc->patch_dim * es, cudaMemcpyHostToDevice, s));
+  int64_t rows = 0;
+  int rc = encode_device(enc, dp, enc->patch_dim, grid_thw, n_images, df, features_capacity_rows, &rows, out_cu_rows, s);
+  if (rc) return rc;
+  if (out_rows) *out_rows = rows;
+  if (rows > 0)
+    EPD_CUDA(cudaMemcpyAsync(host_features, df, (size_t)rows * c.out_dim * es, cudaMemcpyDeviceToHost, s));
+  return EPD_OK;
+}
+
+int epd_encoder_last_status(epd_encoder_t* enc) {
+  if (!enc) return EPD_EINVAL;
+  int32_t st = 0;
+  EPD_CUDA(cudaDeviceSynchronize());
+  EPD_CUDA(cudaMemcpy(&st, enc->ws + enc->lay.status, sizeof(st), cudaMemcpyDeviceToHost));
+  if (st != 0) EPD_CUDA(cudaMemset(enc->ws + enc->lay.status, 0, sizeof(st)));
+  return st;
+}
+
+int64_t epd_encoder_last_launch_count(const epd_encoder_t* enc) { return enc ? enc->launches : 0; }
+
+int epd_encoder_uses_tensor_cores(const epd_encoder_t* enc) { return enc && enc->use_tc ? 1 : 0; }
+
+int epd_encoder_destroy(epd_encoder_t* enc) {
+  if (!enc) return EPD_OK;
+  cudaDeviceSynchronize();
+  if (enc->staged) cudaEventDestroy(enc->staged);
+  for (cudaEvent_t ev : enc->prof_events) cudaEventDestroy(ev);
+  if (enc->pinned) cudaFreeHost(enc->pinned);
+  delete enc;
+  return EPD_OK;
+}
+
+const char* epd_strerror(int status) {
+  switch (status) {
+    case EPD_OK: return "ok";
+    case EPD_EINVAL: return "invalid argument";
+    case EPD_ENOMEM: return "workspace too small or out of host memory";
+    case EPD_ECUDA: return "CUDA call failed";
+    case EPD_ECAPACITY: return "batch exceeds configured capacity";
+    case EPD_EUNSUPPORTED: return "unsupported shape";
+    case EPD_ETIMEOUT: return "bounded device-side wait expired";
+    default: return "unknown status";
+  }
+}
+
+int epd_debug_bookkeeping(epd_encoder_t* enc, int32_t* cu_seqlens, int32_t* pos_row, int32_t* pos_col,
+                          int32_t* merge_idx) {
+  if (!enc || enc->last_T < 0) return EPD_EINVAL;
+  EPD_CUDA(cudaDeviceSynchronize());
+  const size_t n = enc->last_grid.size() / 3, T = (size_t)enc->last_T;
+  if (cu_seqlens) EPD_CUDA(cudaMemcpy(cu_seqlens, enc->ws + enc->lay.cu, (n + 1) * 4, cudaMemcpyDeviceToHost));
+  if (pos_row) EPD_CUDA(cudaMemcpy(pos_row, enc->ws + enc->lay.pos_row, T * 4, cudaMemcpyDeviceToHost));
+  if (pos_col) EPD_CUDA(cudaMemcpy(pos_col, enc->ws + enc->lay.pos_col, T * 4, cudaMemcpyDeviceToHost));
+  if (merge_idx) EPD_CUDA(cudaMemcpy(merge_idx, enc->ws + enc->lay.merge_idx, T * 4, cudaMemcpyDeviceToHost));
+  return EPD_OK;
+}
+
+int epd_debug_set_taps(epd_encoder_t* enc, void* const* taps) {
+  if (!enc) return EPD_EINVAL;
+  enc->taps.clear();
+  if (taps) enc->taps.assign(taps, taps + enc->cfg.layers + 1);
+  return EPD_OK;
+}
+
+int epd_debug_run_block(epd_encoder_t* enc, int32_t layer, void* x, const int32_t* grid_thw, int32_t n_images,
+                        void* stream) {
+  if (!enc || !x || layer < 0 || layer >= enc->cfg.layers) return EPD_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int64_t T = 0;
+  enc->launches = 0;
+  enc->prof_used = 0;
+  int rc = prepare_batch(enc, grid_thw, n_images, -1, nullptr, nullptr, &T, s);
+  if (rc) return rc;
+  if (T == 0) return EPD_OK;
+  if ((rc = run_block(enc, layer, static_cast<float*>(x), T, n_images, s))) return rc;
+  return finish_profile(enc, s);
+}
+
+int epd_debug_profile(epd_encoder_t* enc, int32_t enable) {
+  if (!enc) return EPD_EINVAL;
+  enc->profile = enable != 0;
+  enc->prof_used = 0;
+  return EPD_OK;
+}
+
+int32_t epd_debug_profile_classes(void) { return KC_COUNT; }
+
+const char* epd_debug_profile_class_name(int32_t cls) {
+  static const char* names[KC_COUNT] = {"token_layout", "patch_embed", "rmsnorm", "qkv_linear", "rope_split",
+                                        "attention", "out_linear", "fc1_linear", "fc2_linear", "merge", "projector"};
+  return (cls >= 0 && cls < KC_COUNT) ? names[cls] : "";
+}
+
+int epd_debug_profile_read(epd_encoder_t* enc, float* ms, int64_t* launches) {
+  if (!enc || !ms || !launches) return EPD_EINVAL;
+  for (int i = 0; i < KC_COUNT; ++i) { ms[i] = 0.0f; launches[i] = 0; }
+  if (enc->prof_used < 2) return EPD_OK;
+  EPD_CUDA(cudaEventSynchronize(enc->prof_events[enc->prof_used - 1]));
+  for (size_t i = 0; i + 1 < enc->prof_used; ++i) {
+    float t = 0.0f;
+    EPD_CUDA(cudaEventElapsedTime(&t, enc->prof_events[i], enc->prof_events[i + 1]));
+    const int cls = enc->prof_class[i];
+    if (cls >= 0 && cls < KC_COUNT) { ms[cls] += t; launches[cls]++; }
+  }
+  return EPD_OK;
+}
+
+// ---- single steps ---------------------------------------------------------------------------
+
+int epd_op_linear(int32_t dtype, const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
+                  int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t flags, void* stream) {
+  if (dtype != EPD_DTYPE_F32 && dtype != EPD_DTYPE_BF16) return EPD_EINVAL;
+  if (M < 0 || N < 0 || K < 1 || ldx < K || ldw < K || ldo < N) return EPD_EINVAL;
+  if (M == 0 || N == 0) return EPD_OK;
+  if (!x || !w || !out) return EPD_EINVAL;
+  return linear_dispatch(nullptr, dtype, x, ldx, w, ldw, bias, out, ldo, M, N, K, flags,
+                         static_cast<cudaStream_t>(stream));
+}
+
+int epd_op_rmsnorm(int32_t dtype, const void* x, const void* gain, void* out, const int32_t* dst_row, int64_t T,
+                   int32_t hidden, float eps, void* stream) {
+  if (dtype != EPD_DTYPE_F32 && dtype != EPD_DTYPE_BF16) return EPD_EINVAL;
+  if (T < 0 || hidden < 1) return EPD_EINVAL;
+  if (T == 0) return EPD_OK;
+  if (!x || !gain || !out || ((uintptr_t)x & 15) || ((uintptr_t)out & 15)) return EPD_EINVAL;
+  EPD_CUDA(rmsnorm(dtype, x, gain, out, dst_row, T, hidden, eps, static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int32_t epd_padded_head_dim(int32_t head_dim) { return padded_head_dim(head_dim); }
+
+int epd_op_rope_split(int32_t dtype, const void* qkv, const int32_t* pos_row, const int32_t* pos_col, void* q,
+                      void* k, void* v, int64_t T, int32_t heads, int32_t head_dim, float theta, float q_scale,
+                      void* stream) {
+  if (dtype != EPD_DTYPE_F32 && dtype != EPD_DTYPE_BF16) return EPD_EINVAL;
+  if (T < 0 || heads < 1 || head_dim < 4 || head_dim % 4 || head_dim > kMaxHeadDim) return EPD_EINVAL;
+  if (T == 0) return EPD_OK;
+  if (!qkv || !pos_row || !pos_col || !q || !k || !v) return EPD_EINVAL;
+  EPD_CUDA(rope_split(dtype, qkv, pos_row, pos_col, nullptr, 0, q, k, v, T, heads, head_dim, theta, q_scale,
+                      static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                     const int32_t* host_cu_seqlens, int32_t n_seg, void* out, int64_t T, int32_t heads,
+                     int32_t head_dim, int32_t flags, void* stream) {
+  if (dtype != EPD_DTYPE_F32 && dtype != EPD_DTYPE_BF16) return EPD_EINVAL;
+  if (T < 0 || n_seg < 0 || heads < 1 || head_dim < 4 || head_dim > kMaxHeadDim) return EPD_EINVAL;
+  if (T == 0 || n_seg == 0) return EPD_OK;
+  if (!q || !k || !v || !cu_seqlens || !host_cu_seqlens || !out) return EPD_EINVAL;
+  if (host_cu_seqlens[0] != 0 || host_cu_seqlens[n_seg] != T) return EPD_EINVAL;
+  for (int i = 0; i < n_seg; ++i)
+    if (host_cu_seqlens[i + 1] <= host_cu_seqlens[i]) return EPD_EINVAL;
+  (void)flags;
+  EPD_CUDA(attention_fma(dtype, q, k, v, cu_seqlens, n_seg, out, T, heads, head_dim,
+                         static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int epd_op_merge(int32_t dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm, int32_t hidden,
+                 void* stream) {
+  if (dtype != EPD_DTYPE_F32 && dtype != EPD_DTYPE_BF16) return EPD_EINVAL;
+  if (Tm < 0 || hidden < 1) return EPD_EINVAL;
+  if (Tm == 0) return EPD_OK;
+  if (!y || !merge_idx || !out) return EPD_EINVAL;
+  EPD_CUDA(merge_gather(dtype, y, merge_idx, out, Tm, hidden, static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+}  // extern "C"

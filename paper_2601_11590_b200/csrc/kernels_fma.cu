@@ -1,0 +1,401 @@
+// Plain-FMA kernels of the Encode stage: the float path of every step, the bandwidth-bound
+// steps of the bf16 path (RMSNorm, rotary + head split, merge), and the integer token layout.
+// The dense contractions of the bf16 path run in gemm_tcgen05.cu / attention kernels instead.
+#include "common.cuh"
+
+namespace epd {
+
+// =============================================================================================
+// Token layout (integers): positions and 2x2-merge slots of every packed token.
+// Token j of item i with local index f*h*w + r*w + c has pos_row = r, pos_col = c and goes to
+// quarter q = 2*(r%2) + (c%2) of merged row o = cu_out[i] + f*(h/2)*(w/2) + (r/2)*(w/2) + c/2.
+// =============================================================================================
+__global__ void token_layout_kernel(const int32_t* __restrict__ grid_thw, const int32_t* __restrict__ cu,
+                                    const int32_t* __restrict__ cu_out, int n, int64_t T,
+                                    int32_t* __restrict__ pos_row, int32_t* __restrict__ pos_col,
+                                    int32_t* __restrict__ merge_slot, int32_t* __restrict__ merge_idx) {
+  for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < T; j += (int64_t)gridDim.x * blockDim.x) {
+    int lo = 0, hi = n;  // largest i with cu[i] <= j
+    while (hi - lo > 1) {
+      int mid = (lo + hi) >> 1;
+      if (cu[mid] <= j) lo = mid; else hi = mid;
+    }
+    const int i = lo;
+    const int h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
+    const int local = (int)(j - cu[i]);
+    const int f = local / (h * w);
+    const int rem = local - f * h * w;
+    const int r = rem / w, c = rem - r * w;
+    pos_row[j] = r;
+    pos_col[j] = c;
+    const int o = cu_out[i] + f * (h / 2) * (w / 2) + (r / 2) * (w / 2) + (c / 2);
+    const int slot = o * 4 + 2 * (r & 1) + (c & 1);
+    merge_slot[j] = slot;
+    merge_idx[slot] = (int32_t)j;
+  }
+}
+
+cudaError_t token_layout(const int32_t* grid_thw, const int32_t* cu_seqlens, const int32_t* cu_out, int n_images,
+                         int64_t T, int32_t* pos_row, int32_t* pos_col, int32_t* merge_slot, int32_t* merge_idx,
+                         cudaStream_t s) {
+  if (T == 0) return cudaSuccess;
+  const int threads = 256;
+  const int blocks = (int)((T + threads - 1) / threads);
+  token_layout_kernel<<<blocks, threads, 0, s>>>(grid_thw, cu_seqlens, cu_out, n_images, T, pos_row, pos_col,
+                                                 merge_slot, merge_idx);
+  return cudaGetLastError();
+}
+
+// =============================================================================================
+// Linear layer with plain FMAs: out = act(x . w^T + bias), 64x64 tile, 4x4 outputs per thread.
+// =============================================================================================
+constexpr int kFmaTile = 64;
+constexpr int kFmaBK = 16;
+
+template <typename TIn, typename TOut, int ACT, bool ACCUM>
+__global__ void __launch_bounds__(256)
+linear_fma_kernel(const TIn* __restrict__ x, int64_t ldx, const TIn* __restrict__ w, int64_t ldw,
+                  const TIn* __restrict__ bias, TOut* __restrict__ out, int64_t ldo, int64_t M, int64_t N,
+                  int64_t K) {
+  __shared__ float sx[kFmaBK][kFmaTile + 1];
+  __shared__ float sw[kFmaBK][kFmaTile + 1];
+  const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+  const int64_t m0 = (int64_t)blockIdx.y * kFmaTile, n0 = (int64_t)blockIdx.x * kFmaTile;
+  float acc[4][4] = {};
+  for (int64_t k0 = 0; k0 < K; k0 += kFmaBK) {
+    for (int e = threadIdx.x; e < kFmaTile * kFmaBK; e += 256) {
+      const int row = e / kFmaBK, kk = e % kFmaBK;
+      const int64_t gk = k0 + kk;
+      sx[kk][row] = (m0 + row < M && gk < K) ? to_float<TIn>(x[(m0 + row) * ldx + gk]) : 0.0f;
+      sw[kk][row] = (n0 + row < N && gk < K) ? to_float<TIn>(w[(n0 + row) * ldw + gk]) : 0.0f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < kFmaBK; ++kk) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { a[i] = sx[kk][ty * 4 + i]; b[i] = sw[kk][tx * 4 + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int64_t m = m0 + ty * 4 + i;
+    if (m >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t n = n0 + tx * 4 + j;
+      if (n >= N) continue;
+      float v = acc[i][j] + (bias ? to_float<TIn>(bias[n]) : 0.0f);
+      if (ACT == 1) v = gelu_tanh_f(v);
+      if (ACT == 2) v = gelu_erf_f(v);
+      if (ACCUM) out[m * ldo + n] = from_float<TOut>(to_float<TOut>(out[m * ldo + n]) + v);
+      else out[m * ldo + n] = from_float<TOut>(v);
+    }
+  }
+}
+
+template <typename TIn, typename TOut>
+static cudaError_t linear_fma_t(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
+                                int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, cudaStream_t s) {
+  dim3 grid((unsigned)((N + kFmaTile - 1) / kFmaTile), (unsigned)((M + kFmaTile - 1) / kFmaTile));
+  const int act = (flags & EPD_LINEAR_GELU_TANH) ? 1 : (flags & EPD_LINEAR_GELU_ERF) ? 2 : 0;
+  const bool accum = flags & EPD_LINEAR_ACCUMULATE;
+#define EPD_LAUNCH(A, C)                                                                                      \
+  linear_fma_kernel<TIn, TOut, A, C><<<grid, 256, 0, s>>>((const TIn*)x, ldx, (const TIn*)w, ldw,             \
+                                                          (const TIn*)bias, (TOut*)out, ldo, M, N, K)
+  if (accum) {
+    if (act == 0) EPD_LAUNCH(0, true); else if (act == 1) EPD_LAUNCH(1, true); else EPD_LAUNCH(2, true);
+  } else {
+    if (act == 0) EPD_LAUNCH(0, false); else if (act == 1) EPD_LAUNCH(1, false); else EPD_LAUNCH(2, false);
+  }
+#undef EPD_LAUNCH
+  return cudaGetLastError();
+}
+
+cudaError_t linear_fma(int dtype, const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias,
+                       void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, cudaStream_t s) {
+  if (M == 0 || N == 0) return cudaSuccess;
+  const bool out_f32 = (dtype == EPD_DTYPE_F32) || (flags & (EPD_LINEAR_OUT_F32 | EPD_LINEAR_ACCUMULATE));
+  if (dtype == EPD_DTYPE_F32) return linear_fma_t<float, float>(x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, s);
+  if (out_f32) return linear_fma_t<__nv_bfloat16, float>(x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, s);
+  return linear_fma_t<__nv_bfloat16, __nv_bfloat16>(x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, s);
+}
+
+// =============================================================================================
+// RMSNorm: one warp per row of the float residual stream; optional scattered destination row.
+// Bytes per row: 4h read + sizeof(T)h written (the second pass re-reads the row from L1/L2).
+// =============================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256)
+rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ out,
+               const int32_t* __restrict__ dst_row, int64_t rows, int hidden, float eps) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const float* xr = x + row * hidden;
+  float ss = 0.0f;
+  if ((hidden & 3) == 0) {
+    const float4* x4 = reinterpret_cast<const float4*>(xr);
+    for (int i = lane; i < hidden / 4; i += 32) {
+      const float4 v = x4[i];
+      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+  } else {
+    for (int i = lane; i < hidden; i += 32) ss += xr[i] * xr[i];
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float inv = 1.0f / sqrtf(ss / (float)hidden + eps);
+  const int64_t drow = dst_row ? (int64_t)dst_row[row] : row;
+  T* orow = out + drow * hidden;
+  if ((hidden & 3) == 0) {
+    const float4* x4 = reinterpret_cast<const float4*>(xr);
+    for (int i = lane; i < hidden / 4; i += 32) {
+      const float4 v = x4[i];
+      const float r0 = v.x * inv * to_float<T>(gain[4 * i + 0]);
+      const float r1 = v.y * inv * to_float<T>(gain[4 * i + 1]);
+      const float r2 = v.z * inv * to_float<T>(gain[4 * i + 2]);
+      const float r3 = v.w * inv * to_float<T>(gain[4 * i + 3]);
+      if constexpr (sizeof(T) == 4) {
+        reinterpret_cast<float4*>(orow)[i] = make_float4(r0, r1, r2, r3);
+      } else {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&lo);
+        pk.y = *reinterpret_cast<uint32_t*>(&hi);
+        reinterpret_cast<uint2*>(orow)[i] = pk;
+      }
+    }
+  } else {
+    for (int i = lane; i < hidden; i += 32) orow[i] = from_float<T>(xr[i] * inv * to_float<T>(gain[i]));
+  }
+}
+
+cudaError_t rmsnorm(int dtype, const void* x, const void* gain, void* out, const int32_t* dst_row, int64_t T,
+                    int hidden, float eps, cudaStream_t s) {
+  if (T == 0) return cudaSuccess;
+  const int warps = 8;
+  const unsigned blocks = (unsigned)((T + warps - 1) / warps);
+  if (dtype == EPD_DTYPE_F32)
+    rmsnorm_kernel<float><<<blocks, warps * 32, 0, s>>>((const float*)x, (const float*)gain, (float*)out, dst_row, T,
+                                                        hidden, eps);
+  else
+    rmsnorm_kernel<__nv_bfloat16><<<blocks, warps * 32, 0, s>>>((const float*)x, (const __nv_bfloat16*)gain,
+                                                                (__nv_bfloat16*)out, dst_row, T, hidden, eps);
+  return cudaGetLastError();
+}
+
+// =============================================================================================
+// Rotary table and rotary + head split.
+// table[p * nf + f] = (cos(p w_f), sin(p w_f)), w_f = theta^(-2f/(head_dim/2)), nf = head_dim/4.
+// =============================================================================================
+__global__ void rope_table_kernel(float2* table, int rows, int nf, int d2, double theta) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= rows * nf) return;
+  const int p = idx / nf, f = idx % nf;
+  const double w = pow(theta, -2.0 * (double)f / (double)d2);
+  double sn, cs;
+  sincos((double)p * w, &sn, &cs);
+  table[idx] = make_float2((float)cs, (float)sn);
+}
+
+cudaError_t rope_table(float2* table, int rows, int head_dim, float theta, cudaStream_t s) {
+  const int nf = head_dim / 4;
+  const int total = rows * nf;
+  if (total == 0) return cudaSuccess;
+  rope_table_kernel<<<(total + 127) / 128, 128, 0, s>>>(table, rows, nf, head_dim / 2, (double)theta);
+  return cudaGetLastError();
+}
+
+// One block per token.  Threads walk the token's q|k|v row in units of 2 adjacent frequencies
+// (so loads and stores are 2-element vectors for bf16): unit u of a head covers pairs
+// (f, f+nf), (f+1, f+1+nf) of one half.
+template <typename T>
+__global__ void __launch_bounds__(128)
+rope_split_kernel(const T* __restrict__ qkv, const int32_t* __restrict__ pos_row,
+                  const int32_t* __restrict__ pos_col, const float2* __restrict__ table, int table_rows,
+                  T* __restrict__ q, T* __restrict__ k, T* __restrict__ v, int64_t Tn, int heads, int dh, int dhp,
+                  float theta, float q_scale) {
+  const int64_t j = blockIdx.x;
+  const int h = heads * dh;
+  const int d2 = dh / 2, nf = dh / 4;
+  const T* row = qkv + j * 3 * (int64_t)h;
+  const int pr = pos_row[j], pc = pos_col[j];
+  const bool rotate = theta > 0.0f;
+  // q and k: heads * 2 halves * nf frequencies, for 2 tensors
+  const int n_rot = 2 * heads * 2 * nf;
+  for (int e = threadIdx.x; e < n_rot; e += blockDim.x) {
+    const int f = e % nf;
+    int rest = e / nf;
+    const int half = rest & 1; rest >>= 1;
+    const int hd = rest % heads;
+    const int which = rest / heads;  // 0 = q, 1 = k
+    const int p = half ? pc : pr;
+    float cs = 1.0f, sn = 0.0f;
+    if (rotate) {
+      if (table != nullptr && p < table_rows) {
+        const float2 t = table[p * nf + f];
+        cs = t.x; sn = t.y;
+      } else {
+        const double w = pow((double)theta, -2.0 * (double)f / (double)d2);
+        double s_, c_;
+        sincos((double)p * w, &s_, &c_);
+        cs = (float)c_; sn = (float)s_;
+      }
+    }
+    const int i0 = half * d2 + f, i1 = i0 + nf;
+    const T* src = row + which * h + hd * dh;
+    const float a = to_float<T>(src[i0]), b = to_float<T>(src[i1]);
+    float ra = a * cs - b * sn, rb = b * cs + a * sn;
+    if (which == 0) { ra *= q_scale; rb *= q_scale; }
+    T* dst = (which == 0 ? q : k) + ((int64_t)hd * Tn + j) * dhp;
+    dst[i0] = from_float<T>(ra);
+    dst[i1] = from_float<T>(rb);
+  }
+  // v copy and zero padding of all three
+  for (int e = threadIdx.x; e < heads * dhp; e += blockDim.x) {
+    const int d = e % dhp, hd = e / dhp;
+    const int64_t o = ((int64_t)hd * Tn + j) * dhp + d;
+    if (d < dh) {
+      v[o] = row[2 * h + hd * dh + d];
+    } else {
+      v[o] = from_float<T>(0.0f);
+      q[o] = from_float<T>(0.0f);
+      k[o] = from_float<T>(0.0f);
+    }
+  }
+}
+
+cudaError_t rope_split(int dtype, const void* qkv, const int32_t* pos_row, const int32_t* pos_col,
+                       const float2* table, int table_rows, void* q, void* k, void* v, int64_t T, int heads,
+                       int head_dim, float theta, float q_scale, cudaStream_t s) {
+  if (T == 0) return cudaSuccess;
+  const int dhp = padded_head_dim(head_dim);
+  if (dtype == EPD_DTYPE_F32)
+    rope_split_kernel<float><<<(unsigned)T, 128, 0, s>>>((const float*)qkv, pos_row, pos_col, table, table_rows,
+                                                         (float*)q, (float*)k, (float*)v, T, heads, head_dim, dhp,
+                                                         theta, q_scale);
+  else
+    rope_split_kernel<__nv_bfloat16><<<(unsigned)T, 128, 0, s>>>(
+        (const __nv_bfloat16*)qkv, pos_row, pos_col, table, table_rows, (__nv_bfloat16*)q, (__nv_bfloat16*)k,
+        (__nv_bfloat16*)v, T, heads, head_dim, dhp, theta, q_scale);
+  return cudaGetLastError();
+}
+
+// =============================================================================================
+// Attention with plain FMAs: one warp per (query token, head).  Keys are visited 32 at a time:
+// lane l scores key l of the chunk, the warp keeps a running max / sum (online softmax, base 2:
+// q arrives multiplied by log2(e)/sqrt(head_dim)), and lane l accumulates output dims l, l+32, ...
+// =============================================================================================
+template <typename T>
+__global__ void __launch_bounds__(256)
+attention_fma_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
+                     const int32_t* __restrict__ cu, int n_seg, T* __restrict__ out, int64_t Tn, int heads, int dh,
+                     int dhp) {
+  __shared__ float sq[8][kMaxHeadDim];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const int64_t j = (int64_t)blockIdx.x * 8 + wid;
+  const int hd = blockIdx.y;
+  if (j >= Tn) return;
+  int lo = 0, hi = n_seg;
+  while (hi - lo > 1) {
+    int mid = (lo + hi) >> 1;
+    if (cu[mid] <= j) lo = mid; else hi = mid;
+  }
+  const int kbeg = cu[lo], kend = cu[lo + 1];
+  const T* qrow = q + ((int64_t)hd * Tn + j) * dhp;
+  for (int d = lane; d < dh; d += 32) sq[wid][d] = to_float<T>(qrow[d]);
+  __syncwarp();
+  float m = -INFINITY, l = 0.0f;
+  float acc[kMaxHeadDim / 32] = {};
+  for (int c0 = kbeg; c0 < kend; c0 += 32) {
+    const int key = c0 + lane;
+    float sc = -INFINITY;
+    if (key < kend) {
+      const T* krow = k + ((int64_t)hd * Tn + key) * dhp;
+      float dot = 0.0f;
+      for (int d = 0; d < dh; ++d) dot = fmaf(sq[wid][d], to_float<T>(krow[d]), dot);
+      sc = dot;
+    }
+    float cmax = sc;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cmax = fmaxf(cmax, __shfl_xor_sync(0xffffffffu, cmax, o));
+    const float m_new = fmaxf(m, cmax);
+    const float scale = exp2f(m - m_new);
+    const float p = exp2f(sc - m_new);
+    float psum = p;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) psum += __shfl_xor_sync(0xffffffffu, psum, o);
+    l = l * scale + psum;
+    m = m_new;
+#pragma unroll
+    for (int i = 0; i < kMaxHeadDim / 32; ++i) acc[i] *= scale;
+    const int nk = min(32, kend - c0);
+    for (int kk = 0; kk < nk; ++kk) {
+      const float pk = __shfl_sync(0xffffffffu, p, kk);
+      const T* vrow = v + ((int64_t)hd * Tn + c0 + kk) * dhp;
+#pragma unroll
+      for (int i = 0; i < kMaxHeadDim / 32; ++i) {
+        const int d = lane + 32 * i;
+        if (d < dh) acc[i] = fmaf(pk, to_float<T>(vrow[d]), acc[i]);
+      }
+    }
+  }
+  const float inv = 1.0f / l;
+  T* orow = out + j * (int64_t)(heads * dh) + hd * dh;
+#pragma unroll
+  for (int i = 0; i < kMaxHeadDim / 32; ++i) {
+    const int d = lane + 32 * i;
+    if (d < dh) orow[d] = from_float<T>(acc[i] * inv);
+  }
+}
+
+cudaError_t attention_fma(int dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                          int n_seg, void* out, int64_t T, int heads, int head_dim, cudaStream_t s) {
+  if (T == 0) return cudaSuccess;
+  const int dhp = padded_head_dim(head_dim);
+  dim3 grid((unsigned)((T + 7) / 8), (unsigned)heads);
+  if (dtype == EPD_DTYPE_F32)
+    attention_fma_kernel<float><<<grid, 256, 0, s>>>((const float*)q, (const float*)k, (const float*)v, cu_seqlens,
+                                                     n_seg, (float*)out, T, heads, head_dim, dhp);
+  else
+    attention_fma_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k,
+                                                             (const __nv_bfloat16*)v, cu_seqlens, n_seg,
+                                                             (__nv_bfloat16*)out, T, heads, head_dim, dhp);
+  return cudaGetLastError();
+}
+
+// =============================================================================================
+// 2x2 merge as a gather: slot s = 4*o + q of the merged matrix copies row merge_idx[s] of y.
+// =============================================================================================
+__global__ void __launch_bounds__(128)
+merge_gather_kernel(const uint8_t* __restrict__ y, const int32_t* __restrict__ merge_idx, uint8_t* __restrict__ out,
+                    int64_t slots, int row_bytes) {
+  const int64_t s = blockIdx.x;
+  if (s >= slots) return;
+  const uint8_t* src = y + (int64_t)merge_idx[s] * row_bytes;
+  uint8_t* dst = out + s * row_bytes;
+  if ((row_bytes & 15) == 0) {
+    for (int i = threadIdx.x; i < row_bytes / 16; i += blockDim.x)
+      reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(src)[i];
+  } else {
+    for (int i = threadIdx.x; i < row_bytes / 2; i += blockDim.x)
+      reinterpret_cast<uint16_t*>(dst)[i] = reinterpret_cast<const uint16_t*>(src)[i];
+  }
+}
+
+cudaError_t merge_gather(int dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm, int hidden,
+                         cudaStream_t s) {
+  if (Tm == 0) return cudaSuccess;
+  const int row_bytes = hidden * (dtype == EPD_DTYPE_F32 ? 4 : 2);
+  merge_gather_kernel<<<(unsigned)(Tm * 4), 128, 0, s>>>((const uint8_t*)y, merge_idx, (uint8_t*)out, Tm * 4,
+                                                         row_bytes);
+  return cudaGetLastError();
+}
+
+}  // namespace epd

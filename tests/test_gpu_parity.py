@@ -1,0 +1,389 @@
+"""GPU parity: every step of the CUDA path and the whole stage against the CPU oracle,
+through the C ABI, on the same seeded inputs.
+
+Tolerances (relative Frobenius error ||G - O||_F / ||O||_F):
+  float configurations     <= 1e-4 (whole stage and every step)
+  bf16 configurations      <= 1e-2 per encoder block (block output for the GPU's own block input),
+                           <= 3e-2 on the final features
+  integer layout           bit-exact
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+import paper_2601_11590_b200 as epd
+from oracle import encoder_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16_BLOCK = 1e-2
+TOL_BF16_FINAL = 3e-2
+# a single bf16 step: inputs are exact, the only roundings are fp32 accumulation and one bf16 store (2^-9)
+TOL_BF16_STEP = 4e-3
+
+
+def rel_err(got, ref):
+    got = np.asarray(got, dtype=np.float64)
+    ref = np.asarray(ref, dtype=np.float64)
+    assert got.shape == ref.shape, (got.shape, ref.shape)
+    return float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300))
+
+
+def to_np(t):
+    return t.detach().float().cpu().numpy().astype(np.float64)
+
+
+def dev(a, dtype):
+    return epd.to_device(a, dtype)
+
+
+def rnd(shape, seed, std, dtype):
+    return synth.normal(seed, f"t{seed}", shape, std, 0.0, dtype)
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    from paper_2601_11590_b200 import build
+    build.build_library()
+    epd.load_library()
+
+
+# ----------------------------------------------------------------------------- single steps
+
+@pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
+@pytest.mark.parametrize("M,N,K", [(1, 8, 8), (77, 40, 24), (200, 136, 72), (300, 1080, 288), (130, 288, 1080)])
+@pytest.mark.parametrize("mode", ["plain", "gelu_tanh", "gelu_erf", "accum", "out_f32", "nobias"])
+def test_linear(dtype, M, N, K, mode):
+    x = rnd((M, K), 1, 1.0, dtype)
+    w = rnd((N, K), 2, 1.0 / np.sqrt(K), dtype)
+    b = None if mode == "nobias" else rnd((N,), 3, 0.5, dtype)
+    flags = {"plain": 0, "nobias": 0, "gelu_tanh": epd.LINEAR_GELU_TANH, "gelu_erf": epd.LINEAR_GELU_ERF,
+             "accum": epd.LINEAR_ACCUMULATE, "out_f32": epd.LINEAR_OUT_F32}[mode]
+    ref = O.linear(x.astype(np.float64), w.astype(np.float64), None if b is None else b.astype(np.float64))
+    if mode == "gelu_tanh":
+        ref = O.gelu(ref, O.ACT_GELU_TANH)
+    if mode == "gelu_erf":
+        ref = O.gelu(ref, O.ACT_GELU_ERF)
+    out_f32 = dtype == epd.DTYPE_F32 or mode in ("accum", "out_f32")
+    r0 = rnd((M, N), 4, 1.0, epd.DTYPE_F32)
+    out = torch.from_numpy(r0.copy()).cuda() if out_f32 else torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    if mode == "accum":
+        ref = ref + r0.astype(np.float64)
+    epd.op_linear(dtype, dev(x, dtype), dev(w, dtype), dev(b, dtype), out, M, N, K, flags)
+    torch.cuda.synchronize()
+    tol = TOL_F32 if dtype == epd.DTYPE_F32 else (1e-5 if out_f32 else TOL_BF16_STEP)
+    assert rel_err(to_np(out), ref) <= tol
+
+
+@pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
+@pytest.mark.parametrize("T,h", [(1, 8), (37, 256), (100, 1152), (9, 3200), (5, 30)])
+def test_rmsnorm(dtype, T, h):
+    x = rnd((T, h), 5, 3.0, epd.DTYPE_F32)
+    g = synth.normal(6, "g", (h,), 0.02, 1.0, dtype)
+    ref = O.rmsnorm(x.astype(np.float64), g.astype(np.float64), 1e-6)
+    out = torch.zeros((T, h), dtype=epd.torch_dtype(dtype), device="cuda")
+    epd.op_rmsnorm(dtype, torch.from_numpy(x).cuda(), dev(g, dtype), out, 1e-6)
+    assert rel_err(to_np(out), ref) <= (1e-6 if dtype == epd.DTYPE_F32 else TOL_BF16_STEP)
+    # scattered destination rows (the fused 2x2 merge)
+    perm = np.random.default_rng(0).permutation(T).astype(np.int32)
+    out2 = torch.zeros_like(out)
+    epd.op_rmsnorm(dtype, torch.from_numpy(x).cuda(), dev(g, dtype), out2, 1e-6,
+                   dst_row=torch.from_numpy(perm).cuda())
+    assert torch.equal(out2[torch.from_numpy(perm.astype(np.int64)).cuda()], out)
+
+
+@pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
+@pytest.mark.parametrize("heads,dh", [(4, 64), (3, 72), (2, 128), (2, 8)])
+def test_rope_split(dtype, heads, dh):
+    T, h = 53, heads * dh
+    qkv = rnd((T, 3 * h), 7, 1.0, dtype)
+    rng = np.random.default_rng(1)
+    pr, pc = rng.integers(0, 128, T).astype(np.int32), rng.integers(0, 128, T).astype(np.int32)
+    scale = 0.37
+    q, k, v = epd.op_rope_split(dtype, dev(qkv, dtype), torch.from_numpy(pr).cuda(), torch.from_numpy(pc).cuda(),
+                                heads, dh, 10000.0, scale)
+    x = qkv.astype(np.float64)
+    qr = O.rope_2d(x[:, :h].reshape(T, heads, dh), pr, pc, 10000.0) * scale
+    kr = O.rope_2d(x[:, h:2 * h].reshape(T, heads, dh), pr, pc, 10000.0)
+    vr = x[:, 2 * h:].reshape(T, heads, dh)
+    dhp = epd.padded_head_dim(dh)
+    assert q.shape == (heads, T, dhp)
+    tol = 1e-6 if dtype == epd.DTYPE_F32 else TOL_BF16_STEP
+    for got, ref in ((q, qr), (k, kr), (v, vr)):
+        g = to_np(got)
+        assert rel_err(g[:, :, :dh].transpose(1, 0, 2), ref) <= tol
+        assert np.all(g[:, :, dh:] == 0.0)
+    assert np.array_equal(to_np(v)[:, :, :dh].transpose(1, 0, 2), vr)  # v is a pure copy
+
+
+def _attention_case(dtype, heads, dh, seglens, seed, logit_scale=1.0, flags=0):
+    T = int(sum(seglens))
+    cu = np.concatenate([[0], np.cumsum(seglens)]).astype(np.int32)
+    dhp = epd.padded_head_dim(dh)
+    qs = 1.4426950408889634 / np.sqrt(dh)
+    q = rnd((heads, T, dh), seed, logit_scale, dtype)
+    k = rnd((heads, T, dh), seed + 1, logit_scale, dtype)
+    v = rnd((heads, T, dh), seed + 2, 1.0, dtype)
+    # the kernel receives q already multiplied by log2(e)/sqrt(dh); round that product the way the
+    # rotary step stores it so both sides start from the same numbers
+    q_scaled = (q.astype(np.float64) * qs).astype(np.float32)
+    if dtype == epd.DTYPE_BF16:
+        q_scaled = synth.round_to_bf16(q_scaled)
+
+    def pad(a):
+        out = np.zeros((heads, T, dhp), np.float32)
+        out[:, :, :dh] = a
+        return dev(out, dtype)
+
+    out = epd.op_attention(dtype, pad(q_scaled), pad(k), pad(v), torch.from_numpy(cu).cuda(), cu, dh, flags)
+    q_eff = q_scaled.astype(np.float64) / qs
+    ref = O.attention_block_diagonal(q_eff.transpose(1, 0, 2), k.astype(np.float64).transpose(1, 0, 2),
+                                     v.astype(np.float64).transpose(1, 0, 2), cu).reshape(T, heads * dh)
+    return to_np(out), ref
+
+
+@pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
+@pytest.mark.parametrize("heads,dh,seglens", [
+    (2, 64, [256, 256]), (3, 72, [4, 196, 300, 33]), (2, 128, [129, 64, 1]), (2, 72, [784]), (1, 8, [5])])
+def test_attention(dtype, heads, dh, seglens):
+    got, ref = _attention_case(dtype, heads, dh, seglens, 10)
+    assert rel_err(got, ref) <= (1e-5 if dtype == epd.DTYPE_F32 else TOL_BF16_STEP)
+
+
+@pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
+def test_attention_peaked_logits(dtype):
+    """Logit standard deviation ~ 50: exercises the running-max rescaling of the online softmax."""
+    got, ref = _attention_case(dtype, 2, 72, [300, 520], 20, logit_scale=2.5)
+    assert rel_err(got, ref) <= (1e-4 if dtype == epd.DTYPE_F32 else 1e-2)
+
+
+@pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
+def test_merge(dtype):
+    grids = [(1, 4, 6), (2, 2, 2), (1, 2, 8)]
+    bk = O.bookkeeping(grids)
+    T, h = int(bk["cu_seqlens"][-1]), 40
+    y = rnd((T, h), 30, 1.0, dtype)
+    out = epd.op_merge(dtype, dev(y, dtype), torch.from_numpy(bk["merge_idx"].reshape(-1).copy()).cuda())
+    assert np.array_equal(to_np(out), O.merge_2x2(y.astype(np.float64), bk["merge_idx"]))
+
+
+# ----------------------------------------------------------------------------- integer layout
+
+def _golden_grids():
+    import os
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", "e2p_feature_rows.txt")) as fh:
+        for line in fh:
+            if line.strip() and not line.startswith("#"):
+                rows.append(tuple(int(v) for v in line.split()))
+    return rows
+
+
+def test_bookkeeping_bit_exact_including_paper_shapes():
+    cfg = synth.tiny_variant(head_dim=8, heads=2, layers=0, mlp=16, patch=1, out_dim=8)
+    w = synth.make_weights(cfg, seed=1)
+    golden = _golden_grids()
+    cases = [
+        [(1, 2, 2)],
+        [(1, 4, 6), (3, 2, 4), (1, 2, 2)],
+        [(2, 6, 2), (1, 16, 16), (1, 2, 30)],
+        [(1, r[2], r[3]) for r in golden],
+    ]
+    maxT = max(synth.num_tokens(g) for g in cases)
+    enc = epd.Encoder(cfg, w, max_tokens=maxT, max_images=8, max_grid=512)
+    for grids in cases:
+        T = synth.num_tokens(grids)
+        patches = dev(synth.make_patches(cfg, grids, seed=2), cfg.dtype)
+        feats, cu_rows = enc.encode(patches, grids)
+        bk = O.bookkeeping(grids)
+        got = enc.debug_bookkeeping(len(grids), T)
+        for key in ("cu_seqlens", "pos_row", "pos_col", "merge_idx"):
+            assert np.array_equal(got[key], bk[key]), key
+        assert np.array_equal(cu_rows, bk["cu_out"])
+        assert feats.shape == (T // 4, cfg.out_dim)
+    assert np.diff(cu_rows).tolist() == [r[4] for r in golden]
+    assert enc.last_status() == epd.EPD_OK
+    enc.close()
+
+
+# ----------------------------------------------------------------------------- whole stage
+
+def _run_stage(cfg, grids, seed=0, qkv_scale=1.0, with_taps=True, max_grid=128):
+    w = synth.make_weights(cfg, seed=seed, qkv_scale=qkv_scale)
+    patches = synth.make_patches(cfg, grids, seed=seed)
+    T = synth.num_tokens(grids)
+    enc = epd.Encoder(cfg, w, max_tokens=T, max_images=max(1, len(grids)), max_grid=max_grid)
+    taps = None
+    if with_taps:
+        taps = [torch.zeros((T, cfg.hidden), dtype=torch.float32, device="cuda") for _ in range(cfg.layers + 1)]
+        enc.set_taps(taps)
+    K = cfg.patch_dim
+    ld = K if cfg.dtype == epd.DTYPE_F32 else (K + 7) // 8 * 8
+    p = torch.zeros((T, ld), dtype=epd.torch_dtype(cfg.dtype), device="cuda")
+    p[:, :K] = dev(patches, cfg.dtype)
+    feats, cu_rows = enc.encode(p, grids)
+    torch.cuda.synchronize()
+    assert enc.last_status() == epd.EPD_OK
+    assert enc.last_launch_count() >= 2
+    return enc, w, patches, feats, cu_rows, taps
+
+
+def _check_stage(cfg, grids, tol_final, tol_block, **kw):
+    enc, w, patches, feats, cu_rows, taps = _run_stage(cfg, grids, **kw)
+    ref, ref_taps = O.encode(cfg, w, patches, grids, return_taps=True)
+    bk = O.bookkeeping(grids)
+    assert np.array_equal(cu_rows, bk["cu_out"])
+    e_final = rel_err(to_np(feats), ref)
+    # per-block error: oracle block applied to the GPU's own block input
+    errs = []
+    for l in range(cfg.layers):
+        x_in = to_np(taps[l])
+        want = O.block(cfg, w["layers"][l], x_in, bk)
+        got = to_np(taps[l + 1])
+        errs.append((rel_err(got, want), rel_err(got - x_in, want - x_in)))
+    assert rel_err(to_np(taps[0]), ref_taps[0]) <= (1e-5 if cfg.dtype == epd.DTYPE_F32 else 1e-5)
+    assert all(e[0] <= tol_block for e in errs), errs
+    assert e_final <= tol_final, e_final
+    enc.close()
+    return e_final, errs
+
+
+def test_stage_tiny_fp32_config():
+    cfg, grids = synth.WORKLOADS["cfg0_tiny_fp32"]
+    e, errs = _check_stage(cfg, grids, TOL_F32, TOL_F32)
+    print("cfg0 final", e, "blocks", errs)
+
+
+def test_stage_fp32_ragged_grids_and_clip():
+    cfg = synth.TINY_FP32
+    _check_stage(cfg, [(1, 2, 2), (2, 6, 10), (1, 18, 14), (1, 4, 2)], TOL_F32, TOL_F32, seed=3)
+
+
+def _small_bf16(layers=2, heads=4, dh=72, mlp=1080, act=synth.ACT_GELU_TANH, tp=1, patch=16):
+    import dataclasses
+    return dataclasses.replace(synth.VIT_06B, name="small-bf16", hidden=heads * dh, heads=heads, head_dim=dh,
+                               layers=layers, mlp=mlp, act=act, temporal_patch=tp, patch=patch,
+                               proj_hidden=4 * heads * dh, out_dim=512)
+
+
+@pytest.mark.parametrize("variant", ["dh72", "dh128_erf", "dh64_video"])
+def test_stage_small_bf16(variant):
+    if variant == "dh72":
+        cfg, grids = _small_bf16(), [(1, 28, 28), (1, 14, 20), (1, 2, 2), (1, 30, 8)]
+    elif variant == "dh128_erf":
+        import dataclasses
+        cfg = dataclasses.replace(_small_bf16(heads=3, dh=128, mlp=1536, act=synth.ACT_GELU_ERF), patch=14)
+        grids = [(1, 16, 16), (1, 32, 32)]
+    else:
+        cfg, grids = _small_bf16(heads=4, dh=64, mlp=1000, tp=2), [(4, 10, 12), (1, 22, 6)]
+    e, errs = _check_stage(cfg, grids, TOL_BF16_FINAL, TOL_BF16_BLOCK, seed=5)
+    print(variant, "final", e, "blocks", errs)
+
+
+def test_stage_small_bf16_peaked_attention():
+    """W_qkv scaled x8 (not a benchmark configuration): sharply peaked softmax rows."""
+    cfg, grids = _small_bf16(), [(1, 20, 24), (1, 12, 12)]
+    _check_stage(cfg, grids, TOL_BF16_FINAL, TOL_BF16_BLOCK, seed=6, qkv_scale=8.0)
+
+
+def test_block_diagonal_isolation_on_gpu():
+    """An item's features do not depend on the rest of the batch (bit-identical on the GPU when the
+    launch geometry is the same; within tolerance against the item encoded alone)."""
+    cfg = _small_bf16()
+    grids = [(1, 12, 12), (1, 8, 16), (1, 20, 6)]
+    w = synth.make_weights(cfg, seed=7)
+    patches = synth.make_patches(cfg, grids, seed=7)
+    T = synth.num_tokens(grids)
+    enc = epd.Encoder(cfg, w, max_tokens=T, max_images=4)
+    p = dev(patches, cfg.dtype)
+    f0, cu_rows = enc.encode(p, grids)
+    f0 = f0.clone()
+    bk = O.bookkeeping(grids)
+    cu = bk["cu_seqlens"]
+    p2 = p.clone()
+    p2[cu[0]:cu[1]] *= -1.5
+    p2[cu[2]:cu[3]] += 1.0
+    f1, _ = enc.encode(p2, grids)
+    torch.cuda.synchronize()
+    assert torch.equal(f0[cu_rows[1]:cu_rows[2]], f1[cu_rows[1]:cu_rows[2]])
+    assert not torch.equal(f0[cu_rows[0]:cu_rows[1]], f1[cu_rows[0]:cu_rows[1]])
+    alone, _ = enc.encode(p[cu[1]:cu[2]].contiguous(), [grids[1]])
+    assert rel_err(to_np(alone), to_np(f0[cu_rows[1]:cu_rows[2]])) <= TOL_BF16_FINAL
+    enc.close()
+
+
+def test_run_to_run_determinism():
+    cfg = _small_bf16()
+    grids = [(1, 16, 16), (1, 10, 30)]
+    enc, w, patches, feats, _, _ = _run_stage(cfg, grids, seed=8, with_taps=False)
+    first = feats.clone()
+    p = dev(patches, cfg.dtype)
+    for _ in range(3):
+        again, _ = enc.encode(p, grids)
+        torch.cuda.synchronize()
+        assert torch.equal(first, again)
+    enc.close()
+
+
+def test_host_buffer_entry_point_matches_device_entry_point():
+    cfg = _small_bf16()
+    grids = [(1, 16, 16), (1, 6, 10)]
+    enc, w, patches, feats, cu_rows, _ = _run_stage(cfg, grids, seed=9, with_taps=False)
+    hp = dev(patches, cfg.dtype).cpu().pin_memory()
+    hf = torch.zeros((feats.shape[0], cfg.out_dim), dtype=feats.dtype).pin_memory()
+    rows, cu2 = enc.encode_host(hp, grids, hf)
+    torch.cuda.synchronize()
+    assert rows == feats.shape[0] and np.array_equal(cu2, cu_rows)
+    assert torch.equal(hf, feats.cpu())
+    enc.close()
+
+
+# ----------------------------------------------------------------------------- edge cases / errors
+
+def test_empty_and_invalid_batches():
+    cfg = synth.tiny_variant(head_dim=8, heads=2, layers=1, mlp=16, patch=1, out_dim=8)
+    w = synth.make_weights(cfg, seed=1)
+    enc = epd.Encoder(cfg, w, max_tokens=64, max_images=2, max_grid=8)
+    feats = torch.zeros((16, cfg.out_dim), device="cuda")
+    out, cu_rows = enc.encode(None, [], features=feats)
+    assert out.shape[0] == 0 and cu_rows.tolist() == [0]
+    p = dev(synth.make_patches(cfg, [(1, 2, 2)]), cfg.dtype)
+    for bad in ([(1, 3, 2)], [(0, 2, 2)], [(1, 2, -2)]):
+        with pytest.raises(epd.EpdError) as ei:
+            enc.encode(p, bad, features=feats)
+        assert ei.value.status == epd.EPD_EINVAL
+    for too_big in ([(1, 2, 2)] * 3, [(1, 10, 2)], [(1, 8, 8), (1, 2, 2)]):
+        with pytest.raises(epd.EpdError) as ei:
+            enc.encode(p, too_big, features=feats)
+        assert ei.value.status == epd.EPD_ECAPACITY
+    with pytest.raises(epd.EpdError) as ei:   # feature buffer too small
+        enc.encode(dev(synth.make_patches(cfg, [(1, 8, 8)]), cfg.dtype), [(1, 8, 8)], features=feats[:8])
+    assert ei.value.status == epd.EPD_ECAPACITY
+    # the encoder still works afterwards, at its maximum size
+    grids = [(1, 8, 8)]
+    out, _ = enc.encode(dev(synth.make_patches(cfg, grids), cfg.dtype), grids, features=feats)
+    ref = O.encode(cfg, w, synth.make_patches(cfg, grids), grids)
+    assert rel_err(to_np(out), ref) <= TOL_F32
+    enc.close()
+
+
+def test_create_rejects_small_workspace():
+    lib = epd.load_library()
+    c = epd.make_config(synth.TINY_FP32, 512, 2, 16)
+    need = lib.epd_encoder_workspace_bytes(ctypes.byref(c))
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    w = epd.WeightsStruct()
+    handle = ctypes.c_void_p()
+    w.patch_w = ws.data_ptr(); w.patch_w_ld = 588; w.proj_w1 = ws.data_ptr(); w.final_norm_w = ws.data_ptr()
+    arr = (ctypes.c_void_p * 2)(ws.data_ptr(), ws.data_ptr())
+    for n in ("norm1_w", "qkv_w", "out_w", "norm2_w", "fc1_w", "fc2_w"):
+        setattr(w, n, ctypes.cast(arr, ctypes.POINTER(ctypes.c_void_p)))
+    base = (ws.data_ptr() + 255) // 256 * 256
+    assert lib.epd_encoder_create(ctypes.byref(c), ctypes.byref(w), base, need - 4096, ctypes.byref(handle)) \
+        == epd.EPD_ENOMEM
+    assert lib.epd_encoder_create(ctypes.byref(c), ctypes.byref(w), base + 8, need, ctypes.byref(handle)) \
+        == epd.EPD_EINVAL
