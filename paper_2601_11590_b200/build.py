@@ -25,11 +25,28 @@ def sources():
     return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cu"))
 
 
-def _stale(target: str, deps) -> bool:
-    if not os.path.exists(target):
+def _digest(paths) -> str:
+    """Content hash of the given files and the compiler flags (file times do not survive a copy)."""
+    import hashlib
+    h = hashlib.sha256(" ".join(NVCC_FLAGS[:-4]).encode())
+    for p in sorted(paths):
+        h.update(os.path.basename(p).encode())
+        with open(p, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def _stale(target: str, digest: str) -> bool:
+    stamp = target + ".sha256"
+    if not (os.path.exists(target) and os.path.exists(stamp)):
         return True
-    t = os.path.getmtime(target)
-    return any(os.path.getmtime(d) > t for d in deps)
+    with open(stamp) as fh:
+        return fh.read().strip() != digest
+
+
+def _stamp(target: str, digest: str) -> None:
+    with open(target + ".sha256", "w") as fh:
+        fh.write(digest)
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
@@ -41,22 +58,26 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     for src in sources():
         obj = os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        if force or _stale(obj, [src] + headers):
+        dig = _digest([src] + headers)
+        if force or _stale(obj, dig):
             cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
-            jobs.append(cmd)
+            jobs.append((cmd, obj, dig))
 
-    def run(cmd):
+    def run(job):
+        cmd, target, dig = job
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             raise RuntimeError("nvcc failed: " + " ".join(cmd) + "\n" + r.stdout + r.stderr)
+        _stamp(target, dig)
         return r.stderr
 
     with ThreadPoolExecutor(max_workers=max(1, min(8, len(jobs) or 1))) as ex:
         for log in ex.map(run, jobs):
             if verbose and log:
                 sys.stderr.write(log)
-    if force or jobs or _stale(LIB, objs):
-        run([_nvcc(), "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"])
+    lib_digest = _digest(sources() + headers)
+    if force or jobs or _stale(LIB, lib_digest):
+        run(([_nvcc(), "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"], LIB, lib_digest))
     return LIB
 
 
