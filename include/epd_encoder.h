@@ -206,12 +206,14 @@ enum {
   EPD_LINEAR_GELU_ERF = 2,   /* apply erf-GELU after the bias */
   EPD_LINEAR_ACCUMULATE = 4, /* out (float) += result: the residual update */
   EPD_LINEAR_OUT_F32 = 8,    /* out is float even when dtype is bf16 */
-  EPD_LINEAR_FORCE_FMA = 16  /* use the plain-FMA kernel even where the tensor-core kernel applies */
+  EPD_LINEAR_FORCE_FMA = 16, /* use the plain-FMA kernel even where the tensor-core kernel applies */
+  EPD_LINEAR_TILE_N_SHIFT = 8 /* bits 8..16: tensor-core tile width override (0 = automatic; 128, 192, 256) */
 };
 
 /* out[M,N] = act(x[M,K] . w[N,K]^T + bias[N]) (optionally accumulated into a float out).
  * x, w: element type per dtype, leading dimensions ldx, ldw (elements); out: leading dimension
- * ldo.  All device pointers, 16-byte aligned. */
+ * ldo.  All device pointers, 16-byte aligned.  In bf16 the tcgen05 kernel is used when every
+ * leading dimension and N are multiples of 8; other shapes run on the plain-FMA kernel. */
 int epd_op_linear(int32_t dtype, const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias,
                   void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t flags, void* stream);
 

@@ -50,4 +50,13 @@ cudaError_t token_layout(const int32_t* grid_thw, const int32_t* cu_seqlens, con
                          int64_t T, int32_t* pos_row, int32_t* pos_col, int32_t* merge_slot, int32_t* merge_idx,
                          cudaStream_t s);
 
+
+// ---- tensor-core kernels (gemm_tcgen05.cu) ---------------------------------------------------
+// bf16 x bf16 -> fp32 linear layer on tcgen05; `status` (device int, may be NULL) receives
+// EPD_ETIMEOUT if a bounded wait expires.  forced_bn: 0 = choose the tile width automatically.
+bool linear_tc_supported(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, const void* out,
+                         int64_t ldo, int64_t M, int64_t N, int64_t K, int flags);
+cudaError_t linear_tc(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out, int64_t ldo,
+                      int64_t M, int64_t N, int64_t K, int flags, int forced_bn, int* status, cudaStream_t s);
+
 }  // namespace epd

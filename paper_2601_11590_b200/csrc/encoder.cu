@@ -132,7 +132,14 @@ int mark(epd_encoder* enc, int cls, cudaStream_t s) {
 int linear_dispatch(epd_encoder* enc, int dtype, const void* x, int64_t ldx, const void* w, int64_t ldw,
                     const void* bias, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int flags,
                     cudaStream_t s) {
-  (void)enc;
+  if (dtype == EPD_DTYPE_BF16 && !(flags & EPD_LINEAR_FORCE_FMA) &&
+      linear_tc_supported(x, ldx, w, ldw, bias, out, ldo, M, N, K, flags)) {
+    int* status = enc ? enc->at<int>(enc->lay.status) : nullptr;
+    const int forced_bn = (flags >> EPD_LINEAR_TILE_N_SHIFT) & 0x1FF;
+    if (forced_bn != 0 && forced_bn != 128 && forced_bn != 192 && forced_bn != 256) return EPD_EINVAL;
+    EPD_CUDA(linear_tc(x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, forced_bn, status, s));
+    return EPD_OK;
+  }
   EPD_CUDA(linear_fma(dtype, x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, s));
   return EPD_OK;
 }
@@ -340,6 +347,7 @@ int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, vo
   e->lay = lay;
   e->ws = static_cast<uint8_t*>(workspace);
   e->patch_dim = K;
+  e->use_tc = cfg->dtype == EPD_DTYPE_BF16;
   auto copy_list = [&](std::vector<const void*>& dst, const void* const* src, bool required) -> bool {
     dst.assign(L, nullptr);
     if (!src) return !required || L == 0;

@@ -79,6 +79,45 @@ def test_linear(dtype, M, N, K, mode):
     assert rel_err(to_np(out), ref) <= tol
 
 
+@pytest.mark.parametrize("tile_n", [0, 128, 192, 256])
+@pytest.mark.parametrize("M,N,K,ldpad", [
+    (1000, 1152, 1152, 0),     # several M tiles, K = 18 blocks
+    (300, 4304, 1152, 0),      # ragged N (4304 = 33*128 + 80)
+    (257, 1152, 4304, 0),      # ragged K (4304 = 67*64 + 16)
+    (2000, 2304, 320, 0),      # more tiles than SMs: every CTA walks several tiles, both accumulators
+    (130, 3200, 588, 4),       # K = 588 with leading dimensions padded to 592
+    (64, 8, 8, 0),             # smaller than one tile in every direction
+])
+@pytest.mark.parametrize("mode", ["plain", "gelu_tanh", "accum"])
+def test_linear_tensor_core_tiles(tile_n, M, N, K, ldpad, mode):
+    """bf16 linear layer on the tcgen05 kernel, every tile width, against the oracle and the FMA kernel."""
+    dtype = epd.DTYPE_BF16
+    ld = K + ldpad
+    x = np.zeros((M, ld), np.float32); x[:, :K] = rnd((M, K), 11, 1.0, dtype)
+    w = np.zeros((N, ld), np.float32); w[:, :K] = rnd((N, K), 12, 1.0 / np.sqrt(K), dtype)
+    if ldpad:   # the padding must be ignored, not multiplied in
+        x[:, K:] = 7.0
+        w[:, K:] = 7.0
+    b = rnd((N,), 13, 0.5, dtype)
+    flags = {"plain": 0, "gelu_tanh": epd.LINEAR_GELU_TANH, "accum": epd.LINEAR_ACCUMULATE}[mode]
+    ref = O.linear(x[:, :K].astype(np.float64), w[:, :K].astype(np.float64), b.astype(np.float64))
+    if mode == "gelu_tanh":
+        ref = O.gelu(ref, O.ACT_GELU_TANH)
+    r0 = rnd((M, N), 14, 1.0, epd.DTYPE_F32)
+    if mode == "accum":
+        ref = ref + r0.astype(np.float64)
+        make_out = lambda: torch.from_numpy(r0.copy()).cuda()
+    else:
+        make_out = lambda: torch.full((M, N), 99.0, dtype=torch.bfloat16, device="cuda")
+    xd, wd, bd = dev(x, dtype), dev(w, dtype), dev(b, dtype)
+    out = epd.op_linear(dtype, xd, wd, bd, make_out(), M, N, K, flags | (tile_n << 8))
+    torch.cuda.synchronize()
+    tol = 1e-5 if mode == "accum" else TOL_BF16_STEP
+    assert rel_err(to_np(out), ref) <= tol
+    out_fma = epd.op_linear(dtype, xd, wd, bd, make_out(), M, N, K, flags | epd.LINEAR_FORCE_FMA)
+    assert rel_err(to_np(out), to_np(out_fma)) <= tol
+
+
 @pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
 @pytest.mark.parametrize("T,h", [(1, 8), (37, 256), (100, 1152), (9, 3200), (5, 30)])
 def test_rmsnorm(dtype, T, h):
