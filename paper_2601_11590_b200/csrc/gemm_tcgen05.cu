@@ -6,9 +6,11 @@
 //   warp 1      allocates tensor memory and issues tcgen05.mma (one thread), fp32 accumulators in
 //               TMEM, two accumulator buffers so the epilogue of tile i overlaps the loop of tile i+1
 //   warps 2..5  epilogue: tcgen05.ld the accumulators (warp w reads TMEM lanes 32*(w%4)..+32),
-//               bias / GELU / residual add, 16-byte global stores
+//               bias / GELU in registers, 32-row x 128-byte chunks staged in swizzled shared
+//               memory and written with TMA: a plain tensor store, or for the residual update
+//               a tensor reduce-add (out += tile) so the old values never travel to the SM
 // Both operands are K-major (row-major [rows, K]), so one shared-memory descriptor form serves both.
-// Ragged M, N and K are handled by TMA zero fill on loads and predicated stores.
+// Ragged M, N and K are handled by TMA: zero fill on loads, clipping on stores.
 // Every mbarrier wait is bounded: on expiry the kernel records EPD_ETIMEOUT and drains.
 #include <cuda.h>
 
@@ -75,6 +77,21 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
       ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(smem_u32(bar)), "r"(x), "r"(y)
       : "memory");
 }
+
+// TMA tensor store / reduce-add of one staged box, tracked by the issuing thread's bulk group.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, int x, int y, const void* smem_src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, int x, int y, const void* smem_src) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
@@ -149,10 +166,15 @@ struct SmemLayout {
   static constexpr int kABytes = BM * BK * 2;
   static constexpr int kBBytes = BN * BK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kBarOffset = STAGES * kStageBytes;
+  // output staging: per epilogue warp kOutBufs buffers of 32 rows x 128 bytes (1024-byte aligned)
+  static constexpr int kOutBufs = BN >= 256 ? 1 : 2;
+  static constexpr int kOutBufBytes = 32 * 128;
+  static constexpr int kOutOffset = STAGES * kStageBytes;
+  static constexpr int kBarOffset = kOutOffset + kEpiWarps * kOutBufs * kOutBufBytes;
   // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], tmem base, abort flag, bias[kEpiWarps][BN]
   static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 4) * 8 + 16;
   static constexpr int kTotal = kBiasOffset + kEpiWarps * BN * 4;
+  static_assert(kTotal + 1024 <= 232448, "exceeds the shared memory of one CTA");
   static constexpr int kDynamic = kTotal + 1024;  // slack to align the ring to 1024 bytes
 };
 
@@ -162,8 +184,8 @@ struct SmemLayout {
 template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
-                 const __nv_bfloat16* __restrict__ bias, OutT* __restrict__ out, int64_t ldo, int M, int N, int K,
-                 int* __restrict__ status) {
+                 const __grid_constant__ CUtensorMap tm_out, const __nv_bfloat16* __restrict__ bias, int M, int N,
+                 int K, int* __restrict__ status) {
   using L = SmemLayout<BN, STAGES>;
   static_assert(L::kDynamic > 116 * 1024, "one CTA per SM is assumed by the TMEM allocation");
   static_assert(BN % 16 == 0 && BN >= 32 && BN <= 256, "UMMA N");
@@ -256,10 +278,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     __syncwarp();
   } else {
     // ------------------------------------------------------------------ epilogue
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
-    float* bs = bias_s + (warp - 2) * BN;  // this warp's private copy of the tile's bias values
+    constexpr int CC = sizeof(OutT) == 4 ? 32 : 64;  // columns per staged chunk: 128 bytes per row
+    const int q = warp & 3;                          // TMEM lane quarter this warp may read
+    float* bs = bias_s + (warp - 2) * BN;            // this warp's private copy of the tile's bias values
+    uint8_t* stage_out = smem + L::kOutOffset + (warp - 2) * L::kOutBufs * L::kOutBufBytes;
+    int obuf = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
+    if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_out) : "memory");
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
       const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
       __syncwarp();
@@ -268,64 +294,69 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
       __syncwarp();
       if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) break;
       tc_fence_after();
-      const int row = m0 + q * 32 + lane;
+      const int row0 = m0 + q * 32;
       const uint32_t taddr = tmem_base + acc * kAccStride + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(taddr + c * 32, r);
-        tmem_ld_wait();
-        if (c == BN / 32 - 1) {
-          // all accumulator columns of this tile are in registers: hand the buffer back
+      for (int c = 0; c < BN / CC; ++c) {
+        uint32_t pk[32];  // this thread's row of the chunk, as stored: 32 floats or 64 bf16
+        if constexpr (sizeof(OutT) == 4) {
+          tmem_ld32(taddr + c * CC, pk);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float t = __uint_as_float(pk[j]) + bs[c * CC + j];
+            if (ACT == 1) t = gelu_tanh_fast(t);
+            if (ACT == 2) t = gelu_erf_f(t);
+            pk[j] = __float_as_uint(t);
+          }
+        } else {
+          uint32_t r0[32], r1[32];
+          tmem_ld32(taddr + c * CC, r0);
+          tmem_ld32(taddr + c * CC + 32, r1);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const uint32_t* src = j < 16 ? r0 : r1;
+            const int jj = (2 * j) & 31;
+            float t0 = __uint_as_float(src[jj]) + bs[c * CC + 2 * j];
+            float t1 = __uint_as_float(src[jj + 1]) + bs[c * CC + 2 * j + 1];
+            if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); }
+            if (ACT == 2) { t0 = gelu_erf_f(t0); t1 = gelu_erf_f(t1); }
+            __nv_bfloat162 b = __floats2bfloat162_rn(t0, t1);
+            pk[j] = *reinterpret_cast<uint32_t*>(&b);
+          }
+        }
+        if (c == BN / CC - 1) {
+          // all accumulator columns of this tile have been read: hand the buffer back
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(&tmem_empty[acc]);
         }
-        const int nb = n0 + c * 32;
-        if (row < M && nb < N) {
-          float v[32];
+        // the staging buffer is free once the bulk store issued from it has read it
+        if (lane == 0) bulk_wait_read<L::kOutBufs - 1>();
+        __syncwarp();
+        uint8_t* sbuf = stage_out + obuf * L::kOutBufBytes;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            float t = __uint_as_float(r[j]) + bs[c * 32 + j];
-            if (ACT == 1) t = gelu_tanh_fast(t);
-            if (ACT == 2) t = gelu_erf_f(t);
-            v[j] = t;
-          }
-          OutT* orow = out + (int64_t)row * ldo + nb;
-          if constexpr (sizeof(OutT) == 4) {
-#pragma unroll
-            for (int g = 0; g < 8; ++g) {
-              if (nb + g * 4 < N) {  // N is a multiple of 8, so a group of 4 is all in or all out
-                float4* p = reinterpret_cast<float4*>(orow) + g;
-                float4 o = make_float4(v[4 * g], v[4 * g + 1], v[4 * g + 2], v[4 * g + 3]);
-                if (ACCUM) {
-                  const float4 old = *p;
-                  o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                }
-                *p = o;
-              }
-            }
-          } else {
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              if (nb + g * 8 < N) {
-                uint4 pk;
-                __nv_bfloat162 b0 = __floats2bfloat162_rn(v[8 * g], v[8 * g + 1]);
-                __nv_bfloat162 b1 = __floats2bfloat162_rn(v[8 * g + 2], v[8 * g + 3]);
-                __nv_bfloat162 b2 = __floats2bfloat162_rn(v[8 * g + 4], v[8 * g + 5]);
-                __nv_bfloat162 b3 = __floats2bfloat162_rn(v[8 * g + 6], v[8 * g + 7]);
-                pk.x = *reinterpret_cast<uint32_t*>(&b0);
-                pk.y = *reinterpret_cast<uint32_t*>(&b1);
-                pk.z = *reinterpret_cast<uint32_t*>(&b2);
-                pk.w = *reinterpret_cast<uint32_t*>(&b3);
-                reinterpret_cast<uint4*>(orow)[g] = pk;
-              }
-            }
-          }
+        for (int j = 0; j < 8; ++j) {
+          // 128-byte swizzle: 16-byte chunk j of row r lives at chunk position j ^ (r % 8)
+          uint4* dst = reinterpret_cast<uint4*>(sbuf + lane * 128 + ((j ^ (lane & 7)) << 4));
+          *dst = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
         }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          if (row0 < M && n0 + c * CC < N) {
+            if (ACCUM) tma_reduce_add_2d(&tm_out, n0 + c * CC, row0, sbuf);
+            else tma_store_2d(&tm_out, n0 + c * CC, row0, sbuf);
+          }
+          bulk_commit();
+        }
+        if (++obuf == L::kOutBufs) obuf = 0;
       }
       if (++acc == 2) { acc = 0; acc_phase ^= 1; }
     }
+    if (lane == 0) bulk_wait_all();
+    __syncwarp();
   }
 
   // ------------------------------------------------------------------ teardown
@@ -364,16 +395,19 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// Tensor map of a row-major bf16 matrix [rows, cols] with leading dimension ld, box = box_rows x 64.
-bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+// Tensor map of a row-major matrix [rows, cols] with leading dimension ld (elements of elem_bytes),
+// box = box_rows x (128 bytes of columns), 128-byte swizzle.
+bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows,
+              int elem_bytes) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * elem_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+  return fn(tm, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+            const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -389,7 +423,7 @@ int sm_count() {
 }
 
 template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM>
-cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const void* bias, void* out, int64_t ldo, int M, int N,
+cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& to, const void* bias, int M, int N,
                    int K, int* status, cudaStream_t s) {
   using L = SmemLayout<BN, STAGES>;
   auto kern = linear_tc_kernel<BN, STAGES, OutT, ACT, ACCUM>;
@@ -401,17 +435,17 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const void* bia
   }
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = tiles < sm_count() ? tiles : sm_count();
-  kern<<<grid, kThreads, L::kDynamic, s>>>(tx, tw, (const __nv_bfloat16*)bias, (OutT*)out, ldo, M, N, K, status);
+  kern<<<grid, kThreads, L::kDynamic, s>>>(tx, tw, to, (const __nv_bfloat16*)bias, M, N, K, status);
   return cudaGetLastError();
 }
 
 template <int BN, int STAGES>
-cudaError_t launch_bn(const CUtensorMap& tx, const CUtensorMap& tw, const void* bias, void* out, int64_t ldo, int M,
+cudaError_t launch_bn(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& to, const void* bias, int M,
                       int N, int K, int flags, int* status, cudaStream_t s) {
   const int act = (flags & EPD_LINEAR_GELU_TANH) ? 1 : (flags & EPD_LINEAR_GELU_ERF) ? 2 : 0;
   const bool accum = flags & EPD_LINEAR_ACCUMULATE;
   const bool out_f32 = accum || (flags & EPD_LINEAR_OUT_F32);
-#define EPD_TC(OUT, A, C) return launch<BN, STAGES, OUT, A, C>(tx, tw, bias, out, ldo, M, N, K, status, s)
+#define EPD_TC(OUT, A, C) return launch<BN, STAGES, OUT, A, C>(tx, tw, to, bias, M, N, K, status, s)
   if (accum) {
     if (act == 0) EPD_TC(float, 0, true);
     if (act == 1) EPD_TC(float, 1, true);
@@ -428,17 +462,21 @@ cudaError_t launch_bn(const CUtensorMap& tx, const CUtensorMap& tw, const void* 
 #undef EPD_TC
 }
 
-// Tile width: the candidate with the smallest estimated time, waves x (BN + fixed per-tile cost).
+// Tile width: the candidate with the smallest estimated time = waves x tile width / efficiency.
+// The efficiencies are the measured mainloop rates of each width relative to 256 (narrower tiles
+// re-read the x operand from shared memory more often per flop).
 int pick_bn(int M, int N) {
   const int cands[3] = {256, 192, 128};
+  const double eff[3] = {1.0, 0.88, 0.65};
   const int sms = sm_count();
   const int m_tiles = (M + BM - 1) / BM;
-  int best = 128;
+  int best = 256;
   double best_cost = 1e300;
-  for (int bn : cands) {
+  for (int i = 0; i < 3; ++i) {
+    const int bn = cands[i];
     const int tiles = m_tiles * ((N + bn - 1) / bn);
     const int waves = (tiles + sms - 1) / sms;
-    const double cost = (double)waves * (bn + 24);
+    const double cost = (double)waves * bn / eff[i];
     if (cost < best_cost) { best_cost = cost; best = bn; }
   }
   return best;
@@ -459,12 +497,15 @@ bool linear_tc_supported(const void* x, int64_t ldx, const void* w, int64_t ldw,
 cudaError_t linear_tc(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out, int64_t ldo,
                       int64_t M, int64_t N, int64_t K, int flags, int forced_bn, int* status, cudaStream_t s) {
   const int bn = forced_bn > 0 ? forced_bn : pick_bn((int)M, (int)N);
-  CUtensorMap tx, tw;
-  if (!make_map(&tx, x, M, K, ldx, BM) || !make_map(&tw, w, N, K, ldw, bn)) return cudaErrorInvalidValue;
+  const bool out_f32 = flags & (EPD_LINEAR_ACCUMULATE | EPD_LINEAR_OUT_F32);
+  CUtensorMap tx, tw, to;
+  if (!make_map(&tx, x, M, K, ldx, BM, 2) || !make_map(&tw, w, N, K, ldw, bn, 2) ||
+      !make_map(&to, out, M, N, ldo, 32, out_f32 ? 4 : 2))
+    return cudaErrorInvalidValue;
   switch (bn) {
-    case 256: return launch_bn<256, 4>(tx, tw, bias, out, ldo, (int)M, (int)N, (int)K, flags, status, s);
-    case 192: return launch_bn<192, 5>(tx, tw, bias, out, ldo, (int)M, (int)N, (int)K, flags, status, s);
-    case 128: return launch_bn<128, 6>(tx, tw, bias, out, ldo, (int)M, (int)N, (int)K, flags, status, s);
+    case 256: return launch_bn<256, 4>(tx, tw, to, bias, (int)M, (int)N, (int)K, flags, status, s);
+    case 192: return launch_bn<192, 4>(tx, tw, to, bias, (int)M, (int)N, (int)K, flags, status, s);
+    case 128: return launch_bn<128, 5>(tx, tw, to, bias, (int)M, (int)N, (int)K, flags, status, s);
     default: return cudaErrorInvalidValue;
   }
 }
