@@ -245,6 +245,36 @@ int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v,
 int epd_op_merge(int32_t dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm,
                  int32_t hidden, void* stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Allocation-free variant (the paper has no counterpart: this is a convenience of this library)
+ * ---------------------------------------------------------------------------------------- */
+
+/*
+ * Rotary embedding + head split + block-diagonal attention on a packed qkv matrix, for callers
+ * that cannot allocate device memory: a process whose own pool already owns all of HBM (so
+ * cudaMalloc fails), or a latency-critical loop that must avoid the device-wide synchronisation
+ * an allocation can trigger.  It computes what epd_op_rope_split() followed by epd_op_attention()
+ * computes (q scaled by log2(e)/sqrt(head_dim)), but the head-major q, k, v intermediates live in
+ * a fixed array inside the library's device image instead of caller-provided buffers; the call
+ * performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   qkv [T, 3*heads*head_dim], out [T, heads*head_dim] per dtype; pos_row, pos_col, cu_seqlens
+ *   device int32; host_cu_seqlens the same prefix sums in HOST memory.
+ * Limits and caveats:
+ *   - 3 * heads * T * epd_padded_head_dim(head_dim) * sizeof(element) (each third rounded up to
+ *     256 bytes) must not exceed epd_static_scratch_bytes() (16 MiB); larger batches return
+ *     EPD_ECAPACITY and launch nothing.
+ *   - Every GPU that loads the library holds the array until the process exits.
+ *   - The first call on a device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the array: calls whose kernels can overlap on the GPU
+ *     (different streams without ordering) race.  Nothing has to be cleared between calls: every
+ *     element that is read, padding included, is rewritten first by the same call.
+ */
+int epd_op_rope_attention_static(int32_t dtype, const void* qkv, const int32_t* pos_row, const int32_t* pos_col,
+                                 const int32_t* cu_seqlens, const int32_t* host_cu_seqlens, int32_t n_seg, void* out,
+                                 int64_t T, int32_t heads, int32_t head_dim, float theta, void* stream);
+size_t epd_static_scratch_bytes(void);
+
 #ifdef __cplusplus
 }
 #endif

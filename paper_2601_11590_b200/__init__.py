@@ -26,7 +26,8 @@ EXPORTED_SYMBOLS = [
     "epd_encoder_destroy", "epd_strerror", "epd_debug_bookkeeping", "epd_debug_set_taps",
     "epd_debug_run_block", "epd_debug_profile", "epd_debug_profile_classes",
     "epd_debug_profile_class_name", "epd_debug_profile_read", "epd_op_linear", "epd_op_rmsnorm", "epd_op_rope_split",
-    "epd_padded_head_dim", "epd_op_attention", "epd_op_merge",
+    "epd_padded_head_dim", "epd_op_attention", "epd_op_merge", "epd_op_rope_attention_static",
+    "epd_static_scratch_bytes",
 ]
 
 
@@ -113,6 +114,10 @@ def load_library() -> ctypes.CDLL:
     lib.epd_op_attention.argtypes = [i32, vp, vp, vp, vp, i32p, i32, vp, i64, i32, i32, i32, vp]
     lib.epd_op_merge.restype = ctypes.c_int
     lib.epd_op_merge.argtypes = [i32, vp, vp, vp, i64, i32, vp]
+    lib.epd_op_rope_attention_static.restype = ctypes.c_int
+    lib.epd_op_rope_attention_static.argtypes = [i32, vp, vp, vp, vp, i32p, i32, vp, i64, i32, i32, f32, vp]
+    lib.epd_static_scratch_bytes.restype = ctypes.c_size_t
+    lib.epd_static_scratch_bytes.argtypes = []
     _lib = lib
     return lib
 
@@ -374,4 +379,24 @@ def op_merge(dtype, y, merge_idx, stream=None):
     out = torch.empty((T // 4, 4 * h), dtype=y.dtype, device=y.device)
     _check(lib.epd_op_merge(dtype, _ptr(y), _ptr(merge_idx), _ptr(out), T // 4, h, _stream_ptr(stream)),
            "epd_op_merge")
+    return out
+
+
+def static_scratch_bytes() -> int:
+    return int(load_library().epd_static_scratch_bytes())
+
+
+def op_rope_attention_static(dtype, qkv, pos_row, pos_col, cu_seqlens_dev, cu_seqlens_host, heads, head_dim,
+                             theta, out=None, stream=None):
+    """Allocation-free rotary + split + attention: intermediates live in the library's fixed device
+    array.  `out` may be passed in so that the call itself allocates nothing at all."""
+    torch = _torch()
+    lib = load_library()
+    T = qkv.shape[0]
+    if out is None:
+        out = torch.empty((T, heads * head_dim), dtype=qkv.dtype, device=qkv.device)
+    hcu, hp = _i32_array(cu_seqlens_host)
+    _check(lib.epd_op_rope_attention_static(dtype, _ptr(qkv), _ptr(pos_row), _ptr(pos_col), _ptr(cu_seqlens_dev),
+                                            hp, hcu.size - 1, _ptr(out), T, heads, head_dim, theta,
+                                            _stream_ptr(stream)), "epd_op_rope_attention_static")
     return out

@@ -44,6 +44,10 @@ cudaError_t rope_split(int dtype, const void* qkv, const int32_t* pos_row, const
 cudaError_t rope_table(float2* table, int rows, int head_dim, float theta, cudaStream_t s);
 cudaError_t attention_fma(int dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
                           int n_seg, void* out, int64_t T, int heads, int head_dim, cudaStream_t s);
+// Chooses the attention kernel for the shape (see attention kernels); `status` may be NULL.
+cudaError_t attention_any(int dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
+                          const int32_t* host_cu_seqlens, int n_seg, void* out, int64_t T, int heads, int head_dim,
+                          int flags, int* status, cudaStream_t s);
 cudaError_t merge_gather(int dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm, int hidden,
                          cudaStream_t s);
 cudaError_t token_layout(const int32_t* grid_thw, const int32_t* cu_seqlens, const int32_t* cu_out, int n_images,

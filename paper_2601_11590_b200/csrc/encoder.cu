@@ -201,8 +201,9 @@ int prepare_batch(epd_encoder* enc, const int32_t* grid_thw, int32_t n, int64_t 
 int attention_dispatch(epd_encoder* enc, int64_t T, int n_seg, cudaStream_t s) {
   const epd_config_t& c = enc->cfg;
   EPD_MARK(KC_ATTENTION);
-  EPD_CUDA(attention_fma(c.dtype, enc->at<void>(enc->lay.qh), enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh),
-                         enc->at<int32_t>(enc->lay.cu), n_seg, enc->at<void>(enc->lay.a), T, c.heads, c.head_dim, s));
+  EPD_CUDA(attention_any(c.dtype, enc->at<void>(enc->lay.qh), enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh),
+                         enc->at<int32_t>(enc->lay.cu), enc->host_cu.data(), n_seg, enc->at<void>(enc->lay.a), T,
+                         c.heads, c.head_dim, 0, enc->at<int>(enc->lay.status), s));
   return EPD_OK;
 }
 
@@ -573,8 +574,7 @@ int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v,
   if (host_cu_seqlens[0] != 0 || host_cu_seqlens[n_seg] != T) return EPD_EINVAL;
   for (int i = 0; i < n_seg; ++i)
     if (host_cu_seqlens[i + 1] <= host_cu_seqlens[i]) return EPD_EINVAL;
-  (void)flags;
-  EPD_CUDA(attention_fma(dtype, q, k, v, cu_seqlens, n_seg, out, T, heads, head_dim,
+  EPD_CUDA(attention_any(dtype, q, k, v, cu_seqlens, host_cu_seqlens, n_seg, out, T, heads, head_dim, flags, nullptr,
                          static_cast<cudaStream_t>(stream)));
   return EPD_OK;
 }
