@@ -233,10 +233,14 @@ int epd_op_rope_split(int32_t dtype, const void* qkv, const int32_t* pos_row, co
 
 int32_t epd_padded_head_dim(int32_t head_dim);
 
+enum { EPD_ATTENTION_FORCE_FMA = 1 /* use the plain-FMA kernel even where the tensor-core kernel applies */ };
+
 /* Block-diagonal bidirectional attention.  q, k, v [heads, T, head_dim_padded] per dtype with q
  * already multiplied by log2(e)/sqrt(head_dim); cu_seqlens device int32 [n_seg+1] and the same
  * values in HOST memory (host_cu_seqlens) for the launch geometry.  out [T, heads*head_dim] per
- * dtype: for each segment and head softmax over all keys of the segment. */
+ * dtype: for each segment and head softmax over all keys of the segment.  In bf16 with head_dim 64,
+ * 72 or 128 (a multiple of 8 whose padded width is 64, 80 or 128) the tcgen05 kernel runs; other
+ * shapes, and flags & EPD_ATTENTION_FORCE_FMA, use the plain-FMA kernel. */
 int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
                      const int32_t* host_cu_seqlens, int32_t n_seg, void* out, int64_t T, int32_t heads,
                      int32_t head_dim, int32_t flags, void* stream);

@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libepd_encoder.so")
 EPD_OK, EPD_EINVAL, EPD_ENOMEM, EPD_ECUDA, EPD_ECAPACITY, EPD_EUNSUPPORTED, EPD_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 DTYPE_F32, DTYPE_BF16 = 0, 1
 LINEAR_GELU_TANH, LINEAR_GELU_ERF, LINEAR_ACCUMULATE, LINEAR_OUT_F32, LINEAR_FORCE_FMA = 1, 2, 4, 8, 16
+ATTENTION_FORCE_FMA = 1
 
 EXPORTED_SYMBOLS = [
     "epd_encoder_workspace_bytes", "epd_encoder_create", "epd_encode", "epd_encode_host",

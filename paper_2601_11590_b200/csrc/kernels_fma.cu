@@ -370,13 +370,6 @@ cudaError_t attention_fma(int dtype, const void* q, const void* k, const void* v
   return cudaGetLastError();
 }
 
-cudaError_t attention_any(int dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
-                          const int32_t* host_cu_seqlens, int n_seg, void* out, int64_t T, int heads, int head_dim,
-                          int flags, int* status, cudaStream_t s) {
-  (void)host_cu_seqlens; (void)flags; (void)status;
-  return attention_fma(dtype, q, k, v, cu_seqlens, n_seg, out, T, heads, head_dim, s);
-}
-
 // =============================================================================================
 // 2x2 merge as a gather: slot s = 4*o + q of the merged matrix copies row merge_idx[s] of y.
 // =============================================================================================

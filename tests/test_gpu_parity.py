@@ -193,6 +193,40 @@ def test_attention(dtype, heads, dh, seglens):
     assert rel_err(got, ref) <= (1e-5 if dtype == epd.DTYPE_F32 else TOL_BF16_STEP)
 
 
+@pytest.mark.parametrize("heads,dh,seglens", [
+    (2, 72, [784, 784]),                 # the benchmark's segment length: 6 full key tiles + a 16-key tail
+    (2, 72, [100, 1300, 128, 129, 4]),   # ragged tails on both the query and the key side
+    (3, 64, [2000]),                     # 16 key tiles
+    (2, 128, [700, 260]),
+])
+def test_attention_tensor_core_long_segments(heads, dh, seglens):
+    got, ref = _attention_case(epd.DTYPE_BF16, heads, dh, seglens, 40)
+    assert rel_err(got, ref) <= TOL_BF16_STEP
+    fma, _ = _attention_case(epd.DTYPE_BF16, heads, dh, seglens, 40, flags=epd.ATTENTION_FORCE_FMA)
+    assert rel_err(got, fma) <= TOL_BF16_STEP
+
+
+def test_attention_rescale_path():
+    """Keys ordered so that the running maximum keeps growing from tile to tile by far more than the
+    rescale threshold: every key tile forces a rescale of the accumulated output."""
+    dtype, heads, dh, T = epd.DTYPE_BF16, 1, 64, 1024
+    dhp = epd.padded_head_dim(dh)
+    rng = np.random.default_rng(0)
+    q = np.zeros((heads, T, dhp), np.float32); q[:, :, 0] = 1.0
+    k = np.zeros((heads, T, dhp), np.float32)
+    k[0, :, 0] = synth.round_to_bf16((np.arange(T) * 0.25).astype(np.float32))       # logits 0 .. 256 (base 2)
+    k[0, :, 1:dh] = synth.round_to_bf16(rng.standard_normal((T, dh - 1)).astype(np.float32))
+    v = np.zeros((heads, T, dhp), np.float32)
+    v[:, :, :dh] = synth.round_to_bf16(rng.standard_normal((heads, T, dh)).astype(np.float32))
+    cu = np.array([0, T], np.int32)
+    out = epd.op_attention(dtype, dev(q, dtype), dev(k, dtype), dev(v, dtype), torch.from_numpy(cu).cuda(), cu, dh)
+    # the kernel's q carries log2(e)/sqrt(dh); hand the oracle the unscaled q it implies
+    q_eff = q[:, :, :dh].astype(np.float64) * np.log(2.0) * np.sqrt(dh)
+    ref = O.attention_block_diagonal(q_eff.transpose(1, 0, 2), k[:, :, :dh].astype(np.float64).transpose(1, 0, 2),
+                                     v[:, :, :dh].astype(np.float64).transpose(1, 0, 2), cu).reshape(T, heads * dh)
+    assert rel_err(to_np(out), ref) <= 1e-2
+
+
 @pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
 def test_attention_peaked_logits(dtype):
     """Logit standard deviation ~ 50: exercises the running-max rescaling of the online softmax."""
