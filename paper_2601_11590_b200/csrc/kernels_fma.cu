@@ -128,8 +128,68 @@ cudaError_t linear_fma(int dtype, const void* x, int64_t ldx, const void* w, int
 
 // =============================================================================================
 // RMSNorm: one warp per row of the float residual stream; optional scattered destination row.
-// Bytes per row: 4h read + sizeof(T)h written (the second pass re-reads the row from L1/L2).
+// Bytes per row: 4h read + sizeof(T)h written.  When the row fits (hidden <= 128*NV) each lane keeps
+// its NV float4 pieces in registers, so the row is read once and all loads are in flight together;
+// longer or unaligned rows take the two-pass kernel, whose second pass re-reads from L1/L2.
 // =============================================================================================
+template <typename T>
+__device__ __forceinline__ void store4(T* orow, int i, float r0, float r1, float r2, float r3) {
+  if constexpr (sizeof(T) == 4) {
+    reinterpret_cast<float4*>(orow)[i] = make_float4(r0, r1, r2, r3);
+  } else {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    reinterpret_cast<uint2*>(orow)[i] = pk;
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ float4 load_gain4(const T* gain, int i) {
+  if constexpr (sizeof(T) == 4) {
+    return reinterpret_cast<const float4*>(gain)[i];
+  } else {
+    const uint2 pk = reinterpret_cast<const uint2*>(gain)[i];
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pk.y));
+    return make_float4(a.x, a.y, b.x, b.y);
+  }
+}
+
+template <typename T, int NV>
+__global__ void __launch_bounds__(256)
+rmsnorm_reg_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ out,
+                   const int32_t* __restrict__ dst_row, int64_t rows, int hidden, float eps) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int nvec = hidden >> 2;
+  const float4* x4 = reinterpret_cast<const float4*>(x + row * hidden);
+  float4 v[NV];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int idx = lane + 32 * i;
+    v[i] = idx < nvec ? x4[idx] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+  }
+  float ss = 0.0f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float inv = 1.0f / sqrtf(ss / (float)hidden + eps);
+  const int64_t drow = dst_row ? (int64_t)dst_row[row] : row;
+  T* orow = out + drow * hidden;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int idx = lane + 32 * i;
+    if (idx < nvec) {
+      const float4 g = load_gain4<T>(gain, idx);
+      store4<T>(orow, idx, v[i].x * inv * g.x, v[i].y * inv * g.y, v[i].z * inv * g.z, v[i].w * inv * g.w);
+    }
+  }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ out,
@@ -139,55 +199,41 @@ rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __res
   if (row >= rows) return;
   const float* xr = x + row * hidden;
   float ss = 0.0f;
-  if ((hidden & 3) == 0) {
-    const float4* x4 = reinterpret_cast<const float4*>(xr);
-    for (int i = lane; i < hidden / 4; i += 32) {
-      const float4 v = x4[i];
-      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-    }
-  } else {
-    for (int i = lane; i < hidden; i += 32) ss += xr[i] * xr[i];
-  }
+  for (int i = lane; i < hidden; i += 32) ss += xr[i] * xr[i];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   const float inv = 1.0f / sqrtf(ss / (float)hidden + eps);
   const int64_t drow = dst_row ? (int64_t)dst_row[row] : row;
   T* orow = out + drow * hidden;
-  if ((hidden & 3) == 0) {
-    const float4* x4 = reinterpret_cast<const float4*>(xr);
-    for (int i = lane; i < hidden / 4; i += 32) {
-      const float4 v = x4[i];
-      const float r0 = v.x * inv * to_float<T>(gain[4 * i + 0]);
-      const float r1 = v.y * inv * to_float<T>(gain[4 * i + 1]);
-      const float r2 = v.z * inv * to_float<T>(gain[4 * i + 2]);
-      const float r3 = v.w * inv * to_float<T>(gain[4 * i + 3]);
-      if constexpr (sizeof(T) == 4) {
-        reinterpret_cast<float4*>(orow)[i] = make_float4(r0, r1, r2, r3);
-      } else {
-        __nv_bfloat162 lo = __floats2bfloat162_rn(r0, r1), hi = __floats2bfloat162_rn(r2, r3);
-        uint2 pk;
-        pk.x = *reinterpret_cast<uint32_t*>(&lo);
-        pk.y = *reinterpret_cast<uint32_t*>(&hi);
-        reinterpret_cast<uint2*>(orow)[i] = pk;
-      }
-    }
-  } else {
-    for (int i = lane; i < hidden; i += 32) orow[i] = from_float<T>(xr[i] * inv * to_float<T>(gain[i]));
-  }
+  for (int i = lane; i < hidden; i += 32) orow[i] = from_float<T>(xr[i] * inv * to_float<T>(gain[i]));
+}
+
+template <typename T>
+static cudaError_t rmsnorm_t(const float* x, const T* gain, T* out, const int32_t* dst_row, int64_t rows, int hidden,
+                             float eps, cudaStream_t s) {
+  const int warps = 8;
+  const unsigned blocks = (unsigned)((rows + warps - 1) / warps);
+  const bool vec_ok = (hidden % 4) == 0 && (((uintptr_t)x | (uintptr_t)out) & 15) == 0 &&
+                      ((uintptr_t)gain & (sizeof(T) == 4 ? 15 : 7)) == 0;
+  const int nv = (hidden / 4 + 31) / 32;
+  if (vec_ok && nv <= 4)
+    rmsnorm_reg_kernel<T, 4><<<blocks, warps * 32, 0, s>>>(x, gain, out, dst_row, rows, hidden, eps);
+  else if (vec_ok && nv <= 10)
+    rmsnorm_reg_kernel<T, 10><<<blocks, warps * 32, 0, s>>>(x, gain, out, dst_row, rows, hidden, eps);
+  else if (vec_ok && nv <= 26)
+    rmsnorm_reg_kernel<T, 26><<<blocks, warps * 32, 0, s>>>(x, gain, out, dst_row, rows, hidden, eps);
+  else
+    rmsnorm_kernel<T><<<blocks, warps * 32, 0, s>>>(x, gain, out, dst_row, rows, hidden, eps);
+  return cudaGetLastError();
 }
 
 cudaError_t rmsnorm(int dtype, const void* x, const void* gain, void* out, const int32_t* dst_row, int64_t T,
                     int hidden, float eps, cudaStream_t s) {
   if (T == 0) return cudaSuccess;
-  const int warps = 8;
-  const unsigned blocks = (unsigned)((T + warps - 1) / warps);
   if (dtype == EPD_DTYPE_F32)
-    rmsnorm_kernel<float><<<blocks, warps * 32, 0, s>>>((const float*)x, (const float*)gain, (float*)out, dst_row, T,
-                                                        hidden, eps);
-  else
-    rmsnorm_kernel<__nv_bfloat16><<<blocks, warps * 32, 0, s>>>((const float*)x, (const __nv_bfloat16*)gain,
-                                                                (__nv_bfloat16*)out, dst_row, T, hidden, eps);
-  return cudaGetLastError();
+    return rmsnorm_t<float>((const float*)x, (const float*)gain, (float*)out, dst_row, T, hidden, eps, s);
+  return rmsnorm_t<__nv_bfloat16>((const float*)x, (const __nv_bfloat16*)gain, (__nv_bfloat16*)out, dst_row, T, hidden,
+                                  eps, s);
 }
 
 // =============================================================================================
@@ -271,20 +317,141 @@ rope_split_kernel(const T* __restrict__ qkv, const int32_t* __restrict__ pos_row
   }
 }
 
+// Vector form of the same step.  A block stages the q|k|v rows of a few consecutive tokens in shared
+// memory with 16-byte loads (the rows are contiguous in global memory) together with the tokens'
+// (cos, sin) values; rotates q and k in place there, two adjacent frequencies per thread (one
+// 2-element load per side of the pair); then copies whole 16-byte pieces out to the head-major rows:
+// consecutive threads write consecutive pieces of (tensor, head, token), so the stores cover runs of
+// tokens * head_dim_padded elements.  Needs head_dim to be a multiple of the 16-byte vector width.
+template <typename T> struct Pair;
+template <> struct Pair<float> {
+  using type = float2;
+  static __device__ __forceinline__ float2 unpack(float2 v) { return v; }
+  static __device__ __forceinline__ float2 pack(float a, float b) { return make_float2(a, b); }
+};
+template <> struct Pair<__nv_bfloat16> {
+  using type = __nv_bfloat162;
+  static __device__ __forceinline__ float2 unpack(__nv_bfloat162 v) { return __bfloat1622float2(v); }
+  static __device__ __forceinline__ __nv_bfloat162 pack(float a, float b) { return __floats2bfloat162_rn(a, b); }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+rope_split_vec_kernel(const T* __restrict__ qkv, const int32_t* __restrict__ pos_row,
+                      const int32_t* __restrict__ pos_col, const float2* __restrict__ table, int table_rows,
+                      T* __restrict__ q, T* __restrict__ k, T* __restrict__ v, int64_t Tn, int heads, int dh, int dhp,
+                      int tok_per_block, float theta, float q_scale) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  using P2 = typename Pair<T>::type;
+  extern __shared__ __align__(16) uint8_t rope_smem[];
+  const int h = heads * dh, row_elems = 3 * h;
+  const int d2 = dh / 2, nf = dh / 4, nf2 = nf / 2;
+  const int64_t j0 = (int64_t)blockIdx.x * tok_per_block;
+  const int ntok = (int)min((int64_t)tok_per_block, Tn - j0);
+  T* s_in = reinterpret_cast<T*>(rope_smem);
+  float2* s_cs = reinterpret_cast<float2*>(rope_smem + (size_t)tok_per_block * row_elems * sizeof(T));
+
+  const uint4* src = reinterpret_cast<const uint4*>(qkv + j0 * row_elems);
+  const int nvec = ntok * (row_elems / VEC);
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) reinterpret_cast<uint4*>(s_in)[i] = src[i];
+  for (int i = threadIdx.x; i < ntok * 2 * nf; i += blockDim.x) {
+    const int f = i % nf, half = (i / nf) & 1, t = i / (2 * nf);
+    const int p = half ? pos_col[j0 + t] : pos_row[j0 + t];
+    float2 cs = make_float2(1.0f, 0.0f);
+    if (theta > 0.0f) {
+      if (table != nullptr && p < table_rows) {
+        cs = table[p * nf + f];
+      } else {
+        const double w = pow((double)theta, -2.0 * (double)f / (double)d2);
+        double s_, c_;
+        sincos((double)p * w, &s_, &c_);
+        cs = make_float2((float)c_, (float)s_);
+      }
+    }
+    s_cs[i] = cs;
+  }
+  __syncthreads();
+
+  // rotate q and k in place: unit i = (head, half, frequency pair); index arithmetic once per unit
+  const int units = heads * 2 * nf2;
+  for (int i = threadIdx.x; i < units; i += blockDim.x) {
+    const int fp = i % nf2;
+    const int rest = i / nf2;
+    const int half = rest & 1, hd = rest >> 1;
+    const int e0 = hd * dh + half * d2 + 2 * fp;   // element of the pair's first member inside q (or k)
+    const int c0 = half * nf + 2 * fp;             // its (cos, sin) entry inside the token's list
+    for (int t = 0; t < ntok; ++t) {
+      const float4 cs = *reinterpret_cast<const float4*>(s_cs + t * 2 * nf + c0);  // cos0 sin0 cos1 sin1
+#pragma unroll
+      for (int which = 0; which < 2; ++which) {
+        T* base = s_in + t * row_elems + which * h + e0;
+        const float2 a = Pair<T>::unpack(*reinterpret_cast<const P2*>(base));
+        const float2 b = Pair<T>::unpack(*reinterpret_cast<const P2*>(base + nf));
+        const float sc = which == 0 ? q_scale : 1.0f;
+        const float ra0 = (a.x * cs.x - b.x * cs.y) * sc, rb0 = (b.x * cs.x + a.x * cs.y) * sc;
+        const float ra1 = (a.y * cs.z - b.y * cs.w) * sc, rb1 = (b.y * cs.z + a.y * cs.w) * sc;
+        *reinterpret_cast<P2*>(base) = Pair<T>::pack(ra0, ra1);
+        *reinterpret_cast<P2*>(base + nf) = Pair<T>::pack(rb0, rb1);
+      }
+    }
+  }
+  __syncthreads();
+
+  // copy out: 16-byte pieces, (tensor, head) outermost, then token, then piece inside the padded row
+  const int vec_per_row = dhp / VEC, data_vecs = dh / VEC;
+  const int per_pair = ntok * vec_per_row;
+  const int total = 3 * heads * per_pair;
+  for (int u = threadIdx.x; u < total; u += blockDim.x) {
+    const int pair = u / per_pair, r = u - pair * per_pair;
+    const int t = r / vec_per_row, ov = r - t * vec_per_row;
+    const int which = pair / heads, hd = pair - which * heads;
+    uint4 pk = make_uint4(0u, 0u, 0u, 0u);
+    if (ov < data_vecs)
+      pk = *reinterpret_cast<const uint4*>(s_in + t * row_elems + which * h + hd * dh + ov * VEC);
+    T* dst = (which == 0 ? q : which == 1 ? k : v) + ((int64_t)hd * Tn + j0 + t) * dhp + ov * VEC;
+    *reinterpret_cast<uint4*>(dst) = pk;
+  }
+}
+
+template <typename T>
+static cudaError_t rope_split_t(const T* qkv, const int32_t* pos_row, const int32_t* pos_col, const float2* table,
+                                int table_rows, T* q, T* k, T* v, int64_t Tn, int heads, int dh, float theta,
+                                float q_scale, cudaStream_t s) {
+  constexpr int VEC = 16 / (int)sizeof(T);
+  const int dhp = padded_head_dim(dh);
+  const size_t row_bytes = (size_t)3 * heads * dh * sizeof(T);
+  const bool aligned = ((((uintptr_t)qkv | (uintptr_t)q | (uintptr_t)k | (uintptr_t)v)) & 15) == 0;
+  if (aligned && dh % 8 == 0 && row_bytes + 2 * (dh / 4) * sizeof(float2) <= 96 * 1024) {
+    // a few tokens per block: about 32 KB of rows, so several blocks share an SM
+    int tok = (int)(32768 / row_bytes);
+    tok = tok < 1 ? 1 : tok > 8 ? 8 : tok;
+    const size_t smem = tok * (row_bytes + 2 * (dh / 4) * sizeof(float2));
+    auto kern = rope_split_vec_kernel<T>;
+    static size_t configured = 48 * 1024;
+    if (smem > configured) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+      if (e != cudaSuccess) return e;
+      configured = 100 * 1024;
+    }
+    kern<<<(unsigned)((Tn + tok - 1) / tok), 256, smem, s>>>(qkv, pos_row, pos_col, table, table_rows, q, k, v, Tn,
+                                                            heads, dh, dhp, tok, theta, q_scale);
+  } else {
+    rope_split_kernel<T><<<(unsigned)Tn, 128, 0, s>>>(qkv, pos_row, pos_col, table, table_rows, q, k, v, Tn, heads, dh,
+                                                      dhp, theta, q_scale);
+  }
+  return cudaGetLastError();
+}
+
 cudaError_t rope_split(int dtype, const void* qkv, const int32_t* pos_row, const int32_t* pos_col,
                        const float2* table, int table_rows, void* q, void* k, void* v, int64_t T, int heads,
                        int head_dim, float theta, float q_scale, cudaStream_t s) {
   if (T == 0) return cudaSuccess;
-  const int dhp = padded_head_dim(head_dim);
   if (dtype == EPD_DTYPE_F32)
-    rope_split_kernel<float><<<(unsigned)T, 128, 0, s>>>((const float*)qkv, pos_row, pos_col, table, table_rows,
-                                                         (float*)q, (float*)k, (float*)v, T, heads, head_dim, dhp,
-                                                         theta, q_scale);
-  else
-    rope_split_kernel<__nv_bfloat16><<<(unsigned)T, 128, 0, s>>>(
-        (const __nv_bfloat16*)qkv, pos_row, pos_col, table, table_rows, (__nv_bfloat16*)q, (__nv_bfloat16*)k,
-        (__nv_bfloat16*)v, T, heads, head_dim, dhp, theta, q_scale);
-  return cudaGetLastError();
+    return rope_split_t<float>((const float*)qkv, pos_row, pos_col, table, table_rows, (float*)q, (float*)k,
+                               (float*)v, T, heads, head_dim, theta, q_scale, s);
+  return rope_split_t<__nv_bfloat16>((const __nv_bfloat16*)qkv, pos_row, pos_col, table, table_rows,
+                                     (__nv_bfloat16*)q, (__nv_bfloat16*)k, (__nv_bfloat16*)v, T, heads, head_dim,
+                                     theta, q_scale, s);
 }
 
 // =============================================================================================

@@ -1,0 +1,172 @@
+"""Time single steps of the Encode-stage library on random device data.
+
+  python -m paper_2601_11590_b200.opbench linear --M 6272 --N 4304 --K 1152 --mode gelu_tanh
+  python -m paper_2601_11590_b200.opbench attention --heads 16 --dh 72 --seglens 784x8
+  python -m paper_2601_11590_b200.opbench rope --T 6272 --heads 16 --dh 72
+  python -m paper_2601_11590_b200.opbench rmsnorm --T 6272 --hidden 1152
+
+Each call goes through the C ABI (epd_op_*), is timed with CUDA events on the launching stream
+after warm-up, and prints one JSON line: average device time, algorithmic FLOP/s or bytes/s.
+Between timed launches a buffer larger than the L2 cache is overwritten unless --no-flush is given
+(the in-pipeline condition, where operands come from the previous step, is closer to --no-flush).
+The same command line with --iters 1 --warmup 1 is a convenient small target for a profiler.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import numpy as np
+
+import paper_2601_11590_b200 as epd
+
+
+def parse_seglens(text: str):
+    """'784x8,300,16384' -> [784]*8 + [300, 16384]"""
+    out = []
+    for part in text.split(","):
+        if "x" in part:
+            a, b = part.split("x")
+            out += [int(a)] * int(b)
+        else:
+            out.append(int(part))
+    return out
+
+
+def time_op(torch, fn, iters: int, warmup: int, flush: bool) -> float:
+    """Average device time of one launch.  With flushing, each launch is timed on its own after the
+    L2 was overwritten; without, `iters` launches run back to back inside one pair of events."""
+    stream = torch.cuda.current_stream()
+    scratch = torch.empty(192 << 20, dtype=torch.uint8, device="cuda") if flush else None
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if not flush:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fn()
+        e0.record(stream)
+        for _ in range(iters):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+    total = 0.0
+    for _ in range(iters):
+        scratch.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        total += e0.elapsed_time(e1)
+    return total / iters
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("op", choices=["linear", "attention", "rope", "rmsnorm", "merge"])
+    ap.add_argument("--M", type=int, default=6272)
+    ap.add_argument("--N", type=int, default=1152)
+    ap.add_argument("--K", type=int, default=1152)
+    ap.add_argument("--mode", default="plain", choices=["plain", "gelu_tanh", "gelu_erf", "accum", "out_f32"])
+    ap.add_argument("--tile-n", type=int, default=0)
+    ap.add_argument("--T", type=int, default=6272)
+    ap.add_argument("--hidden", type=int, default=1152)
+    ap.add_argument("--heads", type=int, default=16)
+    ap.add_argument("--dh", type=int, default=72)
+    ap.add_argument("--seglens", default="784x8")
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--fma", action="store_true", help="force the plain-FMA kernel")
+    args = ap.parse_args()
+
+    import torch
+    from paper_2601_11590_b200 import build
+    build.build_library()
+    epd.load_library()
+    dt = epd.DTYPE_BF16
+    bf = torch.bfloat16
+    g = torch.Generator(device="cuda").manual_seed(0)
+    rnd = lambda *shape, std=1.0, dtype=bf: (torch.randn(*shape, generator=g, device="cuda") * std).to(dtype)
+    res = {"op": args.op}
+
+    if args.op == "linear":
+        M, N, K = args.M, args.N, args.K
+        x, w, b = rnd(M, K), rnd(N, K, std=K ** -0.5), rnd(N, std=0.5)
+        flags = {"plain": 0, "gelu_tanh": epd.LINEAR_GELU_TANH, "gelu_erf": epd.LINEAR_GELU_ERF,
+                 "accum": epd.LINEAR_ACCUMULATE, "out_f32": epd.LINEAR_OUT_F32}[args.mode]
+        flags |= args.tile_n << 8
+        if args.fma:
+            flags |= epd.LINEAR_FORCE_FMA
+        f32 = args.mode in ("accum", "out_f32")
+        out = torch.zeros((M, N), dtype=torch.float32 if f32 else bf, device="cuda")
+        fn = lambda: epd.op_linear(dt, x, w, b, out, M, N, K, flags)
+        res.update(M=M, N=N, K=K, mode=args.mode, tile_n=args.tile_n, flops=2.0 * M * N * K,
+                   bytes=2.0 * (M * K + N * K) + (8.0 if args.mode == "accum" else 4.0 if f32 else 2.0) * M * N)
+    elif args.op == "attention":
+        seg = parse_seglens(args.seglens)
+        T = sum(seg)
+        cu = np.concatenate([[0], np.cumsum(seg)]).astype(np.int32)
+        cu_dev = torch.from_numpy(cu).cuda()
+        dhp = epd.padded_head_dim(args.dh)
+        q, k, v = (torch.zeros((args.heads, T, dhp), dtype=bf, device="cuda") for _ in range(3))
+        for t in (q, k, v):
+            t[:, :, :args.dh] = rnd(args.heads, T, args.dh, std=0.5)
+        lib = epd.load_library()
+        out = torch.empty((T, args.heads * args.dh), dtype=bf, device="cuda")
+        hcu, hp = epd._i32_array(cu)
+        flags = epd.ATTENTION_FORCE_FMA if args.fma else 0
+
+        def fn():
+            epd._check(lib.epd_op_attention(dt, epd._ptr(q), epd._ptr(k), epd._ptr(v), epd._ptr(cu_dev), hp,
+                                            hcu.size - 1, epd._ptr(out), T, args.heads, args.dh, flags,
+                                            epd._stream_ptr(None)), "epd_op_attention")
+        res.update(heads=args.heads, dh=args.dh, T=T, n_seg=len(seg),
+                   flops=4.0 * args.heads * args.dh * float(sum(s * s for s in seg)),
+                   bytes=2.0 * args.heads * T * (3 * dhp + args.dh))
+    elif args.op == "rope":
+        T, heads, dh = args.T, args.heads, args.dh
+        h = heads * dh
+        dhp = epd.padded_head_dim(dh)
+        qkv = rnd(T, 3 * h)
+        pr = torch.randint(0, 28, (T,), generator=g, device="cuda", dtype=torch.int32)
+        pc = torch.randint(0, 28, (T,), generator=g, device="cuda", dtype=torch.int32)
+        lib = epd.load_library()
+        q, k, v = (torch.empty((heads, T, dhp), dtype=bf, device="cuda") for _ in range(3))
+
+        def fn():
+            epd._check(lib.epd_op_rope_split(dt, epd._ptr(qkv), epd._ptr(pr), epd._ptr(pc), epd._ptr(q), epd._ptr(k),
+                                             epd._ptr(v), T, heads, dh, 10000.0, 0.17, epd._stream_ptr(None)),
+                       "epd_op_rope_split")
+        res.update(T=T, heads=heads, dh=dh, bytes=2.0 * T * 3 * h + 2.0 * 3 * heads * T * dhp + 8.0 * T)
+    elif args.op == "rmsnorm":
+        T, h = args.T, args.hidden
+        x = rnd(T, h, dtype=torch.float32)
+        gain = rnd(h, std=0.02) + 1
+        out = torch.empty((T, h), dtype=bf, device="cuda")
+        fn = lambda: epd.op_rmsnorm(dt, x, gain, out, 1e-6)
+        res.update(T=T, hidden=h, bytes=6.0 * T * h)
+    else:
+        T, h = args.T // 4 * 4, args.hidden
+        y = rnd(T, h)
+        idx = torch.randperm(T, generator=g, device="cuda").to(torch.int32)
+        lib = epd.load_library()
+        out = torch.empty((T // 4, 4 * h), dtype=bf, device="cuda")
+
+        def fn():
+            epd._check(lib.epd_op_merge(dt, epd._ptr(y), epd._ptr(idx), epd._ptr(out), T // 4, h,
+                                        epd._stream_ptr(None)), "epd_op_merge")
+        res.update(T=T, hidden=h, bytes=4.0 * T * h + 4.0 * T)
+
+    ms = time_op(torch, fn, args.iters, args.warmup, not args.no_flush)
+    res["ms"] = ms
+    res["l2_flush"] = not args.no_flush
+    if "flops" in res:
+        res["tflops"] = res["flops"] / (ms * 1e-3) / 1e12
+    res["gbs"] = res["bytes"] / (ms * 1e-3) / 1e9
+    print(json.dumps(res))
+
+
+if __name__ == "__main__":
+    main()
