@@ -166,6 +166,10 @@ int epd_encoder_destroy(epd_encoder_t* enc);
 
 const char* epd_strerror(int status);
 
+/* Name of the CUDA runtime error behind the calling thread's most recent EPD_ECUDA return
+ * ("cudaSuccess" if there was none): a diagnostic aid, the string is static. */
+const char* epd_last_cuda_error(void);
+
 /* ------------------------------------------------------------------------------------------
  * Test hooks on an encoder
  * ---------------------------------------------------------------------------------------- */

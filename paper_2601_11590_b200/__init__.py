@@ -28,14 +28,17 @@ EXPORTED_SYMBOLS = [
     "epd_debug_run_block", "epd_debug_profile", "epd_debug_profile_classes",
     "epd_debug_profile_class_name", "epd_debug_profile_read", "epd_op_linear", "epd_op_rmsnorm", "epd_op_rope_split",
     "epd_padded_head_dim", "epd_op_attention", "epd_op_merge", "epd_op_rope_attention_static",
-    "epd_static_scratch_bytes",
+    "epd_static_scratch_bytes", "epd_last_cuda_error",
 ]
 
 
 class EpdError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
-        super().__init__(f"{what}: {strerror(status)} ({status})")
+        detail = ""
+        if status == EPD_ECUDA and _lib is not None:
+            detail = " [" + _lib.epd_last_cuda_error().decode() + "]"
+        super().__init__(f"{what}: {strerror(status)} ({status}){detail}")
 
 
 class ConfigStruct(ctypes.Structure):
@@ -89,6 +92,8 @@ def load_library() -> ctypes.CDLL:
     lib.epd_encoder_destroy.argtypes = [vp]
     lib.epd_strerror.restype = ctypes.c_char_p
     lib.epd_strerror.argtypes = [ctypes.c_int]
+    lib.epd_last_cuda_error.restype = ctypes.c_char_p
+    lib.epd_last_cuda_error.argtypes = []
     lib.epd_debug_bookkeeping.restype = ctypes.c_int
     lib.epd_debug_bookkeeping.argtypes = [vp, i32p, i32p, i32p, i32p]
     lib.epd_debug_set_taps.restype = ctypes.c_int

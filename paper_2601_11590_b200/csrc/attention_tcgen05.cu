@@ -1,33 +1,54 @@
 // Block-diagonal bidirectional flash attention on the 5th-generation tensor cores.
 //
-// One CTA handles one (segment, head, 128-query tile) and streams the segment's keys/values in
-// tiles of 128.  Per key tile:
-//   S = Q K^T          tcgen05.mma, both operands K-major in shared memory, fp32 S in TMEM
-//   online softmax     4 warps, one thread per query row: tcgen05.ld S, running max / sum in
-//                      registers (base-2 exponentials; q arrives scaled by log2(e)/sqrt(head_dim)),
-//                      P = exp2(S - m) written back over S in TMEM as bf16 (tcgen05.st)
-//   O += P V           tcgen05.mma with P as the TMEM operand and V read MN-major from shared memory
-// The running max is only advanced (and O rescaled in TMEM) when it grows by more than 2^8; until
-// then the stale max is used for P, the row sum and O alike, so the result is unchanged.
-// Warp roles: warp 0 TMA producer, warp 1 TMEM allocation + MMA issue, warps 2..5 softmax /
-// rescale / epilogue.  Q, K and V tiles are single-buffered (K is reloaded while P V runs, V while
-// the next Q K^T and softmax run); two CTAs share an SM so one CTA's softmax overlaps the other's
-// MMAs.  head_dim 72 is stored padded to 80: columns 0..63 form a 128-byte-swizzled box, columns
-// 64..79 a 32-byte-swizzled box, each fed to its own MMA.
+// Persistent kernel, one CTA per SM.  A work item is one (segment, head, 128-query tile); items are
+// ordered longest segment first and dealt round-robin to the CTAs.  Inside an item the segment's
+// keys/values stream through shared memory in tiles of BKV keys, and the two softmax warpgroups take
+// alternate key tiles, each with its own running max / sum and its own output accumulator:
+//   S_w = Q K^T        tcgen05.mma, both operands K-major in shared memory, fp32 S_w in TMEM (w = tile parity)
+//   online softmax     warpgroup w, one thread per query row: the S row is read once into registers
+//                      (tcgen05.ld) and the S_w buffer handed back at once, so the next S_w is computed
+//                      while this tile's exponentials run; P = exp2(S - m) goes to a separate bf16
+//                      buffer P_w (tcgen05.st).  q arrives scaled by log2(e)/sqrt(head_dim), so base-2
+//                      exponentials suffice
+//   O_w += P_w V       one tcgen05.mma per 16 keys with P_w as the TMEM operand and V read MN-major
+//                      from shared memory
+// Two threads feed the tensor pipe, one issuing the score products and one the P V products (the
+// waits and commits around a product cost more issue time than the product itself, so one thread
+// cannot keep up).  Score tiles run ahead of the P V products by as much as the S_w buffers and the
+// K ring allow, so a warpgroup does not wait for the tensor pipe in steady state and the exponential
+// unit stays busy.  That unit delivers 16 results per clock per SM, which bounds the softmax, so one
+// exponential in kFmaExpEvery is evaluated on the FMA pipe instead (cubic for 2^fraction).
+// The running max only advances (and O_w is rescaled in TMEM) when it grows by more than 2^8; until
+// then the stale max serves P, the row sum and O_w alike, which leaves the result unchanged.  At the
+// end of an item the two partial results are merged:
+//   m = max(m0, m1),  O = (2^(m0-m) O0 + 2^(m1-m) O1) / (2^(m0-m) l0 + 2^(m1-m) l1).
+// TMEM (512 columns): S0 | P0 | S1 | P1 | O0 | O1, with BKV chosen so that this fits: 112 keys for a
+// padded head width of 80, 80 keys for 128, 128 keys for 64.
+// Warp roles: warp 0 TMA producer of Q (double-buffered across items) and the K ring, warp 3 TMA
+// producer of the V ring (a V tile stays resident much longer than a K tile, so the two rings must
+// not throttle each other), warp 1 TMEM allocation + Q K^T issue, warp 2 P V issue, warps 4..7 and
+// 8..11 the two softmax warpgroups (also merge + epilogue).
+// head_dim 72 is stored padded to 80.  Q and K tiles: columns 0..63 form a 128-byte-swizzled box,
+// columns 64..79 a 32-byte-swizzled box, each contraction step its own MMA.  V tiles: five
+// 32-byte-swizzled boxes of 16 columns, so that one MMA covers all 80 output columns (an MMA costs
+// max(45, N/2) clocks whatever its width, so few wide ones beat many narrow ones).
 // Every mbarrier wait is bounded: on expiry the kernel records EPD_ETIMEOUT and drains.
 #include <cuda.h>
 
+#include <algorithm>
 #include <mutex>
+#include <vector>
 
 #include "common.cuh"
 
 namespace epd {
 namespace {
 
-constexpr int BQ = 128;   // query rows per CTA
-constexpr int BKV = 128;  // keys per tile
-constexpr int kThreads = 192;
+constexpr int BQ = 128;          // query rows per work item
+constexpr int kThreads = 384;    // warps 0..3: loaders and MMA issuers; warps 4..11: two softmax warpgroups
+constexpr int kMaxSegs = 128;    // segments one launch can describe
 constexpr long long kWaitCycles = 4000000000LL;
+constexpr int kFmaExpEvery = 4;            // 1 in 4 exponentials is computed with FMAs (must be even)
 constexpr float kRescaleThreshold = 8.0f;  // log2 of the largest P value tolerated before rescaling
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -51,6 +72,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Bounded wait.  Returns false (and raises *abort_flag) if the phase did not complete in time or
+// another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
@@ -105,37 +128,92 @@ __device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64
       ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// mbarrier arrives once all tcgen05.mma issued so far by this thread have completed.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
 
-#define EPD_R16(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), \
-    "=r"(r[o + 6]), "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]),                \
-    "=r"(r[o + 12]), "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15])
-#define EPD_W16(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]),       \
-    "r"(r[o + 6]), "r"(r[o + 7]), "r"(r[o + 8]), "r"(r[o + 9]), "r"(r[o + 10]), "r"(r[o + 11]), "r"(r[o + 12]),       \
-    "r"(r[o + 13]), "r"(r[o + 14]), "r"(r[o + 15])
+#define EPD_R8(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), \
+    "=r"(r[o + 6]), "=r"(r[o + 7])
+#define EPD_W8(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]),       \
+    "r"(r[o + 6]), "r"(r[o + 7])
+#define EPD_R16(r, o) EPD_R8(r, o), EPD_R8(r, o + 8)
+#define EPD_W16(r, o) EPD_W8(r, o), EPD_W8(r, o + 8)
+#define EPD_R32(r, o) EPD_R16(r, o), EPD_R16(r, o + 16)
+#define EPD_W32(r, o) EPD_W16(r, o), EPD_W16(r, o + 16)
+#define EPD_R64(r, o) EPD_R32(r, o), EPD_R32(r, o + 32)
+#define EPD_W64(r, o) EPD_W32(r, o), EPD_W32(r, o + 32)
 
-// 32 lanes x 16 consecutive 32-bit columns: thread i of the warp owns lane (base + i).
+// tcgen05.ld / tcgen05.st, shape 32x32b: thread i of the warp owns TMEM lane (base + i) and moves
+// N consecutive 32-bit columns.  One instruction per call; a wide form costs about the same issue
+// time as a narrow one, so callers use the widest that fits.
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : EPD_R8(r, 0) : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : EPD_R16(r, 0)
-      : "r"(taddr)
-      : "memory");
+      : EPD_R16(r, 0) : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-  tmem_ld16(taddr, r);
-  tmem_ld16(taddr + 16, r + 16);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : EPD_R32(r, 0) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+      : EPD_R64(r, 0) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), EPD_W8(r, 0) : "memory");
 }
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
       "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), EPD_W16(r, 0)
-      : "memory");
+      ::"r"(taddr), EPD_W16(r, 0) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), EPD_W32(r, 0) : "memory");
+}
+__device__ __forceinline__ void tmem_st64(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x64.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, "
+      "%33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, "
+      "%49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63, %64};"
+      ::"r"(taddr), EPD_W64(r, 0) : "memory");
+}
+// N columns (a multiple of 8) with as few instructions as possible.
+template <int N>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t* r) {
+  if constexpr (N >= 64) { tmem_ld64(taddr, r); tmem_ld_cols<N - 64>(taddr + 64, r + 64); }
+  else if constexpr (N >= 32) { tmem_ld32(taddr, r); tmem_ld_cols<N - 32>(taddr + 32, r + 32); }
+  else if constexpr (N >= 16) { tmem_ld16(taddr, r); tmem_ld_cols<N - 16>(taddr + 16, r + 16); }
+  else if constexpr (N >= 8) { tmem_ld8(taddr, r); tmem_ld_cols<N - 8>(taddr + 8, r + 8); }
+}
+template <int N>
+__device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t* r) {
+  if constexpr (N >= 64) { tmem_st64(taddr, r); tmem_st_cols<N - 64>(taddr + 64, r + 64); }
+  else if constexpr (N >= 32) { tmem_st32(taddr, r); tmem_st_cols<N - 32>(taddr + 32, r + 32); }
+  else if constexpr (N >= 16) { tmem_st16(taddr, r); tmem_st_cols<N - 16>(taddr + 16, r + 16); }
+  else if constexpr (N >= 8) { tmem_st8(taddr, r); tmem_st_cols<N - 8>(taddr + 8, r + 8); }
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -145,8 +223,23 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// 2^x for x <= 0 without the special-function unit: x = n + f with n integer and f in [-0.5, 0.5],
+// 2^f from a cubic (relative error 1.2e-4, far below the bf16 rounding of P), and n added into the
+// exponent field.
+__device__ __forceinline__ float ex2_fma(float x) {
+  x = fmaxf(x, -125.0f);
+  const float t = x + 12582912.0f;     // 1.5 * 2^23: the sum's low mantissa bits hold round(x)
+  const float f = x - (t - 12582912.0f);
+  float p = 0.05459282547235489f;
+  p = fmaf(p, f, 0.24221783876419067f);
+  p = fmaf(p, f, 0.6933686137199402f);
+  p = fmaf(p, f, 1.0f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
 
 // Shared-memory matrix descriptor.  layout: 2 = 128-byte swizzle, 6 = 32-byte swizzle.
+// K-major operand: sbo = distance between 8-row groups.  MN-major operand: lbo = distance between
+// swizzle-wide column groups, sbo = distance between 8-row (contraction) groups.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
   uint64_t d = 0;
   d |= (uint64_t)((addr & 0x3FFFF) >> 4);
@@ -157,244 +250,439 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
   return d;
 }
 // bf16 x bf16 -> fp32, M = 128; b_mn = 1 when the B operand is MN-major (V: head_dim contiguous).
-__device__ __forceinline__ uint32_t instr_desc(int n, int b_mn) {
+__host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) |
          ((uint32_t)(128 >> 4) << 24);
 }
 
-// Shared-memory plan for a padded head width DHP (64, 80 or 128).
+// Shared-memory and tensor-memory plan for a padded head width DHP (64, 80 or 128).
 template <int DHP>
 struct Plan {
-  static constexpr int kMainBoxes = DHP / 64;          // 128-byte-swizzled boxes of 64 columns
-  static constexpr int kTail = DHP % 64;               // 0 or 16 columns, 32-byte swizzle
+  static constexpr int BKV = DHP == 80 ? 112 : DHP == 128 ? 80 : 128;   // keys per tile
+  static constexpr int kPCols = (BKV / 2 + 15) / 16 * 16;              // TMEM columns reserved for P_w
+  static constexpr int kS0 = 0, kP0 = BKV, kS1 = BKV + kPCols, kP1 = kS1 + BKV;
+  static constexpr int kO0 = 2 * (BKV + kPCols), kO1 = kO0 + DHP;
+  static_assert(kO1 + DHP <= 512, "tensor memory plan does not fit");
+  static constexpr int kMainBoxes = DHP / 64;          // Q, K: 128-byte-swizzled boxes of 64 columns
+  static constexpr int kTail = DHP % 64;               // Q, K: 0 or 16 columns, 32-byte swizzle
   static_assert(kTail == 0 || kTail == 16, "padded head width must be 64*a or 64*a + 16");
-  static constexpr int kMainBytes = BKV * 128;         // one main box: 128 rows x 128 bytes
-  static constexpr int kTailBytes = kTail ? BKV * 32 : 0;
-  static constexpr int kTileBytes = kMainBoxes * kMainBytes + kTailBytes;  // one of Q / K / V
-  static constexpr int kQ = 0, kK = kTileBytes, kV = 2 * kTileBytes;
-  static constexpr int kBar = 3 * kTileBytes;          // 9 mbarriers, tmem slot, abort flag, segment info
-  static constexpr int kTotal = kBar + 9 * 8 + 32;
-  // at most two CTAs per SM: each allocates 256 of the 512 TMEM columns
-  static constexpr int kDynamic = (kTotal + 1024 > 78 * 1024) ? kTotal + 1024 : 78 * 1024;
-  static constexpr int kOCols = DHP;                   // O accumulator columns, after the 128 S columns
+  static constexpr bool kV32 = kTail != 0;             // V as 32-byte-swizzled boxes of 16 columns
+  static constexpr int kQMain = BQ * 128, kQTail = kTail ? BQ * 32 : 0;
+  static constexpr int kQBytes = kMainBoxes * kQMain + kQTail;
+  static constexpr int kKMain = BKV * 128, kKTail = kTail ? BKV * 32 : 0;
+  static constexpr int kKBytes = kMainBoxes * kKMain + kKTail;          // bytes TMA writes per K (or V) tile
+  static constexpr int kKStride = (kKBytes + 1023) / 1024 * 1024;       // ring slot pitch (1024-byte aligned)
+  static constexpr int kVBox = kV32 ? BKV * 32 : BKV * 128;             // one V box
+  static constexpr int kVBoxes = kV32 ? DHP / 16 : DHP / 64;
+  static_assert(kVBox * kVBoxes == kKBytes, "K and V tiles have the same size");
+  static constexpr int KS = DHP == 128 ? 3 : 4;        // K ring depth
+  static constexpr int VS = DHP == 128 ? 3 : 4;        // V ring depth
+  static constexpr int kQ = 0;                         // two Q buffers
+  static constexpr int kK = 2 * kQBytes;
+  static constexpr int kV = kK + KS * kKStride;
+  static constexpr int kMl = kV + VS * kKStride;       // (m, l) of both warpgroups, by item parity: float2[2][2][128]
+  static constexpr int kBar = kMl + 4 * BQ * 8;
+  // q_full[2] q_empty[2] k_full[KS] k_empty[KS] v_full[VS] v_empty[VS] s_full[2] s_free[2] p_full[2] p_free[2]
+  // o_final o_free ml_ready
+  static constexpr int kNumBars = 4 + 2 * KS + 2 * VS + 11;
+  static constexpr int kTotal = kBar + kNumBars * 8 + 32;
+  static constexpr int kDynamic = kTotal + 1024;       // slack to align the tiles to 1024 bytes
+  static_assert(kQBytes % 1024 == 0, "Q buffers keep the rings 1024-byte aligned");
+  static_assert(kDynamic > 116 * 1024, "one CTA per SM is assumed by the TMEM allocation");
+  static_assert(kDynamic <= 232448, "exceeds the shared memory of one CTA");
+  static constexpr int kOChunks = DHP / 16;            // 16-column pieces of an O accumulator
+  static constexpr int kSChunks = BKV / 16;            // 16-column pieces of a score row
 };
 
 struct Maps {
-  CUtensorMap q_main, q_tail, k_main, k_tail, v_main, v_tail;
+  CUtensorMap q_main, q_tail, k_main, k_tail, v;
 };
 
+// Segments of one launch, longest first (host-sorted).
+struct SegList {
+  int n;
+  int beg[kMaxSegs];
+  int len[kMaxSegs];
+};
+
+struct Item {
+  int head, seg_beg, seg_len, q0, n_kv;
+};
+
+// Item i -> (segment, head, query tile): segments in list order, then head, then query tile, so
+// that neighbouring items (which run at the same time on different SMs) share K and V in L2.
+template <int BKV>
+__device__ __forceinline__ Item decode_item(const SegList& segs, int heads, int i) {
+  Item it{0, 0, 0, 0, 0};
+  for (int s = 0; s < segs.n; ++s) {
+    const int qt = (segs.len[s] + BQ - 1) / BQ;
+    const int cnt = qt * heads;
+    if (i < cnt) {
+      it.head = i / qt;
+      it.seg_beg = segs.beg[s];
+      it.seg_len = segs.len[s];
+      it.q0 = it.seg_beg + (i - it.head * qt) * BQ;
+      it.n_kv = (it.seg_len + BKV - 1) / BKV;
+      return it;
+    }
+    i -= cnt;
+  }
+  return it;
+}
+
 template <int DHP>
-__global__ void __launch_bounds__(kThreads, 2)
-attention_tc_kernel(const __grid_constant__ Maps maps, const int32_t* __restrict__ cu, int n_seg,
+__global__ void __launch_bounds__(kThreads, 1)
+attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ SegList segs, int n_items,
                     __nv_bfloat16* __restrict__ out, int T, int heads, int dh, int* __restrict__ status) {
   using P = Plan<DHP>;
+  constexpr int BKV = P::BKV;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + P::kBar);
-  uint64_t *q_full = bars, *k_full = bars + 1, *k_empty = bars + 2, *v_full = bars + 3, *v_empty = bars + 4,
-           *s_full = bars + 5, *p_full = bars + 6, *o_done = bars + 7;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 9);
+  uint64_t* q_full = bars;                    // [2]
+  uint64_t* q_empty = bars + 2;               // [2]
+  uint64_t* k_full = bars + 4;                // [KS]
+  uint64_t* k_empty = k_full + P::KS;         // [KS]
+  uint64_t* v_full = k_empty + P::KS;         // [VS]
+  uint64_t* v_empty = v_full + P::VS;         // [VS]
+  uint64_t* s_full = v_empty + P::VS;         // [2]  S_w complete
+  uint64_t* s_free = s_full + 2;              // [2]  S_w copied to registers (4 warp arrivals)
+  uint64_t* p_full = s_free + 2;              // [2]  P_w written (4 warp arrivals)
+  uint64_t* p_free = p_full + 2;              // [2]  P_w consumed: the warpgroup's last P V is complete
+  uint64_t* o_final = p_free + 2;             // all P V products of the item complete
+  uint64_t* o_free = o_final + 1;             // both accumulators read out (8 warp arrivals)
+  uint64_t* ml_ready = o_free + 1;            // both warpgroups published (m, l) (8 warp arrivals)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + P::kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float2* ml_all = reinterpret_cast<float2*>(smem + P::kMl);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int head = blockIdx.y;
-
-  // which segment and query tile: walk the segments (a few dozen at most)
-  int tile = blockIdx.x, seg_beg = 0, seg_end = 0;
-  for (int i = 0; i < n_seg; ++i) {
-    const int b = cu[i], e = cu[i + 1];
-    const int nt = (e - b + BQ - 1) / BQ;
-    if (tile < nt) { seg_beg = b; seg_end = e; break; }
-    tile -= nt;
-  }
-  const int q0 = seg_beg + tile * BQ;            // first query token of this CTA
-  const int seg_len = seg_end - seg_beg;
-  const int n_kv = (seg_len + BKV - 1) / BKV;
-  const int row_base = head * T;                 // row of token 0 of this head in the [heads*T, DHP] matrices
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 8; ++i) mbar_init(&bars[i], i == 6 ? 4 : 1);  // p_full: one arrival per softmax warp
+    for (int i = 0; i < P::kNumBars; ++i) mbar_init(&bars[i], 1);
+    for (int w = 0; w < 2; ++w) { mbar_init(&s_free[w], 4); mbar_init(&p_full[w], 4); }
+    mbar_init(o_free, 8);
+    mbar_init(ml_ready, 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, 256);
+    tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base;        // S (fp32, 128 columns), overwritten by P (bf16 pairs, 64 columns)
-  const uint32_t tmem_o = tmem_base + 128;  // O (fp32, DHP columns)
 
   if (warp == 0) {
-    // ---------------------------------------------------------------- TMA producer
-    if (lane == 0 && seg_len > 0) {
-      auto load_tile = [&](uint8_t* dst, const CUtensorMap* mm, const CUtensorMap* mt, int row, uint64_t* bar) {
-        mbar_expect_tx(bar, P::kTileBytes);
+    // ---------------------------------------------------------------- TMA producer of Q and K
+    if (lane == 0) {
+      uint32_t kc = 0, n = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
+        const Item it = decode_item<BKV>(segs, heads, item);
+        const int row_base = it.head * T;
+        const int qb = n & 1;
+        if (!mbar_wait(&q_empty[qb], ((n >> 1) & 1) ^ 1, abort_flag)) break;
+        {
+          uint8_t* dst = smem + P::kQ + qb * P::kQBytes;
+          mbar_expect_tx(&q_full[qb], P::kQBytes);
 #pragma unroll
-        for (int b = 0; b < P::kMainBoxes; ++b) tma_load_2d(dst + b * P::kMainBytes, mm, b * 64, row, bar);
-        if (P::kTail) tma_load_2d(dst + P::kMainBoxes * P::kMainBytes, mt, P::kMainBoxes * 64, row, bar);
-      };
-      load_tile(smem + P::kQ, &maps.q_main, &maps.q_tail, row_base + q0, q_full);
-      for (int j = 0; j < n_kv; ++j) {
-        const int row = row_base + seg_beg + j * BKV;
-        if (!mbar_wait(k_empty, (j & 1) ^ 1, abort_flag)) break;
-        load_tile(smem + P::kK, &maps.k_main, &maps.k_tail, row, k_full);
-        if (!mbar_wait(v_empty, (j & 1) ^ 1, abort_flag)) break;
-        load_tile(smem + P::kV, &maps.v_main, &maps.v_tail, row, v_full);
+          for (int b = 0; b < P::kMainBoxes; ++b)
+            tma_load_2d(dst + b * P::kQMain, &maps.q_main, b * 64, row_base + it.q0, &q_full[qb]);
+          if (P::kTail)
+            tma_load_2d(dst + P::kMainBoxes * P::kQMain, &maps.q_tail, P::kMainBoxes * 64, row_base + it.q0, &q_full[qb]);
+        }
+        for (int j = 0; j < it.n_kv; ++j, ++kc) {
+          const int row = row_base + it.seg_beg + j * BKV;
+          const int ks = kc % P::KS;
+          if (!mbar_wait(&k_empty[ks], ((kc / P::KS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          uint8_t* dk = smem + P::kK + ks * P::kKStride;
+          mbar_expect_tx(&k_full[ks], P::kKBytes);
+#pragma unroll
+          for (int b = 0; b < P::kMainBoxes; ++b) tma_load_2d(dk + b * P::kKMain, &maps.k_main, b * 64, row, &k_full[ks]);
+          if (P::kTail) tma_load_2d(dk + P::kMainBoxes * P::kKMain, &maps.k_tail, P::kMainBoxes * 64, row, &k_full[ks]);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 3) {
+    // ---------------------------------------------------------------- TMA producer of V
+    if (lane == 0) {
+      uint32_t vc = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const Item it = decode_item<BKV>(segs, heads, item);
+        const int row_base = it.head * T;
+        for (int j = 0; j < it.n_kv; ++j, ++vc) {
+          const int row = row_base + it.seg_beg + j * BKV;
+          const int vs = vc % P::VS;
+          if (!mbar_wait(&v_empty[vs], ((vc / P::VS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          uint8_t* dv = smem + P::kV + vs * P::kKStride;
+          mbar_expect_tx(&v_full[vs], P::kKBytes);
+#pragma unroll
+          for (int b = 0; b < P::kVBoxes; ++b)
+            tma_load_2d(dv + b * P::kVBox, &maps.v, b * (P::kV32 ? 16 : 64), row, &v_full[vs]);
+        }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ---------------------------------------------------------------- MMA issuer
-    if (lane == 0 && seg_len > 0) {
-      const uint32_t sq = smem_u32(smem + P::kQ), sk = smem_u32(smem + P::kK), sv = smem_u32(smem + P::kV);
-      bool ok = mbar_wait(q_full, 0, abort_flag);
-      for (int j = 0; j < n_kv && ok; ++j) {
-        const int kv_valid = min(BKV, seg_len - j * BKV);
-        const int n16 = (kv_valid + 15) & ~15;  // keys taking part in this tile's MMAs
-        // S and O of the previous tile must be complete before S is overwritten
-        if (j > 0 && !mbar_wait(o_done, (j - 1) & 1, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(k_full, j & 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        {
-          const uint32_t idesc = instr_desc(n16, 0);
-          uint32_t accum = 0;
+    // ---------------------------------------------------------------- Q K^T issuer:  S_w(j) = Q K_j^T
+    if (lane == 0) {
+      uint32_t kc = 0, n = 0, sc0 = 0, sc1 = 0;        // sc_w: score tiles issued for warpgroup w
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
+        const Item it = decode_item<BKV>(segs, heads, item);
+        const int qb = n & 1;
+        if (!mbar_wait(&q_full[qb], (n >> 1) & 1, abort_flag)) break;
+        const uint32_t sq = smem_u32(smem + P::kQ + qb * P::kQBytes);
+        const uint64_t dq_main = smem_desc(sq, 16, 1024, 2);
+        const uint64_t dq_tail = smem_desc(sq + P::kMainBoxes * P::kQMain, 16, 256, 6);
+        for (int j = 0; j < it.n_kv; ++j, ++kc) {
+          const int w = j & 1;
+          const int ks = kc % P::KS;
+          if (!mbar_wait(&k_full[ks], (kc / P::KS) & 1, abort_flag)) { ok = false; break; }
+          uint32_t& sc = w ? sc1 : sc0;
+          // the warpgroup must have copied its previous score tile out of S_w
+          if (sc > 0 && !mbar_wait(&s_free[w], (sc - 1) & 1, abort_flag)) { ok = false; break; }
+          ++sc;
+          tc_fence_after();
+          const uint32_t sk = smem_u32(smem + P::kK + ks * P::kKStride);
+          const uint64_t dk_main = smem_desc(sk, 16, 1024, 2);
+          const uint64_t dk_tail = smem_desc(sk + P::kMainBoxes * P::kKMain, 16, 256, 6);
+          const uint32_t tmem_s = tmem_base + (w ? P::kS1 : P::kS0);
+          const int kv_valid = min(BKV, it.seg_len - j * BKV);
+          const uint32_t idesc = kv_valid == BKV ? instr_desc(BKV, 0) : instr_desc((kv_valid + 15) & ~15, 0);
+          // descriptor addresses count 16-byte units: one 16-element step inside a swizzled row is +2
 #pragma unroll
           for (int b = 0; b < P::kMainBoxes; ++b) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              umma_ss(tmem_s, smem_desc(sq + b * P::kMainBytes + k * 32, 16, 1024, 2),
-                      smem_desc(sk + b * P::kMainBytes + k * 32, 16, 1024, 2), idesc, accum);
-              accum = 1;
-            }
+            for (int k = 0; k < 4; ++k)
+              umma_ss(tmem_s, dq_main + (b * P::kQMain / 16 + 2 * k), dk_main + (b * P::kKMain / 16 + 2 * k), idesc,
+                      (b | k) != 0);
           }
-          if (P::kTail)
-            umma_ss(tmem_s, smem_desc(sq + P::kMainBoxes * P::kMainBytes, 16, 256, 6),
-                    smem_desc(sk + P::kMainBoxes * P::kMainBytes, 16, 256, 6), idesc, accum);
+          if (P::kTail) umma_ss(tmem_s, dq_tail, dk_tail, idesc, 1);
+          umma_commit(&s_full[w]);
+          umma_commit(&k_empty[ks]);
+          if (j == it.n_kv - 1) umma_commit(&q_empty[qb]);
         }
-        umma_commit(s_full);
-        umma_commit(k_empty);
-        if (!mbar_wait(p_full, j & 1, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(v_full, j & 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-        {
-          const uint32_t idesc_main = instr_desc(64, 1), idesc_tail = instr_desc(16, 1);
-          for (int ks = 0; ks < n16 / 16; ++ks) {
-            const uint32_t accum = (j | ks) != 0;
-            const uint32_t a_tmem = tmem_s + ks * 8;  // 16 bf16 of P = 8 columns
-#pragma unroll
-            for (int b = 0; b < P::kMainBoxes; ++b)
-              umma_ts(tmem_o + b * 64, a_tmem, smem_desc(sv + b * P::kMainBytes + ks * 2048, 16384, 1024, 2),
-                      idesc_main, accum);
-            if (P::kTail)
-              umma_ts(tmem_o + P::kMainBoxes * 64, a_tmem,
-                      smem_desc(sv + P::kMainBoxes * P::kMainBytes + ks * 512, 4096, 256, 6), idesc_tail, accum);
-          }
-        }
-        umma_commit(v_empty);
-        umma_commit(o_done);
       }
     }
     __syncwarp();
-  } else if (seg_len > 0) {
-    // ---------------------------------------------------------------- softmax / rescale / epilogue
-    const int q = warp & 3;
-    const int r = q * 32 + lane;                       // query row inside the tile
-    const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-    float m = -INFINITY, l = 0.0f;
-    bool ok = true;
-    for (int j = 0; j < n_kv; ++j) {
-      const int kv_valid = min(BKV, seg_len - j * BKV);
-      const int n_chunks = (kv_valid + 31) >> 5;       // 32-column chunks that hold valid keys
-      if (!mbar_wait(s_full, j & 1, abort_flag)) { ok = false; break; }
-      tc_fence_after();
-      // pass 1: row max over the valid keys
-      float m_tile = -INFINITY;
-      for (int c = 0; c < n_chunks; ++c) {
-        uint32_t s[32];
-        tmem_ld32(tmem_s + lane_off + c * 32, s);
-        tmem_ld_wait();
+  } else if (warp == 2) {
+    // ---------------------------------------------------------------- P V issuer:  O_w += P_w(j) V_j
+    if (lane == 0) {
+      uint32_t vc = 0, n = 0, pc0 = 0, pc1 = 0;        // pc_w: P tiles consumed for warpgroup w
+      constexpr uint32_t idesc = instr_desc(DHP, 1);
+      constexpr uint32_t kStep = P::kV32 ? 512 / 16 : 2048 / 16;   // 16 keys further down the V tile, 16-byte units
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
+        const Item it = decode_item<BKV>(segs, heads, item);
+        // the accumulators of the previous item must have been read out before they are overwritten
+        if (n > 0 && !mbar_wait(o_free, (n - 1) & 1, abort_flag)) break;
+        for (int j = 0; j < it.n_kv; ++j, ++vc) {
+          const int w = j & 1;
+          const int vs = vc % P::VS;
+          uint32_t& pc = w ? pc1 : pc0;
+          if (!mbar_wait(&p_full[w], pc & 1, abort_flag)) { ok = false; break; }
+          ++pc;
+          if (!mbar_wait(&v_full[vs], (vc / P::VS) & 1, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sv = smem_u32(smem + P::kV + vs * P::kKStride);
+          // MN-major V: boxes (16 or 64 columns wide) are kVBox apart, 8-row groups 256 / 1024 bytes apart
+          const uint64_t dv = P::kV32 ? smem_desc(sv, P::kVBox, 256, 6) : smem_desc(sv, P::kVBox, 1024, 2);
+          const uint32_t tmem_p = tmem_base + (w ? P::kP1 : P::kP0), tmem_o = tmem_base + (w ? P::kO1 : P::kO0);
+          const uint32_t first = j >= 2 ? 1u : 0u;     // a warpgroup's first tile starts O_w afresh
+          const int kv_valid = min(BKV, it.seg_len - j * BKV);
+          if (kv_valid == BKV) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (c * 32 + i < kv_valid) m_tile = fmaxf(m_tile, __uint_as_float(s[i]));
-      }
-      // advance the running max only when it would grow by more than the threshold
-      float scale = 1.0f;
-      bool grow = false;
-      if (j == 0) {
-        m = m_tile;
-      } else if (m_tile - m > kRescaleThreshold) {
-        scale = ex2(m - m_tile);
-        m = m_tile;
-        l *= scale;
-        grow = true;
-      }
-      if (__any_sync(0xffffffffu, grow)) {
-        // O of the previous tiles is complete (the S we just read was issued after it): rescale it
-#pragma unroll
-        for (int c = 0; c < P::kOCols / 16; ++c) {
-          uint32_t o[16];
-          tmem_ld16(tmem_o + lane_off + c * 16, o);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * scale);
-          tmem_st16(tmem_o + lane_off + c * 16, o);
+            for (int ks = 0; ks < BKV / 16; ++ks)       // 16 bf16 of P = 8 columns
+              umma_ts(tmem_o, tmem_p + ks * 8, dv + ks * kStep, idesc, ks == 0 ? first : 1u);
+          } else {
+            const int steps = (kv_valid + 15) >> 4;
+            for (int ks = 0; ks < steps; ++ks)
+              umma_ts(tmem_o, tmem_p + ks * 8, dv + ks * kStep, idesc, ks == 0 ? first : 1u);
+          }
+          umma_commit(&v_empty[vs]);
+          umma_commit(&p_free[w]);
         }
+        if (!ok) break;
+        umma_commit(o_final);
       }
-      // pass 2: P = exp2(S - m) as bf16 pairs over the S columns already consumed
-      for (int c = 0; c < n_chunks; ++c) {
-        uint32_t s[32], pk[16];
-        tmem_ld32(tmem_s + lane_off + c * 32, s);
+    }
+    __syncwarp();
+  } else if (warp >= 4) {
+    // ---------------------------------------------------------------- softmax / rescale / merge / epilogue
+    const int w = (warp - 4) >> 2;                      // warpgroup = key-tile parity
+    const int qr = warp & 3;                            // TMEM lane quarter this warp may access
+    const int r = qr * 32 + lane;                       // query row inside the tile
+    const uint32_t lane_off = (uint32_t)(qr * 32) << 16;
+    const uint32_t tmem_s = tmem_base + (w ? P::kS1 : P::kS0) + lane_off;
+    const uint32_t tmem_p = tmem_base + (w ? P::kP1 : P::kP0) + lane_off;
+    const uint32_t tmem_o = tmem_base + (w ? P::kO1 : P::kO0) + lane_off;
+    uint32_t tc = 0, n = 0;                             // score tiles processed, items processed
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
+      const Item it = decode_item<BKV>(segs, heads, item);
+      float m = -INFINITY, l = 0.0f;
+      uint32_t s[BKV];
+      // The loop is software-pipelined: the tcgen05.ld of the next score tile is issued right after
+      // the tcgen05.st of this tile's P, so the two TMEM round trips overlap.
+      auto load_scores = [&](int j) -> bool {
+        const int kv_valid = min(BKV, it.seg_len - j * BKV);
+        if (!mbar_wait(&s_full[w], tc & 1, abort_flag)) return false;
+        tc_fence_after();
+        if (kv_valid == BKV) {
+          tmem_ld_cols<BKV>(tmem_s, s);
+        } else {
+#pragma unroll
+          for (int c = 0; c < P::kSChunks; ++c)
+            if (c * 16 < kv_valid) tmem_ld16(tmem_s + c * 16, s + c * 16);
+        }
+        return true;
+      };
+      if (w < it.n_kv && !load_scores(w)) { ok = false; break; }
+      for (int j = w; j < it.n_kv; j += 2) {
+        const int kv_valid = min(BKV, it.seg_len - j * BKV);
         tmem_ld_wait();
+        // S_w may be overwritten by the next score tile from here on
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_free[w]);
+
+        float mx[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mx[i] = -INFINITY;
+        if (kv_valid == BKV) {
+#pragma unroll
+          for (int i = 0; i < BKV; ++i) mx[i & 7] = fmaxf(mx[i & 7], __uint_as_float(s[i]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < BKV; ++i)
+            if (i < kv_valid) mx[i & 7] = fmaxf(mx[i & 7], __uint_as_float(s[i]));
+        }
+        const float m_tile = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                   fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7])));
+        // advance the running max only when it would grow by more than the threshold
+        float scale = 1.0f;
+        bool grow = false;
+        if (j == w) {
+          m = m_tile;
+        } else if (m_tile - m > kRescaleThreshold) {
+          scale = ex2(m - m_tile);
+          m = m_tile;
+          l *= scale;
+          grow = true;
+        }
+        // P = exp2(S - m) as bf16 pairs
+        const float neg_m = -m;
+        float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (kv_valid == BKV) {
+#pragma unroll
+          for (int i = 0; i < BKV / 2; ++i) {
+            // one exponential in kFmaExpEvery goes to the FMA pipe
+            const float p0 = ex2(__uint_as_float(s[2 * i]) + neg_m);
+            const float p1 = (i % (kFmaExpEvery / 2) == kFmaExpEvery / 2 - 1)
+                                 ? ex2_fma(__uint_as_float(s[2 * i + 1]) + neg_m)
+                                 : ex2(__uint_as_float(s[2 * i + 1]) + neg_m);
+            sum[i & 3] += p0 + p1;
+            __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+            s[i] = *reinterpret_cast<uint32_t*>(&b);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < BKV / 2; ++i) {
+            const float p0 = 2 * i < kv_valid ? ex2(__uint_as_float(s[2 * i]) + neg_m) : 0.0f;
+            const float p1 = 2 * i + 1 < kv_valid ? ex2(__uint_as_float(s[2 * i + 1]) + neg_m) : 0.0f;
+            sum[i & 3] += p0 + p1;
+            __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
+            s[i] = *reinterpret_cast<uint32_t*>(&b);
+          }
+        }
+        l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+        // P_w and O_w are free once this warpgroup's previous P V has completed
+        if (tc > 0 && !mbar_wait(&p_free[w], (tc - 1) & 1, abort_flag)) { ok = false; break; }
+        ++tc;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, grow)) {
+#pragma unroll
+          for (int c = 0; c < P::kOChunks; ++c) {
+            uint32_t o[16];
+            tmem_ld16(tmem_o + c * 16, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * scale);
+            tmem_st16(tmem_o + c * 16, o);
+          }
+        }
+        // 8 packed columns hold 16 keys; a store reads its registers when it is issued
+        if (kv_valid == BKV) {
+          tmem_st_cols<BKV / 2>(tmem_p, s);
+        } else {
+#pragma unroll
+          for (int c = 0; c < P::kSChunks; ++c)
+            if (c * 16 < kv_valid) tmem_st8(tmem_p + c * 8, s + c * 8);
+        }
+        if (j + 2 < it.n_kv && !load_scores(j + 2)) { ok = false; break; }
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full[w]);
+      }
+      if (!ok) break;
+      // merge the two partial results and write the item's rows; (m, l) are double-buffered by item
+      // parity because a warpgroup without key tiles in the next item may publish early
+      float2* ml = ml_all + (n & 1) * 2 * BQ;
+      ml[w * BQ + r] = make_float2(m, l);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(ml_ready);
+      if (!mbar_wait(ml_ready, n & 1, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(o_final, n & 1, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const bool has1 = it.n_kv > 1;
+      const float2 ml0 = ml[r], ml1 = ml[BQ + r];
+      const float mm = has1 ? fmaxf(ml0.x, ml1.x) : ml0.x;
+      const float a0 = ex2(ml0.x - mm), a1 = has1 ? ex2(ml1.x - mm) : 0.0f;
+      const float inv = 1.0f / (a0 * ml0.y + a1 * ml1.y);
+      const float f0 = a0 * inv, f1 = a1 * inv;
+      const int token = it.q0 + r;
+      const bool row_ok = token < it.seg_beg + it.seg_len;
+      __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + it.head * dh;
+      const uint32_t tmem_o0 = tmem_base + P::kO0 + lane_off, tmem_o1 = tmem_base + P::kO1 + lane_off;
+      constexpr int kSplit = (P::kOChunks + 1) / 2;    // warpgroup 0 writes chunks [0, kSplit), warpgroup 1 the rest
+      const int c_beg = w == 0 ? 0 : kSplit, c_end = w == 0 ? kSplit : P::kOChunks;
+      for (int c = c_beg; c < c_end; ++c) {
+        uint32_t o0[16], o1[16];
+        tmem_ld16(tmem_o0 + c * 16, o0);
+        if (has1) tmem_ld16(tmem_o1 + c * 16, o1);
+        tmem_ld_wait();
+        float v[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
-          const int col = c * 32 + 2 * i;
-          const float p0 = col < kv_valid ? ex2(__uint_as_float(s[2 * i]) - m) : 0.0f;
-          const float p1 = col + 1 < kv_valid ? ex2(__uint_as_float(s[2 * i + 1]) - m) : 0.0f;
-          l += p0 + p1;
-          __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
-          pk[i] = *reinterpret_cast<uint32_t*>(&b);
+          v[i] = __uint_as_float(o0[i]) * f0;
+          if (has1) v[i] = fmaf(__uint_as_float(o1[i]), f1, v[i]);
         }
-        tmem_st16(tmem_s + lane_off + c * 16, pk);
-      }
-      tmem_st_wait();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(p_full);
-    }
-    // epilogue: O / l -> bf16 -> out[token, head*dh ..]
-    if (ok && mbar_wait(o_done, (n_kv - 1) & 1, abort_flag)) {
-      tc_fence_after();
-      const float inv = 1.0f / l;
-      const int token = q0 + r;
-      __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + head * dh;
-#pragma unroll
-      for (int c = 0; c < P::kOCols / 16; ++c) {
-        uint32_t o[16];
-        tmem_ld16(tmem_o + lane_off + c * 16, o);
-        tmem_ld_wait();
-        if (token < seg_end) {
+        if (row_ok) {
 #pragma unroll
           for (int g = 0; g < 2; ++g) {
             if (c * 16 + g * 8 < dh) {  // dh is a multiple of 8
-              uint4 pk;
-              __nv_bfloat162 b0 = __floats2bfloat162_rn(__uint_as_float(o[8 * g]) * inv, __uint_as_float(o[8 * g + 1]) * inv);
-              __nv_bfloat162 b1 = __floats2bfloat162_rn(__uint_as_float(o[8 * g + 2]) * inv, __uint_as_float(o[8 * g + 3]) * inv);
-              __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[8 * g + 4]) * inv, __uint_as_float(o[8 * g + 5]) * inv);
-              __nv_bfloat162 b3 = __floats2bfloat162_rn(__uint_as_float(o[8 * g + 6]) * inv, __uint_as_float(o[8 * g + 7]) * inv);
-              pk.x = *reinterpret_cast<uint32_t*>(&b0);
-              pk.y = *reinterpret_cast<uint32_t*>(&b1);
-              pk.z = *reinterpret_cast<uint32_t*>(&b2);
-              pk.w = *reinterpret_cast<uint32_t*>(&b3);
-              *reinterpret_cast<uint4*>(orow + c * 16 + g * 8) = pk;
+              uint32_t pk[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * g + 2 * e], v[8 * g + 2 * e + 1]);
+                pk[e] = *reinterpret_cast<uint32_t*>(&b);
+              }
+              *reinterpret_cast<uint4*>(orow + c * 16 + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
           }
         }
       }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(o_free);
     }
   }
 
@@ -408,7 +696,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const int32_t* __restrict
   }
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, 256);
+    tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -432,21 +720,33 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// Map over a bf16 matrix [rows, dhp] (row pitch dhp*2 bytes): box = 128 rows x box_cols columns.
-bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int dhp, int box_cols, CUtensorMapSwizzle swz) {
+// Map over a bf16 matrix [rows, dhp] (row pitch dhp*2 bytes): box = box_rows rows x box_cols columns.
+bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int dhp, int box_cols, int box_rows,
+              CUtensorMapSwizzle swz) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)dhp, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)dhp * 2};
-  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)BKV};
+  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
 template <int DHP>
-cudaError_t launch(const Maps& maps, const int32_t* cu, int n_seg, int q_tiles, void* out, int T, int heads, int dh,
+cudaError_t launch(const Maps& maps, const SegList& segs, int n_items, void* out, int T, int heads, int dh,
                    int* status, cudaStream_t s) {
   using P = Plan<DHP>;
   auto kern = attention_tc_kernel<DHP>;
@@ -456,8 +756,8 @@ cudaError_t launch(const Maps& maps, const int32_t* cu, int n_seg, int q_tiles, 
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  dim3 grid((unsigned)q_tiles, (unsigned)heads);
-  kern<<<grid, kThreads, P::kDynamic, s>>>(maps, cu, n_seg, (__nv_bfloat16*)out, T, heads, dh, status);
+  const int grid = n_items < sm_count() ? n_items : sm_count();
+  kern<<<grid, kThreads, P::kDynamic, s>>>(maps, segs, n_items, (__nv_bfloat16*)out, T, heads, dh, status);
   return cudaGetLastError();
 }
 
@@ -471,28 +771,49 @@ bool attention_tc_supported(const void* q, const void* k, const void* v, const v
   return encode_tiled_fn() != nullptr;
 }
 
-cudaError_t attention_tc(const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
-                         const int32_t* host_cu_seqlens, int n_seg, void* out, int64_t T, int heads, int head_dim,
-                         int* status, cudaStream_t s) {
+cudaError_t attention_tc(const void* q, const void* k, const void* v, const int32_t* host_cu_seqlens, int n_seg,
+                         void* out, int64_t T, int heads, int head_dim, int* status, cudaStream_t s) {
   const int dhp = padded_head_dim(head_dim);
-  int q_tiles = 0;
-  for (int i = 0; i < n_seg; ++i) q_tiles += (host_cu_seqlens[i + 1] - host_cu_seqlens[i] + BQ - 1) / BQ;
-  if (q_tiles == 0) return cudaSuccess;
+  if (n_seg <= 0) return cudaSuccess;
   const int64_t rows = (int64_t)heads * T;
   Maps maps;
-  const void* ptr[3] = {q, k, v};
-  CUtensorMap* mains[3] = {&maps.q_main, &maps.k_main, &maps.v_main};
-  CUtensorMap* tails[3] = {&maps.q_tail, &maps.k_tail, &maps.v_tail};
-  for (int i = 0; i < 3; ++i) {
-    if (!make_map(mains[i], ptr[i], rows, dhp, 64, CU_TENSOR_MAP_SWIZZLE_128B)) return cudaErrorInvalidValue;
-    if (!make_map(tails[i], ptr[i], rows, dhp, 16, CU_TENSOR_MAP_SWIZZLE_32B)) return cudaErrorInvalidValue;
+  const int bkv = dhp == 80 ? Plan<80>::BKV : dhp == 128 ? Plan<128>::BKV : Plan<64>::BKV;
+  if (!make_map(&maps.q_main, q, rows, dhp, 64, BQ, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&maps.q_tail, q, rows, dhp, 16, BQ, CU_TENSOR_MAP_SWIZZLE_32B) ||
+      !make_map(&maps.k_main, k, rows, dhp, 64, bkv, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&maps.k_tail, k, rows, dhp, 16, bkv, CU_TENSOR_MAP_SWIZZLE_32B))
+    return cudaErrorInvalidValue;
+  if (dhp % 64 ? !make_map(&maps.v, v, rows, dhp, 16, bkv, CU_TENSOR_MAP_SWIZZLE_32B)
+               : !make_map(&maps.v, v, rows, dhp, 64, bkv, CU_TENSOR_MAP_SWIZZLE_128B))
+    return cudaErrorInvalidValue;
+  // longest segments first: items are dealt round-robin, so the long ones spread evenly and the
+  // short ones fill the tail
+  std::vector<int> order(n_seg);
+  for (int i = 0; i < n_seg; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+    return host_cu_seqlens[a + 1] - host_cu_seqlens[a] > host_cu_seqlens[b + 1] - host_cu_seqlens[b];
+  });
+  for (int first = 0; first < n_seg; first += kMaxSegs) {
+    SegList segs;
+    segs.n = n_seg - first < kMaxSegs ? n_seg - first : kMaxSegs;
+    int n_items = 0;
+    for (int i = 0; i < segs.n; ++i) {
+      const int sg = order[first + i];
+      segs.beg[i] = host_cu_seqlens[sg];
+      segs.len[i] = host_cu_seqlens[sg + 1] - host_cu_seqlens[sg];
+      n_items += (segs.len[i] + BQ - 1) / BQ * heads;
+    }
+    for (int i = segs.n; i < kMaxSegs; ++i) segs.beg[i] = segs.len[i] = 0;
+    cudaError_t e;
+    switch (dhp) {
+      case 64: e = launch<64>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s); break;
+      case 80: e = launch<80>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s); break;
+      case 128: e = launch<128>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s); break;
+      default: return cudaErrorInvalidValue;
+    }
+    if (e != cudaSuccess) return e;
   }
-  switch (dhp) {
-    case 64: return launch<64>(maps, cu_seqlens, n_seg, q_tiles, out, (int)T, heads, head_dim, status, s);
-    case 80: return launch<80>(maps, cu_seqlens, n_seg, q_tiles, out, (int)T, heads, head_dim, status, s);
-    case 128: return launch<128>(maps, cu_seqlens, n_seg, q_tiles, out, (int)T, heads, head_dim, status, s);
-    default: return cudaErrorInvalidValue;
-  }
+  return cudaSuccess;
 }
 
 }  // namespace
@@ -502,7 +823,7 @@ cudaError_t attention_any(int dtype, const void* q, const void* k, const void* v
                           int flags, int* status, cudaStream_t s) {
   if (dtype == EPD_DTYPE_BF16 && !(flags & EPD_ATTENTION_FORCE_FMA) &&
       attention_tc_supported(q, k, v, out, T, heads, head_dim))
-    return attention_tc(q, k, v, cu_seqlens, host_cu_seqlens, n_seg, out, T, heads, head_dim, status, s);
+    return attention_tc(q, k, v, host_cu_seqlens, n_seg, out, T, heads, head_dim, status, s);
   return attention_fma(dtype, q, k, v, cu_seqlens, n_seg, out, T, heads, head_dim, s);
 }
 

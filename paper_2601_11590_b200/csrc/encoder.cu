@@ -102,10 +102,16 @@ struct epd_encoder {
 
 namespace {
 
+// The CUDA error behind the most recent EPD_ECUDA of this thread (see epd_last_cuda_error()).
+thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+
 #define EPD_CUDA(expr)                        \
   do {                                        \
     cudaError_t e__ = (expr);                 \
-    if (e__ != cudaSuccess) return EPD_ECUDA; \
+    if (e__ != cudaSuccess) {                 \
+      g_last_cuda_error = e__;                \
+      return EPD_ECUDA;                       \
+    }                                         \
   } while (0)
 
 // Counts a launch of step class `cls` and, in profiling mode, records an event before it.
@@ -452,6 +458,8 @@ int epd_encoder_destroy(epd_encoder_t* enc) {
   delete enc;
   return EPD_OK;
 }
+
+const char* epd_last_cuda_error(void) { return cudaGetErrorName(g_last_cuda_error); }
 
 const char* epd_strerror(int status) {
   switch (status) {
