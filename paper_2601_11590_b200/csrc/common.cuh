@@ -63,4 +63,8 @@ bool linear_tc_supported(const void* x, int64_t ldx, const void* w, int64_t ldw,
 cudaError_t linear_tc(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out, int64_t ldo,
                       int64_t M, int64_t N, int64_t K, int flags, int forced_bn, int* status, cudaStream_t s);
 
+// Same contract on CTA pairs (256 x 256 tiles, tcgen05.mma.cta_group::2); gemm_tcgen05_pair.cu.
+cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
+                           int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, int* status, cudaStream_t s);
+
 }  // namespace epd

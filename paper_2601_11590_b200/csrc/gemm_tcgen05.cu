@@ -496,6 +496,8 @@ bool linear_tc_supported(const void* x, int64_t ldx, const void* w, int64_t ldw,
 
 cudaError_t linear_tc(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out, int64_t ldo,
                       int64_t M, int64_t N, int64_t K, int flags, int forced_bn, int* status, cudaStream_t s) {
+  // Without a forced tile width, anything taller than one 128-row tile goes to the CTA-pair kernel.
+  if (forced_bn == 0 && M > BM) return linear_tc_pair(x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, status, s);
   const int bn = forced_bn > 0 ? forced_bn : pick_bn((int)M, (int)N);
   const bool out_f32 = flags & (EPD_LINEAR_ACCUMULATE | EPD_LINEAR_OUT_F32);
   CUtensorMap tx, tw, to;

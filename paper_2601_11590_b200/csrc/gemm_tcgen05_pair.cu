@@ -1,0 +1,520 @@
+// bf16 linear layer on the 5th-generation tensor cores with CTA pairs:  out = act(x . w^T + bias) (+ out).
+//
+// Why pairs: with one CTA per tile the main loop is bound by shared-memory bandwidth, not by the
+// tensor pipe.  Per 64-wide contraction block a 128 x 256 tile has TMA write 48 KB into shared
+// memory and the MMAs read the same 48 KB back in the 512 clocks the MMAs need: 192 B/clk against
+// the 128 B/clk an SM's shared memory moves (measured: ~63 % of the MMA rate, which alone reaches
+// 8165 FLOP/clk/SM).  A pair of CTAs on neighbouring SMs (a cluster of 2) computes a 256 x 256 tile
+// with tcgen05.mma.cta_group::2: each CTA stages its own 128 rows of x and only HALF of the w tile
+// (128 of the 256 output columns); the hardware feeds both halves of w to both tensor cores.  That is
+// 32 KB written + 32 KB read per SM per block = 128 B/clk.
+//
+// Roles per CTA (10 warps):
+//   warp 0      TMA producer: loads its x tile and its half of the w tile into a STAGES-deep ring; the
+//               bytes of both CTAs are counted on the LEADER's (cluster rank 0) "full" barrier
+//   warp 1      allocates tensor memory (pair-wide allocation); in the leader one thread issues the MMAs
+//               for both CTAs and commits to the "empty" / "accumulator full" barriers of both
+//   warps 2..9  epilogue, two warps per TMEM lane quarter, each taking half of the tile's columns:
+//               tcgen05.ld, bias / GELU, 32-row x 128-byte chunks staged in swizzled shared memory and
+//               written with TMA (plain store, or reduce-add for the residual update)
+// Each CTA holds the accumulator rows of its own 128 rows of x (two accumulators of 256 columns, so
+// the epilogue of tile i overlaps the main loop of tile i+1).  Ragged M, N, K are handled by TMA
+// (zero fill on loads, clipping on stores).  No load in this file is a multicast load.
+// Every mbarrier wait is bounded: on expiry the CTA records EPD_ETIMEOUT and drains; the two cluster
+// barriers (start, end) are reached by both CTAs on every path.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace epd {
+namespace {
+
+constexpr int BM = 128;         // rows of x per CTA (256 per pair)
+constexpr int BK = 64;          // 64 bf16 = 128 bytes = one swizzle row
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 32 * (2 + kEpiWarps);
+constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address, in the cluster's shared-memory window, of the same variable in CTA `rank` of the pair.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Arrive on a barrier given by its cluster-window address (own CTA's or the peer's).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+// Tensor load into this CTA's shared memory whose completion bytes are counted on a barrier that may
+// live in the other CTA of the pair (given by its cluster-window address).
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* tm, int x, int y,
+                                                 uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, int x, int y, const void* smem_src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, int x, int y, const void* smem_src) {
+  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
+               "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem, both CTAs] (+)= A[smem, 128 rows per CTA] . B[smem, half the columns per CTA]^T; issued by
+// one thread of the leader CTA.
+__device__ __forceinline__ void umma_pair_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Once all MMAs issued so far by this thread have completed, arrive on the barrier at this offset in
+// both CTAs of the pair.
+__device__ __forceinline__ void umma_commit_both(uint64_t* bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(smem_u32(bar)), "h"((uint16_t)3)
+      : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major tile whose rows are 128 bytes, 128-byte swizzled: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)1 << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 256 over the pair, N = BN.
+__host__ __device__ constexpr uint32_t instr_desc_pair(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+__device__ __forceinline__ float gelu_tanh_fast(float x) {
+  const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+  return 0.5f * x * (1.0f + t);
+}
+
+template <int BN, int STAGES>
+struct PairLayout {
+  static constexpr int kABytes = BM * BK * 2;
+  static constexpr int kBBytes = (BN / 2) * BK * 2;     // this CTA's half of the w tile
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kOutBufBytes = 32 * 128;         // one staging buffer per epilogue warp
+  static constexpr int kOutOffset = STAGES * kStageBytes;
+  static constexpr int kBarOffset = kOutOffset + kEpiWarps * kOutBufBytes;
+  // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], tmem base, abort flag, bias[kEpiWarps][BN/2]
+  static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 4) * 8 + 16;
+  static constexpr int kTotal = kBiasOffset + kEpiWarps * (BN / 2) * 4;
+  static constexpr int kDynamic = kTotal + 1024;
+  static_assert(kDynamic <= 232448, "exceeds the shared memory of one CTA");
+  static_assert(kDynamic > 116 * 1024, "one CTA per SM is assumed by the TMEM allocation");
+};
+
+// ---------------------------------------------------------------------------------------------
+// Kernel
+// ---------------------------------------------------------------------------------------------
+template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
+                   const __grid_constant__ CUtensorMap tm_out, const __nv_bfloat16* __restrict__ bias, int M, int N,
+                   int K, int* __restrict__ status) {
+  using L = PairLayout<BN, STAGES>;
+  static_assert(BN == 256 || BN == 128, "tile width");
+  constexpr int kAccStride = BN;                 // TMEM columns between the two accumulators
+  constexpr int kTmemCols = 2 * kAccStride;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);   // used in the leader only
+  uint64_t* empty = full + STAGES;                                      // one set per CTA
+  uint64_t* tmem_full = empty + STAGES;                                 // one set per CTA
+  uint64_t* tmem_empty = tmem_full + 2;                                 // used in the leader only
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
+  float* bias_s = reinterpret_cast<float*>(smem + L::kBiasOffset);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();          // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int m_tiles = (M + 2 * BM - 1) / (2 * BM), n_tiles = (N + BN - 1) / BN;
+  const int num_tiles = m_tiles * n_tiles;
+  const int k_blocks = (K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 2 * kEpiWarps); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_base_slot, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync();                                 // both CTAs' barriers exist before either signals the other
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer (both CTAs)
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_x) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
+        const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;        // this CTA's rows of x
+        const int n0 = (tile / m_tiles) * BN + (int)rank * (BN / 2);       // this CTA's half of the w tile
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          uint8_t* sa = smem + stage * L::kStageBytes;
+          // the leader's barrier counts the bytes of both CTAs
+          if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
+          const uint32_t bar = map_to_rank(smem_u32(&full[stage]), 0);
+          tma_load_2d_pair(sa, &tm_x, kb * BK, m0, bar);
+          tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BK, n0, bar);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (leader only)
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = instr_desc_pair(BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      int acc = 0;
+      uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
+        if (!mbar_wait(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * kAccStride;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+          const uint64_t da = smem_desc_k_sw128(sa), db = smem_desc_k_sw128(sa + L::kABytes);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)   // 16 bf16 along K inside the swizzled row = 32 bytes = 2 descriptor units
+            umma_pair_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+          umma_commit_both(&empty[stage]);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        umma_commit_both(&tmem_full[acc]);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------------ epilogue (both CTAs)
+    constexpr int CC = sizeof(OutT) == 4 ? 32 : 64;  // columns per staged chunk: 128 bytes per row
+    constexpr int kChunks = (BN / 2) / CC;           // chunks per warp: a warp owns half of the tile's columns
+    const int q = warp & 3;                          // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;                // which half of the columns
+    float* bs = bias_s + (warp - 2) * (BN / 2);
+    uint8_t* sbuf = smem + L::kOutOffset + (warp - 2) * L::kOutBufBytes;
+    const uint32_t tmem_empty_leader0 = map_to_rank(smem_u32(&tmem_empty[0]), 0);
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_out) : "memory");
+    for (int tile = pair; tile < num_tiles; tile += n_pairs) {
+      const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;
+      const int n0 = (tile / m_tiles) * BN + half * (BN / 2);
+      __syncwarp();
+      for (int i = lane; i < BN / 2; i += 32)
+        bs[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
+      __syncwarp();
+      if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) break;
+      tc_fence_after();
+      const int row0 = m0 + q * 32;
+      const uint32_t taddr = tmem_base + acc * kAccStride + half * (BN / 2) + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < kChunks; ++c) {
+        uint32_t pk[32];  // this thread's row of the chunk, as stored: 32 floats or 64 bf16
+        if constexpr (sizeof(OutT) == 4) {
+          tmem_ld32(taddr + c * CC, pk);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float t = __uint_as_float(pk[j]) + bs[c * CC + j];
+            if (ACT == 1) t = gelu_tanh_fast(t);
+            if (ACT == 2) t = gelu_erf_f(t);
+            pk[j] = __float_as_uint(t);
+          }
+        } else {
+          uint32_t r0[32], r1[32];
+          tmem_ld32(taddr + c * CC, r0);
+          tmem_ld32(taddr + c * CC + 32, r1);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const uint32_t* src = j < 16 ? r0 : r1;
+            const int jj = (2 * j) & 31;
+            float t0 = __uint_as_float(src[jj]) + bs[c * CC + 2 * j];
+            float t1 = __uint_as_float(src[jj + 1]) + bs[c * CC + 2 * j + 1];
+            if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); }
+            if (ACT == 2) { t0 = gelu_erf_f(t0); t1 = gelu_erf_f(t1); }
+            __nv_bfloat162 b = __floats2bfloat162_rn(t0, t1);
+            pk[j] = *reinterpret_cast<uint32_t*>(&b);
+          }
+        }
+        if (c == kChunks - 1) {
+          // this warp has read all of its accumulator columns: tell the leader's MMA thread
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(tmem_empty_leader0 + acc * 8);
+        }
+        // the staging buffer is free once the bulk store issued from it has read it
+        if (lane == 0) bulk_wait_read_all();
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          // 128-byte swizzle: 16-byte chunk j of row r lives at chunk position j ^ (r % 8)
+          uint4* dst = reinterpret_cast<uint4*>(sbuf + lane * 128 + ((j ^ (lane & 7)) << 4));
+          *dst = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          if (row0 < M && n0 + c * CC < N) {
+            if (ACCUM) tma_reduce_add_2d(&tm_out, n0 + c * CC, row0, sbuf);
+            else tma_store_2d(&tm_out, n0 + c * CC, row0, sbuf);
+          }
+          bulk_commit();
+        }
+      }
+      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+    }
+    if (lane == 0) bulk_wait_all();
+    __syncwarp();
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, 0, kStatusTimeout);
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  cluster_sync();   // neither CTA's shared memory or tensor memory goes away while the other may still touch it
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// Tensor map of a row-major matrix [rows, cols] with leading dimension ld (elements of elem_bytes),
+// box = box_rows x (128 bytes of columns), 128-byte swizzle.
+bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows,
+              int elem_bytes) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * elem_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(tm, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+            const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM>
+cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& to, const void* bias, int M, int N,
+                   int K, int* status, cudaStream_t s) {
+  using L = PairLayout<BN, STAGES>;
+  auto kern = linear_pair_kernel<BN, STAGES, OutT, ACT, ACCUM>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
+  // pairs that can be resident at once (SMs pair up inside a GPC, so this can be below SMs / 2)
+  static int max_pairs = 0;
+  if (max_pairs == 0) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(sm_count() / 2 * 2);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = L::kDynamic;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
+      (void)cudaGetLastError();
+      n = sm_count() / 2;
+    }
+    max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
+  }
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  kern<<<2 * pairs, kThreads, L::kDynamic, s>>>(tx, tw, to, (const __nv_bfloat16*)bias, M, N, K, status);
+  return cudaGetLastError();
+}
+
+template <int BN, int STAGES>
+cudaError_t launch_bn(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& to, const void* bias, int M,
+                      int N, int K, int flags, int* status, cudaStream_t s) {
+  const int act = (flags & EPD_LINEAR_GELU_TANH) ? 1 : (flags & EPD_LINEAR_GELU_ERF) ? 2 : 0;
+  const bool accum = flags & EPD_LINEAR_ACCUMULATE;
+  const bool out_f32 = accum || (flags & EPD_LINEAR_OUT_F32);
+#define EPD_TC(OUT, A, C) return launch<BN, STAGES, OUT, A, C>(tx, tw, to, bias, M, N, K, status, s)
+  if (accum) {
+    if (act == 0) EPD_TC(float, 0, true);
+    if (act == 1) EPD_TC(float, 1, true);
+    EPD_TC(float, 2, true);
+  }
+  if (out_f32) {
+    if (act == 0) EPD_TC(float, 0, false);
+    if (act == 1) EPD_TC(float, 1, false);
+    EPD_TC(float, 2, false);
+  }
+  if (act == 0) EPD_TC(__nv_bfloat16, 0, false);
+  if (act == 1) EPD_TC(__nv_bfloat16, 1, false);
+  EPD_TC(__nv_bfloat16, 2, false);
+#undef EPD_TC
+}
+
+}  // namespace
+
+// 256 x 256 tiles on CTA pairs.  Same argument contract as linear_tc().
+cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
+                           int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, int* status, cudaStream_t s) {
+  const bool out_f32 = flags & (EPD_LINEAR_ACCUMULATE | EPD_LINEAR_OUT_F32);
+  constexpr int BN = 256;
+  CUtensorMap tx, tw, to;
+  if (!make_map(&tx, x, M, K, ldx, BM, 2) || !make_map(&tw, w, N, K, ldw, BN / 2, 2) ||
+      !make_map(&to, out, M, N, ldo, 32, out_f32 ? 4 : 2))
+    return cudaErrorInvalidValue;
+  return launch_bn<BN, 5>(tx, tw, to, bias, (int)M, (int)N, (int)K, flags, status, s);
+}
+
+}  // namespace epd
