@@ -162,6 +162,54 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ----------------------------------------------------------------------------- replicas (N > 1)
+
+def rank_env():
+    """(world size, rank, local rank) as torch.distributed.run exports them; (1, 0, 0) when run alone."""
+    return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def replica_seed(rank: int) -> int:
+    """Every replica encodes its own batch: same shapes, pixels drawn from a stream of its own."""
+    return rank
+
+
+def max_over_ranks(ms: float, device) -> float:
+    """The slowest rank's time (the job's time); a no-op without a process group."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank: int, world: int, steps: int, ms_total: float) -> float:
+    """Aggregate image-tokens/s of `world` independent replicas over the slowest rank's time."""
+    return world * tokens_per_rank * steps / (ms_total * 1e-3)
+
+
+def run_dist_selftest(args):
+    """CPU check of the N > 1 plumbing (gloo): per-rank seeds differ, the time is the max over ranks,
+    rank 0 alone prints."""
+    import torch
+    import torch.distributed as dist
+    world, rank, _ = rank_env()
+    dist.init_process_group("gloo")
+    cfg, grids = synth.WORKLOADS["cfg0_tiny_fp32"]
+    patches = synth.make_patches(cfg, grids, seed=replica_seed(rank))
+    digest = float(np.abs(patches).sum())
+    digests = [None] * world
+    dist.all_gather_object(digests, digest)
+    ms = max_over_ranks(10.0 * (rank + 1), torch.device("cpu"))
+    dist.barrier()
+    if rank == 0:
+        print(json.dumps({"selftest": "dist", "world": world, "ms_max": ms, "distinct_batches": len(set(digests)),
+                          "value": whole_job_value(synth.num_tokens(grids), world, 1, ms)}))
+    dist.destroy_process_group()
+
+
 # ----------------------------------------------------------------------------- CUDA path
 
 def run_cuda(args):
@@ -170,9 +218,7 @@ def run_cuda(args):
     import paper_2601_11590_b200 as epd
     from paper_2601_11590_b200 import build
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local_rank = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the Encode-stage library has no CPU path")
     torch.cuda.set_device(local_rank)
@@ -195,7 +241,7 @@ def run_cuda(args):
     enc = epd.Encoder(cfg, w, max_tokens=T, max_images=len(grids), max_grid=max(max(g[1], g[2]) for g in grids))
     del w
     # every rank encodes its own batch (same shapes, different pixels)
-    patches_np = synth.make_patches(cfg, grids, seed=rank)
+    patches_np = synth.make_patches(cfg, grids, seed=replica_seed(rank))
     host_patches = torch.zeros((T, ld), dtype=tdt).pin_memory()
     host_patches[:, :K] = torch.from_numpy(patches_np).to(tdt)
     dev_patches = host_patches.cuda()
@@ -217,10 +263,7 @@ def run_cuda(args):
             fn()
         e1.record(stream)
         barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return max_over_ranks(e0.elapsed_time(e1), "cuda")
 
     def step_device():
         enc.encode(dev_patches, grids, features=feats, stream=stream)
@@ -264,11 +307,11 @@ def run_cuda(args):
     peaks = load_peaks()
     flops = algorithmic_flops(cfg, grids)
     ms_step = ms_total / args.steps
-    value = world * T * args.steps / (ms_total * 1e-3)
-    e2e_value = world * T * args.steps / (ms_e2e * 1e-3)
+    value = whole_job_value(T, world, args.steps, ms_total)
+    e2e_value = whole_job_value(T, world, args.steps, ms_e2e)
     es = 2 if cfg.dtype == synth.DTYPE_BF16 else 4
 
-    # dominant kernel: the tcgen05 linear kernel (all linear launches of a step)
+    # dominant kernel: the tcgen05 linear kernels (all linear launches of a step)
     lin_classes = ["patch_embed", "qkv_linear", "out_linear", "fc1_linear", "fc2_linear", "projector"]
     lin_ms = sum(prof[c]["ms"] for c in lin_classes) / prof_steps
     lin_launches = sum(prof[c]["launches"] for c in lin_classes) // prof_steps
@@ -276,7 +319,7 @@ def run_cuda(args):
     peak_tf = peaks["bf16_tflops_sustained"]
     achieved_tf = flops["linear"] / (lin_ms * 1e-3) / 1e12 if lin_ms > 0 else 0.0
     roofline = {
-        "bound": "tensor", "kernel": "linear_tc_kernel (all linear layers of a step)",
+        "bound": "tensor", "kernel": "linear_pair_kernel / linear_tc_kernel (all linear layers of a step)",
         "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
         "peak_source": f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
         "flops_per_launch": flops["linear"] / max(lin_launches, 1),
@@ -331,7 +374,11 @@ def main():
     ap.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(synth.WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dist-selftest", action="store_true", help="CPU/gloo check of the multi-rank plumbing")
     args = ap.parse_args()
+    if args.dist_selftest:
+        run_dist_selftest(args)
+        return
     if args.impl == "reference":
         if args.steps == 20:
             args.steps = 3

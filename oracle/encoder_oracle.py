@@ -193,6 +193,40 @@ def block(cfg, lw: Dict, x: np.ndarray, bk: Dict) -> np.ndarray:
     return mlp_sublayer(cfg, lw, attention_sublayer(cfg, lw, _f64(x), bk))
 
 
+def block_rows(cfg, lw: Dict, x: np.ndarray, bk: Dict, rows: Sequence[int]) -> np.ndarray:
+    """Rows `rows` of block(cfg, lw, x, bk): the same definition (O2-O7) evaluated only for the chosen
+    query tokens.  Keys and values are still formed for every token of the images those rows belong
+    to; everything after attention is row-wise.  Lets a large batch be checked on sampled rows."""
+    x = _f64(x)
+    rows = np.asarray(rows, dtype=np.int64)
+    h, nH, dh = cfg.hidden, cfg.heads, cfg.head_dim
+    cu = bk["cu_seqlens"]
+    out = np.empty((len(rows), h), dtype=np.float64)
+    seg_of = np.searchsorted(cu, rows, side="right") - 1
+    for i in np.unique(seg_of):
+        a, b = int(cu[i]), int(cu[i + 1])
+        sel = np.nonzero(seg_of == i)[0]
+        local = rows[sel] - a
+        an = rmsnorm(x[a:b], _f64(lw["norm1_w"]), cfg.eps)
+        qkv = linear(an, _f64(lw["qkv_w"]), _f64(lw["qkv_b"]))
+        q = qkv[:, 0:h].reshape(b - a, nH, dh)
+        k = qkv[:, h:2 * h].reshape(b - a, nH, dh)
+        v = qkv[:, 2 * h:3 * h].reshape(b - a, nH, dh)
+        if cfg.rope_theta > 0:
+            q = rope_2d(q, bk["pos_row"][a:b], bk["pos_col"][a:b], cfg.rope_theta)
+            k = rope_2d(k, bk["pos_row"][a:b], bk["pos_col"][a:b], cfg.rope_theta)
+        o = np.empty((len(local), nH, dh), dtype=np.float64)
+        for hd in range(nH):
+            sc = (q[local, hd, :] @ k[:, hd, :].T) / np.sqrt(float(dh))
+            sc = sc - sc.max(axis=1, keepdims=True)
+            p = np.exp(sc)
+            p = p / p.sum(axis=1, keepdims=True)
+            o[:, hd, :] = p @ v[:, hd, :]
+        x1 = x[rows[sel]] + linear(o.reshape(len(local), h), _f64(lw["out_w"]), _f64(lw["out_b"]))
+        out[sel] = mlp_sublayer(cfg, lw, x1)
+    return out
+
+
 def head(cfg, weights: Dict, x: np.ndarray, bk: Dict) -> np.ndarray:
     """Steps O8-O10 on the residual stream after the last block."""
     y = rmsnorm(_f64(x), _f64(weights["final_norm_w"]), cfg.eps) if cfg.final_norm else _f64(x)

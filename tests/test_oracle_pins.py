@@ -397,3 +397,17 @@ def test_synthetic_recipe():
     assert synth.num_tokens(synth.WORKLOADS["cfg1_vit06b_b8_448"][1]) == 6272
     assert synth.num_tokens(synth.WORKLOADS["cfg3_vit06b_long"][1]) == 16384 + 6272
     assert synth.num_tokens(synth.WORKLOADS["cfg4_vit6b_b16_448"][1]) == 16384
+
+
+def test_block_rows_is_block_restricted_to_rows():
+    """The sampled-row form used for large batches equals the full block on those rows."""
+    cfg = synth.tiny_variant(head_dim=8, heads=2, layers=1, mlp=24, patch=2)
+    grids = [(1, 4, 6), (2, 2, 4), (1, 6, 2)]
+    w = synth.make_weights(cfg, seed=11)
+    bk = O.bookkeeping(grids)
+    T = int(bk["cu_seqlens"][-1])
+    x = synth.normal(12, "x", (T, cfg.hidden), 1.0, 0.0, synth.DTYPE_FP32).astype(np.float64)
+    full = O.block(cfg, w["layers"][0], x, bk)
+    rows = [0, 5, 23, 24, 30, 39, 40, T - 1]
+    got = O.block_rows(cfg, w["layers"][0], x, bk, rows)
+    assert np.allclose(got, full[rows], rtol=0, atol=1e-12)
