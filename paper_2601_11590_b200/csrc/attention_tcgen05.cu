@@ -16,8 +16,10 @@
 // waits and commits around a product cost more issue time than the product itself, so one thread
 // cannot keep up).  Score tiles run ahead of the P V products by as much as the S_w buffers and the
 // K ring allow, so a warpgroup does not wait for the tensor pipe in steady state and the exponential
-// unit stays busy.  That unit delivers 16 results per clock per SM, which bounds the softmax, so one
-// exponential in kFmaExpEvery is evaluated on the FMA pipe instead (cubic for 2^fraction).
+// unit stays busy.  That unit delivers 16 results per clock per SM; evaluating part of the exponentials
+// on the FMA pipe instead (cubic for 2^fraction, kFmaExpEvery) is implemented but off: measured on
+// B200 the softmax warps are bound by instruction issue as much as by that unit, and the extra FMAs
+// cost more than they save (16k-token segment: 660 TFLOP/s without, 622 with one in four, 517 with one in two).
 // The running max only advances (and O_w is rescaled in TMEM) when it grows by more than 2^8; until
 // then the stale max serves P, the row sum and O_w alike, which leaves the result unchanged.  At the
 // end of an item the two partial results are merged:
@@ -48,7 +50,7 @@ constexpr int BQ = 128;          // query rows per work item
 constexpr int kThreads = 384;    // warps 0..3: loaders and MMA issuers; warps 4..11: two softmax warpgroups
 constexpr int kMaxSegs = 128;    // segments one launch can describe
 constexpr long long kWaitCycles = 4000000000LL;
-constexpr int kFmaExpEvery = 4;            // 1 in 4 exponentials is computed with FMAs (must be even)
+constexpr int kFmaExpEvery = 0;            // 1 in this many exponentials is computed with FMAs (even; 0 = none)
 constexpr float kRescaleThreshold = 8.0f;  // log2 of the largest P value tolerated before rescaling
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -585,7 +587,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           for (int i = 0; i < BKV / 2; ++i) {
             // one exponential in kFmaExpEvery goes to the FMA pipe
             const float p0 = ex2(__uint_as_float(s[2 * i]) + neg_m);
-            const float p1 = (i % (kFmaExpEvery / 2) == kFmaExpEvery / 2 - 1)
+            const float p1 = (kFmaExpEvery > 0 && i % (kFmaExpEvery > 0 ? kFmaExpEvery / 2 : 1) == kFmaExpEvery / 2 - 1)
                                  ? ex2_fma(__uint_as_float(s[2 * i + 1]) + neg_m)
                                  : ex2(__uint_as_float(s[2 * i + 1]) + neg_m);
             sum[i & 3] += p0 + p1;
