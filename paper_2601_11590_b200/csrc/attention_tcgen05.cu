@@ -338,6 +338,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
                     __nv_bfloat16* __restrict__ out, int T, int heads, int dh, int* __restrict__ status) {
   using P = Plan<DHP>;
   constexpr int BKV = P::BKV;
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + P::kBar);
@@ -377,6 +378,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();   // nothing above touches global memory
 
   if (warp == 0) {
     // ---------------------------------------------------------------- TMA producer of Q and K
@@ -759,8 +761,8 @@ cudaError_t launch(const Maps& maps, const SegList& segs, int n_items, void* out
     configured = true;
   }
   const int grid = n_items < sm_count() ? n_items : sm_count();
-  kern<<<grid, kThreads, P::kDynamic, s>>>(maps, segs, n_items, (__nv_bfloat16*)out, T, heads, dh, status);
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(grid), dim3(kThreads), P::kDynamic, s, maps, segs, n_items, (__nv_bfloat16*)out, T, heads, dh,
+                    status);
 }
 
 bool attention_tc_supported(const void* q, const void* k, const void* v, const void* out, int64_t T, int heads,

@@ -33,6 +33,32 @@ __device__ __forceinline__ float gelu_tanh_f(float x) {
 }
 __device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f)); }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// The kernels of one encode run back to back on one stream.  Launched with the programmatic-stream-
+// serialization attribute, a kernel's CTAs may become resident as soon as every CTA of the previous
+// kernel has started (pdl_launch_dependents, called first thing) and SM resources are free; they run
+// their set-up (barrier init, tensor-memory allocation, descriptor prefetch) and then block in
+// pdl_wait() until the previous kernel has completed and its writes are visible.  No global memory is
+// read or written before pdl_wait().  A kernel launched the ordinary way ignores both instructions.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                              Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 // ---- plain-FMA kernels (kernels_fma.cu) -----------------------------------------------------
 cudaError_t linear_fma(int dtype, const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias,
                        void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, cudaStream_t s);

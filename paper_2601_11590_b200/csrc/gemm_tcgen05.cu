@@ -192,6 +192,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
   constexpr int kAccStride = BN <= 128 ? 128 : 256;  // TMEM columns between the two accumulators
   constexpr int kTmemCols = 2 * kAccStride;
 
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
@@ -222,6 +223,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_slot;
+  pdl_wait();   // nothing above touches global memory
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -435,8 +437,7 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
   }
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
   const int grid = tiles < sm_count() ? tiles : sm_count();
-  kern<<<grid, kThreads, L::kDynamic, s>>>(tx, tw, to, (const __nv_bfloat16*)bias, M, N, K, status);
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(grid), dim3(kThreads), L::kDynamic, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K, status);
 }
 
 template <int BN, int STAGES>

@@ -208,6 +208,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   constexpr int kAccStride = BN;                 // TMEM columns between the two accumulators
   constexpr int kTmemCols = 2 * kAccStride;
 
+  pdl_launch_dependents();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);   // used in the leader only
@@ -241,6 +242,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   cluster_sync();                                 // both CTAs' barriers exist before either signals the other
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_slot;
+  pdl_wait();   // nothing above touches global memory
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -476,8 +478,8 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
     max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
   }
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  kern<<<2 * pairs, kThreads, L::kDynamic, s>>>(tx, tw, to, (const __nv_bfloat16*)bias, M, N, K, status);
-  return cudaGetLastError();
+  return launch_pdl(kern, dim3(2 * pairs), dim3(kThreads), L::kDynamic, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K,
+                    status);
 }
 
 template <int BN, int STAGES>

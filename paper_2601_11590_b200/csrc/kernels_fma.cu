@@ -161,6 +161,8 @@ template <typename T, int NV>
 __global__ void __launch_bounds__(256)
 rmsnorm_reg_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ out,
                    const int32_t* __restrict__ dst_row, int64_t rows, int hidden, float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -194,6 +196,8 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ out,
                const int32_t* __restrict__ dst_row, int64_t rows, int hidden, float eps) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -217,14 +221,13 @@ static cudaError_t rmsnorm_t(const float* x, const T* gain, T* out, const int32_
                       ((uintptr_t)gain & (sizeof(T) == 4 ? 15 : 7)) == 0;
   const int nv = (hidden / 4 + 31) / 32;
   if (vec_ok && nv <= 4)
-    rmsnorm_reg_kernel<T, 4><<<blocks, warps * 32, 0, s>>>(x, gain, out, dst_row, rows, hidden, eps);
+    return launch_pdl(rmsnorm_reg_kernel<T, 4>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
   else if (vec_ok && nv <= 10)
-    rmsnorm_reg_kernel<T, 10><<<blocks, warps * 32, 0, s>>>(x, gain, out, dst_row, rows, hidden, eps);
+    return launch_pdl(rmsnorm_reg_kernel<T, 10>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
   else if (vec_ok && nv <= 26)
-    rmsnorm_reg_kernel<T, 26><<<blocks, warps * 32, 0, s>>>(x, gain, out, dst_row, rows, hidden, eps);
+    return launch_pdl(rmsnorm_reg_kernel<T, 26>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
   else
-    rmsnorm_kernel<T><<<blocks, warps * 32, 0, s>>>(x, gain, out, dst_row, rows, hidden, eps);
-  return cudaGetLastError();
+    return launch_pdl(rmsnorm_kernel<T>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
 }
 
 cudaError_t rmsnorm(int dtype, const void* x, const void* gain, void* out, const int32_t* dst_row, int64_t T,
@@ -341,6 +344,8 @@ rope_split_vec_kernel(const T* __restrict__ qkv, const int32_t* __restrict__ pos
                       const int32_t* __restrict__ pos_col, const float2* __restrict__ table, int table_rows,
                       T* __restrict__ q, T* __restrict__ k, T* __restrict__ v, int64_t Tn, int heads, int dh, int dhp,
                       int tok_per_block, float theta, float q_scale) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr int VEC = 16 / (int)sizeof(T);
   using P2 = typename Pair<T>::type;
   extern __shared__ __align__(16) uint8_t rope_smem[];
@@ -433,8 +438,8 @@ static cudaError_t rope_split_t(const T* qkv, const int32_t* pos_row, const int3
       if (e != cudaSuccess) return e;
       configured = 100 * 1024;
     }
-    kern<<<(unsigned)((Tn + tok - 1) / tok), 256, smem, s>>>(qkv, pos_row, pos_col, table, table_rows, q, k, v, Tn,
-                                                            heads, dh, dhp, tok, theta, q_scale);
+    return launch_pdl(kern, dim3((unsigned)((Tn + tok - 1) / tok)), dim3(256), smem, s, qkv, pos_row, pos_col, table,
+                      table_rows, q, k, v, Tn, heads, dh, dhp, tok, theta, q_scale);
   } else {
     rope_split_kernel<T><<<(unsigned)Tn, 128, 0, s>>>(qkv, pos_row, pos_col, table, table_rows, q, k, v, Tn, heads, dh,
                                                       dhp, theta, q_scale);
