@@ -158,7 +158,7 @@ __device__ __forceinline__ float4 load_gain4(const T* gain, int i) {
 }
 
 template <typename T, int NV>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, NV <= 9 ? 5 : 1)
 rmsnorm_reg_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ out,
                    const int32_t* __restrict__ dst_row, int64_t rows, int hidden, float eps) {
   pdl_launch_dependents();
@@ -222,8 +222,10 @@ static cudaError_t rmsnorm_t(const float* x, const T* gain, T* out, const int32_
   const int nv = (hidden / 4 + 31) / 32;
   if (vec_ok && nv <= 4)
     return launch_pdl(rmsnorm_reg_kernel<T, 4>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
-  else if (vec_ok && nv <= 10)
-    return launch_pdl(rmsnorm_reg_kernel<T, 10>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
+  else if (vec_ok && nv <= 9)   // hidden <= 1152: 48 registers, five blocks per SM
+    return launch_pdl(rmsnorm_reg_kernel<T, 9>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
+  else if (vec_ok && nv <= 13)
+    return launch_pdl(rmsnorm_reg_kernel<T, 13>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
   else if (vec_ok && nv <= 26)
     return launch_pdl(rmsnorm_reg_kernel<T, 26>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
   else
@@ -339,7 +341,7 @@ template <> struct Pair<__nv_bfloat16> {
 };
 
 template <typename T>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(512)
 rope_split_vec_kernel(const T* __restrict__ qkv, const int32_t* __restrict__ pos_row,
                       const int32_t* __restrict__ pos_col, const float2* __restrict__ table, int table_rows,
                       T* __restrict__ q, T* __restrict__ k, T* __restrict__ v, int64_t Tn, int heads, int dh, int dhp,
@@ -402,19 +404,22 @@ rope_split_vec_kernel(const T* __restrict__ qkv, const int32_t* __restrict__ pos
   }
   __syncthreads();
 
-  // copy out: 16-byte pieces, (tensor, head) outermost, then token, then piece inside the padded row
+  // copy out: a warp takes whole (tensor, head) pairs; the ntok padded rows of a pair are contiguous in
+  // global memory, so consecutive lanes write consecutive 16-byte pieces
   const int vec_per_row = dhp / VEC, data_vecs = dh / VEC;
   const int per_pair = ntok * vec_per_row;
-  const int total = 3 * heads * per_pair;
-  for (int u = threadIdx.x; u < total; u += blockDim.x) {
-    const int pair = u / per_pair, r = u - pair * per_pair;
-    const int t = r / vec_per_row, ov = r - t * vec_per_row;
+  const unsigned inv_vpr = (65536u + vec_per_row - 1) / vec_per_row;   // r / vec_per_row for r < 4096
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  for (int pair = warp; pair < 3 * heads; pair += nwarps) {
     const int which = pair / heads, hd = pair - which * heads;
-    uint4 pk = make_uint4(0u, 0u, 0u, 0u);
-    if (ov < data_vecs)
-      pk = *reinterpret_cast<const uint4*>(s_in + t * row_elems + which * h + hd * dh + ov * VEC);
-    T* dst = (which == 0 ? q : which == 1 ? k : v) + ((int64_t)hd * Tn + j0 + t) * dhp + ov * VEC;
-    *reinterpret_cast<uint4*>(dst) = pk;
+    const T* sbase = s_in + which * h + hd * dh;
+    T* gbase = (which == 0 ? q : which == 1 ? k : v) + ((int64_t)hd * Tn + j0) * dhp;
+    for (int r = lane; r < per_pair; r += 32) {
+      const int t = (int)((r * inv_vpr) >> 16), ov = r - t * vec_per_row;
+      uint4 pk = make_uint4(0u, 0u, 0u, 0u);
+      if (ov < data_vecs) pk = *reinterpret_cast<const uint4*>(sbase + t * row_elems + ov * VEC);
+      *reinterpret_cast<uint4*>(gbase + r * VEC) = pk;
+    }
   }
 }
 
@@ -427,10 +432,15 @@ static cudaError_t rope_split_t(const T* qkv, const int32_t* pos_row, const int3
   const size_t row_bytes = (size_t)3 * heads * dh * sizeof(T);
   const bool aligned = ((((uintptr_t)qkv | (uintptr_t)q | (uintptr_t)k | (uintptr_t)v)) & 15) == 0;
   if (aligned && dh % 8 == 0 && row_bytes + 2 * (dh / 4) * sizeof(float2) <= 96 * 1024) {
-    // a few tokens per block: about 32 KB of rows, so several blocks share an SM
-    int tok = (int)(32768 / row_bytes);
+    // 8 tokens per block (fewer for very wide rows); as many threads as there are rotation units
+    // (head, half, frequency pair), so that the rotation takes whole passes
+    int tok = (int)(65536 / row_bytes);
     tok = tok < 1 ? 1 : tok > 8 ? 8 : tok;
     const size_t smem = tok * (row_bytes + 2 * (dh / 4) * sizeof(float2));
+    const int units = heads * 2 * (dh / 8);
+    const int passes = (units + 511) / 512;
+    int threads = ((units + passes - 1) / passes + 31) / 32 * 32;
+    threads = threads < 128 ? 128 : threads;
     auto kern = rope_split_vec_kernel<T>;
     static size_t configured = 48 * 1024;
     if (smem > configured) {
@@ -438,7 +448,7 @@ static cudaError_t rope_split_t(const T* qkv, const int32_t* pos_row, const int3
       if (e != cudaSuccess) return e;
       configured = 100 * 1024;
     }
-    return launch_pdl(kern, dim3((unsigned)((Tn + tok - 1) / tok)), dim3(256), smem, s, qkv, pos_row, pos_col, table,
+    return launch_pdl(kern, dim3((unsigned)((Tn + tok - 1) / tok)), dim3(threads), smem, s, qkv, pos_row, pos_col, table,
                       table_rows, q, k, v, Tn, heads, dh, dhp, tok, theta, q_scale);
   } else {
     rope_split_kernel<T><<<(unsigned)Tn, 128, 0, s>>>(qkv, pos_row, pos_col, table, table_rows, q, k, v, Tn, heads, dh,
