@@ -228,8 +228,9 @@ int epd_op_rmsnorm(int32_t dtype, const void* x, const void* gain, void* out, co
                    int64_t T, int32_t hidden, float eps, void* stream);
 
 /* Rotary embedding + head split.  qkv [T, 3*hidden] per dtype -> q, k, v each
- * [heads, T, head_dim_padded] per dtype (head_dim_padded = epd_padded_head_dim(head_dim), pad
- * columns zero).  q and k are rotated by (pos_row, pos_col) (device int32 [T]); q is also
+ * [heads, T, head_dim_padded] per dtype (head_dim_padded = epd_padded_head_dim(head_dim); pad
+ * columns zero, except that column head_dim of v is 1 when there is padding: the attention
+ * step's P.V product then also delivers the softmax row sums).  q and k are rotated by (pos_row, pos_col) (device int32 [T]); q is also
  * multiplied by q_scale.  theta <= 0 skips the rotation. */
 int epd_op_rope_split(int32_t dtype, const void* qkv, const int32_t* pos_row, const int32_t* pos_col,
                       void* q, void* k, void* v, int64_t T, int32_t heads, int32_t head_dim, float theta,
@@ -239,8 +240,9 @@ int32_t epd_padded_head_dim(int32_t head_dim);
 
 enum { EPD_ATTENTION_FORCE_FMA = 1 /* use the plain-FMA kernel even where the tensor-core kernel applies */ };
 
-/* Block-diagonal bidirectional attention.  q, k, v [heads, T, head_dim_padded] per dtype with q
- * already multiplied by log2(e)/sqrt(head_dim); cu_seqlens device int32 [n_seg+1] and the same
+/* Block-diagonal bidirectional attention.  q, k, v [heads, T, head_dim_padded] per dtype as written
+ * by epd_op_rope_split(): q already multiplied by log2(e)/sqrt(head_dim), pad columns zero except
+ * v[.., head_dim] = 1 when head_dim_padded > head_dim (required by the tensor-core kernel); cu_seqlens device int32 [n_seg+1] and the same
  * values in HOST memory (host_cu_seqlens) for the launch geometry.  out [T, heads*head_dim] per
  * dtype: for each segment and head softmax over all keys of the segment.  In bf16 with head_dim 64,
  * 72 or 128 (a multiple of 8 whose padded width is 64, 80 or 128) the tcgen05 kernel runs; other

@@ -220,6 +220,11 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t* r) 
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -332,7 +337,10 @@ __device__ __forceinline__ Item decode_item(const SegList& segs, int heads, int 
   return it;
 }
 
-template <int DHP>
+// ONES: head_dim < DHP and column head_dim of every V row holds 1.0, so column head_dim of O_w is the
+// row sum of P_w (summed by the tensor core from the same bf16 values as the numerator) and the
+// softmax threads need not add it up.
+template <int DHP, bool ONES>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ SegList segs, int n_items,
                     __nv_bfloat16* __restrict__ out, int T, int heads, int dh, int* __restrict__ status) {
@@ -562,7 +570,8 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         for (int i = 0; i < 8; ++i) mx[i] = -INFINITY;
         if (kv_valid == BKV) {
 #pragma unroll
-          for (int i = 0; i < BKV; ++i) mx[i & 7] = fmaxf(mx[i & 7], __uint_as_float(s[i]));
+          for (int i = 0; i < BKV / 2; ++i)
+            mx[i & 7] = max3(mx[i & 7], __uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
         } else {
 #pragma unroll
           for (int i = 0; i < BKV; ++i)
@@ -592,7 +601,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
             const float p1 = (kFmaExpEvery > 0 && i % (kFmaExpEvery > 0 ? kFmaExpEvery / 2 : 1) == kFmaExpEvery / 2 - 1)
                                  ? ex2_fma(__uint_as_float(s[2 * i + 1]) + neg_m)
                                  : ex2(__uint_as_float(s[2 * i + 1]) + neg_m);
-            sum[i & 3] += p0 + p1;
+            if (!ONES) sum[i & 3] += p0 + p1;
             __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
             s[i] = *reinterpret_cast<uint32_t*>(&b);
           }
@@ -601,12 +610,12 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           for (int i = 0; i < BKV / 2; ++i) {
             const float p0 = 2 * i < kv_valid ? ex2(__uint_as_float(s[2 * i]) + neg_m) : 0.0f;
             const float p1 = 2 * i + 1 < kv_valid ? ex2(__uint_as_float(s[2 * i + 1]) + neg_m) : 0.0f;
-            sum[i & 3] += p0 + p1;
+            if (!ONES) sum[i & 3] += p0 + p1;
             __nv_bfloat162 b = __floats2bfloat162_rn(p0, p1);
             s[i] = *reinterpret_cast<uint32_t*>(&b);
           }
         }
-        l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+        if (!ONES) l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
         // P_w and O_w are free once this warpgroup's previous P V has completed
         if (tc > 0 && !mbar_wait(&p_free[w], (tc - 1) & 1, abort_flag)) { ok = false; break; }
         ++tc;
@@ -647,7 +656,21 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
       if (!mbar_wait(o_final, n & 1, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const bool has1 = it.n_kv > 1;
-      const float2 ml0 = ml[r], ml1 = ml[BQ + r];
+      float2 ml0 = ml[r], ml1 = ml[BQ + r];
+      if (ONES) {
+        // the row sums sit in column head_dim of the accumulators
+        uint32_t t0[8], t1[8];
+        tmem_ld8(tmem_base + P::kO0 + lane_off + (dh & ~7), t0);
+        if (has1) tmem_ld8(tmem_base + P::kO1 + lane_off + (dh & ~7), t1);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (i == (dh & 7)) {
+            ml0.y = __uint_as_float(t0[i]);
+            ml1.y = has1 ? __uint_as_float(t1[i]) : 0.0f;
+          }
+        }
+      }
       const float mm = has1 ? fmaxf(ml0.x, ml1.x) : ml0.x;
       const float a0 = ex2(ml0.x - mm), a1 = has1 ? ex2(ml1.x - mm) : 0.0f;
       const float inv = 1.0f / (a0 * ml0.y + a1 * ml1.y);
@@ -749,11 +772,11 @@ int sm_count() {
   return n;
 }
 
-template <int DHP>
+template <int DHP, bool ONES>
 cudaError_t launch(const Maps& maps, const SegList& segs, int n_items, void* out, int T, int heads, int dh,
                    int* status, cudaStream_t s) {
   using P = Plan<DHP>;
-  auto kern = attention_tc_kernel<DHP>;
+  auto kern = attention_tc_kernel<DHP, ONES>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P::kDynamic);
@@ -810,9 +833,13 @@ cudaError_t attention_tc(const void* q, const void* k, const void* v, const int3
     for (int i = segs.n; i < kMaxSegs; ++i) segs.beg[i] = segs.len[i] = 0;
     cudaError_t e;
     switch (dhp) {
-      case 64: e = launch<64>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s); break;
-      case 80: e = launch<80>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s); break;
-      case 128: e = launch<128>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s); break;
+#define EPD_ATT(D)                                                                                          \
+  e = head_dim < D ? launch<D, true>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s)          \
+                   : launch<D, false>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s)
+      case 64: EPD_ATT(64); break;
+      case 80: EPD_ATT(80); break;
+      case 128: EPD_ATT(128); break;
+#undef EPD_ATT
       default: return cudaErrorInvalidValue;
     }
     if (e != cudaSuccess) return e;

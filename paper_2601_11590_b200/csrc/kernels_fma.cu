@@ -315,7 +315,7 @@ rope_split_kernel(const T* __restrict__ qkv, const int32_t* __restrict__ pos_row
     if (d < dh) {
       v[o] = row[2 * h + hd * dh + d];
     } else {
-      v[o] = from_float<T>(0.0f);
+      v[o] = from_float<T>(d == dh ? 1.0f : 0.0f);   // column head_dim of v is 1: P V then also yields the row sums
       q[o] = from_float<T>(0.0f);
       k[o] = from_float<T>(0.0f);
     }
@@ -418,6 +418,8 @@ rope_split_vec_kernel(const T* __restrict__ qkv, const int32_t* __restrict__ pos
       const int t = (int)((r * inv_vpr) >> 16), ov = r - t * vec_per_row;
       uint4 pk = make_uint4(0u, 0u, 0u, 0u);
       if (ov < data_vecs) pk = *reinterpret_cast<const uint4*>(sbase + t * row_elems + ov * VEC);
+      // column head_dim of v is 1 (the rest of the padding 0): P V then also yields the row sums
+      else if (which == 2 && ov == data_vecs) pk.x = sizeof(T) == 4 ? 0x3F800000u : 0x00003F80u;
       *reinterpret_cast<uint4*>(gbase + r * VEC) = pk;
     }
   }

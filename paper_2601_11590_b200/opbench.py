@@ -113,6 +113,8 @@ def main():
         q, k, v = (torch.zeros((args.heads, T, dhp), dtype=bf, device="cuda") for _ in range(3))
         for t in (q, k, v):
             t[:, :, :args.dh] = rnd(args.heads, T, args.dh, std=0.5)
+        if dhp > args.dh:
+            v[:, :, args.dh] = 1.0
         lib = epd.load_library()
         out = torch.empty((T, args.heads * args.dh), dtype=bf, device="cuda")
         hcu, hp = epd._i32_array(cu)

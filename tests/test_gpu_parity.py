@@ -155,7 +155,10 @@ def test_rope_split(dtype, heads, dh):
     for got, ref in ((q, qr), (k, kr), (v, vr)):
         g = to_np(got)
         assert rel_err(g[:, :, :dh].transpose(1, 0, 2), ref) <= tol
-        assert np.all(g[:, :, dh:] == 0.0)
+        if got is v and dhp > dh:   # v's first padding column is 1 (it makes P V deliver the row sums)
+            assert np.all(g[:, :, dh] == 1.0) and np.all(g[:, :, dh + 1:] == 0.0)
+        else:
+            assert np.all(g[:, :, dh:] == 0.0)
     assert np.array_equal(to_np(v)[:, :, :dh].transpose(1, 0, 2), vr)  # v is a pure copy
 
 
@@ -173,12 +176,14 @@ def _attention_case(dtype, heads, dh, seglens, seed, logit_scale=1.0, flags=0):
     if dtype == epd.DTYPE_BF16:
         q_scaled = synth.round_to_bf16(q_scaled)
 
-    def pad(a):
+    def pad(a, ones_column=False):
         out = np.zeros((heads, T, dhp), np.float32)
         out[:, :, :dh] = a
+        if ones_column and dhp > dh:
+            out[:, :, dh] = 1.0
         return dev(out, dtype)
 
-    out = epd.op_attention(dtype, pad(q_scaled), pad(k), pad(v), torch.from_numpy(cu).cuda(), cu, dh, flags)
+    out = epd.op_attention(dtype, pad(q_scaled), pad(k), pad(v, True), torch.from_numpy(cu).cuda(), cu, dh, flags)
     q_eff = q_scaled.astype(np.float64) / qs
     ref = O.attention_block_diagonal(q_eff.transpose(1, 0, 2), k.astype(np.float64).transpose(1, 0, 2),
                                      v.astype(np.float64).transpose(1, 0, 2), cu).reshape(T, heads * dh)
