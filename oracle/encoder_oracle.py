@@ -12,6 +12,8 @@ formulae, so the encoder evaluated here is the standard pre-norm ViT the benchma
 configurations name, written out step by step in float64 with no blocking, fusion or
 intermediate rounding:
 
+  P0  (optional front end) raw uint8 frames -> patch vectors: per-channel normalisation and
+      patch extraction, element order (channel, temporal, y, x)
   O0  packing: image i has grid (t, h, w); its tokens are raster-ordered (frame, row, col)
       and occupy rows cu[i]..cu[i+1] of every activation matrix; every frame reuses the
       image's (row, col) positions.
@@ -85,6 +87,32 @@ def bookkeeping(grid_thw: Sequence[Sequence[int]], merge: int = 2) -> Dict[str, 
         "pos_col": cat(pos_col).astype(np.int32),
         "merge_idx": cat(idx, merge * merge).astype(np.int32).reshape(-1, merge * merge),
     }
+
+
+# ----------------------------------------------------------------------------- pixels -> patch vectors
+
+def patchify(frames: Sequence[np.ndarray], grid_thw: Sequence[Sequence[int]], patch: int, temporal_patch: int,
+             mean: Sequence[float], std: Sequence[float]) -> np.ndarray:
+    """The step in front of the stage: raw frames -> the packed patch matrix [T, C*Tp*P*P] that O1 consumes.
+
+    frames[i] is item i as uint8 [t*Tp, C, h*P, w*P] (frame, channel, y, x).  Pixel value v of channel c
+    becomes (v/255 - mean[c]) / std[c]; token (f, r, c) of the item gathers frames f*Tp .. f*Tp+Tp-1,
+    rows r*P .. r*P+P-1, columns c*P .. c*P+P-1 in element order (channel, temporal, y, x).
+    Resizing an image to a multiple of the patch size is preprocessing and happens before this.
+    """
+    P, Tp = int(patch), int(temporal_patch)
+    mean = np.asarray(mean, dtype=np.float64)
+    std = np.asarray(std, dtype=np.float64)
+    rows = []
+    for fr, (t, h, w) in zip(frames, grid_thw):
+        fr = np.asarray(fr)
+        C = fr.shape[1]
+        assert fr.shape == (t * Tp, C, h * P, w * P), (fr.shape, (t, h, w))
+        x = (fr.astype(np.float64) / 255.0 - mean[None, :, None, None]) / std[None, :, None, None]
+        x = x.reshape(t, Tp, C, h, P, w, P)              # f, tp, c, r, y, col, xx
+        x = x.transpose(0, 3, 5, 2, 1, 4, 6)             # f, r, col, c, tp, y, xx
+        rows.append(x.reshape(t * h * w, C * Tp * P * P))
+    return np.concatenate(rows, axis=0) if rows else np.zeros((0, 0))
 
 
 # ----------------------------------------------------------------------------- elementwise pieces

@@ -183,6 +183,20 @@ def make_patches(cfg: EncoderConfig, grid_thw: Sequence[Sequence[int]], seed: in
     return normal(seed, tensor_id, (num_tokens(grid_thw), cfg.patch_dim), 1.0, 0.0, cfg.dtype)
 
 
+PIXEL_MEAN = (0.5, 0.5, 0.5)
+PIXEL_STD = (0.5, 0.5, 0.5)
+
+
+def make_frames(cfg: EncoderConfig, grid_thw: Sequence[Sequence[int]], seed: int = 0) -> List[np.ndarray]:
+    """Raw frames of every item: uint8 [t*Tp, C, h*P, w*P], pixel values uniform over 0..255."""
+    out = []
+    for i, (t, h, w) in enumerate(grid_thw):
+        g = generator(seed, f"frames{i}")
+        out.append(g.integers(0, 256, size=(t * cfg.temporal_patch, cfg.in_channels, h * cfg.patch, w * cfg.patch),
+                              dtype=np.uint8))
+    return out
+
+
 # ----------------------------------------------------------------------------- workloads
 
 def grid_batch_fixed(n_images: int, height: int, width: int, patch: int, frames_t: int = 1

@@ -411,3 +411,46 @@ def test_block_rows_is_block_restricted_to_rows():
     rows = [0, 5, 23, 24, 30, 39, 40, T - 1]
     got = O.block_rows(cfg, w["layers"][0], x, bk, rows)
     assert np.allclose(got, full[rows], rtol=0, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- pixels -> patches
+
+def test_patchify_matches_brute_force_loops():
+    cfg = synth.tiny_variant(patch=2, temporal_patch=2)
+    grids = [(1, 2, 4), (2, 4, 2)]
+    frames = synth.make_frames(cfg, grids, seed=3)
+    mean, std = (0.4, 0.5, 0.6), (0.2, 0.25, 0.3)
+    got = O.patchify(frames, grids, cfg.patch, cfg.temporal_patch, mean, std)
+    P, Tp, C = cfg.patch, cfg.temporal_patch, cfg.in_channels
+    want = []
+    for fr, (t, h, w) in zip(frames, grids):
+        for f in range(t):
+            for r in range(h):
+                for c in range(w):
+                    vec = []
+                    for ch in range(C):
+                        for tp in range(Tp):
+                            for y in range(P):
+                                for x in range(P):
+                                    v = float(fr[f * Tp + tp, ch, r * P + y, c * P + x])
+                                    vec.append((v / 255.0 - mean[ch]) / std[ch])
+                    want.append(vec)
+    assert got.shape == (synth.num_tokens(grids), cfg.patch_dim)
+    assert np.allclose(got, np.asarray(want), rtol=0, atol=1e-14)
+
+
+def test_patchify_constant_and_position_coded_frames():
+    P, Tp, C = 4, 1, 3
+    grids = [(1, 2, 3)]
+    # constant image: every element of every patch is (v/255 - mean)/std of its channel
+    fr = np.full((1, C, 2 * P, 3 * P), 51, dtype=np.uint8)
+    out = O.patchify([fr], grids, P, Tp, (0.2, 0.2, 0.2), (0.5, 1.0, 2.0))
+    assert np.allclose(out[:, : P * P], 0.0) and np.allclose(out.reshape(6, C, P * P)[:, 1], 0.0)
+    # pixel value codes (row, column): patch (r, c) must hold exactly its own window, row-major
+    yy, xx = np.meshgrid(np.arange(2 * P), np.arange(3 * P), indexing="ij")
+    fr = np.broadcast_to((yy * 12 + xx).astype(np.uint8), (1, C, 2 * P, 3 * P)).copy()
+    out = O.patchify([fr], grids, P, Tp, (0.0,) * 3, (1.0 / 255.0,) * 3)     # identity scaling
+    for r in range(2):
+        for c in range(3):
+            win = fr[0, 0, r * P:(r + 1) * P, c * P:(c + 1) * P].astype(np.float64).reshape(-1)
+            assert np.allclose(out[r * 3 + c, : P * P], win)
