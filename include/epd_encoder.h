@@ -151,6 +151,20 @@ int epd_encode_host(epd_encoder_t* enc, const void* host_patches, const int32_t*
                     int32_t n_images, void* host_features, int64_t features_capacity_rows,
                     int64_t* out_rows, int32_t* out_cu_rows, void* stream);
 
+/*
+ * The same stage fed with raw pixels: the step immediately in front of Eq. 1's E.  `frames` is a
+ * device buffer of uint8 pixels holding the items back to back, item i as [t*Tp, C, h*P, w*P]
+ * (frame, channel, y, x; t, h, w from grid_thw, Tp = temporal_patch, P = patch, C = in_channels <= 4).
+ * Pixel v of channel c becomes (v/255 - mean[c]) * inv_std[c] (mean, inv_std: HOST arrays of C floats)
+ * and token (frame f, row r, column c) gathers its patch in element order (channel, temporal, y, x)
+ * -- the patch matrix epd_encode() takes -- in a buffer inside the workspace; then the stage runs as
+ * in epd_encode().  Resizing images to a multiple of the patch size is preprocessing and stays with
+ * the caller.  Errors as epd_encode(), plus EPD_EUNSUPPORTED for more than 4 channels.
+ */
+int epd_encode_frames(epd_encoder_t* enc, const void* frames, const int32_t* grid_thw, int32_t n_images,
+                      const float* mean, const float* inv_std, void* features, int64_t features_capacity_rows,
+                      int64_t* out_rows, int32_t* out_cu_rows, void* stream);
+
 /* Reads the encoder's device status word (synchronises the device): EPD_OK or the first
  * device-side error (EPD_ETIMEOUT), then clears it. */
 int epd_encoder_last_status(epd_encoder_t* enc);
@@ -250,6 +264,15 @@ enum { EPD_ATTENTION_FORCE_FMA = 1 /* use the plain-FMA kernel even where the te
 int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
                      const int32_t* host_cu_seqlens, int32_t n_seg, void* out, int64_t T, int32_t heads,
                      int32_t head_dim, int32_t flags, void* stream);
+
+/* Pixels -> patch vectors (the front end of epd_encode_frames()).  frames: device uint8 as described
+ * there; item_offsets: device int64 [n_images+1] byte offsets of the items inside frames; grid_thw:
+ * device int32 [n_images, 3]; cu_seqlens: device int32 [n_images+1]; patches: device [T, ld] per
+ * dtype, ld >= C*Tp*P*P (columns beyond are zeroed); mean, inv_std: HOST arrays of in_channels floats. */
+int epd_op_patchify(int32_t dtype, const void* frames, const int64_t* item_offsets, const int32_t* grid_thw,
+                    const int32_t* cu_seqlens, int32_t n_images, int64_t T, void* patches, int64_t ld,
+                    int32_t in_channels, int32_t patch, int32_t temporal_patch, const float* mean, const float* inv_std,
+                    void* stream);
 
 /* out[o, q*hidden:(q+1)*hidden] = y[merge_idx[o*4+q], :], y [T, hidden], out [T/4, 4*hidden] per dtype. */
 int epd_op_merge(int32_t dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm,

@@ -28,7 +28,7 @@ EXPORTED_SYMBOLS = [
     "epd_debug_run_block", "epd_debug_profile", "epd_debug_profile_classes",
     "epd_debug_profile_class_name", "epd_debug_profile_read", "epd_op_linear", "epd_op_rmsnorm", "epd_op_rope_split",
     "epd_padded_head_dim", "epd_op_attention", "epd_op_merge", "epd_op_rope_attention_static",
-    "epd_static_scratch_bytes", "epd_last_cuda_error",
+    "epd_static_scratch_bytes", "epd_last_cuda_error", "epd_encode_frames", "epd_op_patchify",
 ]
 
 
@@ -84,6 +84,11 @@ def load_library() -> ctypes.CDLL:
     lib.epd_encode_host.argtypes = [vp, vp, i32p, i32, vp, i64, i64p, i32p, vp]
     lib.epd_encoder_last_status.restype = ctypes.c_int
     lib.epd_encoder_last_status.argtypes = [vp]
+    f32p = ctypes.POINTER(ctypes.c_float)
+    lib.epd_encode_frames.restype = ctypes.c_int
+    lib.epd_encode_frames.argtypes = [vp, vp, i32p, i32, f32p, f32p, vp, i64, i64p, i32p, vp]
+    lib.epd_op_patchify.restype = ctypes.c_int
+    lib.epd_op_patchify.argtypes = [i32, vp, vp, vp, vp, i32, i64, vp, i64, i32, i32, i32, f32p, f32p, vp]
     lib.epd_encoder_last_launch_count.restype = ctypes.c_int64
     lib.epd_encoder_last_launch_count.argtypes = [vp]
     lib.epd_encoder_uses_tensor_cores.restype = ctypes.c_int
@@ -264,6 +269,25 @@ class Encoder:
                                    _stream_ptr(stream)), "epd_encode")
         return features[: rows.value], cu_rows
 
+    def encode_frames(self, frames, grid_thw, mean, std, features=None, stream=None):
+        """frames: device uint8 tensor, the items' [t*Tp, C, H, W] frames back to back (flattened)."""
+        torch = _torch()
+        g, gp = _i32_array(grid_thw)
+        n = g.size // 3
+        T = int(sum(int(g[3 * i]) * int(g[3 * i + 1]) * int(g[3 * i + 2]) for i in range(n)))
+        if features is None:
+            features = torch.empty((max(T // 4, 1), self.cfg.out_dim), dtype=torch_dtype(self.dtype),
+                                   device=self.device)
+        rows = ctypes.c_int64(0)
+        cu_rows = np.zeros(n + 1, dtype=np.int32)
+        m = (ctypes.c_float * len(mean))(*[float(v) for v in mean])
+        istd = (ctypes.c_float * len(std))(*[1.0 / float(v) for v in std])
+        _check(self.lib.epd_encode_frames(self._h, _ptr(frames), gp, n, m, istd, _ptr(features),
+                                          int(features.shape[0]), ctypes.byref(rows),
+                                          cu_rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                          _stream_ptr(stream)), "epd_encode_frames")
+        return features[: rows.value], cu_rows
+
     def encode_host(self, host_patches, grid_thw, host_features, stream=None):
         """host_patches / host_features: CPU tensors (pinned for asynchronous copies)."""
         g, gp = _i32_array(grid_thw)
@@ -385,6 +409,36 @@ def op_merge(dtype, y, merge_idx, stream=None):
     out = torch.empty((T // 4, 4 * h), dtype=y.dtype, device=y.device)
     _check(lib.epd_op_merge(dtype, _ptr(y), _ptr(merge_idx), _ptr(out), T // 4, h, _stream_ptr(stream)),
            "epd_op_merge")
+    return out
+
+
+def pack_frames(frames: Sequence[np.ndarray]):
+    """List of uint8 [t*Tp, C, H, W] arrays -> one flat device tensor (items back to back) and the
+    int64 byte offsets of the items."""
+    torch = _torch()
+    flat = np.concatenate([np.ascontiguousarray(f, dtype=np.uint8).reshape(-1) for f in frames]) if frames \
+        else np.zeros(0, np.uint8)
+    off = np.concatenate([[0], np.cumsum([f.size for f in frames])]).astype(np.int64)
+    return torch.from_numpy(flat).cuda(), off
+
+
+def op_patchify(dtype, frames_dev, item_off, grid_thw, cu_seqlens, in_channels, patch, temporal_patch, mean, std,
+                ld=None, stream=None):
+    torch = _torch()
+    lib = load_library()
+    g = np.asarray(grid_thw, dtype=np.int32).reshape(-1, 3)
+    n = g.shape[0]
+    T = int(cu_seqlens[-1])
+    K = in_channels * temporal_patch * patch * patch
+    ld = K if ld is None else ld
+    out = torch.full((T, ld), 7.0, dtype=torch_dtype(dtype), device="cuda")
+    m = (ctypes.c_float * len(mean))(*[float(v) for v in mean])
+    istd = (ctypes.c_float * len(std))(*[1.0 / float(v) for v in std])
+    off_d = torch.from_numpy(np.asarray(item_off, dtype=np.int64)).cuda()
+    g_d = torch.from_numpy(g.copy()).cuda()
+    cu_d = torch.from_numpy(np.asarray(cu_seqlens, dtype=np.int32)).cuda()
+    _check(lib.epd_op_patchify(dtype, _ptr(frames_dev), _ptr(off_d), _ptr(g_d), _ptr(cu_d), n, T, _ptr(out), ld,
+                               in_channels, patch, temporal_patch, m, istd, _stream_ptr(stream)), "epd_op_patchify")
     return out
 
 

@@ -19,8 +19,8 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Offsets of every activation buffer inside the caller's workspace.
 struct Layout {
-  size_t x, a, qkv, qh, kh, vh, u, merged, proj_hidden, stage_patches, stage_features;
-  size_t grid, cu, cu_out, pos_row, pos_col, merge_slot, merge_idx, rope, status, aux, total;
+  size_t x, a, qkv, qh, kh, vh, u, merged, proj_hidden, stage_patches, stage_features, pix_patches;
+  size_t grid, cu, cu_out, item_off, pos_row, pos_col, merge_slot, merge_idx, rope, status, aux, total;
 };
 
 bool config_ok(const epd_config_t* c) {
@@ -59,9 +59,11 @@ Layout make_layout(const epd_config_t& c) {
   L.proj_hidden = take(c.proj_kind == EPD_PROJ_MLP ? Tm * (size_t)c.proj_hidden * es : 0);
   L.stage_patches = take(T * K * es);
   L.stage_features = take(Tm * (size_t)c.out_dim * es);
+  L.pix_patches = take(T * ((K + 7) / 8 * 8) * es);   // patch vectors built from raw frames
   L.grid = take((size_t)c.max_images * 3 * 4);
   L.cu = take(((size_t)c.max_images + 1) * 4);
   L.cu_out = take(((size_t)c.max_images + 1) * 4);
+  L.item_off = take(((size_t)c.max_images + 1) * 8);
   L.pos_row = take(T * 4);
   L.pos_col = take(T * 4);
   L.merge_slot = take(T * 4);
@@ -82,6 +84,9 @@ struct epd_encoder {
   Layout lay;
   uint8_t* ws = nullptr;
   int32_t* pinned = nullptr;       // [3*max_images | max_images+1 | max_images+1]
+  int64_t* pinned_off = nullptr;   // [max_images+1] byte offsets of the items' frames
+  cudaEvent_t staged_off = nullptr;
+  bool staged_off_valid = false;
   cudaEvent_t staged = nullptr;    // recorded after the layout copy of the last batch
   bool staged_valid = false;
   std::vector<int32_t> last_grid;  // grids of the batch whose layout is on the device
@@ -379,7 +384,12 @@ int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, vo
     delete e;
     return EPD_ECUDA;
   }
-  if (cudaEventCreateWithFlags(&e->staged, cudaEventDisableTiming) != cudaSuccess) {
+  if (cudaEventCreateWithFlags(&e->staged, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&e->staged_off, cudaEventDisableTiming) != cudaSuccess ||
+      cudaMallocHost(reinterpret_cast<void**>(&e->pinned_off), ((size_t)cfg->max_images + 1) * sizeof(int64_t)) !=
+          cudaSuccess) {
+    if (e->staged) cudaEventDestroy(e->staged);
+    if (e->staged_off) cudaEventDestroy(e->staged_off);
     cudaFreeHost(e->pinned);
     delete e;
     return EPD_ECUDA;
@@ -390,6 +400,8 @@ int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, vo
   if (err == cudaSuccess) err = cudaDeviceSynchronize();
   if (err != cudaSuccess) {
     cudaEventDestroy(e->staged);
+    cudaEventDestroy(e->staged_off);
+    cudaFreeHost(e->pinned_off);
     cudaFreeHost(e->pinned);
     delete e;
     return EPD_ECUDA;
@@ -436,6 +448,50 @@ int epd_encode_host(epd_encoder_t* enc, const void* host_patches, const int32_t*
   return EPD_OK;
 }
 
+int epd_encode_frames(epd_encoder_t* enc, const void* frames, const int32_t* grid_thw, int32_t n_images,
+                      const float* mean, const float* inv_std, void* features, int64_t features_capacity_rows,
+                      int64_t* out_rows, int32_t* out_cu_rows, void* stream) {
+  if (!enc) return EPD_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const epd_config_t& c = enc->cfg;
+  if (n_images < 0 || (n_images > 0 && (!grid_thw || !frames || !mean || !inv_std))) return EPD_EINVAL;
+  if (c.in_channels > 4) return EPD_EUNSUPPORTED;
+  if (n_images > c.max_images) return EPD_ECAPACITY;
+  // byte offset of every item's frames in the packed buffer
+  if (enc->staged_off_valid) EPD_CUDA(cudaEventSynchronize(enc->staged_off));
+  int64_t off = 0, T = 0;
+  for (int i = 0; i < n_images; ++i) {
+    const int64_t t = grid_thw[3 * i], h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
+    if (t < 1 || h < 1 || w < 1) return EPD_EINVAL;
+    if (t > c.max_tokens || t * h > c.max_tokens || t * h * w > c.max_tokens) return EPD_ECAPACITY;
+    T += t * h * w;
+    if (T > c.max_tokens) return EPD_ECAPACITY;
+    enc->pinned_off[i] = off;
+    off += t * c.temporal_patch * c.in_channels * (h * c.patch) * (w * c.patch);
+  }
+  enc->pinned_off[n_images] = off;
+  // the integer layout (grid, cu_seqlens) must be on the device before the patch kernel reads it
+  enc->launches = 0;
+  enc->prof_used = 0;
+  int64_t T2 = 0;
+  int rc = prepare_batch(enc, grid_thw, n_images, features_capacity_rows, out_rows, out_cu_rows, &T2, s);
+  if (rc) return rc;
+  if (T2 == 0) return EPD_OK;
+  const int64_t launches_layout = enc->launches;
+  EPD_CUDA(cudaMemcpyAsync(enc->at<int64_t>(enc->lay.item_off), enc->pinned_off, ((size_t)n_images + 1) * sizeof(int64_t),
+                           cudaMemcpyHostToDevice, s));
+  EPD_CUDA(cudaEventRecord(enc->staged_off, s));
+  enc->staged_off_valid = true;
+  const int64_t ld = (enc->patch_dim + 7) / 8 * 8;
+  EPD_CUDA(patchify(c.dtype, static_cast<const uint8_t*>(frames), enc->at<int64_t>(enc->lay.item_off),
+                    enc->at<int32_t>(enc->lay.grid), enc->at<int32_t>(enc->lay.cu), n_images, T2,
+                    enc->at<void>(enc->lay.pix_patches), ld, c.in_channels, c.patch, c.temporal_patch, mean, inv_std, s));
+  rc = encode_device(enc, enc->at<void>(enc->lay.pix_patches), ld, grid_thw, n_images, features, features_capacity_rows,
+                     out_rows, out_cu_rows, s);
+  enc->launches += launches_layout + 1;
+  return rc;
+}
+
 int epd_encoder_last_status(epd_encoder_t* enc) {
   if (!enc) return EPD_EINVAL;
   int32_t st = 0;
@@ -453,6 +509,8 @@ int epd_encoder_destroy(epd_encoder_t* enc) {
   if (!enc) return EPD_OK;
   cudaDeviceSynchronize();
   if (enc->staged) cudaEventDestroy(enc->staged);
+  if (enc->staged_off) cudaEventDestroy(enc->staged_off);
+  if (enc->pinned_off) cudaFreeHost(enc->pinned_off);
   for (cudaEvent_t ev : enc->prof_events) cudaEventDestroy(ev);
   if (enc->pinned) cudaFreeHost(enc->pinned);
   delete enc;
@@ -584,6 +642,20 @@ int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v,
     if (host_cu_seqlens[i + 1] <= host_cu_seqlens[i]) return EPD_EINVAL;
   EPD_CUDA(attention_any(dtype, q, k, v, cu_seqlens, host_cu_seqlens, n_seg, out, T, heads, head_dim, flags, nullptr,
                          static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int epd_op_patchify(int32_t dtype, const void* frames, const int64_t* item_offsets, const int32_t* grid_thw,
+                    const int32_t* cu_seqlens, int32_t n_images, int64_t T, void* patches, int64_t ld,
+                    int32_t in_channels, int32_t patch, int32_t temporal_patch, const float* mean, const float* inv_std,
+                    void* stream) {
+  if (dtype != EPD_DTYPE_F32 && dtype != EPD_DTYPE_BF16) return EPD_EINVAL;
+  if (n_images < 0 || T < 0 || in_channels < 1 || in_channels > 4 || patch < 1 || temporal_patch < 1) return EPD_EINVAL;
+  if (T == 0 || n_images == 0) return EPD_OK;
+  if (!frames || !item_offsets || !grid_thw || !cu_seqlens || !patches || !mean || !inv_std) return EPD_EINVAL;
+  if (ld < (int64_t)in_channels * temporal_patch * patch * patch) return EPD_EINVAL;
+  EPD_CUDA(patchify(dtype, static_cast<const uint8_t*>(frames), item_offsets, grid_thw, cu_seqlens, n_images, T, patches,
+                    ld, in_channels, patch, temporal_patch, mean, inv_std, static_cast<cudaStream_t>(stream)));
   return EPD_OK;
 }
 

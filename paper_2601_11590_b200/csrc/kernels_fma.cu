@@ -47,6 +47,69 @@ cudaError_t token_layout(const int32_t* grid_thw, const int32_t* cu_seqlens, con
 }
 
 // =============================================================================================
+// Pixels -> patch vectors: token j = (item, frame f, row r, column c) gathers, from the item's uint8
+// frames [t*Tp, C, h*P, w*P], the window rows r*P.., columns c*P.. of frames f*Tp.. in element order
+// (channel, temporal, y, x); value = (pixel/255 - mean[channel]) * inv_std[channel].
+// One block per token, one thread per (channel, temporal, y) pixel row: P contiguous bytes in, P
+// contiguous elements out.  Bytes per token: K read + K*sizeof(T) written.
+// =============================================================================================
+struct PixelNorm {
+  float mean[4], inv_std[4];
+};
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+patchify_kernel(const uint8_t* __restrict__ frames, const int64_t* __restrict__ item_off,
+                const int32_t* __restrict__ grid_thw, const int32_t* __restrict__ cu, int n, T* __restrict__ patches,
+                int64_t ld, int C, int P, int Tp, PixelNorm norm) {
+  const int64_t j = blockIdx.x;
+  int lo = 0, hi = n;  // largest i with cu[i] <= j
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (cu[mid] <= j) lo = mid; else hi = mid;
+  }
+  const int i = lo;
+  const int h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
+  const int local = (int)(j - cu[i]);
+  const int f = local / (h * w);
+  const int rem = local - f * h * w;
+  const int r = rem / w, c = rem - r * w;
+  const int64_t H = (int64_t)h * P, W = (int64_t)w * P;
+  const uint8_t* base = frames + item_off[i];
+  T* out = patches + j * ld;
+  const int rows = C * Tp * P;
+  for (int e = threadIdx.x; e < rows; e += blockDim.x) {
+    const int y = e % P;
+    const int tp = (e / P) % Tp;
+    const int ch = e / (P * Tp);
+    const uint8_t* src = base + (((int64_t)(f * Tp + tp) * C + ch) * H + (int64_t)r * P + y) * W + (int64_t)c * P;
+    const float m = norm.mean[ch], is = norm.inv_std[ch];
+    T* dst = out + (int64_t)e * P;
+    for (int x = 0; x < P; ++x) dst[x] = from_float<T>(((float)src[x] * (1.0f / 255.0f) - m) * is);
+  }
+  // padding columns of the row (leading dimension > K) are zeroed so that they are never garbage
+  for (int e = rows * P + threadIdx.x; e < ld; e += blockDim.x) out[e] = from_float<T>(0.0f);
+}
+
+cudaError_t patchify(int dtype, const uint8_t* frames, const int64_t* item_off, const int32_t* grid_thw,
+                     const int32_t* cu_seqlens, int n_images, int64_t T, void* patches, int64_t ld, int C, int P, int Tp,
+                     const float* mean, const float* inv_std, cudaStream_t s) {
+  if (T == 0) return cudaSuccess;
+  PixelNorm norm;
+  for (int c = 0; c < 4; ++c) {
+    norm.mean[c] = c < C ? mean[c] : 0.0f;
+    norm.inv_std[c] = c < C ? inv_std[c] : 1.0f;
+  }
+  if (dtype == EPD_DTYPE_F32)
+    patchify_kernel<float><<<(unsigned)T, 128, 0, s>>>(frames, item_off, grid_thw, cu_seqlens, n_images, (float*)patches,
+                                                       ld, C, P, Tp, norm);
+  else
+    patchify_kernel<__nv_bfloat16><<<(unsigned)T, 128, 0, s>>>(frames, item_off, grid_thw, cu_seqlens, n_images,
+                                                               (__nv_bfloat16*)patches, ld, C, P, Tp, norm);
+  return cudaGetLastError();
+}
+
+// =============================================================================================
 // Linear layer with plain FMAs: out = act(x . w^T + bias), 64x64 tile, 4x4 outputs per thread.
 // =============================================================================================
 constexpr int kFmaTile = 64;

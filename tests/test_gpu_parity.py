@@ -249,6 +249,47 @@ def test_merge(dtype):
     assert np.array_equal(to_np(out), O.merge_2x2(y.astype(np.float64), bk["merge_idx"]))
 
 
+@pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
+@pytest.mark.parametrize("P,Tp,grids,ldpad", [(16, 1, [(1, 4, 6), (1, 2, 2)], 0), (14, 1, [(1, 2, 4)], 4),
+                                              (16, 2, [(3, 2, 4), (1, 6, 2)], 0), (2, 2, [(2, 2, 2)], 8)])
+def test_patchify(dtype, P, Tp, grids, ldpad):
+    """Raw uint8 frames -> patch vectors against the oracle (one rounding to the element type)."""
+    cfg = synth.tiny_variant(patch=P, temporal_patch=Tp)
+    frames = synth.make_frames(cfg, grids, seed=21)
+    mean, std = (0.48, 0.46, 0.41), (0.27, 0.26, 0.28)
+    ref = O.patchify(frames, grids, P, Tp, mean, std)
+    bk = O.bookkeeping(grids)
+    fd, off = epd.pack_frames(frames)
+    K = cfg.patch_dim
+    got = epd.op_patchify(dtype, fd, off, grids, bk["cu_seqlens"], cfg.in_channels, P, Tp, mean, std, ld=K + ldpad)
+    g = to_np(got)
+    assert rel_err(g[:, :K], ref) <= (1e-6 if dtype == epd.DTYPE_F32 else TOL_BF16_STEP)
+    assert np.all(g[:, K:] == 0.0)
+
+
+def test_stage_from_raw_frames():
+    """epd_encode_frames: pixels in, features out, against the oracle's patchify + encode."""
+    cfg = _small_bf16(tp=2)
+    grids = [(2, 6, 8), (1, 10, 4)]
+    w = synth.make_weights(cfg, seed=12)
+    frames = synth.make_frames(cfg, grids, seed=12)
+    T = synth.num_tokens(grids)
+    enc = epd.Encoder(cfg, w, max_tokens=T, max_images=2, max_grid=16)
+    fd, _ = epd.pack_frames(frames)
+    feats, cu_rows = enc.encode_frames(fd, grids, synth.PIXEL_MEAN, synth.PIXEL_STD)
+    torch.cuda.synchronize()
+    assert enc.last_status() == epd.EPD_OK
+    patches = O.patchify(frames, grids, cfg.patch, cfg.temporal_patch, synth.PIXEL_MEAN, synth.PIXEL_STD)
+    ref = O.encode(cfg, w, patches, grids)
+    assert np.array_equal(cu_rows, O.bookkeeping(grids)["cu_out"])
+    assert rel_err(to_np(feats), ref) <= TOL_BF16_FINAL
+    # a second call with the same grids (layout already staged) gives the same bits
+    again, _ = enc.encode_frames(fd, grids, synth.PIXEL_MEAN, synth.PIXEL_STD)
+    torch.cuda.synchronize()
+    assert torch.equal(feats, again)
+    enc.close()
+
+
 # ----------------------------------------------------------------------------- integer layout
 
 def _golden_grids():
