@@ -57,7 +57,7 @@ Layout make_layout(const epd_config_t& c) {
   L.u = take(T * (size_t)c.mlp * es);
   L.merged = take(Tm * 4 * h * es);
   L.proj_hidden = take(c.proj_kind == EPD_PROJ_MLP ? Tm * (size_t)c.proj_hidden * es : 0);
-  L.stage_patches = take(T * K * es);
+  L.stage_patches = take(T * ((K + 7) / 8 * 8) * es);
   L.stage_features = take(Tm * (size_t)c.out_dim * es);
   L.pix_patches = take(T * ((K + 7) / 8 * 8) * es);   // patch vectors built from raw frames
   L.grid = take((size_t)c.max_images * 3 * 4);
@@ -437,10 +437,13 @@ int epd_encode_host(epd_encoder_t* enc, const void* host_patches, const int32_t*
   if (T > 0 && (!host_patches || !host_features)) return EPD_EINVAL;
   void* dp = enc->at<void>(enc->lay.stage_patches);
   void* df = enc->at<void>(enc->lay.stage_features);
+  // the staged copy gets a leading dimension the tensor-core path accepts (a multiple of 8 elements)
+  const int64_t ld = c.dtype == EPD_DTYPE_BF16 ? (enc->patch_dim + 7) / 8 * 8 : enc->patch_dim;
   if (T > 0)
-    EPD_CUDA(cudaMemcpyAsync(dp, host_patches, (size_t)T * enc->patch_dim * es, cudaMemcpyHostToDevice, s));
+    EPD_CUDA(cudaMemcpy2DAsync(dp, (size_t)ld * es, host_patches, (size_t)enc->patch_dim * es,
+                               (size_t)enc->patch_dim * es, (size_t)T, cudaMemcpyHostToDevice, s));
   int64_t rows = 0;
-  int rc = encode_device(enc, dp, enc->patch_dim, grid_thw, n_images, df, features_capacity_rows, &rows, out_cu_rows, s);
+  int rc = encode_device(enc, dp, ld, grid_thw, n_images, df, features_capacity_rows, &rows, out_cu_rows, s);
   if (rc) return rc;
   if (out_rows) *out_rows = rows;
   if (rows > 0)

@@ -461,6 +461,21 @@ def test_host_buffer_entry_point_matches_device_entry_point():
     enc.close()
 
 
+def test_host_buffer_entry_point_with_patch_length_not_a_multiple_of_8():
+    """patch 14 gives K = 588: the host entry point re-pitches the staged copy for the tensor-core path."""
+    import dataclasses
+    cfg = dataclasses.replace(_small_bf16(), patch=14)
+    grids = [(1, 8, 8), (1, 4, 6)]
+    enc, w, patches, feats, cu_rows, _ = _run_stage(cfg, grids, seed=10, with_taps=False)
+    hp = dev(patches, cfg.dtype).cpu().pin_memory()
+    hf = torch.zeros((feats.shape[0], cfg.out_dim), dtype=feats.dtype).pin_memory()
+    rows, cu2 = enc.encode_host(hp, grids, hf)
+    torch.cuda.synchronize()
+    assert rows == feats.shape[0] and np.array_equal(cu2, cu_rows)
+    assert torch.equal(hf, feats.cpu())
+    enc.close()
+
+
 # ----------------------------------------------------------------------------- edge cases / errors
 
 def test_empty_and_invalid_batches():
