@@ -337,6 +337,40 @@ __device__ __forceinline__ Item decode_item(const SegList& segs, int heads, int 
   return it;
 }
 
+// Epilogue of one query row: columns [col0, col0 + N) of (f0 O0 + f1 O1) as bf16, 16 bytes per store.
+// buf holds 2 MAXB registers; N columns are done in batches of at most MAXB.
+template <int N, int MAXB>
+__device__ __forceinline__ void write_output_cols(uint32_t tmem_o0, uint32_t tmem_o1, int col0, bool has1, bool row_ok,
+                                                  float f0, float f1, int dh, __nv_bfloat16* orow, uint32_t* buf) {
+  if constexpr (N > MAXB) {
+    write_output_cols<MAXB, MAXB>(tmem_o0, tmem_o1, col0, has1, row_ok, f0, f1, dh, orow, buf);
+    write_output_cols<N - MAXB, MAXB>(tmem_o0, tmem_o1, col0 + MAXB, has1, row_ok, f0, f1, dh, orow, buf);
+    return;
+  }
+  tmem_ld_cols<N>(tmem_o0 + col0, buf);
+  if (has1) tmem_ld_cols<N>(tmem_o1 + col0, buf + N);
+  tmem_ld_wait();
+  if (row_ok) {
+#pragma unroll
+    for (int g = 0; g < N / 8; ++g) {
+      if (col0 + g * 8 < dh) {  // dh is a multiple of 8
+        uint32_t pk[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float v0 = __uint_as_float(buf[8 * g + 2 * e]) * f0, v1 = __uint_as_float(buf[8 * g + 2 * e + 1]) * f0;
+          if (has1) {
+            v0 = fmaf(__uint_as_float(buf[N + 8 * g + 2 * e]), f1, v0);
+            v1 = fmaf(__uint_as_float(buf[N + 8 * g + 2 * e + 1]), f1, v1);
+          }
+          __nv_bfloat162 b = __floats2bfloat162_rn(v0, v1);
+          pk[e] = *reinterpret_cast<uint32_t*>(&b);
+        }
+        *reinterpret_cast<uint4*>(orow + col0 + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      }
+    }
+  }
+}
+
 // ONES: head_dim < DHP and column head_dim of every V row holds 1.0, so column head_dim of O_w is the
 // row sum of P_w (summed by the tensor core from the same bf16 values as the numerator) and the
 // softmax threads need not add it up.
@@ -679,34 +713,12 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
       const bool row_ok = token < it.seg_beg + it.seg_len;
       __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + it.head * dh;
       const uint32_t tmem_o0 = tmem_base + P::kO0 + lane_off, tmem_o1 = tmem_base + P::kO1 + lane_off;
-      constexpr int kSplit = (P::kOChunks + 1) / 2;    // warpgroup 0 writes chunks [0, kSplit), warpgroup 1 the rest
-      const int c_beg = w == 0 ? 0 : kSplit, c_end = w == 0 ? kSplit : P::kOChunks;
-      for (int c = c_beg; c < c_end; ++c) {
-        uint32_t o0[16], o1[16];
-        tmem_ld16(tmem_o0 + c * 16, o0);
-        if (has1) tmem_ld16(tmem_o1 + c * 16, o1);
-        tmem_ld_wait();
-        float v[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          v[i] = __uint_as_float(o0[i]) * f0;
-          if (has1) v[i] = fmaf(__uint_as_float(o1[i]), f1, v[i]);
-        }
-        if (row_ok) {
-#pragma unroll
-          for (int g = 0; g < 2; ++g) {
-            if (c * 16 + g * 8 < dh) {  // dh is a multiple of 8
-              uint32_t pk[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * g + 2 * e], v[8 * g + 2 * e + 1]);
-                pk[e] = *reinterpret_cast<uint32_t*>(&b);
-              }
-              *reinterpret_cast<uint4*>(orow + c * 16 + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-            }
-          }
-        }
-      }
+      // warpgroup 0 writes columns [0, kSplitCols), warpgroup 1 the rest.  The score registers are dead
+      // here and serve as the landing buffer, so that all TMEM loads of a thread are in flight together.
+      constexpr int kSplitCols = (P::kOChunks + 1) / 2 * 16;
+      constexpr int kMaxB = BKV / 2 / 16 * 16;   // columns of each accumulator that fit the score registers
+      if (w == 0) write_output_cols<kSplitCols, kMaxB>(tmem_o0, tmem_o1, 0, has1, row_ok, f0, f1, dh, orow, s);
+      else write_output_cols<DHP - kSplitCols, kMaxB>(tmem_o0, tmem_o1, kSplitCols, has1, row_ok, f0, f1, dh, orow, s);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(o_free);
