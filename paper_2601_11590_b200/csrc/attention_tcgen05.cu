@@ -533,9 +533,10 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           const int w = j & 1;
           const int vs = vc % P::VS;
           uint32_t& pc = w ? pc1 : pc0;
+          // V arrives long before P: take that wait first so that only P's is on the critical path
+          if (!mbar_wait(&v_full[vs], (vc / P::VS) & 1, abort_flag)) { ok = false; break; }
           if (!mbar_wait(&p_full[w], pc & 1, abort_flag)) { ok = false; break; }
           ++pc;
-          if (!mbar_wait(&v_full[vs], (vc / P::VS) & 1, abort_flag)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sv = smem_u32(smem + P::kV + vs * P::kKStride);
           // MN-major V: boxes (16 or 64 columns wide) are kVBox apart, 8-row groups 256 / 1024 bytes apart
