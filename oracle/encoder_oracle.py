@@ -89,6 +89,38 @@ def bookkeeping(grid_thw: Sequence[Sequence[int]], merge: int = 2) -> Dict[str, 
     }
 
 
+# ----------------------------------------------------------------------------- content hash (feature key)
+
+_MASK64 = (1 << 64) - 1
+_GOLDEN = 0x9E3779B97F4A7C15
+
+
+def _mix64(z: int) -> int:
+    """The finalizer of the SplitMix64 generator (Steele, Lea, Flood 2014; constants of Stafford's mix 13)."""
+    z &= _MASK64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _MASK64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _MASK64
+    return z ^ (z >> 31)
+
+
+def content_hash(data: bytes) -> int:
+    """64-bit key of one item's input bytes (the key under which its features are cached; the paper's
+    MM Store keys features by a hash of the multimodal input, Section 3.2, without naming the hash).
+
+    The bytes (length a multiple of 8) are read as little-endian 64-bit words w_1 .. w_n:
+        key = mix( (sum_k mix(w_k xor k*GOLDEN)) + 8n )   (all arithmetic mod 2^64)
+    The sum makes the key independent of evaluation order (it can be formed in parallel), the
+    position salt k*GOLDEN makes it depend on word order, the length term on trailing zeros.
+    Plain Python integers, one word at a time."""
+    if len(data) % 8:
+        raise ValueError("length must be a multiple of 8 bytes")
+    acc = 0
+    for k in range(len(data) // 8):
+        w = int.from_bytes(data[8 * k: 8 * k + 8], "little")
+        acc = (acc + _mix64(w ^ (((k + 1) * _GOLDEN) & _MASK64))) & _MASK64
+    return _mix64((acc + len(data)) & _MASK64)
+
+
 # ----------------------------------------------------------------------------- pixels -> patch vectors
 
 def patchify(frames: Sequence[np.ndarray], grid_thw: Sequence[Sequence[int]], patch: int, temporal_patch: int,
