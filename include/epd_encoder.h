@@ -279,6 +279,37 @@ int epd_op_merge(int32_t dtype, const void* y, const int32_t* merge_idx, void* o
                  int32_t hidden, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * After the stage: feature keys and a feature cache (the encoder's side of the multimodal store of
+ * Section 3.2, "Asynchronous Feature Prefetching": features are kept under a hash of the input so
+ * that a repeated input is not encoded again and only the key travels with the request)
+ * ---------------------------------------------------------------------------------------- */
+
+/* 64-bit content key of each item.  data: device bytes (8-byte aligned); item_offsets: device int64
+ * [n_items+1] byte offsets of the items inside data, multiples of 8; hashes: device uint64 [n_items].
+ * With w_1..w_n the item's bytes as little-endian 64-bit words and mix the SplitMix64 finalizer,
+ *   key = mix( (sum_k mix(w_k xor k*0x9E3779B97F4A7C15)) + 8n )  mod 2^64.
+ * Enqueued on the stream (a memset and two kernels); bit-exact whatever the launch geometry. */
+int epd_op_content_hash(const void* data, const int64_t* item_offsets, int32_t n_items, uint64_t* hashes,
+                        void* stream);
+
+typedef struct epd_feature_cache epd_feature_cache_t;
+
+/* A cache of feature matrices by key inside `pool` (device memory, 256-byte aligned, owned by the
+ * caller and reserved for the cache until destroy).  row_bytes = out_dim * sizeof(element).  The index
+ * lives on the host; entries are evicted first-in-first-out when the pool wraps.  Not thread-safe. */
+int epd_feature_cache_create(void* pool, size_t pool_bytes, size_t row_bytes, epd_feature_cache_t** out);
+int epd_feature_cache_destroy(epd_feature_cache_t* cache);
+/* Returns EPD_OK on a hit (and, if dst != NULL, enqueues the copy of the `rows` feature rows to dst on
+ * the stream), 1 on a miss (no entry with this key and row count), < 0 on error. */
+int epd_feature_cache_lookup(epd_feature_cache_t* cache, uint64_t key, int64_t rows, void* dst, void* stream);
+/* Enqueues the copy of `rows` feature rows from src (device) into the pool and records them under
+ * key; evicts the oldest entries if room is needed.  EPD_ECAPACITY if they can never fit.  The copy is
+ * stream-ordered: a lookup on the same stream afterwards sees the data. */
+int epd_feature_cache_insert(epd_feature_cache_t* cache, uint64_t key, int64_t rows, const void* src, void* stream);
+int epd_feature_cache_stats(const epd_feature_cache_t* cache, int64_t* hits, int64_t* misses, int64_t* evictions,
+                            int64_t* entries);
+
+/* ------------------------------------------------------------------------------------------
  * Allocation-free variant (the paper has no counterpart: this is a convenience of this library)
  * ---------------------------------------------------------------------------------------- */
 

@@ -29,6 +29,8 @@ EXPORTED_SYMBOLS = [
     "epd_debug_profile_class_name", "epd_debug_profile_read", "epd_op_linear", "epd_op_rmsnorm", "epd_op_rope_split",
     "epd_padded_head_dim", "epd_op_attention", "epd_op_merge", "epd_op_rope_attention_static",
     "epd_static_scratch_bytes", "epd_last_cuda_error", "epd_encode_frames", "epd_op_patchify",
+    "epd_op_content_hash", "epd_feature_cache_create", "epd_feature_cache_destroy",
+    "epd_feature_cache_lookup", "epd_feature_cache_insert", "epd_feature_cache_stats",
 ]
 
 
@@ -89,6 +91,18 @@ def load_library() -> ctypes.CDLL:
     lib.epd_encode_frames.argtypes = [vp, vp, i32p, i32, f32p, f32p, vp, i64, i64p, i32p, vp]
     lib.epd_op_patchify.restype = ctypes.c_int
     lib.epd_op_patchify.argtypes = [i32, vp, vp, vp, vp, i32, i64, vp, i64, i32, i32, i32, f32p, f32p, vp]
+    lib.epd_op_content_hash.restype = ctypes.c_int
+    lib.epd_op_content_hash.argtypes = [vp, vp, i32, vp, vp]
+    lib.epd_feature_cache_create.restype = ctypes.c_int
+    lib.epd_feature_cache_create.argtypes = [vp, ctypes.c_size_t, ctypes.c_size_t, ctypes.POINTER(vp)]
+    lib.epd_feature_cache_destroy.restype = ctypes.c_int
+    lib.epd_feature_cache_destroy.argtypes = [vp]
+    lib.epd_feature_cache_lookup.restype = ctypes.c_int
+    lib.epd_feature_cache_lookup.argtypes = [vp, ctypes.c_uint64, i64, vp, vp]
+    lib.epd_feature_cache_insert.restype = ctypes.c_int
+    lib.epd_feature_cache_insert.argtypes = [vp, ctypes.c_uint64, i64, vp, vp]
+    lib.epd_feature_cache_stats.restype = ctypes.c_int
+    lib.epd_feature_cache_stats.argtypes = [vp, i64p, i64p, i64p, i64p]
     lib.epd_encoder_last_launch_count.restype = ctypes.c_int64
     lib.epd_encoder_last_launch_count.argtypes = [vp]
     lib.epd_encoder_uses_tensor_cores.restype = ctypes.c_int
@@ -288,6 +302,35 @@ class Encoder:
                                           _stream_ptr(stream)), "epd_encode_frames")
         return features[: rows.value], cu_rows
 
+    def encode_frames_cached(self, cache: "FeatureCache", frames, item_off, grid_thw, mean, std, stream=None):
+        """encode_frames with a feature cache in front: items whose content key is cached are not
+        encoded again.  Returns (list of per-item feature tensors, keys uint64 [n], hit mask)."""
+        torch = _torch()
+        g = np.asarray(grid_thw, dtype=np.int32).reshape(-1, 3)
+        n = g.shape[0]
+        off = np.asarray(item_off, dtype=np.int64)
+        keys = op_content_hash(frames, off, stream)
+        rows = [int(t) * int(h) * int(w) // 4 for t, h, w in g]
+        out = [cache.lookup(int(keys[i]), rows[i], stream) for i in range(n)]
+        hit = np.array([o is not None for o in out], dtype=bool)
+        # one encode per distinct missing key
+        todo = {}
+        for i in range(n):
+            if not hit[i]:
+                todo.setdefault(int(keys[i]), i)
+        if todo:
+            idx = list(todo.values())
+            sub = torch.cat([frames[int(off[i]):int(off[i + 1])] for i in idx])
+            feats, cu = self.encode_frames(sub, g[idx], mean, std, stream=stream)
+            for j, i in enumerate(idx):
+                f = feats[int(cu[j]):int(cu[j + 1])].contiguous()
+                cache.insert(int(keys[i]), f, stream)
+                todo[int(keys[i])] = f
+            for i in range(n):
+                if not hit[i]:
+                    out[i] = todo[int(keys[i])]
+        return out, keys, hit
+
     def encode_host(self, host_patches, grid_thw, host_features, stream=None):
         """host_patches / host_features: CPU tensors (pinned for asynchronous copies)."""
         g, gp = _i32_array(grid_thw)
@@ -440,6 +483,73 @@ def op_patchify(dtype, frames_dev, item_off, grid_thw, cu_seqlens, in_channels, 
     _check(lib.epd_op_patchify(dtype, _ptr(frames_dev), _ptr(off_d), _ptr(g_d), _ptr(cu_d), n, T, _ptr(out), ld,
                                in_channels, patch, temporal_patch, m, istd, _stream_ptr(stream)), "epd_op_patchify")
     return out
+
+
+def op_content_hash(data_dev, item_off, stream=None) -> np.ndarray:
+    """64-bit content keys of the items of a packed device byte buffer (item_off: byte offsets,
+    multiples of 8, length n+1).  Returns uint64 [n] on the host."""
+    torch = _torch()
+    lib = load_library()
+    off = np.asarray(item_off, dtype=np.int64).reshape(-1)
+    n = off.size - 1
+    if n <= 0:
+        return np.zeros(0, dtype=np.uint64)
+    if np.any(off % 8) or np.any(np.diff(off) < 0):
+        raise ValueError("item offsets must be non-decreasing multiples of 8")
+    off_d = torch.from_numpy(off).cuda()
+    out = torch.empty(n, dtype=torch.int64, device="cuda")
+    _check(lib.epd_op_content_hash(_ptr(data_dev), _ptr(off_d), n, _ptr(out), _stream_ptr(stream)),
+           "epd_op_content_hash")
+    return out.cpu().numpy().view(np.uint64)
+
+
+class FeatureCache:
+    """Feature matrices by content key in a device pool owned by this object (first-in-first-out)."""
+
+    def __init__(self, pool_bytes: int, out_dim: int, dtype: int):
+        torch = _torch()
+        lib = load_library()
+        self._lib = lib
+        self.out_dim = out_dim
+        self.tdtype = torch_dtype(dtype)
+        self._pool = torch.empty(pool_bytes, dtype=torch.uint8, device="cuda")
+        h = ctypes.c_void_p()
+        row_bytes = out_dim * (4 if dtype == DTYPE_F32 else 2)
+        _check(lib.epd_feature_cache_create(_ptr(self._pool), pool_bytes, row_bytes, ctypes.byref(h)),
+               "epd_feature_cache_create")
+        self._h = h
+
+    def lookup(self, key: int, rows: int, stream=None):
+        """The cached [rows, out_dim] features, or None."""
+        torch = _torch()
+        dst = torch.empty((rows, self.out_dim), dtype=self.tdtype, device="cuda")
+        st = self._lib.epd_feature_cache_lookup(self._h, int(key), rows, _ptr(dst), _stream_ptr(stream))
+        if st == 1:
+            return None
+        _check(st, "epd_feature_cache_lookup")
+        return dst
+
+    def insert(self, key: int, feats, stream=None) -> None:
+        assert feats.is_contiguous() and feats.shape[1] == self.out_dim and feats.dtype == self.tdtype
+        _check(self._lib.epd_feature_cache_insert(self._h, int(key), feats.shape[0], _ptr(feats),
+                                                  _stream_ptr(stream)), "epd_feature_cache_insert")
+
+    def stats(self) -> dict:
+        v = [ctypes.c_int64() for _ in range(4)]
+        _check(self._lib.epd_feature_cache_stats(self._h, *[ctypes.byref(x) for x in v]), "epd_feature_cache_stats")
+        return dict(zip(("hits", "misses", "evictions", "entries"), (int(x.value) for x in v)))
+
+    def close(self) -> None:
+        if self._h:
+            self._lib.epd_feature_cache_destroy(self._h)
+            self._h = None
+            self._pool = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def static_scratch_bytes() -> int:

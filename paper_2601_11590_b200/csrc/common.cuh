@@ -77,6 +77,7 @@ cudaError_t attention_any(int dtype, const void* q, const void* k, const void* v
 cudaError_t patchify(int dtype, const uint8_t* frames, const int64_t* item_off, const int32_t* grid_thw,
                      const int32_t* cu_seqlens, int n_images, int64_t T, void* patches, int64_t ld, int C, int P, int Tp,
                      const float* mean, const float* inv_std, cudaStream_t s);
+cudaError_t content_hash(const void* data, const int64_t* item_off, int n_items, uint64_t* hashes, cudaStream_t s);
 cudaError_t merge_gather(int dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm, int hidden,
                          cudaStream_t s);
 cudaError_t token_layout(const int32_t* grid_thw, const int32_t* cu_seqlens, const int32_t* cu_out, int n_images,

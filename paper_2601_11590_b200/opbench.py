@@ -4,6 +4,7 @@
   python -m paper_2601_11590_b200.opbench attention --heads 16 --dh 72 --seglens 784x8
   python -m paper_2601_11590_b200.opbench rope --T 6272 --heads 16 --dh 72
   python -m paper_2601_11590_b200.opbench rmsnorm --T 6272 --hidden 1152
+  python -m paper_2601_11590_b200.opbench hash --items 64 --item-bytes 4816896
 
 Each call goes through the C ABI (epd_op_*), is timed with CUDA events on the launching stream
 after warm-up, and prints one JSON line: average device time, algorithmic FLOP/s or bytes/s.
@@ -64,7 +65,7 @@ def time_op(torch, fn, iters: int, warmup: int, flush: bool) -> float:
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "attention", "rope", "rmsnorm", "merge"])
+    ap.add_argument("op", choices=["linear", "attention", "rope", "rmsnorm", "merge", "hash"])
     ap.add_argument("--M", type=int, default=6272)
     ap.add_argument("--N", type=int, default=1152)
     ap.add_argument("--K", type=int, default=1152)
@@ -75,6 +76,8 @@ def main():
     ap.add_argument("--heads", type=int, default=16)
     ap.add_argument("--dh", type=int, default=72)
     ap.add_argument("--seglens", default="784x8")
+    ap.add_argument("--items", type=int, default=64)
+    ap.add_argument("--item-bytes", type=int, default=4816896)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--no-flush", action="store_true")
@@ -149,6 +152,17 @@ def main():
         out = torch.empty((T, h), dtype=bf, device="cuda")
         fn = lambda: epd.op_rmsnorm(dt, x, gain, out, 1e-6)
         res.update(T=T, hidden=h, bytes=6.0 * T * h)
+    elif args.op == "hash":
+        n, nb = args.items, args.item_bytes // 8 * 8
+        data = torch.randint(0, 256, (n * nb,), generator=g, device="cuda", dtype=torch.uint8)
+        off = torch.arange(n + 1, device="cuda", dtype=torch.int64) * nb
+        keys = torch.empty(n, dtype=torch.int64, device="cuda")
+        lib = epd.load_library()
+
+        def fn():
+            epd._check(lib.epd_op_content_hash(epd._ptr(data), epd._ptr(off), n, epd._ptr(keys),
+                                               epd._stream_ptr(None)), "epd_op_content_hash")
+        res.update(items=n, item_bytes=nb, bytes=float(n) * nb + 16.0 * n)
     else:
         T, h = args.T // 4 * 4, args.hidden
         y = rnd(T, h)

@@ -521,3 +521,69 @@ def test_create_rejects_small_workspace():
         == epd.EPD_ENOMEM
     assert lib.epd_encoder_create(ctypes.byref(c), ctypes.byref(w), base + 8, need, ctypes.byref(handle)) \
         == epd.EPD_EINVAL
+
+
+# ---------------------------------------------------------------------------------------------
+# Feature keys and the feature cache
+# ---------------------------------------------------------------------------------------------
+def test_content_hash_bit_exact():
+    """Keys of items of very different sizes (empty, one word, several blocks' worth, ragged against
+    the launch width) equal the oracle's, bit for bit."""
+    rng = np.random.default_rng(11)
+    sizes = [0, 8, 16, 8 * 255, 8 * 256, 8 * 257, 8 * 64 * 256, 8 * (64 * 256 + 1), 8 * 150001, 1176 * 4 * 1024]
+    items = [rng.integers(0, 256, size=s, dtype=np.uint8) for s in sizes]
+    items[3][:] = 0                                     # an all-zero item still has a non-trivial key
+    flat = np.concatenate(items)
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    got = epd.op_content_hash(torch.from_numpy(flat).cuda(), off)
+    want = np.array([O.content_hash(it.tobytes()) for it in items], dtype=np.uint64)
+    assert got.dtype == np.uint64 and np.array_equal(got, want), (got, want)
+    assert epd.op_content_hash(torch.zeros(8, dtype=torch.uint8, device="cuda"), [0]).size == 0
+    with pytest.raises(ValueError):
+        epd.op_content_hash(torch.zeros(16, dtype=torch.uint8, device="cuda"), [0, 12])
+
+
+def test_feature_cache_hits_misses_and_eviction():
+    cache = epd.FeatureCache(pool_bytes=4096, out_dim=64, dtype=epd.DTYPE_BF16)   # 128 bytes per row
+    mk = lambda rows, val: torch.full((rows, 64), float(val), dtype=torch.bfloat16, device="cuda")
+    assert cache.lookup(1, 8) is None
+    cache.insert(1, mk(8, 1))           # 1024 bytes
+    cache.insert(2, mk(16, 2))          # 2048
+    cache.insert(2, mk(16, 9))          # same key: kept as is
+    assert torch.equal(cache.lookup(1, 8), mk(8, 1)) and torch.equal(cache.lookup(2, 16), mk(16, 2))
+    assert cache.lookup(1, 4) is None   # same key, other row count: a miss
+    cache.insert(3, mk(12, 3))          # 1536 bytes: does not fit behind key 2, wraps and evicts 1 and 2
+    st = cache.stats()
+    assert cache.lookup(1, 8) is None and torch.equal(cache.lookup(3, 12), mk(12, 3))
+    assert st["evictions"] >= 1 and st["entries"] == cache.stats()["entries"]
+    cache.insert(4, mk(0, 0))           # an item without rows
+    assert cache.lookup(4, 0).shape == (0, 64)
+    with pytest.raises(epd.EpdError):
+        cache.insert(5, mk(64, 5))      # 8192 bytes can never fit
+    torch.cuda.synchronize()
+    cache.close()
+
+
+def test_encode_frames_cached_matches_uncached():
+    """A batch with a repeated image: the repeat is served from the cache, every item's features are
+    bit-identical to the uncached encode of the same item, and a second call hits for every item."""
+    cfg = _small_bf16()
+    grids = [(1, 4, 6), (1, 8, 4), (1, 4, 6)]
+    w = synth.make_weights(cfg, seed=21)
+    frames = synth.make_frames(cfg, grids, seed=22)
+    frames[2] = frames[0].copy()
+    enc = epd.Encoder(cfg, w, max_tokens=synth.num_tokens(grids), max_images=len(grids), max_grid=8)
+    dev, off = epd.pack_frames(frames)
+    ref, cu = enc.encode_frames(dev, grids, synth.PIXEL_MEAN, synth.PIXEL_STD)
+    ref = ref.clone()
+    cache = epd.FeatureCache(pool_bytes=1 << 20, out_dim=cfg.out_dim, dtype=cfg.dtype)
+    out, keys, hit = enc.encode_frames_cached(cache, dev, off, grids, synth.PIXEL_MEAN, synth.PIXEL_STD)
+    assert keys[0] == keys[2] != keys[1] and not hit.any()
+    assert [int(k) for k in keys] == [O.content_hash(f.tobytes()) for f in frames]
+    for i in range(3):
+        assert torch.equal(out[i], ref[cu[i]:cu[i + 1]]), i
+    out2, _, hit2 = enc.encode_frames_cached(cache, dev, off, grids, synth.PIXEL_MEAN, synth.PIXEL_STD)
+    assert hit2.all() and all(torch.equal(a, b) for a, b in zip(out, out2))
+    assert cache.stats()["entries"] == 2
+    cache.close()
+    enc.close()
