@@ -27,16 +27,32 @@ __host__ __device__ inline unsigned long long mix64(unsigned long long z) {
   return z ^ (z >> 31);
 }
 
-// grid (chunks, items): block (c, i) sums the mixed words c*blockDim.x + t, stepping by the grid's width
+// grid (chunks, items): the item's words are read as 16-byte pairs from the first 16-byte boundary on;
+// thread t of chunk c takes pairs c*blockDim.x + t, stepping by the grid's width.  k*GOLDEN advances
+// by addition.  A leading or trailing single word is taken by the first thread of chunk 0.
 __global__ void __launch_bounds__(256)
 hash_accumulate_kernel(const uint8_t* __restrict__ data, const int64_t* __restrict__ item_off,
                        unsigned long long* __restrict__ acc) {
   const int i = blockIdx.y;
   const int64_t beg = item_off[i], words = (item_off[i + 1] - beg) >> 3;
   const unsigned long long* w = reinterpret_cast<const unsigned long long*>(data + beg);
+  const int64_t head = (words > 0 && (reinterpret_cast<uintptr_t>(w) & 8)) ? 1 : 0;
+  const int64_t pairs = (words - head) >> 1;
+  const ulonglong2* w2 = reinterpret_cast<const ulonglong2*>(w + head);
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  unsigned long long c = (unsigned long long)(head + 2 * p + 1) * kGolden;   // (1-based index of the pair's first word) * GOLDEN
+  const unsigned long long cstep = (unsigned long long)(2 * stride) * kGolden;
   unsigned long long sum = 0;
-  for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < words; k += (int64_t)gridDim.x * blockDim.x)
-    sum += mix64(w[k] ^ ((unsigned long long)(k + 1) * kGolden));
+#pragma unroll 4
+  for (; p < pairs; p += stride, c += cstep) {
+    const ulonglong2 v = __ldg(w2 + p);
+    sum += mix64(v.x ^ c) + mix64(v.y ^ (c + kGolden));
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (head) sum += mix64(w[0] ^ kGolden);
+    if ((words - head) & 1) sum += mix64(w[words - 1] ^ ((unsigned long long)words * kGolden));
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
   __shared__ unsigned long long part[8];
