@@ -252,6 +252,33 @@ int epd_op_rope_split(int32_t dtype, const void* qkv, const int32_t* pos_row, co
 
 int32_t epd_padded_head_dim(int32_t head_dim);
 
+/* The fused form of "QKV projection, rotary embedding, head split" that the encoder uses for bf16
+ * batches of more than 128 tokens (head_dim a multiple of 8): the rotation runs in the projection's
+ * epilogue on the fp32 accumulators, so the [T, 3*hidden] intermediate is never written.
+ *
+ * epd_op_qkv_prepare: w [3*hidden, hidden] (leading dimension ldw, a multiple of 8), bias [3*hidden] or
+ *   NULL -> w_prepared [3*hidden, hidden] contiguous, bias_prepared [3*hidden]: the q and k rows
+ *   reordered inside each head so that position 2p holds the first member of rotation pair p and 2p+1
+ *   its partner (pairs of the row half first, then the column half); v rows unchanged.  q.k^T does not
+ *   depend on the order of the head dimensions as long as q and k share it.
+ * epd_op_rope_table: table float [rows, head_dim/4, 2] = (cos, sin)(p * theta^(-2f/(head_dim/2))) for
+ *   position p < rows and frequency f, evaluated in double precision.
+ * epd_op_qkv_pad_init: writes the padding columns of q, k, v [rows, head_dim_padded] (zeros; 1 in v's
+ *   first padding column).  Needed once per buffer: epd_op_qkv_rope never writes them.
+ * epd_op_qkv_rope: x bf16 [T, hidden] (leading dimension ldx) -> q, k, v bf16
+ *   [heads, T, head_dim_padded]; q additionally multiplied by q_scale; q and k keep the prepared
+ *   (pair) order of their head dimensions, v the natural one.  pos_row / pos_col device int32 [T] with
+ *   values < table_rows.  All pointers device, 16-byte aligned.  EPD_EINVAL for other dtypes or
+ *   head_dim not a multiple of 8. */
+int epd_op_qkv_prepare(const void* w, int64_t ldw, const void* bias, void* w_prepared, void* bias_prepared,
+                       int32_t heads, int32_t head_dim, void* stream);
+int epd_op_rope_table(float* table, int32_t rows, int32_t head_dim, float theta, void* stream);
+int epd_op_qkv_pad_init(void* q, void* k, void* v, int64_t rows, int32_t head_dim, void* stream);
+int epd_op_qkv_rope(const void* x, int64_t ldx, const void* w_prepared, const void* bias_prepared,
+                    const int32_t* pos_row, const int32_t* pos_col, const float* table, int32_t table_rows,
+                    void* q, void* k, void* v, int64_t T, int32_t heads, int32_t head_dim, float q_scale,
+                    void* stream);
+
 enum { EPD_ATTENTION_FORCE_FMA = 1 /* use the plain-FMA kernel even where the tensor-core kernel applies */ };
 
 /* Block-diagonal bidirectional attention.  q, k, v [heads, T, head_dim_padded] per dtype as written

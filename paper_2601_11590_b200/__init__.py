@@ -29,6 +29,7 @@ EXPORTED_SYMBOLS = [
     "epd_debug_profile_class_name", "epd_debug_profile_read", "epd_op_linear", "epd_op_rmsnorm", "epd_op_rope_split",
     "epd_padded_head_dim", "epd_op_attention", "epd_op_merge", "epd_op_rope_attention_static",
     "epd_static_scratch_bytes", "epd_last_cuda_error", "epd_encode_frames", "epd_op_patchify",
+    "epd_op_qkv_prepare", "epd_op_rope_table", "epd_op_qkv_pad_init", "epd_op_qkv_rope",
     "epd_op_content_hash", "epd_feature_cache_create", "epd_feature_cache_destroy",
     "epd_feature_cache_lookup", "epd_feature_cache_insert", "epd_feature_cache_stats",
 ]
@@ -91,6 +92,14 @@ def load_library() -> ctypes.CDLL:
     lib.epd_encode_frames.argtypes = [vp, vp, i32p, i32, f32p, f32p, vp, i64, i64p, i32p, vp]
     lib.epd_op_patchify.restype = ctypes.c_int
     lib.epd_op_patchify.argtypes = [i32, vp, vp, vp, vp, i32, i64, vp, i64, i32, i32, i32, f32p, f32p, vp]
+    lib.epd_op_qkv_prepare.restype = ctypes.c_int
+    lib.epd_op_qkv_prepare.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp]
+    lib.epd_op_rope_table.restype = ctypes.c_int
+    lib.epd_op_rope_table.argtypes = [vp, i32, i32, ctypes.c_float, vp]
+    lib.epd_op_qkv_pad_init.restype = ctypes.c_int
+    lib.epd_op_qkv_pad_init.argtypes = [vp, vp, vp, i64, i32, vp]
+    lib.epd_op_qkv_rope.restype = ctypes.c_int
+    lib.epd_op_qkv_rope.argtypes = [vp, i64, vp, vp, vp, vp, vp, i32, vp, vp, vp, i64, i32, i32, ctypes.c_float, vp]
     lib.epd_op_content_hash.restype = ctypes.c_int
     lib.epd_op_content_hash.argtypes = [vp, vp, i32, vp, vp]
     lib.epd_feature_cache_create.restype = ctypes.c_int
@@ -483,6 +492,39 @@ def op_patchify(dtype, frames_dev, item_off, grid_thw, cu_seqlens, in_channels, 
     _check(lib.epd_op_patchify(dtype, _ptr(frames_dev), _ptr(off_d), _ptr(g_d), _ptr(cu_d), n, T, _ptr(out), ld,
                                in_channels, patch, temporal_patch, m, istd, _stream_ptr(stream)), "epd_op_patchify")
     return out
+
+
+def qkv_pair_order(heads: int, head_dim: int) -> np.ndarray:
+    """Index map of epd_op_qkv_prepare for one of q / k: element j of the prepared order is element
+    order[j] of the natural one (argument marshalling for tests: no arithmetic of the method)."""
+    nf = head_dim // 4
+    j = np.arange(head_dim)
+    p = j // 2
+    hf, f = p // nf, p % nf
+    inside = hf * (head_dim // 2) + f + (j % 2) * nf
+    return (np.arange(heads)[:, None] * head_dim + inside[None, :]).reshape(-1)
+
+
+def op_qkv_rope(x, w, bias, pos_row, pos_col, heads, head_dim, theta, q_scale, table_rows, stream=None):
+    """Fused QKV projection + rotary + head split (bf16).  Returns q, k, v [heads, T, padded]; q and k in
+    the prepared (pair) order of qkv_pair_order()."""
+    torch = _torch()
+    lib = load_library()
+    T, h = x.shape[0], heads * head_dim
+    sp = _stream_ptr(stream)
+    wp = torch.empty((3 * h, h), dtype=torch.bfloat16, device="cuda")
+    bp = torch.empty(3 * h, dtype=torch.bfloat16, device="cuda")
+    _check(lib.epd_op_qkv_prepare(_ptr(w), w.stride(0), _ptr(bias), _ptr(wp), _ptr(bp), heads, head_dim, sp),
+           "epd_op_qkv_prepare")
+    table = torch.empty((table_rows, head_dim // 4, 2), dtype=torch.float32, device="cuda")
+    _check(lib.epd_op_rope_table(_ptr(table), table_rows, head_dim, theta, sp), "epd_op_rope_table")
+    dhp = padded_head_dim(head_dim)
+    q, k, v = (torch.full((heads, T, dhp), 7.0, dtype=torch.bfloat16, device="cuda") for _ in range(3))
+    _check(lib.epd_op_qkv_pad_init(_ptr(q), _ptr(k), _ptr(v), heads * T, head_dim, sp), "epd_op_qkv_pad_init")
+    _check(lib.epd_op_qkv_rope(_ptr(x), x.stride(0), _ptr(wp), _ptr(bp), _ptr(pos_row), _ptr(pos_col), _ptr(table),
+                               table_rows, _ptr(q), _ptr(k), _ptr(v), T, heads, head_dim, q_scale, sp),
+           "epd_op_qkv_rope")
+    return q, k, v
 
 
 def op_content_hash(data_dev, item_off, stream=None) -> np.ndarray:

@@ -97,4 +97,16 @@ cudaError_t linear_tc(const void* x, int64_t ldx, const void* w, int64_t ldw, co
 cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
                            int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, int* status, cudaStream_t s);
 
+
+// QKV projection whose epilogue applies the rotary embedding and writes head-major q, k, v (the
+// padding columns are left as the caller initialised them with qkv_pad_init).  w_perm / bias_perm come
+// from qkv_permute (pair order inside each head of q and k).
+cudaError_t linear_tc_pair_qkv(const void* x, int64_t ldx, const void* w_perm, int64_t ldw, const void* bias_perm,
+                               void* q, void* k, void* v, const int32_t* pos_row, const int32_t* pos_col,
+                               const float2* table, int table_rows, int64_t M, int heads, int head_dim, float q_scale,
+                               int* status, cudaStream_t s);
+cudaError_t qkv_permute(const void* w, int64_t ldw, const void* bias, void* w_out, void* bias_out, int heads,
+                        int head_dim, cudaStream_t s);
+cudaError_t qkv_pad_init(void* q, void* k, void* v, int64_t rows, int head_dim, cudaStream_t s);
+
 }  // namespace epd

@@ -21,7 +21,13 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct Layout {
   size_t x, a, qkv, qh, kh, vh, u, merged, proj_hidden, stage_patches, stage_features, pix_patches;
   size_t grid, cu, cu_out, item_off, pos_row, pos_col, merge_slot, merge_idx, rope, status, aux, total;
+  size_t qkv_perm_w, qkv_perm_b;   // per layer: QKV weight / bias with q and k rows in rotation-pair order
 };
+
+// The QKV projection can apply the rotary embedding and the head split in its epilogue.
+bool fused_rope_possible(const epd_config_t& c) {
+  return c.dtype == EPD_DTYPE_BF16 && c.head_dim % 8 == 0 && c.rope_theta > 0.0f && c.layers > 0;
+}
 
 bool config_ok(const epd_config_t* c) {
   if (!c) return false;
@@ -70,6 +76,9 @@ Layout make_layout(const epd_config_t& c) {
   L.merge_idx = take(T * 4);
   L.rope = take((size_t)c.max_grid * (c.head_dim / 4) * sizeof(float2));
   L.status = take(256);
+  const bool fused = fused_rope_possible(c);
+  L.qkv_perm_w = take(fused ? (size_t)c.layers * 3 * h * h * es : 0);
+  L.qkv_perm_b = take(fused ? (size_t)c.layers * align_up(3 * h * es, 256) : 0);
   L.aux = take(0);
   L.total = off;
   return L;
@@ -101,6 +110,7 @@ struct epd_encoder {
   std::vector<int> prof_class;
   size_t prof_used = 0;
   bool use_tc = false;
+  bool fused_rope = false;         // QKV epilogue does rotary + split (batches of more than 128 tokens)
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -231,13 +241,25 @@ int run_block(epd_encoder* enc, int l, float* x, int64_t T, int n_seg, cudaStrea
   EPD_MARK(KC_RMSNORM);
   EPD_CUDA(rmsnorm(dt, x, enc->norm1_w[l], a, nullptr, T, h, c.eps, s));
   EPD_MARK(KC_QKV);
-  if ((rc = linear_dispatch(enc, dt, a, h, enc->qkv_w[l], h, enc->qkv_b[l], qkv, 3 * h, T, 3 * h, h, 0, s))) return rc;
   const float q_scale = 1.4426950408889634f / sqrtf((float)c.head_dim);
-  EPD_MARK(KC_ROPE);
-  EPD_CUDA(rope_split(dt, qkv, enc->at<int32_t>(enc->lay.pos_row), enc->at<int32_t>(enc->lay.pos_col),
-                      enc->at<float2>(enc->lay.rope), c.max_grid, enc->at<void>(enc->lay.qh),
-                      enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh), T, c.heads, c.head_dim, c.rope_theta,
-                      q_scale, s));
+  if (enc->fused_rope && T > 128) {
+    // rotary embedding and head split in the projection's epilogue
+    const size_t hh = (size_t)h;
+    EPD_CUDA(linear_tc_pair_qkv(a, h, enc->ws + enc->lay.qkv_perm_w + (size_t)l * 3 * hh * hh * 2, h,
+                                enc->ws + enc->lay.qkv_perm_b + (size_t)l * align_up(3 * hh * 2, 256),
+                                enc->at<void>(enc->lay.qh), enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh),
+                                enc->at<int32_t>(enc->lay.pos_row), enc->at<int32_t>(enc->lay.pos_col),
+                                enc->at<float2>(enc->lay.rope), c.max_grid, T, c.heads, c.head_dim, q_scale,
+                                enc->at<int>(enc->lay.status), s));
+  } else {
+    if ((rc = linear_dispatch(enc, dt, a, h, enc->qkv_w[l], h, enc->qkv_b[l], qkv, 3 * h, T, 3 * h, h, 0, s)))
+      return rc;
+    EPD_MARK(KC_ROPE);
+    EPD_CUDA(rope_split(dt, qkv, enc->at<int32_t>(enc->lay.pos_row), enc->at<int32_t>(enc->lay.pos_col),
+                        enc->at<float2>(enc->lay.rope), c.max_grid, enc->at<void>(enc->lay.qh),
+                        enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh), T, c.heads, c.head_dim, c.rope_theta,
+                        q_scale, s));
+  }
   if ((rc = attention_dispatch(enc, T, n_seg, s))) return rc;
   EPD_MARK(KC_OUT);
   if ((rc = linear_dispatch(enc, dt, a, h, enc->out_w[l], h, enc->out_b[l], x, h, T, h, h, EPD_LINEAR_ACCUMULATE, s)))
@@ -397,6 +419,19 @@ int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, vo
   cudaError_t err = cudaMemset(e->ws + lay.status, 0, 256);
   if (err == cudaSuccess && cfg->rope_theta > 0.0f)
     err = rope_table(e->at<float2>(lay.rope), cfg->max_grid, cfg->head_dim, cfg->rope_theta, 0);
+  // permuted QKV weights and the padding columns of q, k, v for the fused rotary epilogue
+  e->fused_rope = fused_rope_possible(*cfg);
+  for (int l = 0; l < L && e->fused_rope; ++l)
+    if (((uintptr_t)e->qkv_w[l] & 15) || (e->qkv_b[l] && ((uintptr_t)e->qkv_b[l] & 1))) e->fused_rope = false;
+  if (e->fused_rope) {
+    const size_t h = (size_t)cfg->hidden;
+    for (int l = 0; l < L && err == cudaSuccess; ++l)
+      err = qkv_permute(e->qkv_w[l], cfg->hidden, e->qkv_b[l], e->ws + lay.qkv_perm_w + (size_t)l * 3 * h * h * 2,
+                        e->ws + lay.qkv_perm_b + (size_t)l * align_up(3 * h * 2, 256), cfg->heads, cfg->head_dim, 0);
+    if (err == cudaSuccess)
+      err = qkv_pad_init(e->at<void>(lay.qh), e->at<void>(lay.kh), e->at<void>(lay.vh),
+                         (int64_t)cfg->heads * cfg->max_tokens, cfg->head_dim, 0);
+  }
   if (err == cudaSuccess) err = cudaDeviceSynchronize();
   if (err != cudaSuccess) {
     cudaEventDestroy(e->staged);
@@ -630,6 +665,46 @@ int epd_op_rope_split(int32_t dtype, const void* qkv, const int32_t* pos_row, co
   if (!qkv || !pos_row || !pos_col || !q || !k || !v) return EPD_EINVAL;
   EPD_CUDA(rope_split(dtype, qkv, pos_row, pos_col, nullptr, 0, q, k, v, T, heads, head_dim, theta, q_scale,
                       static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int epd_op_qkv_prepare(const void* w, int64_t ldw, const void* bias, void* w_prepared, void* bias_prepared,
+                       int32_t heads, int32_t head_dim, void* stream) {
+  if (heads < 1 || head_dim < 8 || head_dim % 8 || head_dim > kMaxHeadDim) return EPD_EINVAL;
+  if (!w || !w_prepared || !bias_prepared || ldw < (int64_t)heads * head_dim || ldw % 8) return EPD_EINVAL;
+  if (((uintptr_t)w | (uintptr_t)w_prepared) & 15) return EPD_EINVAL;
+  EPD_CUDA(qkv_permute(w, ldw, bias, w_prepared, bias_prepared, heads, head_dim, static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int epd_op_rope_table(float* table, int32_t rows, int32_t head_dim, float theta, void* stream) {
+  if (!table || rows < 1 || head_dim < 4 || head_dim % 4 || head_dim > kMaxHeadDim || !(theta > 0.0f)) return EPD_EINVAL;
+  EPD_CUDA(rope_table(reinterpret_cast<float2*>(table), rows, head_dim, theta, static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int epd_op_qkv_pad_init(void* q, void* k, void* v, int64_t rows, int32_t head_dim, void* stream) {
+  if (rows < 0 || head_dim < 4 || head_dim > kMaxHeadDim) return EPD_EINVAL;
+  if (rows == 0) return EPD_OK;
+  if (!q || !k || !v) return EPD_EINVAL;
+  EPD_CUDA(qkv_pad_init(q, k, v, rows, head_dim, static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int epd_op_qkv_rope(const void* x, int64_t ldx, const void* w_prepared, const void* bias_prepared,
+                    const int32_t* pos_row, const int32_t* pos_col, const float* table, int32_t table_rows,
+                    void* q, void* k, void* v, int64_t T, int32_t heads, int32_t head_dim, float q_scale,
+                    void* stream) {
+  if (T < 0 || T > (1 << 30) || heads < 1 || head_dim < 8 || head_dim % 8 || head_dim > kMaxHeadDim) return EPD_EINVAL;
+  if (T == 0) return EPD_OK;
+  const int64_t h = (int64_t)heads * head_dim;
+  if (!x || !w_prepared || !pos_row || !pos_col || !table || table_rows < 1 || !q || !k || !v) return EPD_EINVAL;
+  if (ldx < h || ldx % 8) return EPD_EINVAL;
+  if (((uintptr_t)x | (uintptr_t)w_prepared | (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)table) & 15)
+    return EPD_EINVAL;
+  EPD_CUDA(linear_tc_pair_qkv(x, ldx, w_prepared, h, bias_prepared, q, k, v, pos_row, pos_col,
+                              reinterpret_cast<const float2*>(table), table_rows, T, heads, head_dim, q_scale, nullptr,
+                              static_cast<cudaStream_t>(stream)));
   return EPD_OK;
 }
 

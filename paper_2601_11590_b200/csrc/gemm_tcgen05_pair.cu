@@ -20,6 +20,13 @@
 // Each CTA holds the accumulator rows of its own 128 rows of x (two accumulators of 256 columns, so
 // the epilogue of tile i overlaps the main loop of tile i+1).  Ragged M, N, K are handled by TMA
 // (zero fill on loads, clipping on stores).  No load in this file is a multicast load.
+//
+// QKV variant (ROPE = true): the epilogue applies the 2-D rotary embedding to the q and k columns and
+// writes q, k, v straight into the head-major padded buffers the attention kernel reads, so the
+// [T, 3h] intermediate and a separate rotary pass disappear.  It expects the q and k rows of the weight
+// (and bias) permuted inside each head so that the two members of a rotation pair are neighbours
+// (qkv_pair_permutation below); q.k^T does not depend on the order of the head dimensions as long as q
+// and k share it.
 // Every mbarrier wait is bounded: on expiry the CTA records EPD_ETIMEOUT and drains; the two cluster
 // barriers (start, end) are reached by both CTAs on every path.
 #include <cuda.h>
@@ -36,6 +43,7 @@ constexpr int BK = 64;          // 64 bf16 = 128 bytes = one swizzle row
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
 constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
+constexpr int kMaxDynamicSmem = 232448;           // 227 KB: the most one CTA can have
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ uint32_t cluster_rank() {
@@ -179,6 +187,17 @@ __device__ __forceinline__ float gelu_tanh_fast(float x) {
   return 0.5f * x * (1.0f + t);
 }
 
+// Destination of the QKV variant's epilogue.
+struct RopeSplitArgs {
+  __nv_bfloat16* qkv[3];        // head-major [heads, T, dhp] each
+  const int32_t* pos_row;       // [T]
+  const int32_t* pos_col;       // [T]
+  const float2* table;          // [table_rows, dh/4] (cos, sin) of position * frequency
+  int table_in_smem;            // entries (float2) copied into shared memory behind the kernel's own layout; 0 = read from global
+  int heads, dh, dhp;
+  float q_scale;
+};
+
 template <int BN, int STAGES>
 struct PairLayout {
   static constexpr int kABytes = BM * BK * 2;
@@ -198,11 +217,12 @@ struct PairLayout {
 // ---------------------------------------------------------------------------------------------
 // Kernel
 // ---------------------------------------------------------------------------------------------
-template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM>
+template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_out, const __nv_bfloat16* __restrict__ bias, int M, int N,
-                   int K, int* __restrict__ status) {
+                   int K, int* __restrict__ status, const RopeSplitArgs rs) {
+  static_assert(!ROPE || (sizeof(OutT) == 2 && ACT == 0 && !ACCUM), "the QKV variant writes bf16, no activation");
   using L = PairLayout<BN, STAGES>;
   static_assert(BN == 256 || BN == 128, "tile width");
   constexpr int kAccStride = BN;                 // TMEM columns between the two accumulators
@@ -309,7 +329,19 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     const uint32_t tmem_empty_leader0 = map_to_rank(smem_u32(&tmem_empty[0]), 0);
     int acc = 0;
     uint32_t acc_phase = 0;
-    if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_out) : "memory");
+    if (!ROPE && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_out) : "memory");
+    const float2* rope_tab = rs.table;
+    if constexpr (ROPE) {
+      if (rs.table_in_smem > 0) {
+        // the (cos, sin) table is small: keep it in shared memory (every epilogue warp reaches this
+        // barrier before any wait that can give up)
+        float4* dst = reinterpret_cast<float4*>(smem + L::kTotal);
+        const float4* srcv = reinterpret_cast<const float4*>(rs.table);
+        for (int i = threadIdx.x - 64; i < rs.table_in_smem / 2; i += 32 * kEpiWarps) dst[i] = srcv[i];
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+        rope_tab = reinterpret_cast<const float2*>(dst);
+      }
+    }
     for (int tile = pair; tile < num_tiles; tile += n_pairs) {
       const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;
       const int n0 = (tile / m_tiles) * BN + half * (BN / 2);
@@ -321,6 +353,16 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       tc_fence_after();
       const int row0 = m0 + q * 32;
       const uint32_t taddr = tmem_base + acc * kAccStride + half * (BN / 2) + ((uint32_t)(q * 32) << 16);
+      // QKV variant: this thread's row positions, and (tensor, head, dim) of its first column
+      int prow = 0, pcol = 0, rt = 0, rhead = 0, rd = 0;
+      if constexpr (ROPE) {
+        if (row0 + lane < M) { prow = rs.pos_row[row0 + lane]; pcol = rs.pos_col[row0 + lane]; }
+        const int hdim = rs.heads * rs.dh;
+        rt = n0 / hdim;
+        const int within = n0 - rt * hdim;
+        rhead = within / rs.dh;
+        rd = within - rhead * rs.dh;
+      }
 #pragma unroll 1
       for (int c = 0; c < kChunks; ++c) {
         uint32_t pk[32];  // this thread's row of the chunk, as stored: 32 floats or 64 bf16
@@ -339,16 +381,52 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           tmem_ld32(taddr + c * CC, r0);
           tmem_ld32(taddr + c * CC + 32, r1);
           tmem_ld_wait();
+          if constexpr (ROPE) {
+            // groups of 8 columns = 4 rotation pairs, never across a head; two pairs share one
+            // 16-byte table read (pairs 2u, 2u+1 of a half use neighbouring frequencies)
+            const int nf = rs.dh >> 2;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const uint32_t* src = j < 16 ? r0 : r1;
-            const int jj = (2 * j) & 31;
-            float t0 = __uint_as_float(src[jj]) + bs[c * CC + 2 * j];
-            float t1 = __uint_as_float(src[jj + 1]) + bs[c * CC + 2 * j + 1];
-            if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); }
-            if (ACT == 2) { t0 = gelu_erf_f(t0); t1 = gelu_erf_f(t1); }
-            __nv_bfloat162 b = __floats2bfloat162_rn(t0, t1);
-            pk[j] = *reinterpret_cast<uint32_t*>(&b);
+            for (int g = 0; g < 8; ++g) {
+              const uint32_t* src = g < 4 ? r0 : r1;
+              const int jj = (8 * g) & 31;
+              float v[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(src[jj + e]) + bs[c * CC + 8 * g + e];
+              if (rt < 2) {
+                const float sc = rt == 0 ? rs.q_scale : 1.0f;
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                  const int p2 = (rd >> 1) + 2 * u;                       // first pair of the unit inside the head
+                  const int hf = p2 >= nf ? 1 : 0;
+                  const int f = p2 - hf * nf;
+                  const float4 cs = *reinterpret_cast<const float4*>(rope_tab + (hf ? pcol : prow) * nf + f);
+                  const float a0 = v[4 * u], b0 = v[4 * u + 1], a1 = v[4 * u + 2], b1 = v[4 * u + 3];
+                  v[4 * u] = (a0 * cs.x - b0 * cs.y) * sc;
+                  v[4 * u + 1] = (b0 * cs.x + a0 * cs.y) * sc;
+                  v[4 * u + 2] = (a1 * cs.z - b1 * cs.w) * sc;
+                  v[4 * u + 3] = (b1 * cs.z + a1 * cs.w) * sc;
+                }
+              }
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                __nv_bfloat162 b = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+                pk[4 * g + e] = *reinterpret_cast<uint32_t*>(&b);
+              }
+              rd += 8;
+              if (rd == rs.dh) { rd = 0; if (++rhead == rs.heads) { rhead = 0; ++rt; } }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const uint32_t* src = j < 16 ? r0 : r1;
+              const int jj = (2 * j) & 31;
+              float t0 = __uint_as_float(src[jj]) + bs[c * CC + 2 * j];
+              float t1 = __uint_as_float(src[jj + 1]) + bs[c * CC + 2 * j + 1];
+              if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); }
+              if (ACT == 2) { t0 = gelu_erf_f(t0); t1 = gelu_erf_f(t1); }
+              __nv_bfloat162 b = __floats2bfloat162_rn(t0, t1);
+              pk[j] = *reinterpret_cast<uint32_t*>(&b);
+            }
           }
         }
         if (c == kChunks - 1) {
@@ -358,13 +436,35 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           if (lane == 0) mbar_arrive_cluster(tmem_empty_leader0 + acc * 8);
         }
         // the staging buffer is free once the bulk store issued from it has read it
-        if (lane == 0) bulk_wait_read_all();
+        if (!ROPE && lane == 0) bulk_wait_read_all();
         __syncwarp();
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           // 128-byte swizzle: 16-byte chunk j of row r lives at chunk position j ^ (r % 8)
           uint4* dst = reinterpret_cast<uint4*>(sbuf + lane * 128 + ((j ^ (lane & 7)) << 4));
           *dst = make_uint4(pk[4 * j], pk[4 * j + 1], pk[4 * j + 2], pk[4 * j + 3]);
+        }
+        if constexpr (ROPE) {
+          // copy out with 8 lanes per row: 128 contiguous bytes of a head-major row per lane group
+          __syncwarp();
+          const int piece = lane & 7;
+          const int col = n0 + c * CC + 8 * piece;
+          const int hdim = rs.heads * rs.dh;
+          const int t = col / hdim;
+          const int within = col - t * hdim;
+          const int head = within / rs.dh;
+          const int d = within - head * rs.dh;
+          if (col < N) {
+            __nv_bfloat16* base = (t == 0 ? rs.qkv[0] : t == 1 ? rs.qkv[1] : rs.qkv[2]) + (int64_t)head * M * rs.dhp + d;
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+              const int r = it * 4 + (lane >> 3);
+              if (row0 + r < M)
+                *reinterpret_cast<uint4*>(base + (int64_t)(row0 + r) * rs.dhp) =
+                    *reinterpret_cast<const uint4*>(sbuf + r * 128 + ((piece ^ (r & 7)) << 4));
+            }
+          }
+          continue;
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
@@ -444,17 +544,19 @@ int sm_count() {
   return n;
 }
 
-template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM>
+template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE = false>
 cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& to, const void* bias, int M, int N,
-                   int K, int* status, cudaStream_t s) {
+                   int K, int* status, cudaStream_t s, const RopeSplitArgs& rs = RopeSplitArgs{}) {
   using L = PairLayout<BN, STAGES>;
-  auto kern = linear_pair_kernel<BN, STAGES, OutT, ACT, ACCUM>;
+  auto kern = linear_pair_kernel<BN, STAGES, OutT, ACT, ACCUM, ROPE>;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         ROPE ? kMaxDynamicSmem : L::kDynamic);
     if (e != cudaSuccess) return e;
     configured = true;
   }
+  const size_t smem_bytes = L::kDynamic + (ROPE ? (size_t)rs.table_in_smem * sizeof(float2) : 0);
   const int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
   // pairs that can be resident at once (SMs pair up inside a GPC, so this can be below SMs / 2)
   static int max_pairs = 0;
@@ -478,8 +580,8 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
     max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
   }
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  return launch_pdl(kern, dim3(2 * pairs), dim3(kThreads), L::kDynamic, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K,
-                    status);
+  return launch_pdl(kern, dim3(2 * pairs), dim3(kThreads), smem_bytes, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K,
+                    status, rs);
 }
 
 template <int BN, int STAGES>
@@ -517,6 +619,91 @@ cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ld
       !make_map(&to, out, M, N, ldo, 32, out_f32 ? 4 : 2))
     return cudaErrorInvalidValue;
   return launch_bn<BN, 5>(tx, tw, to, bias, (int)M, (int)N, (int)K, flags, status, s);
+}
+
+// QKV projection with the rotary embedding and the head split in its epilogue.  w and bias hold the q
+// and k rows in pair order (qkv_pair_permutation); q, k, v are head-major [heads, M, padded head_dim]
+// whose padding columns the caller has initialised (they are not written here).
+cudaError_t linear_tc_pair_qkv(const void* x, int64_t ldx, const void* w_perm, int64_t ldw, const void* bias_perm,
+                               void* q, void* k, void* v, const int32_t* pos_row, const int32_t* pos_col,
+                               const float2* table, int table_rows, int64_t M, int heads, int head_dim, float q_scale,
+                               int* status, cudaStream_t s) {
+  constexpr int BN = 256;
+  const int64_t hdim = (int64_t)heads * head_dim, N = 3 * hdim, K = hdim;
+  if (head_dim % 8 || !table) return cudaErrorInvalidValue;
+  CUtensorMap tx, tw;
+  if (!make_map(&tx, x, M, K, ldx, BM, 2) || !make_map(&tw, w_perm, N, K, ldw, BN / 2, 2)) return cudaErrorInvalidValue;
+  RopeSplitArgs rs;
+  rs.qkv[0] = static_cast<__nv_bfloat16*>(q);
+  rs.qkv[1] = static_cast<__nv_bfloat16*>(k);
+  rs.qkv[2] = static_cast<__nv_bfloat16*>(v);
+  rs.pos_row = pos_row;
+  rs.pos_col = pos_col;
+  rs.table = table;
+  const int64_t entries = (int64_t)table_rows * (head_dim / 4);
+  rs.table_in_smem =
+      (entries % 2 == 0 && entries * (int64_t)sizeof(float2) <= kMaxDynamicSmem - PairLayout<BN, 5>::kDynamic) ? (int)entries : 0;
+  rs.heads = heads;
+  rs.dh = head_dim;
+  rs.dhp = padded_head_dim(head_dim);
+  rs.q_scale = q_scale;
+  // the output tensor map is not used by this variant
+  return launch<BN, 5, __nv_bfloat16, 0, false, true>(tx, tw, tx, bias_perm, (int)M, (int)N, (int)K, status, s, rs);
+}
+
+namespace {
+
+// Row n of the permuted QKV weight is row qkv_source_row(n) of the original: inside each head of q and
+// k, position 2p holds the first member of rotation pair p and 2p + 1 its partner (pairs counted over
+// the row half, then the column half); v rows stay.
+__global__ void qkv_permute_kernel(const __nv_bfloat16* __restrict__ w, const __nv_bfloat16* __restrict__ b,
+                                   __nv_bfloat16* __restrict__ w_out, __nv_bfloat16* __restrict__ b_out, int heads,
+                                   int dh, int64_t ldw) {
+  const int hdim = heads * dh, n = blockIdx.x;
+  int src = n;
+  if (n < 2 * hdim) {
+    const int j = n % dh, p = j >> 1, nf = dh >> 2;
+    const int hf = p / nf, f = p - hf * nf;
+    src = n - j + hf * (dh >> 1) + f + (j & 1) * nf;
+  }
+  const uint4* in = reinterpret_cast<const uint4*>(w + (int64_t)src * ldw);
+  uint4* out = reinterpret_cast<uint4*>(w_out + (int64_t)n * hdim);
+  for (int i = threadIdx.x; i < hdim / 8; i += blockDim.x) out[i] = in[i];
+  if (threadIdx.x == 0) b_out[n] = b ? b[src] : __float2bfloat16(0.0f);
+}
+
+// Padding columns of the head-major buffers: zeros, and 1 in v's first padding column.
+__global__ void qkv_pad_init_kernel(__nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ k,
+                                    __nv_bfloat16* __restrict__ v, int64_t rows, int dh, int dhp) {
+  const int pad = dhp - dh;
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= rows * pad) return;
+  const int64_t r = i / pad;
+  const int c = (int)(i - r * pad);
+  const int64_t at = r * dhp + dh + c;
+  q[at] = __float2bfloat16(0.0f);
+  k[at] = __float2bfloat16(0.0f);
+  v[at] = __float2bfloat16(c == 0 ? 1.0f : 0.0f);
+}
+
+}  // namespace
+
+cudaError_t qkv_permute(const void* w, int64_t ldw, const void* bias, void* w_out, void* bias_out, int heads,
+                        int head_dim, cudaStream_t s) {
+  const int hdim = heads * head_dim;
+  if (head_dim % 8 || (ldw % 8) || ((uintptr_t)w & 15) || ((uintptr_t)w_out & 15)) return cudaErrorInvalidValue;
+  qkv_permute_kernel<<<3 * hdim, 128, 0, s>>>((const __nv_bfloat16*)w, (const __nv_bfloat16*)bias, (__nv_bfloat16*)w_out,
+                                             (__nv_bfloat16*)bias_out, heads, head_dim, ldw);
+  return cudaGetLastError();
+}
+
+cudaError_t qkv_pad_init(void* q, void* k, void* v, int64_t rows, int head_dim, cudaStream_t s) {
+  const int dhp = padded_head_dim(head_dim), pad = dhp - head_dim;
+  if (pad == 0 || rows == 0) return cudaSuccess;
+  const int64_t n = rows * pad;
+  qkv_pad_init_kernel<<<(unsigned)((n + 255) / 256), 256, 0, s>>>((__nv_bfloat16*)q, (__nv_bfloat16*)k, (__nv_bfloat16*)v,
+                                                                 rows, head_dim, dhp);
+  return cudaGetLastError();
 }
 
 }  // namespace epd

@@ -5,6 +5,7 @@
   python -m paper_2601_11590_b200.opbench rope --T 6272 --heads 16 --dh 72
   python -m paper_2601_11590_b200.opbench rmsnorm --T 6272 --hidden 1152
   python -m paper_2601_11590_b200.opbench hash --items 64 --item-bytes 4816896
+  python -m paper_2601_11590_b200.opbench qkv --T 6272 --heads 16 --dh 72        (projection + rotary + split, fused)
 
 Each call goes through the C ABI (epd_op_*), is timed with CUDA events on the launching stream
 after warm-up, and prints one JSON line: average device time, algorithmic FLOP/s or bytes/s.
@@ -65,7 +66,7 @@ def time_op(torch, fn, iters: int, warmup: int, flush: bool) -> float:
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "attention", "rope", "rmsnorm", "merge", "hash"])
+    ap.add_argument("op", choices=["linear", "attention", "rope", "rmsnorm", "merge", "hash", "qkv"])
     ap.add_argument("--M", type=int, default=6272)
     ap.add_argument("--N", type=int, default=1152)
     ap.add_argument("--K", type=int, default=1152)
@@ -152,6 +153,28 @@ def main():
         out = torch.empty((T, h), dtype=bf, device="cuda")
         fn = lambda: epd.op_rmsnorm(dt, x, gain, out, 1e-6)
         res.update(T=T, hidden=h, bytes=6.0 * T * h)
+    elif args.op == "qkv":
+        T, heads, dh = args.T, args.heads, args.dh
+        h = heads * dh
+        dhp = epd.padded_head_dim(dh)
+        x, w, b = rnd(T, h), rnd(3 * h, h, std=h ** -0.5), rnd(3 * h, std=0.5)
+        pr = torch.randint(0, 28, (T,), generator=g, device="cuda", dtype=torch.int32)
+        pc = torch.randint(0, 28, (T,), generator=g, device="cuda", dtype=torch.int32)
+        lib = epd.load_library()
+        sp = epd._stream_ptr(None)
+        wp, bp = torch.empty_like(w), torch.empty_like(b)
+        epd._check(lib.epd_op_qkv_prepare(epd._ptr(w), h, epd._ptr(b), epd._ptr(wp), epd._ptr(bp), heads, dh, sp),
+                   "epd_op_qkv_prepare")
+        table = torch.empty((28, dh // 4, 2), dtype=torch.float32, device="cuda")
+        epd._check(lib.epd_op_rope_table(epd._ptr(table), 28, dh, 10000.0, sp), "epd_op_rope_table")
+        q, k, v = (torch.zeros((heads, T, dhp), dtype=bf, device="cuda") for _ in range(3))
+
+        def fn():
+            epd._check(lib.epd_op_qkv_rope(epd._ptr(x), h, epd._ptr(wp), epd._ptr(bp), epd._ptr(pr), epd._ptr(pc),
+                                           epd._ptr(table), 28, epd._ptr(q), epd._ptr(k), epd._ptr(v), T, heads, dh,
+                                           0.17, sp), "epd_op_qkv_rope")
+        res.update(T=T, heads=heads, dh=dh, flops=2.0 * T * 3 * h * h,
+                   bytes=2.0 * (T * h + 3 * h * h) + 2.0 * 3 * T * h + 8.0 * T)
     elif args.op == "hash":
         n, nb = args.items, args.item_bytes // 8 * 8
         data = torch.randint(0, 256, (n * nb,), generator=g, device="cuda", dtype=torch.uint8)

@@ -162,6 +162,44 @@ def test_rope_split(dtype, heads, dh):
     assert np.array_equal(to_np(v)[:, :, :dh].transpose(1, 0, 2), vr)  # v is a pure copy
 
 
+@pytest.mark.parametrize("heads,dh,T", [(16, 72, 784), (3, 72, 300), (4, 64, 129), (25, 128, 260), (2, 8, 40), (16, 72, 1)])
+def test_qkv_rope_fused(heads, dh, T):
+    """Projection + rotary + head split in one kernel against the oracle's linear, rope_2d and split.
+    Tile-ragged T, heads whose 72 columns straddle the 128-column halves and 256-column tiles, the
+    q / k / v boundaries inside a tile (3 heads), padded and unpadded head widths."""
+    dtype = epd.DTYPE_BF16
+    h = heads * dh
+    x = rnd((T, h), 31, 1.0, dtype)
+    w = rnd((3 * h, h), 32, h ** -0.5, dtype)
+    b = rnd((3 * h,), 33, 0.5, dtype)
+    rng = np.random.default_rng(2)
+    rows = 97
+    pr, pc = rng.integers(0, rows, T).astype(np.int32), rng.integers(0, rows, T).astype(np.int32)
+    scale = 0.21
+    q, k, v = epd.op_qkv_rope(dev(x, dtype), dev(w, dtype), dev(b, dtype), torch.from_numpy(pr).cuda(),
+                              torch.from_numpy(pc).cuda(), heads, dh, 10000.0, scale, rows)
+    y = O.linear(x.astype(np.float64), w.astype(np.float64), b.astype(np.float64))
+    qr = O.rope_2d(y[:, :h].reshape(T, heads, dh), pr, pc, 10000.0) * scale
+    kr = O.rope_2d(y[:, h:2 * h].reshape(T, heads, dh), pr, pc, 10000.0)
+    vr = y[:, 2 * h:].reshape(T, heads, dh)
+    order = epd.qkv_pair_order(heads, dh)          # q and k come back in the prepared order of head dims
+    qr = qr.reshape(T, h)[:, order].reshape(T, heads, dh)
+    kr = kr.reshape(T, h)[:, order].reshape(T, heads, dh)
+    dhp = epd.padded_head_dim(dh)
+    for got, ref in ((q, qr), (k, kr), (v, vr)):
+        g = to_np(got)
+        assert g.shape == (heads, T, dhp)
+        assert rel_err(g[:, :, :dh].transpose(1, 0, 2), ref) <= TOL_BF16_STEP
+        if got is v and dhp > dh:
+            assert np.all(g[:, :, dh] == 1.0) and np.all(g[:, :, dh + 1:] == 0.0)
+        else:
+            assert np.all(g[:, :, dh:] == 0.0)
+    # the scores do not depend on the order of the head dimensions
+    s_fused = np.einsum("htd,hud->htu", to_np(q)[:, :, :dh], to_np(k)[:, :, :dh])
+    s_ref = np.einsum("thd,uhd->htu", qr, kr)
+    assert rel_err(s_fused, s_ref) <= TOL_BF16_STEP
+
+
 def _attention_case(dtype, heads, dh, seglens, seed, logit_scale=1.0, flags=0):
     T = int(sum(seglens))
     cu = np.concatenate([[0], np.cumsum(seglens)]).astype(np.int32)
