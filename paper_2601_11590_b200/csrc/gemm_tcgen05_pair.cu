@@ -369,12 +369,18 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         if constexpr (sizeof(OutT) == 4) {
           tmem_ld32(taddr + c * CC, pk);
           tmem_ld_wait();
+          const float4* bs4 = reinterpret_cast<const float4*>(bs + c * CC);   // broadcast reads, 16 bytes each
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            float t = __uint_as_float(pk[j]) + bs[c * CC + j];
-            if (ACT == 1) t = gelu_tanh_fast(t);
-            if (ACT == 2) t = gelu_erf_f(t);
-            pk[j] = __float_as_uint(t);
+          for (int j4 = 0; j4 < 8; ++j4) {
+            const float4 bv = bs4[j4];
+            const float bb[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float t = __uint_as_float(pk[4 * j4 + e]) + bb[e];
+              if (ACT == 1) t = gelu_tanh_fast(t);
+              if (ACT == 2) t = gelu_erf_f(t);
+              pk[4 * j4 + e] = __float_as_uint(t);
+            }
           }
         } else {
           uint32_t r0[32], r1[32];
@@ -389,9 +395,12 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             for (int g = 0; g < 8; ++g) {
               const uint32_t* src = g < 4 ? r0 : r1;
               const int jj = (8 * g) & 31;
+              const float4 ba = *reinterpret_cast<const float4*>(bs + c * CC + 8 * g);
+              const float4 bb = *reinterpret_cast<const float4*>(bs + c * CC + 8 * g + 4);
+              const float bias8[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
               float v[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(src[jj + e]) + bs[c * CC + 8 * g + e];
+              for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(src[jj + e]) + bias8[e];
               if (rt < 2) {
                 const float sc = rt == 0 ? rs.q_scale : 1.0f;
 #pragma unroll
@@ -416,16 +425,19 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
               if (rd == rs.dh) { rd = 0; if (++rhead == rs.heads) { rhead = 0; ++rt; } }
             }
           } else {
+            const float4* bs4 = reinterpret_cast<const float4*>(bs + c * CC);   // broadcast reads, 16 bytes each
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const uint32_t* src = j < 16 ? r0 : r1;
-              const int jj = (2 * j) & 31;
-              float t0 = __uint_as_float(src[jj]) + bs[c * CC + 2 * j];
-              float t1 = __uint_as_float(src[jj + 1]) + bs[c * CC + 2 * j + 1];
-              if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); }
-              if (ACT == 2) { t0 = gelu_erf_f(t0); t1 = gelu_erf_f(t1); }
-              __nv_bfloat162 b = __floats2bfloat162_rn(t0, t1);
-              pk[j] = *reinterpret_cast<uint32_t*>(&b);
+            for (int j2 = 0; j2 < 16; ++j2) {
+              const uint32_t* src = j2 < 8 ? r0 : r1;
+              const int jj = (4 * j2) & 31;
+              const float4 bv = bs4[j2];
+              float t0 = __uint_as_float(src[jj]) + bv.x, t1 = __uint_as_float(src[jj + 1]) + bv.y;
+              float t2 = __uint_as_float(src[jj + 2]) + bv.z, t3 = __uint_as_float(src[jj + 3]) + bv.w;
+              if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); t2 = gelu_tanh_fast(t2); t3 = gelu_tanh_fast(t3); }
+              if (ACT == 2) { t0 = gelu_erf_f(t0); t1 = gelu_erf_f(t1); t2 = gelu_erf_f(t2); t3 = gelu_erf_f(t3); }
+              __nv_bfloat162 b0 = __floats2bfloat162_rn(t0, t1), b1 = __floats2bfloat162_rn(t2, t3);
+              pk[2 * j2] = *reinterpret_cast<uint32_t*>(&b0);
+              pk[2 * j2 + 1] = *reinterpret_cast<uint32_t*>(&b1);
             }
           }
         }
