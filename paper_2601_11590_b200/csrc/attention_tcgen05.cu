@@ -4,7 +4,7 @@
 // ordered longest segment first and dealt round-robin to the CTAs.  Inside an item the segment's
 // keys/values stream through shared memory in tiles of BKV keys, and the two softmax warpgroups take
 // alternate key tiles, each with its own running max / sum and its own output accumulator:
-//   S_w = Q K^T        tcgen05.mma, both operands K-major in shared memory, fp32 S_w in TMEM (w = tile parity)
+//   S_w = Q K^T        tcgen05.mma, both operands K-major in shared memory, fp32 S_w in TMEM (w = warpgroup)
 //   online softmax     warpgroup w, one thread per query row: the S row is read once into registers
 //                      (tcgen05.ld) and the S_w buffer handed back at once, so the next S_w is computed
 //                      while this tile's exponentials run; P = exp2(S - m) goes to a separate bf16
@@ -23,7 +23,10 @@
 // The running max only advances (and O_w is rescaled in TMEM) when it grows by more than 2^8; until
 // then the stale max serves P, the row sum and O_w alike, which leaves the result unchanged.  At the
 // end of an item the two partial results are merged:
-//   m = max(m0, m1),  O = (2^(m0-m) O0 + 2^(m1-m) O1) / (2^(m0-m) l0 + 2^(m1-m) l1).
+//   m = max(m0, m1),  O = (2^(m0-m) O0 + 2^(m1-m) O1) / (2^(m0-m) l0 + 2^(m1-m) l1)
+// by the warpgroup that owns the item's last key tile; the other one publishes its (m, l) and starts on
+// the next item's score tiles at once.  The warpgroups swap key-tile parities every item, so with an odd
+// number of key tiles (7 for a 784-token image) the extra tile and the merge alternate between them.
 // TMEM (512 columns): S0 | P0 | S1 | P1 | O0 | O1, with BKV chosen so that this fits: 112 keys for a
 // padded head width of 80, 80 keys for 128, 128 keys for 64.
 // Warp roles: warp 0 TMA producer of Q (double-buffered across items) and the K ring, warp 3 TMA
@@ -291,7 +294,7 @@ struct Plan {
   static constexpr int kBar = kMl + 4 * BQ * 8;
   // q_full[2] q_empty[2] k_full[KS] k_empty[KS] v_full[VS] v_empty[VS] s_full[2] s_free[2] p_full[2] p_free[2]
   // o_final o_free ml_ready
-  static constexpr int kNumBars = 4 + 2 * KS + 2 * VS + 11;
+  static constexpr int kNumBars = 4 + 2 * KS + 2 * VS + 12;
   static constexpr int kTotal = kBar + kNumBars * 8 + 32;
   static constexpr int kDynamic = kTotal + 1024;       // slack to align the tiles to 1024 bytes
   static_assert(kQBytes % 1024 == 0, "Q buffers keep the rings 1024-byte aligned");
@@ -395,8 +398,8 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
   uint64_t* p_full = s_free + 2;              // [2]  P_w written (4 warp arrivals)
   uint64_t* p_free = p_full + 2;              // [2]  P_w consumed: the warpgroup's last P V is complete
   uint64_t* o_final = p_free + 2;             // all P V products of the item complete
-  uint64_t* o_free = o_final + 1;             // both accumulators read out (8 warp arrivals)
-  uint64_t* ml_ready = o_free + 1;            // both warpgroups published (m, l) (8 warp arrivals)
+  uint64_t* o_free = o_final + 1;             // both accumulators read out by the closing warpgroup (4 warp arrivals)
+  uint64_t* ml_pub = o_free + 1;              // [2]  warpgroup w published its (m, l) of the item (4 warp arrivals)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + P::kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float2* ml_all = reinterpret_cast<float2*>(smem + P::kMl);
@@ -406,8 +409,9 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
   if (threadIdx.x == 0) {
     for (int i = 0; i < P::kNumBars; ++i) mbar_init(&bars[i], 1);
     for (int w = 0; w < 2; ++w) { mbar_init(&s_free[w], 4); mbar_init(&p_full[w], 4); }
-    mbar_init(o_free, 8);
-    mbar_init(ml_ready, 8);
+    mbar_init(o_free, 4);
+    mbar_init(&ml_pub[0], 4);
+    mbar_init(&ml_pub[1], 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -488,7 +492,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         const uint64_t dq_main = smem_desc(sq, 16, 1024, 2);
         const uint64_t dq_tail = smem_desc(sq + P::kMainBoxes * P::kQMain, 16, 256, 6);
         for (int j = 0; j < it.n_kv; ++j, ++kc) {
-          const int w = j & 1;
+          const int w = (j ^ n) & 1;                    // the warpgroups swap key-tile parities every item
           const int ks = kc % P::KS;
           if (!mbar_wait(&k_full[ks], (kc / P::KS) & 1, abort_flag)) { ok = false; break; }
           uint32_t& sc = w ? sc1 : sc0;
@@ -530,7 +534,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         // the accumulators of the previous item must have been read out before they are overwritten
         if (n > 0 && !mbar_wait(o_free, (n - 1) & 1, abort_flag)) break;
         for (int j = 0; j < it.n_kv; ++j, ++vc) {
-          const int w = j & 1;
+          const int w = (j ^ n) & 1;
           const int vs = vc % P::VS;
           uint32_t& pc = w ? pc1 : pc0;
           // V arrives long before P: take that wait first so that only P's is on the critical path
@@ -563,7 +567,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     __syncwarp();
   } else if (warp >= 4) {
     // ---------------------------------------------------------------- softmax / rescale / merge / epilogue
-    const int w = (warp - 4) >> 2;                      // warpgroup = key-tile parity
+    const int w = (warp - 4) >> 2;                      // warpgroup; takes key tiles of parity w ^ (item count & 1)
     const int qr = warp & 3;                            // TMEM lane quarter this warp may access
     const int r = qr * 32 + lane;                       // query row inside the tile
     const uint32_t lane_off = (uint32_t)(qr * 32) << 16;
@@ -571,7 +575,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     const uint32_t tmem_p = tmem_base + (w ? P::kP1 : P::kP0) + lane_off;
     const uint32_t tmem_o = tmem_base + (w ? P::kO1 : P::kO0) + lane_off;
     uint32_t tc = 0, n = 0;                             // score tiles processed, items processed
-    bool ok = true;
+    bool ok = true, closed_prev = false;                // closed_prev: this warpgroup merged the previous item
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
       const Item it = decode_item<BKV>(segs, heads, item);
       float m = -INFINITY, l = 0.0f;
@@ -591,8 +595,13 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         }
         return true;
       };
-      if (w < it.n_kv && !load_scores(w)) { ok = false; break; }
-      for (int j = w; j < it.n_kv; j += 2) {
+      // With an odd number of key tiles one warpgroup has one more than the other; swapping parities every
+      // item evens that out over two items, because a warpgroup that is done does not wait for the other:
+      // it publishes (m, l) and goes on to the next item, and the warpgroup that owns the item's last key
+      // tile (the "closing" one) merges and writes the rows alone.
+      const int j0 = (w ^ n) & 1;                       // this warpgroup's first key tile of the item
+      if (j0 < it.n_kv && !load_scores(j0)) { ok = false; break; }
+      for (int j = j0; j < it.n_kv; j += 2) {
         const int kv_valid = min(BKV, it.seg_len - j * BKV);
         tmem_ld_wait();
         // S_w may be overwritten by the next score tile from here on
@@ -617,7 +626,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         // advance the running max only when it would grow by more than the threshold
         float scale = 1.0f;
         bool grow = false;
-        if (j == w) {
+        if (j == j0) {
           m = m_tile;
         } else if (m_tile - m > kRescaleThreshold) {
           scale = ex2(m - m_tile);
@@ -681,45 +690,52 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         if (lane == 0) mbar_arrive(&p_full[w]);
       }
       if (!ok) break;
-      // merge the two partial results and write the item's rows; (m, l) are double-buffered by item
-      // parity because a warpgroup without key tiles in the next item may publish early
+      // publish (m, l); they are double-buffered by item parity because the other warpgroup may still be
+      // reading the previous item's while this one is already an item ahead
+      // A publication must not overtake the reader of the previous one by a whole barrier phase: unless this
+      // warpgroup merged the previous item itself, it first sees that merge finished (with two or more
+      // key tiles in this item it already has, through its P V products).
+      if (n > 0 && !closed_prev && !mbar_wait(o_free, (n - 1) & 1, abort_flag)) { ok = false; break; }
       float2* ml = ml_all + (n & 1) * 2 * BQ;
       ml[w * BQ + r] = make_float2(m, l);
       __syncwarp();
-      if (lane == 0) mbar_arrive(ml_ready);
-      if (!mbar_wait(ml_ready, n & 1, abort_flag)) { ok = false; break; }
+      if (lane == 0) mbar_arrive(&ml_pub[w]);
+      const int closing = ((it.n_kv - 1) ^ n) & 1;      // owner of the last key tile
+      closed_prev = w == closing;
+      if (!closed_prev) continue;
+      if (!mbar_wait(&ml_pub[w ^ 1], n & 1, abort_flag)) { ok = false; break; }
       if (!mbar_wait(o_final, n & 1, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const bool has1 = it.n_kv > 1;
-      float2 ml0 = ml[r], ml1 = ml[BQ + r];
+      // "a" is this warpgroup's accumulator (it has at least the last key tile), "b" the other's
+      const bool has_b = it.n_kv > 1;
+      float2 ml_a = ml[w * BQ + r], ml_b = ml[(w ^ 1) * BQ + r];
+      const uint32_t tmem_oa = tmem_base + (w ? P::kO1 : P::kO0) + lane_off;
+      const uint32_t tmem_ob = tmem_base + (w ? P::kO0 : P::kO1) + lane_off;
       if (ONES) {
         // the row sums sit in column head_dim of the accumulators
         uint32_t t0[8], t1[8];
-        tmem_ld8(tmem_base + P::kO0 + lane_off + (dh & ~7), t0);
-        if (has1) tmem_ld8(tmem_base + P::kO1 + lane_off + (dh & ~7), t1);
+        tmem_ld8(tmem_oa + (dh & ~7), t0);
+        if (has_b) tmem_ld8(tmem_ob + (dh & ~7), t1);
         tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           if (i == (dh & 7)) {
-            ml0.y = __uint_as_float(t0[i]);
-            ml1.y = has1 ? __uint_as_float(t1[i]) : 0.0f;
+            ml_a.y = __uint_as_float(t0[i]);
+            ml_b.y = has_b ? __uint_as_float(t1[i]) : 0.0f;
           }
         }
       }
-      const float mm = has1 ? fmaxf(ml0.x, ml1.x) : ml0.x;
-      const float a0 = ex2(ml0.x - mm), a1 = has1 ? ex2(ml1.x - mm) : 0.0f;
-      const float inv = 1.0f / (a0 * ml0.y + a1 * ml1.y);
-      const float f0 = a0 * inv, f1 = a1 * inv;
+      const float mm = has_b ? fmaxf(ml_a.x, ml_b.x) : ml_a.x;
+      const float ea = ex2(ml_a.x - mm), eb = has_b ? ex2(ml_b.x - mm) : 0.0f;
+      const float inv = 1.0f / (ea * ml_a.y + eb * ml_b.y);
+      const float fa = ea * inv, fb = eb * inv;
       const int token = it.q0 + r;
       const bool row_ok = token < it.seg_beg + it.seg_len;
       __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + it.head * dh;
-      const uint32_t tmem_o0 = tmem_base + P::kO0 + lane_off, tmem_o1 = tmem_base + P::kO1 + lane_off;
-      // warpgroup 0 writes columns [0, kSplitCols), warpgroup 1 the rest.  The score registers are dead
-      // here and serve as the landing buffer, so that all TMEM loads of a thread are in flight together.
-      constexpr int kSplitCols = (P::kOChunks + 1) / 2 * 16;
+      // The score registers are dead here and serve as the landing buffer, so that all TMEM loads of a
+      // batch of columns are in flight together.
       constexpr int kMaxB = BKV / 2 / 16 * 16;   // columns of each accumulator that fit the score registers
-      if (w == 0) write_output_cols<kSplitCols, kMaxB>(tmem_o0, tmem_o1, 0, has1, row_ok, f0, f1, dh, orow, s);
-      else write_output_cols<DHP - kSplitCols, kMaxB>(tmem_o0, tmem_o1, kSplitCols, has1, row_ok, f0, f1, dh, orow, s);
+      write_output_cols<DHP, kMaxB>(tmem_oa, tmem_ob, 0, has_b, row_ok, fa, fb, dh, orow, s);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(o_free);
