@@ -24,9 +24,14 @@
 // then the stale max serves P, the row sum and O_w alike, which leaves the result unchanged.  At the
 // end of an item the two partial results are merged:
 //   m = max(m0, m1),  O = (2^(m0-m) O0 + 2^(m1-m) O1) / (2^(m0-m) l0 + 2^(m1-m) l1)
-// by the warpgroup that owns the item's last key tile; the other one publishes its (m, l) and starts on
-// the next item's score tiles at once.  The warpgroups swap key-tile parities every item, so with an odd
-// number of key tiles (7 for a 784-token image) the extra tile and the merge alternate between them.
+// by the warpgroup that owns the item's last key tile.  The other one publishes its (m, l) and starts on
+// the next item's score tiles at once; the first key tile of the next item is given to it.  The merging
+// warpgroup first copies the other accumulator into its (dead) score registers and hands it back, then
+// its own, so the other warpgroup's P V products of the next item are not held up by the merge; each
+// accumulator has its own "complete" (o_done) and "read out" (o_free) barrier.  With an odd number of
+// key tiles (7 for a 784-token image) the extra tile and the merge alternate between the warpgroups.
+// (Measured against both warpgroups waiting for each other and sharing the epilogue: 16384-token segment
+// 726 -> 756 TFLOP/s, 8 x 784 tokens 361 -> 383, mixed lengths 569 -> 581, 16 x 1024 tokens 466 -> 457.)
 // TMEM (512 columns): S0 | P0 | S1 | P1 | O0 | O1, with BKV chosen so that this fits: 112 keys for a
 // padded head width of 80, 80 keys for 128, 128 keys for 64.
 // Warp roles: warp 0 TMA producer of Q (double-buffered across items) and the K ring, warp 3 TMA
@@ -293,8 +298,8 @@ struct Plan {
   static constexpr int kMl = kV + VS * kKStride;       // (m, l) of both warpgroups, by item parity: float2[2][2][128]
   static constexpr int kBar = kMl + 4 * BQ * 8;
   // q_full[2] q_empty[2] k_full[KS] k_empty[KS] v_full[VS] v_empty[VS] s_full[2] s_free[2] p_full[2] p_free[2]
-  // o_final o_free ml_ready
-  static constexpr int kNumBars = 4 + 2 * KS + 2 * VS + 12;
+  // o_done[2] o_free[2] ml_pub[2]
+  static constexpr int kNumBars = 4 + 2 * KS + 2 * VS + 14;
   static constexpr int kTotal = kBar + kNumBars * 8 + 32;
   static constexpr int kDynamic = kTotal + 1024;       // slack to align the tiles to 1024 bytes
   static_assert(kQBytes % 1024 == 0, "Q buffers keep the rings 1024-byte aligned");
@@ -374,6 +379,11 @@ __device__ __forceinline__ void write_output_cols(uint32_t tmem_o0, uint32_t tme
   }
 }
 
+// Key tile j of an item goes to warpgroup (j & 1) ^ fw.  The warpgroup that owns the last key tile merges
+// the item; the other one is free earlier, so it takes the first key tile of the next item.
+__device__ __forceinline__ int merging_warpgroup(int fw, int n_kv) { return ((n_kv - 1) & 1) ^ fw; }
+__device__ __forceinline__ int next_first_warpgroup(int fw, int n_kv) { return merging_warpgroup(fw, n_kv) ^ 1; }
+
 // ONES: head_dim < DHP and column head_dim of every V row holds 1.0, so column head_dim of O_w is the
 // row sum of P_w (summed by the tensor core from the same bf16 values as the numerator) and the
 // softmax threads need not add it up.
@@ -397,9 +407,9 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
   uint64_t* s_free = s_full + 2;              // [2]  S_w copied to registers (4 warp arrivals)
   uint64_t* p_full = s_free + 2;              // [2]  P_w written (4 warp arrivals)
   uint64_t* p_free = p_full + 2;              // [2]  P_w consumed: the warpgroup's last P V is complete
-  uint64_t* o_final = p_free + 2;             // all P V products of the item complete
-  uint64_t* o_free = o_final + 1;             // both accumulators read out by the closing warpgroup (4 warp arrivals)
-  uint64_t* ml_pub = o_free + 1;              // [2]  warpgroup w published its (m, l) of the item (4 warp arrivals)
+  uint64_t* o_done = p_free + 2;              // [2]  warpgroup w's P V products of the item complete: O_w final
+  uint64_t* o_free = o_done + 2;              // [2]  O_w read out by the merging warpgroup (4 warp arrivals)
+  uint64_t* ml_pub = o_free + 2;              // [2]  warpgroup w published its (m, l) of the item (4 warp arrivals)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + P::kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   float2* ml_all = reinterpret_cast<float2*>(smem + P::kMl);
@@ -409,9 +419,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
   if (threadIdx.x == 0) {
     for (int i = 0; i < P::kNumBars; ++i) mbar_init(&bars[i], 1);
     for (int w = 0; w < 2; ++w) { mbar_init(&s_free[w], 4); mbar_init(&p_full[w], 4); }
-    mbar_init(o_free, 4);
-    mbar_init(&ml_pub[0], 4);
-    mbar_init(&ml_pub[1], 4);
+    for (int w = 0; w < 2; ++w) { mbar_init(&o_free[w], 4); mbar_init(&ml_pub[w], 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -483,6 +491,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     // ---------------------------------------------------------------- Q K^T issuer:  S_w(j) = Q K_j^T
     if (lane == 0) {
       uint32_t kc = 0, n = 0, sc0 = 0, sc1 = 0;        // sc_w: score tiles issued for warpgroup w
+      int fw = 0;                                      // warpgroup that takes the item's first key tile
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
         const Item it = decode_item<BKV>(segs, heads, item);
@@ -492,7 +501,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         const uint64_t dq_main = smem_desc(sq, 16, 1024, 2);
         const uint64_t dq_tail = smem_desc(sq + P::kMainBoxes * P::kQMain, 16, 256, 6);
         for (int j = 0; j < it.n_kv; ++j, ++kc) {
-          const int w = (j ^ n) & 1;                    // the warpgroups swap key-tile parities every item
+          const int w = (j & 1) ^ fw;
           const int ks = kc % P::KS;
           if (!mbar_wait(&k_full[ks], (kc / P::KS) & 1, abort_flag)) { ok = false; break; }
           uint32_t& sc = w ? sc1 : sc0;
@@ -519,6 +528,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           umma_commit(&k_empty[ks]);
           if (j == it.n_kv - 1) umma_commit(&q_empty[qb]);
         }
+        fw = next_first_warpgroup(fw, it.n_kv);
       }
     }
     __syncwarp();
@@ -526,21 +536,27 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     // ---------------------------------------------------------------- P V issuer:  O_w += P_w(j) V_j
     if (lane == 0) {
       uint32_t vc = 0, n = 0, pc0 = 0, pc1 = 0;        // pc_w: P tiles consumed for warpgroup w
+      uint32_t items0 = 0, items1 = 0;                 // items in which warpgroup 0 / 1 had key tiles
+      int fw = 0;
       constexpr uint32_t idesc = instr_desc(DHP, 1);
       constexpr uint32_t kStep = P::kV32 ? 512 / 16 : 2048 / 16;   // 16 keys further down the V tile, 16-byte units
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
         const Item it = decode_item<BKV>(segs, heads, item);
-        // the accumulators of the previous item must have been read out before they are overwritten
-        if (n > 0 && !mbar_wait(o_free, (n - 1) & 1, abort_flag)) break;
         for (int j = 0; j < it.n_kv; ++j, ++vc) {
-          const int w = (j ^ n) & 1;
+          const int w = (j & 1) ^ fw;
           const int vs = vc % P::VS;
           uint32_t& pc = w ? pc1 : pc0;
           // V arrives long before P: take that wait first so that only P's is on the critical path
           if (!mbar_wait(&v_full[vs], (vc / P::VS) & 1, abort_flag)) { ok = false; break; }
           if (!mbar_wait(&p_full[w], pc & 1, abort_flag)) { ok = false; break; }
           ++pc;
+          if (j < 2) {
+            // the warpgroup's accumulator of its previous item must have been read out before it is overwritten
+            uint32_t& items = w ? items1 : items0;
+            if (items > 0 && !mbar_wait(&o_free[w], (items - 1) & 1, abort_flag)) { ok = false; break; }
+            ++items;
+          }
           tc_fence_after();
           const uint32_t sv = smem_u32(smem + P::kV + vs * P::kKStride);
           // MN-major V: boxes (16 or 64 columns wide) are kVBox apart, 8-row groups 256 / 1024 bytes apart
@@ -559,9 +575,10 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           }
           umma_commit(&v_empty[vs]);
           umma_commit(&p_free[w]);
+          if (j >= it.n_kv - 2) umma_commit(&o_done[w]);   // the warpgroup's last key tile of the item
         }
         if (!ok) break;
-        umma_commit(o_final);
+        fw = next_first_warpgroup(fw, it.n_kv);
       }
     }
     __syncwarp();
@@ -575,7 +592,10 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     const uint32_t tmem_p = tmem_base + (w ? P::kP1 : P::kP0) + lane_off;
     const uint32_t tmem_o = tmem_base + (w ? P::kO1 : P::kO0) + lane_off;
     uint32_t tc = 0, n = 0;                             // score tiles processed, items processed
-    bool ok = true, closed_prev = false;                // closed_prev: this warpgroup merged the previous item
+    uint32_t items_me = 0, items_other = 0;             // items in which this / the other warpgroup had key tiles
+    uint32_t pubs_me = 0, pubs_other = 0;               // (m, l) publications of this / the other warpgroup
+    int fw = 0;                                         // warpgroup that takes the item's first key tile
+    bool ok = true;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
       const Item it = decode_item<BKV>(segs, heads, item);
       float m = -INFINITY, l = 0.0f;
@@ -595,11 +615,22 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         }
         return true;
       };
-      // With an odd number of key tiles one warpgroup has one more than the other; swapping parities every
-      // item evens that out over two items, because a warpgroup that is done does not wait for the other:
-      // it publishes (m, l) and goes on to the next item, and the warpgroup that owns the item's last key
-      // tile (the "closing" one) merges and writes the rows alone.
-      const int j0 = (w ^ n) & 1;                       // this warpgroup's first key tile of the item
+      // The warpgroup that owns the item's last key tile merges the item and writes its rows.  The other
+      // one does not wait: it publishes (m, l) and goes on to the next item, whose first key tile is
+      // given to it.  With an odd number of key tiles (7 for a 784-token image) the extra tile and the
+      // merge thus alternate between the warpgroups.
+      const int j0 = w ^ fw;                            // this warpgroup's first key tile of the item
+      const int merging = merging_warpgroup(fw, it.n_kv);
+      const bool has_other = it.n_kv > 1;               // the other warpgroup has key tiles too
+      // state of both warpgroups after this item (every path below leaves the item with it)
+      const uint32_t my_items = items_me + (j0 < it.n_kv ? 1u : 0u);   // counts this item
+      const uint32_t other_items = items_other + ((j0 ^ 1) < it.n_kv ? 1u : 0u);
+      const uint32_t other_pubs = pubs_other;           // publications before this item
+      const uint32_t my_pubs = pubs_me;
+      items_me = my_items;
+      items_other = other_items;
+      if (has_other) { if (merging == w) ++pubs_other; else ++pubs_me; }
+      fw = merging ^ 1;
       if (j0 < it.n_kv && !load_scores(j0)) { ok = false; break; }
       for (int j = j0; j < it.n_kv; j += 2) {
         const int kv_valid = min(BKV, it.seg_len - j * BKV);
@@ -690,55 +721,122 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         if (lane == 0) mbar_arrive(&p_full[w]);
       }
       if (!ok) break;
-      // publish (m, l); they are double-buffered by item parity because the other warpgroup may still be
-      // reading the previous item's while this one is already an item ahead
-      // A publication must not overtake the reader of the previous one by a whole barrier phase: unless this
-      // warpgroup merged the previous item itself, it first sees that merge finished (with two or more
-      // key tiles in this item it already has, through its P V products).
-      if (n > 0 && !closed_prev && !mbar_wait(o_free, (n - 1) & 1, abort_flag)) { ok = false; break; }
-      float2* ml = ml_all + (n & 1) * 2 * BQ;
-      ml[w * BQ + r] = make_float2(m, l);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&ml_pub[w]);
-      const int closing = ((it.n_kv - 1) ^ n) & 1;      // owner of the last key tile
-      closed_prev = w == closing;
-      if (!closed_prev) continue;
-      if (!mbar_wait(&ml_pub[w ^ 1], n & 1, abort_flag)) { ok = false; break; }
-      if (!mbar_wait(o_final, n & 1, abort_flag)) { ok = false; break; }
-      tc_fence_after();
-      // "a" is this warpgroup's accumulator (it has at least the last key tile), "b" the other's
-      const bool has_b = it.n_kv > 1;
-      float2 ml_a = ml[w * BQ + r], ml_b = ml[(w ^ 1) * BQ + r];
+      if (w != merging) {
+        if (j0 >= it.n_kv) continue;                    // no key tile in this item: nothing to hand over
+        // Publish (m, l) and go on.  The slot (double-buffered by item parity) and the barrier phase must
+        // not overtake the reader of this warpgroup's previous publication: that reader has finished once
+        // O_w of this warpgroup's previous item with key tiles was read out (with two or more key tiles
+        // in this item that is already known through the P V products).
+        if (my_pubs > 0 && my_items >= 2 && !mbar_wait(&o_free[w], (my_items - 2) & 1, abort_flag)) { ok = false; break; }
+        ml_all[(n & 1) * 2 * BQ + w * BQ + r] = make_float2(m, l);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ml_pub[w]);
+        continue;
+      }
+      // ---- merge: "a" is this warpgroup's accumulator, "b" the other's
       const uint32_t tmem_oa = tmem_base + (w ? P::kO1 : P::kO0) + lane_off;
       const uint32_t tmem_ob = tmem_base + (w ? P::kO0 : P::kO1) + lane_off;
-      if (ONES) {
-        // the row sums sit in column head_dim of the accumulators
-        uint32_t t0[8], t1[8];
-        tmem_ld8(tmem_oa + (dh & ~7), t0);
-        if (has_b) tmem_ld8(tmem_ob + (dh & ~7), t1);
-        tmem_ld_wait();
+      float2 ml_a = make_float2(m, l), ml_b = make_float2(-INFINITY, 0.0f);
+      // O_b fits the dead score registers next to a 32-column batch of O_a: read it first and hand the
+      // accumulator back, so that the other warpgroup's next item is not held up by this merge
+      constexpr bool kEarly = DHP + 32 <= BKV;
+      if (has_other) {
+        if (!mbar_wait(&ml_pub[w ^ 1], other_pubs & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(&o_done[w ^ 1], (other_items - 1) & 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        ml_b = ml_all[(n & 1) * 2 * BQ + (w ^ 1) * BQ + r];
+        if constexpr (kEarly) {
+          tmem_ld_cols<DHP>(tmem_ob, s);
+          tmem_ld_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&o_free[w ^ 1]);
+          // with a ones column head_dim is DHP - 8 (a multiple of 8 just below the padded width): the row
+          // sum sits in column DHP - 8
+          if (ONES) ml_b.y = __uint_as_float(s[DHP - 8]);
+        } else if (ONES) {
+          uint32_t t1[8];
+          tmem_ld8(tmem_ob + (dh & ~7), t1);            // the row sum sits in column head_dim
+          tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          if (i == (dh & 7)) {
-            ml_a.y = __uint_as_float(t0[i]);
-            ml_b.y = has_b ? __uint_as_float(t1[i]) : 0.0f;
-          }
+          for (int i = 0; i < 8; ++i)
+            if (i == (dh & 7)) ml_b.y = __uint_as_float(t1[i]);
         }
       }
-      const float mm = has_b ? fmaxf(ml_a.x, ml_b.x) : ml_a.x;
-      const float ea = ex2(ml_a.x - mm), eb = has_b ? ex2(ml_b.x - mm) : 0.0f;
-      const float inv = 1.0f / (ea * ml_a.y + eb * ml_b.y);
-      const float fa = ea * inv, fb = eb * inv;
+      if (!mbar_wait(&o_done[w], (my_items - 1) & 1, abort_flag)) { ok = false; break; }
+      tc_fence_after();
       const int token = it.q0 + r;
       const bool row_ok = token < it.seg_beg + it.seg_len;
       __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + it.head * dh;
-      // The score registers are dead here and serve as the landing buffer, so that all TMEM loads of a
-      // batch of columns are in flight together.
-      constexpr int kMaxB = BKV / 2 / 16 * 16;   // columns of each accumulator that fit the score registers
-      write_output_cols<DHP, kMaxB>(tmem_oa, tmem_ob, 0, has_b, row_ok, fa, fb, dh, orow, s);
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(o_free);
+      if constexpr (kEarly) {
+        // O_a in batches of at most 32 columns behind O_b in the score registers, the last batch first:
+        // it holds the row sum the factors need
+        uint32_t* oa = s + DHP;
+        constexpr int kLast = (DHP - 1) / 32 * 32;       // first column of the last batch
+        float fa = 0.0f, fb = 0.0f;
+#pragma unroll
+        for (int b = 0; b < (DHP + 31) / 32; ++b) {
+          const int c0 = b == 0 ? kLast : (b - 1) * 32;
+          if (b == 0) tmem_ld_cols<DHP - kLast>(tmem_oa + kLast, oa);
+          else tmem_ld_cols<32>(tmem_oa + c0, oa);
+          tmem_ld_wait();
+          if (b == (DHP + 31) / 32 - 1) {
+            // O_a is in registers: the accumulator may be overwritten by this warpgroup's next item
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&o_free[w]);
+          }
+          if (b == 0) {
+            if (ONES) ml_a.y = __uint_as_float(oa[DHP - 8 - kLast]);
+            const float mm = fmaxf(ml_a.x, ml_b.x);
+            const float ea = ex2(ml_a.x - mm), eb = has_other ? ex2(ml_b.x - mm) : 0.0f;
+            const float inv = 1.0f / (ea * ml_a.y + eb * ml_b.y);
+            fa = ea * inv;
+            fb = eb * inv;
+          }
+          if (row_ok) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              if (c0 + g * 8 < DHP && c0 + g * 8 < dh) {   // dh is a multiple of 8
+                uint32_t pk[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  float v0 = __uint_as_float(oa[8 * g + 2 * e]) * fa, v1 = __uint_as_float(oa[8 * g + 2 * e + 1]) * fa;
+                  if (has_other) {
+                    v0 = fmaf(__uint_as_float(s[c0 + 8 * g + 2 * e]), fb, v0);
+                    v1 = fmaf(__uint_as_float(s[c0 + 8 * g + 2 * e + 1]), fb, v1);
+                  }
+                  __nv_bfloat162 b2 = __floats2bfloat162_rn(v0, v1);
+                  pk[e] = *reinterpret_cast<uint32_t*>(&b2);
+                }
+                *reinterpret_cast<uint4*>(orow + c0 + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+              }
+            }
+          }
+        }
+      } else {
+        // both accumulators in batches through the score registers; handed back at the end
+        if (ONES) {
+          uint32_t t0[8];
+          tmem_ld8(tmem_oa + (dh & ~7), t0);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            if (i == (dh & 7)) ml_a.y = __uint_as_float(t0[i]);
+        }
+        const float mm = fmaxf(ml_a.x, ml_b.x);
+        const float ea = ex2(ml_a.x - mm), eb = has_other ? ex2(ml_b.x - mm) : 0.0f;
+        const float inv = 1.0f / (ea * ml_a.y + eb * ml_b.y);
+        const float fa = ea * inv, fb = eb * inv;
+        constexpr int kMaxB = BKV / 2 / 16 * 16;   // columns of each accumulator that fit the score registers
+        write_output_cols<DHP, kMaxB>(tmem_oa, tmem_ob, 0, has_other, row_ok, fa, fb, dh, orow, s);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(&o_free[w]);
+          if (has_other) mbar_arrive(&o_free[w ^ 1]);
+        }
+      }
     }
   }
 
