@@ -384,6 +384,20 @@ __device__ __forceinline__ void write_output_cols(uint32_t tmem_o0, uint32_t tme
 __device__ __forceinline__ int merging_warpgroup(int fw, int n_kv) { return ((n_kv - 1) & 1) ^ fw; }
 __device__ __forceinline__ int next_first_warpgroup(int fw, int n_kv) { return merging_warpgroup(fw, n_kv) ^ 1; }
 
+// Order in which the two issuing threads walk an item's key tiles: 0, 2, 1, 4, 3, 6, 5, ... for items of
+// at most 32 key tiles, 0, 1, 2, ... for longer ones.
+// The warpgroup that takes tile 0 is the one that did not merge the previous item; giving it its first
+// tiles one step early lets it work through three of them while the other warpgroup is still merging
+// (with the plain order 0, 1, 2, ... it stalls after one, behind the first product the merging
+// warpgroup is not ready for).  Each warpgroup still sees its own tiles in ascending order.  Measured:
+// 8 x 784 tokens 378 -> 393 TFLOP/s, 16 x 1024 tokens 456 -> 471; a 16384-token segment, where item
+// boundaries are rare, lost 1 % in that order and keeps the plain one.
+__device__ __forceinline__ int issue_order(int i, int n_kv) {
+  if (i == 0 || n_kv > 32) return i;
+  const int j = (i & 1) ? i + 1 : i - 1;
+  return j < n_kv ? j : i;
+}
+
 // ONES: head_dim < DHP and column head_dim of every V row holds 1.0, so column head_dim of O_w is the
 // row sum of P_w (summed by the tensor core from the same bf16 values as the numerator) and the
 // softmax threads need not add it up.
@@ -500,10 +514,12 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         const uint32_t sq = smem_u32(smem + P::kQ + qb * P::kQBytes);
         const uint64_t dq_main = smem_desc(sq, 16, 1024, 2);
         const uint64_t dq_tail = smem_desc(sq + P::kMainBoxes * P::kQMain, 16, 256, 6);
-        for (int j = 0; j < it.n_kv; ++j, ++kc) {
+        for (int i = 0; i < it.n_kv; ++i) {
+          const int j = issue_order(i, it.n_kv);
+          const uint32_t kt = kc + j;                   // the tile's number in the K ring
           const int w = (j & 1) ^ fw;
-          const int ks = kc % P::KS;
-          if (!mbar_wait(&k_full[ks], (kc / P::KS) & 1, abort_flag)) { ok = false; break; }
+          const int ks = kt % P::KS;
+          if (!mbar_wait(&k_full[ks], (kt / P::KS) & 1, abort_flag)) { ok = false; break; }
           uint32_t& sc = w ? sc1 : sc0;
           // the warpgroup must have copied its previous score tile out of S_w
           if (sc > 0 && !mbar_wait(&s_free[w], (sc - 1) & 1, abort_flag)) { ok = false; break; }
@@ -526,8 +542,9 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           if (P::kTail) umma_ss(tmem_s, dq_tail, dk_tail, idesc, 1);
           umma_commit(&s_full[w]);
           umma_commit(&k_empty[ks]);
-          if (j == it.n_kv - 1) umma_commit(&q_empty[qb]);
+          if (i == it.n_kv - 1) umma_commit(&q_empty[qb]);
         }
+        kc += it.n_kv;
         fw = next_first_warpgroup(fw, it.n_kv);
       }
     }
@@ -543,12 +560,14 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
       bool ok = true;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
         const Item it = decode_item<BKV>(segs, heads, item);
-        for (int j = 0; j < it.n_kv; ++j, ++vc) {
+        for (int i = 0; i < it.n_kv; ++i) {
+          const int j = issue_order(i, it.n_kv);
+          const uint32_t vt = vc + j;                   // the tile's number in the V ring
           const int w = (j & 1) ^ fw;
-          const int vs = vc % P::VS;
+          const int vs = vt % P::VS;
           uint32_t& pc = w ? pc1 : pc0;
           // V arrives long before P: take that wait first so that only P's is on the critical path
-          if (!mbar_wait(&v_full[vs], (vc / P::VS) & 1, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(&v_full[vs], (vt / P::VS) & 1, abort_flag)) { ok = false; break; }
           if (!mbar_wait(&p_full[w], pc & 1, abort_flag)) { ok = false; break; }
           ++pc;
           if (j < 2) {
@@ -578,6 +597,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           if (j >= it.n_kv - 2) umma_commit(&o_done[w]);   // the warpgroup's last key tile of the item
         }
         if (!ok) break;
+        vc += it.n_kv;
         fw = next_first_warpgroup(fw, it.n_kv);
       }
     }
