@@ -22,12 +22,12 @@
 // (zero fill on loads, clipping on stores).  No load in this file is a multicast load.
 //
 // RMSNorm folded into the neighbouring linear layers (NORM):
-//   NORM = 1, residual update  x += a w^T + b  whose result feeds an RMSNorm: the epilogue reads the old
-//     x tile, adds, stores the new x (fp32) and, from the same registers, xg = bf16(x_new * gain[col]) and
-//     the tile's contribution to each row's sum of squares, partials[row][2 * n_tile + half] (one
-//     writer per entry: the row statistics are bit-reproducible).  Plain loads and stores of 128-byte
-//     row pieces, 8 lanes per row; the old values of the next 32-column chunk are in flight while the
-//     current one is processed.
+//   NORM = 1, residual update  x += a w^T + b  whose result feeds an RMSNorm: besides the reduce-add of the
+//     staged chunk into x, the epilogue reads the old x values (plain loads of 128-byte row pieces, 8 lanes
+//     per row, in flight during the accumulator read), forms the new x in registers and writes
+//     xg = bf16(x_new * gain[col]) and the tile's contribution to each row's sum of squares,
+//     partials[row][2 * n_tile + half] (one writer per entry: the row statistics are bit-reproducible).
+//     The reduce-add is issued after the old values have arrived.
 //   NORM = 2, the consumer  y = act(RMSNorm(x) w^T + b) = act(rinv[row] * (xg w^T) + b): the epilogue
 //     multiplies its accumulator row by rinv = 1 / sqrt(sum(partials[row][:]) / h + eps).
 // The separate normalisation pass (read 4 bytes, write 2 per element, ~12 us per call at 6272 x 1152) and
@@ -519,7 +519,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           if (lane == 0) mbar_arrive_cluster(tmem_empty_leader0 + acc * 8);
         }
         // the staging buffer is free once the bulk store issued from it has read it
-        if (!ROPE && NORM != 1 && lane == 0) bulk_wait_read_all();
+        if (!ROPE && lane == 0) bulk_wait_read_all();
         __syncwarp();
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -561,8 +561,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             if (col_ok && row0 + r < M) {
               const float4 t = *reinterpret_cast<const float4*>(sbuf + r * 128 + ((piece ^ (r & 7)) << 4));
               const float4 o = old_cur[it];
+              // the new x: memory receives the same sum through the reduce-add issued below
               const float4 xn = make_float4(o.x + t.x, o.y + t.y, o.z + t.z, o.w + t.w);
-              *reinterpret_cast<float4*>(out_f32 + (long long)(row0 + r) * ldo + col) = xn;
               const __nv_bfloat162 g01 = __floats2bfloat162_rn(xn.x * gain_cur[0], xn.y * gain_cur[1]);
               const __nv_bfloat162 g23 = __floats2bfloat162_rn(xn.z * gain_cur[2], xn.w * gain_cur[3]);
               *reinterpret_cast<uint2*>(nm.xg + (long long)(row0 + r) * N + col) =
@@ -583,6 +583,13 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
               const int r = row0 + it * 4 + (lane >> 3);
               if (piece == 0 && r < M) nm.partials[(long long)r * nm.n_parts + part] = ss;
             }
+          }
+          // x += staged chunk in L2; only now, when the old values have arrived in registers
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) {
+            if (row0 < M && n0 + c * CC < N) tma_reduce_add_2d(&tm_out, n0 + c * CC, row0, sbuf);
+            bulk_commit();
           }
           continue;
         }
@@ -788,15 +795,16 @@ cudaError_t linear_tc_pair_residual_norm(const void* a, int64_t lda, const void*
                                          float* x, int64_t ldo, int64_t M, int64_t N, int64_t K, const void* gain,
                                          void* xg, float* row_partials, int* status, cudaStream_t s) {
   constexpr int BN = 256;
-  CUtensorMap ta, tw;
-  if (!make_map(&ta, a, M, K, lda, BM, 2) || !make_map(&tw, w, N, K, ldw, BN / 2, 2)) return cudaErrorInvalidValue;
+  CUtensorMap ta, tw, to;
+  if (!make_map(&ta, a, M, K, lda, BM, 2) || !make_map(&tw, w, N, K, ldw, BN / 2, 2) || !make_map(&to, x, M, N, ldo, 32, 4))
+    return cudaErrorInvalidValue;
   if ((ldo % 4) || (N % 8) || ((uintptr_t)x & 15) || ((uintptr_t)xg & 15) || ((uintptr_t)gain & 7)) return cudaErrorInvalidValue;
   NormArgs nm{};
   nm.partials = row_partials;
   nm.n_parts = norm_parts(N);
   nm.xg = static_cast<__nv_bfloat16*>(xg);
   nm.gain = static_cast<const __nv_bfloat16*>(gain);
-  return launch<BN, 5, float, 0, true, false, 1>(ta, tw, ta, bias, (int)M, (int)N, (int)K, status, s, RopeSplitArgs{}, nm, x,
+  return launch<BN, 5, float, 0, true, false, 1>(ta, tw, to, bias, (int)M, (int)N, (int)K, status, s, RopeSplitArgs{}, nm, x,
                                                  ldo);
 }
 
