@@ -771,6 +771,37 @@ int epd_op_qkv_rope(const void* x, int64_t ldx, const void* w_prepared, const vo
   return EPD_OK;
 }
 
+int32_t epd_norm_parts(int64_t N) { return N > 0 ? norm_parts(N) : 0; }
+
+int epd_op_linear_residual_norm(const void* a, int64_t lda, const void* w, int64_t ldw, const void* bias, float* x,
+                                int64_t ldx, int64_t M, int64_t N, int64_t K, const void* gain, void* xg,
+                                float* row_partials, void* stream) {
+  if (M < 0 || N < 1 || K < 1 || M > (1 << 30) || lda < K || ldw < K || ldx < N) return EPD_EINVAL;
+  if (M == 0) return EPD_OK;
+  if (!a || !w || !x || !gain || !xg || !row_partials) return EPD_EINVAL;
+  if ((lda % 8) || (ldw % 8) || (ldx % 4) || (N % 8)) return EPD_EINVAL;
+  if (((uintptr_t)a | (uintptr_t)w | (uintptr_t)x | (uintptr_t)xg) & 15) return EPD_EINVAL;
+  if (((uintptr_t)gain & 7) || ((uintptr_t)row_partials & 3) || ((uintptr_t)bias & 1)) return EPD_EINVAL;
+  EPD_CUDA(linear_tc_pair_residual_norm(a, lda, w, ldw, bias, x, ldx, M, N, K, gain, xg, row_partials, nullptr,
+                                        static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int epd_op_linear_normed(const void* xg, int64_t ldxg, const void* w, int64_t ldw, const void* bias, void* out,
+                         int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t flags, const float* row_partials,
+                         int32_t n_parts, float eps, void* stream) {
+  if (M < 0 || N < 1 || K < 1 || M > (1 << 30) || ldxg < K || ldw < K || ldo < N || n_parts < 1 || !(eps >= 0.0f))
+    return EPD_EINVAL;
+  if (M == 0) return EPD_OK;
+  if (!xg || !w || !out || !row_partials) return EPD_EINVAL;
+  if ((ldxg % 8) || (ldw % 8) || (ldo % 8) || (N % 8)) return EPD_EINVAL;
+  if (((uintptr_t)xg | (uintptr_t)w | (uintptr_t)out) & 15) return EPD_EINVAL;
+  if (flags & ~(EPD_LINEAR_GELU_TANH | EPD_LINEAR_GELU_ERF)) return EPD_EINVAL;
+  EPD_CUDA(linear_tc_pair_normed(xg, ldxg, w, ldw, bias, out, ldo, M, N, K, flags, row_partials, n_parts, eps, nullptr,
+                                 static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
 int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
                      const int32_t* host_cu_seqlens, int32_t n_seg, void* out, int64_t T, int32_t heads,
                      int32_t head_dim, int32_t flags, void* stream) {
