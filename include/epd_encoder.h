@@ -305,24 +305,6 @@ int epd_op_patchify(int32_t dtype, const void* frames, const int64_t* item_offse
 int epd_op_merge(int32_t dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm,
                  int32_t hidden, void* stream);
 
-/* RMSNorm folded into the linear layers around it (bf16 tensor-core path; what the encoder runs for
- * batches of more than 128 tokens).  For a residual update whose result feeds an RMSNorm,
- *   epd_op_linear_residual_norm:  x[M,N] (float, leading dimension ldx) += a[M,K] . w[N,K]^T + bias, and from
- *     the new x: xg[M,N] = bf16(x * gain[col]) (contiguous) and row_partials[M, epd_norm_parts(N)] (float), whose
- *     sum over a row is the row's sum of squares (one 128-column half tile per entry, fixed order: the
- *     statistics are bit-reproducible);
- *   epd_op_linear_normed:  out[M,N] (bf16) = act(rinv[row] * (xg . w^T) + bias) with
- *     rinv = 1 / sqrt(sum(row_partials[row, :n_parts]) / K + eps), which equals act(RMSNorm(x) . w^T + bias)
- *     for the x, gain that produced xg.  flags: 0, EPD_LINEAR_GELU_TANH or EPD_LINEAR_GELU_ERF.
- * All pointers device, 16-byte aligned (gain 8-byte); lda, ldw, ldxg, ldo multiples of 8, ldx of 4, N of 8. */
-int32_t epd_norm_parts(int64_t N);
-int epd_op_linear_residual_norm(const void* a, int64_t lda, const void* w, int64_t ldw, const void* bias, float* x,
-                                int64_t ldx, int64_t M, int64_t N, int64_t K, const void* gain, void* xg,
-                                float* row_partials, void* stream);
-int epd_op_linear_normed(const void* xg, int64_t ldxg, const void* w, int64_t ldw, const void* bias, void* out,
-                         int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t flags, const float* row_partials,
-                         int32_t n_parts, float eps, void* stream);
-
 /* ------------------------------------------------------------------------------------------
  * After the stage: feature keys and a feature cache (the encoder's side of the multimodal store of
  * Section 3.2, "Asynchronous Feature Prefetching": features are kept under a hash of the input so

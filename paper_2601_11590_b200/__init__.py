@@ -29,7 +29,7 @@ EXPORTED_SYMBOLS = [
     "epd_debug_profile_class_name", "epd_debug_profile_read", "epd_op_linear", "epd_op_rmsnorm", "epd_op_rope_split",
     "epd_padded_head_dim", "epd_op_attention", "epd_op_merge", "epd_op_rope_attention_static",
     "epd_static_scratch_bytes", "epd_last_cuda_error", "epd_encode_frames", "epd_op_patchify",
-    "epd_norm_parts", "epd_op_linear_residual_norm", "epd_op_linear_normed", "epd_op_qkv_prepare", "epd_op_rope_table", "epd_op_qkv_pad_init", "epd_op_qkv_rope",
+    "epd_op_qkv_prepare", "epd_op_rope_table", "epd_op_qkv_pad_init", "epd_op_qkv_rope",
     "epd_op_content_hash", "epd_feature_cache_create", "epd_feature_cache_destroy",
     "epd_feature_cache_lookup", "epd_feature_cache_insert", "epd_feature_cache_stats",
 ]
@@ -92,12 +92,6 @@ def load_library() -> ctypes.CDLL:
     lib.epd_encode_frames.argtypes = [vp, vp, i32p, i32, f32p, f32p, vp, i64, i64p, i32p, vp]
     lib.epd_op_patchify.restype = ctypes.c_int
     lib.epd_op_patchify.argtypes = [i32, vp, vp, vp, vp, i32, i64, vp, i64, i32, i32, i32, f32p, f32p, vp]
-    lib.epd_norm_parts.restype = i32
-    lib.epd_norm_parts.argtypes = [i64]
-    lib.epd_op_linear_residual_norm.restype = ctypes.c_int
-    lib.epd_op_linear_residual_norm.argtypes = [vp, i64, vp, i64, vp, vp, i64, i64, i64, i64, vp, vp, vp, vp]
-    lib.epd_op_linear_normed.restype = ctypes.c_int
-    lib.epd_op_linear_normed.argtypes = [vp, i64, vp, i64, vp, vp, i64, i64, i64, i64, i32, vp, i32, ctypes.c_float, vp]
     lib.epd_op_qkv_prepare.restype = ctypes.c_int
     lib.epd_op_qkv_prepare.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp]
     lib.epd_op_rope_table.restype = ctypes.c_int
@@ -497,34 +491,6 @@ def op_patchify(dtype, frames_dev, item_off, grid_thw, cu_seqlens, in_channels, 
     cu_d = torch.from_numpy(np.asarray(cu_seqlens, dtype=np.int32)).cuda()
     _check(lib.epd_op_patchify(dtype, _ptr(frames_dev), _ptr(off_d), _ptr(g_d), _ptr(cu_d), n, T, _ptr(out), ld,
                                in_channels, patch, temporal_patch, m, istd, _stream_ptr(stream)), "epd_op_patchify")
-    return out
-
-
-def op_linear_residual_norm(a, w, bias, x, gain, stream=None):
-    """x (float [M, N], updated in place) += a w^T + bias; returns (xg bf16 [M, N], row_partials float [M, parts])."""
-    torch = _torch()
-    lib = load_library()
-    M, K = a.shape
-    N = w.shape[0]
-    parts = int(lib.epd_norm_parts(N))
-    xg = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
-    partials = torch.full((M, parts), -1.0, dtype=torch.float32, device="cuda")
-    _check(lib.epd_op_linear_residual_norm(_ptr(a), a.stride(0), _ptr(w), w.stride(0), _ptr(bias), _ptr(x), x.stride(0),
-                                           M, N, K, _ptr(gain), _ptr(xg), _ptr(partials), _stream_ptr(stream)),
-           "epd_op_linear_residual_norm")
-    return xg, partials
-
-
-def op_linear_normed(xg, w, bias, partials, eps, flags=0, stream=None):
-    """bf16 [M, N] = act(rinv[row] * (xg w^T) + bias), rinv from the row partials."""
-    torch = _torch()
-    lib = load_library()
-    M, K = xg.shape
-    N = w.shape[0]
-    out = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
-    _check(lib.epd_op_linear_normed(_ptr(xg), xg.stride(0), _ptr(w), w.stride(0), _ptr(bias), _ptr(out), out.stride(0),
-                                    M, N, K, flags, _ptr(partials), partials.shape[1], eps, _stream_ptr(stream)),
-           "epd_op_linear_normed")
     return out
 
 

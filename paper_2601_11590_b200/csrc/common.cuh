@@ -64,8 +64,6 @@ cudaError_t linear_fma(int dtype, const void* x, int64_t ldx, const void* w, int
                        void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, cudaStream_t s);
 cudaError_t rmsnorm(int dtype, const void* x, const void* gain, void* out, const int32_t* dst_row, int64_t T,
                     int hidden, float eps, cudaStream_t s);
-cudaError_t rmsnorm_prepare(const float* x, const void* gain, void* xg, float* partials, int n_parts, int64_t T,
-                            int hidden, cudaStream_t s);
 cudaError_t rope_split(int dtype, const void* qkv, const int32_t* pos_row, const int32_t* pos_col,
                        const float2* table, int table_rows, void* q, void* k, void* v, int64_t T, int heads,
                        int head_dim, float theta, float q_scale, cudaStream_t s);
@@ -106,18 +104,7 @@ cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ld
 cudaError_t linear_tc_pair_qkv(const void* x, int64_t ldx, const void* w_perm, int64_t ldw, const void* bias_perm,
                                void* q, void* k, void* v, const int32_t* pos_row, const int32_t* pos_col,
                                const float2* table, int table_rows, int64_t M, int heads, int head_dim, float q_scale,
-                               const float* row_partials, int n_parts, float eps, int* status, cudaStream_t s);
-// RMSNorm folded into the neighbouring linear layers.  linear_tc_pair_residual_norm: x += a w^T + bias
-// (x float [M, N]), and from the new x: xg = bf16(x * gain) [M, N] and row_partials [M, norm_parts(N)] whose
-// sum over a row is the row's sum of squares.  linear_tc_pair_normed (and linear_tc_pair_qkv with
-// row_partials != NULL) then compute act(rinv[row] * (xg w^T) + bias) with rinv = 1 / sqrt(sum / K + eps).
-int norm_parts(int64_t N);
-cudaError_t linear_tc_pair_residual_norm(const void* a, int64_t lda, const void* w, int64_t ldw, const void* bias,
-                                         float* x, int64_t ldo, int64_t M, int64_t N, int64_t K, const void* gain,
-                                         void* xg, float* row_partials, int* status, cudaStream_t s);
-cudaError_t linear_tc_pair_normed(const void* xg, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
-                                  int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, const float* row_partials,
-                                  int n_parts, float eps, int* status, cudaStream_t s);
+                               int* status, cudaStream_t s);
 cudaError_t qkv_permute(const void* w, int64_t ldw, const void* bias, void* w_out, void* bias_out, int heads,
                         int head_dim, cudaStream_t s);
 cudaError_t qkv_pad_init(void* q, void* k, void* v, int64_t rows, int head_dim, cudaStream_t s);

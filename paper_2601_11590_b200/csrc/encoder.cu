@@ -22,7 +22,6 @@ struct Layout {
   size_t x, a, qkv, qh, kh, vh, u, merged, proj_hidden, stage_patches, stage_features, pix_patches;
   size_t grid, cu, cu_out, item_off, pos_row, pos_col, merge_slot, merge_idx, rope, status, aux, total;
   size_t qkv_perm_w, qkv_perm_b;   // per layer: QKV weight / bias with q and k rows in rotation-pair order
-  size_t norm_partials;            // [max_tokens, norm_parts(hidden)] row sums of squares (RMSNorm folded into the linears)
 };
 
 // The QKV projection can apply the rotary embedding and the head split in its epilogue.
@@ -78,7 +77,6 @@ Layout make_layout(const epd_config_t& c) {
   L.rope = take((size_t)c.max_grid * (c.head_dim / 4) * sizeof(float2));
   L.status = take(256);
   const bool fused = fused_rope_possible(c);
-  L.norm_partials = take(fused ? T * (size_t)norm_parts(c.hidden) * sizeof(float) : 0);
   L.qkv_perm_w = take(fused ? (size_t)c.layers * 3 * h * h * es : 0);
   L.qkv_perm_b = take(fused ? (size_t)c.layers * align_up(3 * h * es, 256) : 0);
   L.aux = take(0);
@@ -113,7 +111,6 @@ struct epd_encoder {
   size_t prof_used = 0;
   bool use_tc = false;
   bool fused_rope = false;         // QKV epilogue does rotary + split (batches of more than 128 tokens)
-  bool fused_norm = false;         // and both RMSNorms of a block are folded into the linear layers around them
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -222,53 +219,12 @@ int prepare_batch(epd_encoder* enc, const int32_t* grid_thw, int32_t n, int64_t 
   return EPD_OK;
 }
 
-int attention_dispatch(epd_encoder* enc, int64_t T, int n_seg, void* out, cudaStream_t s) {
+int attention_dispatch(epd_encoder* enc, int64_t T, int n_seg, cudaStream_t s) {
   const epd_config_t& c = enc->cfg;
   EPD_MARK(KC_ATTENTION);
   EPD_CUDA(attention_any(c.dtype, enc->at<void>(enc->lay.qh), enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh),
-                         enc->at<int32_t>(enc->lay.cu), enc->host_cu.data(), n_seg, out, T,
+                         enc->at<int32_t>(enc->lay.cu), enc->host_cu.data(), n_seg, enc->at<void>(enc->lay.a), T,
                          c.heads, c.head_dim, 0, enc->at<int>(enc->lay.status), s));
-  return EPD_OK;
-}
-
-// Block l with both RMSNorms folded into the linear layers around them (bf16, more than 128 tokens).
-// prepared: the producer of x (patch embedding or the previous block's fc2) has already left
-// xg = bf16(x * norm1 gain) in `a` and the row sums of squares in the partials buffer.
-int run_block_fused(epd_encoder* enc, int l, float* x, int64_t T, int n_seg, bool prepared, cudaStream_t s) {
-  const epd_config_t& c = enc->cfg;
-  const int h = c.hidden, m = c.mlp;
-  void* a = enc->at<void>(enc->lay.a);
-  void* att = enc->at<void>(enc->lay.qkv);           // the [T, 3h] buffer is free in this path: attention output
-  void* u = enc->at<void>(enc->lay.u);
-  float* partials = enc->at<float>(enc->lay.norm_partials);
-  int* status = enc->at<int>(enc->lay.status);
-  const int np = norm_parts(h);
-  const int gelu = c.act == EPD_ACT_GELU_TANH ? EPD_LINEAR_GELU_TANH : EPD_LINEAR_GELU_ERF;
-  const size_t hh = (size_t)h;
-  int rc;
-  if (!prepared) {
-    EPD_MARK(KC_RMSNORM);
-    EPD_CUDA(rmsnorm_prepare(x, enc->norm1_w[l], a, partials, np, T, h, s));
-  }
-  EPD_MARK(KC_QKV);
-  const float q_scale = 1.4426950408889634f / sqrtf((float)c.head_dim);
-  EPD_CUDA(linear_tc_pair_qkv(a, h, enc->ws + enc->lay.qkv_perm_w + (size_t)l * 3 * hh * hh * 2, h,
-                              enc->ws + enc->lay.qkv_perm_b + (size_t)l * align_up(3 * hh * 2, 256),
-                              enc->at<void>(enc->lay.qh), enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh),
-                              enc->at<int32_t>(enc->lay.pos_row), enc->at<int32_t>(enc->lay.pos_col),
-                              enc->at<float2>(enc->lay.rope), c.max_grid, T, c.heads, c.head_dim, q_scale, partials, np,
-                              c.eps, status, s));
-  if ((rc = attention_dispatch(enc, T, n_seg, att, s))) return rc;
-  EPD_MARK(KC_OUT);
-  EPD_CUDA(linear_tc_pair_residual_norm(att, h, enc->out_w[l], h, enc->out_b[l], x, h, T, h, h, enc->norm2_w[l], a,
-                                        partials, status, s));
-  EPD_MARK(KC_FC1);
-  EPD_CUDA(linear_tc_pair_normed(a, h, enc->fc1_w[l], h, enc->fc1_b[l], u, m, T, m, h, gelu, partials, np, c.eps, status,
-                                 s));
-  EPD_MARK(KC_FC2);
-  const void* next_gain = l + 1 < c.layers ? enc->norm1_w[l + 1] : enc->norm1_w[l];   // unused after the last block
-  EPD_CUDA(linear_tc_pair_residual_norm(u, m, enc->fc2_w[l], m, enc->fc2_b[l], x, h, T, h, m, next_gain, a, partials,
-                                        status, s));
   return EPD_OK;
 }
 
@@ -277,7 +233,6 @@ int run_block(epd_encoder* enc, int l, float* x, int64_t T, int n_seg, cudaStrea
   const epd_config_t& c = enc->cfg;
   const int h = c.hidden, m = c.mlp;
   const int dt = c.dtype;
-  if (enc->fused_norm && T > 128) return run_block_fused(enc, l, x, T, n_seg, false, s);
   void* a = enc->at<void>(enc->lay.a);
   void* qkv = enc->at<void>(enc->lay.qkv);
   void* u = enc->at<void>(enc->lay.u);
@@ -294,8 +249,8 @@ int run_block(epd_encoder* enc, int l, float* x, int64_t T, int n_seg, cudaStrea
                                 enc->ws + enc->lay.qkv_perm_b + (size_t)l * align_up(3 * hh * 2, 256),
                                 enc->at<void>(enc->lay.qh), enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh),
                                 enc->at<int32_t>(enc->lay.pos_row), enc->at<int32_t>(enc->lay.pos_col),
-                                enc->at<float2>(enc->lay.rope), c.max_grid, T, c.heads, c.head_dim, q_scale, nullptr, 0,
-                                0.0f, enc->at<int>(enc->lay.status), s));
+                                enc->at<float2>(enc->lay.rope), c.max_grid, T, c.heads, c.head_dim, q_scale,
+                                enc->at<int>(enc->lay.status), s));
   } else {
     if ((rc = linear_dispatch(enc, dt, a, h, enc->qkv_w[l], h, enc->qkv_b[l], qkv, 3 * h, T, 3 * h, h, 0, s)))
       return rc;
@@ -305,7 +260,7 @@ int run_block(epd_encoder* enc, int l, float* x, int64_t T, int n_seg, cudaStrea
                         enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh), T, c.heads, c.head_dim, c.rope_theta,
                         q_scale, s));
   }
-  if ((rc = attention_dispatch(enc, T, n_seg, a, s))) return rc;
+  if ((rc = attention_dispatch(enc, T, n_seg, s))) return rc;
   EPD_MARK(KC_OUT);
   if ((rc = linear_dispatch(enc, dt, a, h, enc->out_w[l], h, enc->out_b[l], x, h, T, h, h, EPD_LINEAR_ACCUMULATE, s)))
     return rc;
@@ -346,24 +301,14 @@ int encode_device(epd_encoder* enc, const void* patches, int64_t patches_ld, con
   float* x = enc->at<float>(enc->lay.x);
 
   // patch embedding -> float residual stream
-  const bool fused = enc->fused_norm && T > 128;
   EPD_MARK(KC_PATCH);
-  if (fused) {
-    // as a residual update of a zeroed stream, so that it also prepares block 0's first RMSNorm
-    EPD_CUDA(cudaMemsetAsync(x, 0, (size_t)T * h * 4, s));
-    EPD_CUDA(linear_tc_pair_residual_norm(patches, patches_ld, enc->w.patch_w, enc->w.patch_w_ld, enc->w.patch_b, x, h, T,
-                                          h, enc->patch_dim, enc->norm1_w[0], enc->at<void>(enc->lay.a),
-                                          enc->at<float>(enc->lay.norm_partials), enc->at<int>(enc->lay.status), s));
-  } else if ((rc = linear_dispatch(enc, dt, patches, patches_ld, enc->w.patch_w, enc->w.patch_w_ld, enc->w.patch_b, x, h,
-                                   T, h, enc->patch_dim, EPD_LINEAR_OUT_F32, s))) {
+  if ((rc = linear_dispatch(enc, dt, patches, patches_ld, enc->w.patch_w, enc->w.patch_w_ld, enc->w.patch_b, x, h, T,
+                            h, enc->patch_dim, EPD_LINEAR_OUT_F32, s)))
     return rc;
-  }
   for (int l = 0; l < c.layers; ++l) {
     if (!enc->taps.empty() && enc->taps[l])
       EPD_CUDA(cudaMemcpyAsync(enc->taps[l], x, (size_t)T * h * 4, cudaMemcpyDeviceToDevice, s));
-    if (fused) rc = run_block_fused(enc, l, x, T, n, true, s);
-    else rc = run_block(enc, l, x, T, n, s);
-    if (rc) return rc;
+    if ((rc = run_block(enc, l, x, T, n, s))) return rc;
   }
   if (!enc->taps.empty() && enc->taps[c.layers])
     EPD_CUDA(cudaMemcpyAsync(enc->taps[c.layers], x, (size_t)T * h * 4, cudaMemcpyDeviceToDevice, s));
@@ -478,14 +423,6 @@ int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, vo
   e->fused_rope = fused_rope_possible(*cfg);
   for (int l = 0; l < L && e->fused_rope; ++l)
     if (((uintptr_t)e->qkv_w[l] & 15) || (e->qkv_b[l] && ((uintptr_t)e->qkv_b[l] & 1))) e->fused_rope = false;
-  // RMSNorm folded into the linear layers: every operand the pair kernel reads must be aligned for it
-  e->fused_norm = e->fused_rope && !((uintptr_t)weights->patch_w & 15) && (weights->patch_w_ld % 8 == 0);
-  for (int l = 0; l < L && e->fused_norm; ++l) {
-    const uintptr_t w16 = (uintptr_t)e->out_w[l] | (uintptr_t)e->fc1_w[l] | (uintptr_t)e->fc2_w[l];
-    const uintptr_t g8 = (uintptr_t)e->norm1_w[l] | (uintptr_t)e->norm2_w[l];
-    const uintptr_t b2 = (uintptr_t)e->out_b[l] | (uintptr_t)e->fc1_b[l] | (uintptr_t)e->fc2_b[l];
-    if ((w16 & 15) || (g8 & 7) || (b2 & 1)) e->fused_norm = false;
-  }
   if (e->fused_rope) {
     const size_t h = (size_t)cfg->hidden;
     for (int l = 0; l < L && err == cudaSuccess; ++l)
@@ -766,39 +703,8 @@ int epd_op_qkv_rope(const void* x, int64_t ldx, const void* w_prepared, const vo
   if (((uintptr_t)x | (uintptr_t)w_prepared | (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)table) & 15)
     return EPD_EINVAL;
   EPD_CUDA(linear_tc_pair_qkv(x, ldx, w_prepared, h, bias_prepared, q, k, v, pos_row, pos_col,
-                              reinterpret_cast<const float2*>(table), table_rows, T, heads, head_dim, q_scale, nullptr, 0,
-                              0.0f, nullptr, static_cast<cudaStream_t>(stream)));
-  return EPD_OK;
-}
-
-int32_t epd_norm_parts(int64_t N) { return N > 0 ? norm_parts(N) : 0; }
-
-int epd_op_linear_residual_norm(const void* a, int64_t lda, const void* w, int64_t ldw, const void* bias, float* x,
-                                int64_t ldx, int64_t M, int64_t N, int64_t K, const void* gain, void* xg,
-                                float* row_partials, void* stream) {
-  if (M < 0 || N < 1 || K < 1 || M > (1 << 30) || lda < K || ldw < K || ldx < N) return EPD_EINVAL;
-  if (M == 0) return EPD_OK;
-  if (!a || !w || !x || !gain || !xg || !row_partials) return EPD_EINVAL;
-  if ((lda % 8) || (ldw % 8) || (ldx % 4) || (N % 8)) return EPD_EINVAL;
-  if (((uintptr_t)a | (uintptr_t)w | (uintptr_t)x | (uintptr_t)xg) & 15) return EPD_EINVAL;
-  if (((uintptr_t)gain & 7) || ((uintptr_t)row_partials & 3) || ((uintptr_t)bias & 1)) return EPD_EINVAL;
-  EPD_CUDA(linear_tc_pair_residual_norm(a, lda, w, ldw, bias, x, ldx, M, N, K, gain, xg, row_partials, nullptr,
-                                        static_cast<cudaStream_t>(stream)));
-  return EPD_OK;
-}
-
-int epd_op_linear_normed(const void* xg, int64_t ldxg, const void* w, int64_t ldw, const void* bias, void* out,
-                         int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t flags, const float* row_partials,
-                         int32_t n_parts, float eps, void* stream) {
-  if (M < 0 || N < 1 || K < 1 || M > (1 << 30) || ldxg < K || ldw < K || ldo < N || n_parts < 1 || !(eps >= 0.0f))
-    return EPD_EINVAL;
-  if (M == 0) return EPD_OK;
-  if (!xg || !w || !out || !row_partials) return EPD_EINVAL;
-  if ((ldxg % 8) || (ldw % 8) || (ldo % 8) || (N % 8)) return EPD_EINVAL;
-  if (((uintptr_t)xg | (uintptr_t)w | (uintptr_t)out) & 15) return EPD_EINVAL;
-  if (flags & ~(EPD_LINEAR_GELU_TANH | EPD_LINEAR_GELU_ERF)) return EPD_EINVAL;
-  EPD_CUDA(linear_tc_pair_normed(xg, ldxg, w, ldw, bias, out, ldo, M, N, K, flags, row_partials, n_parts, eps, nullptr,
-                                 static_cast<cudaStream_t>(stream)));
+                              reinterpret_cast<const float2*>(table), table_rows, T, heads, head_dim, q_scale, nullptr,
+                              static_cast<cudaStream_t>(stream)));
   return EPD_OK;
 }
 

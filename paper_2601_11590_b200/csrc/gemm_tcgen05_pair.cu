@@ -21,18 +21,6 @@
 // the epilogue of tile i overlaps the main loop of tile i+1).  Ragged M, N, K are handled by TMA
 // (zero fill on loads, clipping on stores).  No load in this file is a multicast load.
 //
-// RMSNorm folded into the neighbouring linear layers (NORM):
-//   NORM = 1, residual update  x += a w^T + b  whose result feeds an RMSNorm: besides the reduce-add of the
-//     staged chunk into x, the epilogue reads the old x values (plain loads of 128-byte row pieces, 8 lanes
-//     per row, in flight during the accumulator read), forms the new x in registers and writes
-//     xg = bf16(x_new * gain[col]) and the tile's contribution to each row's sum of squares,
-//     partials[row][2 * n_tile + half] (one writer per entry: the row statistics are bit-reproducible).
-//     The reduce-add is issued after the old values have arrived.
-//   NORM = 2, the consumer  y = act(RMSNorm(x) w^T + b) = act(rinv[row] * (xg w^T) + b): the epilogue
-//     multiplies its accumulator row by rinv = 1 / sqrt(sum(partials[row][:]) / h + eps).
-// The separate normalisation pass (read 4 bytes, write 2 per element, ~12 us per call at 6272 x 1152) and
-// its launch disappear.
-//
 // QKV variant (ROPE = true): the epilogue applies the 2-D rotary embedding to the q and k columns and
 // writes q, k, v straight into the head-major padded buffers the attention kernel reads, so the
 // [T, 3h] intermediate and a separate rotary pass disappear.  It expects the q and k rows of the weight
@@ -213,15 +201,6 @@ struct RopeSplitArgs {
   float q_scale;
 };
 
-// RMSNorm folded into the linear layers (see the file header).
-struct NormArgs {
-  float* partials;              // [M, n_parts] per-row sums of squares of x, one entry per 128-column half tile
-  int n_parts;                  // entries per row (consumer: of the matrix it reads; producer: 2 * tiles along N)
-  float inv_h, eps;             // consumer: 1 / row width of x, epsilon
-  __nv_bfloat16* xg;            // producer: [M, N] bf16(x_new * gain), leading dimension N
-  const __nv_bfloat16* gain;    // producer: [N]
-};
-
 template <int BN, int STAGES>
 struct PairLayout {
   static constexpr int kABytes = BM * BK * 2;
@@ -241,15 +220,12 @@ struct PairLayout {
 // ---------------------------------------------------------------------------------------------
 // Kernel
 // ---------------------------------------------------------------------------------------------
-template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE, int NORM>
+template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_out, const __nv_bfloat16* __restrict__ bias, int M, int N,
-                   int K, int* __restrict__ status, const RopeSplitArgs rs, const NormArgs nm, float* __restrict__ out_f32,
-                   long long ldo) {
+                   int K, int* __restrict__ status, const RopeSplitArgs rs) {
   static_assert(!ROPE || (sizeof(OutT) == 2 && ACT == 0 && !ACCUM), "the QKV variant writes bf16, no activation");
-  static_assert(NORM != 1 || (ACCUM && ACT == 0 && sizeof(OutT) == 4), "the norm-producing variant is a residual update");
-  static_assert(NORM != 2 || (!ACCUM && sizeof(OutT) == 2), "the norm-consuming variant writes bf16");
   using L = PairLayout<BN, STAGES>;
   static_assert(BN == 256 || BN == 128, "tile width");
   constexpr int kAccStride = BN;                 // TMEM columns between the two accumulators
@@ -376,45 +352,9 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       for (int i = lane; i < BN / 2; i += 32)
         bs[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
       __syncwarp();
-      const int row0 = m0 + q * 32;
-      // NORM = 2: 1 / rms of this thread's row from the producer's partial sums (fixed order)
-      [[maybe_unused]] float rinv = 1.0f;
-      if constexpr (NORM == 2) {
-        if (row0 + lane < M) {
-          const float* pr = nm.partials + (long long)(row0 + lane) * nm.n_parts;
-          float ss = 0.0f;
-          for (int i = 0; i < nm.n_parts; ++i) ss += pr[i];
-          rinv = rsqrtf(ss * nm.inv_h + nm.eps);
-        }
-      }
-      // NORM = 1: lane l handles 16-byte piece l % 8 (4 columns) of rows l / 8 + 4 i of a staged chunk
-      [[maybe_unused]] float4 old_cur[8];
-      [[maybe_unused]] float gain_cur[4], row_ss[8];
-      [[maybe_unused]] const int piece_col = n0 + 4 * (lane & 7);   // + 32 c
-      auto load_old = [&](int c, float4 (&dst)[8], float (&g)[4]) {
-        const int col = piece_col + 32 * c;
-        const bool col_ok = col < N;
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int r = row0 + it * 4 + (lane >> 3);
-          dst[it] = (col_ok && r < M) ? *reinterpret_cast<const float4*>(out_f32 + (long long)r * ldo + col)
-                                      : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-        }
-        if (col_ok) {
-          const uint2 gv = *reinterpret_cast<const uint2*>(nm.gain + col);
-          const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.x));
-          const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv.y));
-          g[0] = g01.x; g[1] = g01.y; g[2] = g23.x; g[3] = g23.y;
-        } else {
-          g[0] = g[1] = g[2] = g[3] = 0.0f;
-        }
-      };
-      if constexpr (NORM == 1) {
-#pragma unroll
-        for (int it = 0; it < 8; ++it) row_ss[it] = 0.0f;
-      }
       if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) break;
       tc_fence_after();
+      const int row0 = m0 + q * 32;
       const uint32_t taddr = tmem_base + acc * kAccStride + half * (BN / 2) + ((uint32_t)(q * 32) << 16);
       // QKV variant: this thread's row positions, and (tensor, head, dim) of its first column
       int prow = 0, pcol = 0, rt = 0, rhead = 0, rd = 0;
@@ -431,7 +371,6 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         uint32_t pk[32];  // this thread's row of the chunk, as stored: 32 floats or 64 bf16
         if constexpr (sizeof(OutT) == 4) {
           tmem_ld32(taddr + c * CC, pk);
-          if constexpr (NORM == 1) load_old(c, old_cur, gain_cur);   // in flight during the accumulator read and the staging
           tmem_ld_wait();
           const float4* bs4 = reinterpret_cast<const float4*>(bs + c * CC);   // broadcast reads, 16 bytes each
 #pragma unroll
@@ -464,8 +403,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
               const float bias8[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
               float v[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e)
-                v[e] = NORM == 2 ? fmaf(__uint_as_float(src[jj + e]), rinv, bias8[e]) : __uint_as_float(src[jj + e]) + bias8[e];
+              for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(src[jj + e]) + bias8[e];
               if (rt < 2) {
                 const float sc = rt == 0 ? rs.q_scale : 1.0f;
 #pragma unroll
@@ -496,14 +434,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
               const uint32_t* src = j2 < 8 ? r0 : r1;
               const int jj = (4 * j2) & 31;
               const float4 bv = bs4[j2];
-              float t0, t1, t2, t3;
-              if constexpr (NORM == 2) {
-                t0 = fmaf(__uint_as_float(src[jj]), rinv, bv.x); t1 = fmaf(__uint_as_float(src[jj + 1]), rinv, bv.y);
-                t2 = fmaf(__uint_as_float(src[jj + 2]), rinv, bv.z); t3 = fmaf(__uint_as_float(src[jj + 3]), rinv, bv.w);
-              } else {
-                t0 = __uint_as_float(src[jj]) + bv.x; t1 = __uint_as_float(src[jj + 1]) + bv.y;
-                t2 = __uint_as_float(src[jj + 2]) + bv.z; t3 = __uint_as_float(src[jj + 3]) + bv.w;
-              }
+              float t0 = __uint_as_float(src[jj]) + bv.x, t1 = __uint_as_float(src[jj + 1]) + bv.y;
+              float t2 = __uint_as_float(src[jj + 2]) + bv.z, t3 = __uint_as_float(src[jj + 3]) + bv.w;
               if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); t2 = gelu_tanh_fast(t2); t3 = gelu_tanh_fast(t3); }
               if (ACT == 2) { t0 = gelu_erf_f(t0); t1 = gelu_erf_f(t1); t2 = gelu_erf_f(t2); t3 = gelu_erf_f(t3); }
               __nv_bfloat162 b0 = __floats2bfloat162_rn(t0, t1), b1 = __floats2bfloat162_rn(t2, t3);
@@ -546,50 +478,6 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
                 *reinterpret_cast<uint4*>(base + (int64_t)(row0 + r) * rs.dhp) =
                     *reinterpret_cast<const uint4*>(sbuf + r * 128 + ((piece ^ (r & 7)) << 4));
             }
-          }
-          continue;
-        }
-        if constexpr (NORM == 1) {
-          __syncwarp();
-          const int piece = lane & 7;
-          const int col = piece_col + 32 * c;
-          const bool col_ok = col < N;
-#pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const int r = it * 4 + (lane >> 3);
-            float ss = 0.0f;
-            if (col_ok && row0 + r < M) {
-              const float4 t = *reinterpret_cast<const float4*>(sbuf + r * 128 + ((piece ^ (r & 7)) << 4));
-              const float4 o = old_cur[it];
-              // the new x: memory receives the same sum through the reduce-add issued below
-              const float4 xn = make_float4(o.x + t.x, o.y + t.y, o.z + t.z, o.w + t.w);
-              const __nv_bfloat162 g01 = __floats2bfloat162_rn(xn.x * gain_cur[0], xn.y * gain_cur[1]);
-              const __nv_bfloat162 g23 = __floats2bfloat162_rn(xn.z * gain_cur[2], xn.w * gain_cur[3]);
-              *reinterpret_cast<uint2*>(nm.xg + (long long)(row0 + r) * N + col) =
-                  make_uint2(*reinterpret_cast<const uint32_t*>(&g01), *reinterpret_cast<const uint32_t*>(&g23));
-              ss = (xn.x * xn.x + xn.y * xn.y) + (xn.z * xn.z + xn.w * xn.w);
-            }
-            row_ss[it] += ss;
-          }
-          if (c == kChunks - 1) {
-            // the 8 lanes of a row piece group together hold the row's 128 columns of this half tile
-            const int part = 2 * (tile / m_tiles) + half;
-#pragma unroll
-            for (int it = 0; it < 8; ++it) {
-              float ss = row_ss[it];
-              ss += __shfl_xor_sync(0xffffffffu, ss, 1);
-              ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-              ss += __shfl_xor_sync(0xffffffffu, ss, 4);
-              const int r = row0 + it * 4 + (lane >> 3);
-              if (piece == 0 && r < M) nm.partials[(long long)r * nm.n_parts + part] = ss;
-            }
-          }
-          // x += staged chunk in L2; only now, when the old values have arrived in registers
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) {
-            if (row0 < M && n0 + c * CC < N) tma_reduce_add_2d(&tm_out, n0 + c * CC, row0, sbuf);
-            bulk_commit();
           }
           continue;
         }
@@ -671,12 +559,11 @@ int sm_count() {
   return n;
 }
 
-template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE = false, int NORM = 0>
+template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE = false>
 cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& to, const void* bias, int M, int N,
-                   int K, int* status, cudaStream_t s, const RopeSplitArgs& rs = RopeSplitArgs{},
-                   const NormArgs& nm = NormArgs{}, float* out_f32 = nullptr, long long ldo = 0) {
+                   int K, int* status, cudaStream_t s, const RopeSplitArgs& rs = RopeSplitArgs{}) {
   using L = PairLayout<BN, STAGES>;
-  auto kern = linear_pair_kernel<BN, STAGES, OutT, ACT, ACCUM, ROPE, NORM>;
+  auto kern = linear_pair_kernel<BN, STAGES, OutT, ACT, ACCUM, ROPE>;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -709,7 +596,7 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
   }
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
   return launch_pdl(kern, dim3(2 * pairs), dim3(kThreads), smem_bytes, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K,
-                    status, rs, nm, out_f32, ldo);
+                    status, rs);
 }
 
 template <int BN, int STAGES>
@@ -755,7 +642,7 @@ cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ld
 cudaError_t linear_tc_pair_qkv(const void* x, int64_t ldx, const void* w_perm, int64_t ldw, const void* bias_perm,
                                void* q, void* k, void* v, const int32_t* pos_row, const int32_t* pos_col,
                                const float2* table, int table_rows, int64_t M, int heads, int head_dim, float q_scale,
-                               const float* row_partials, int n_parts, float eps, int* status, cudaStream_t s) {
+                               int* status, cudaStream_t s) {
   constexpr int BN = 256;
   const int64_t hdim = (int64_t)heads * head_dim, N = 3 * hdim, K = hdim;
   if (head_dim % 8 || !table) return cudaErrorInvalidValue;
@@ -776,57 +663,7 @@ cudaError_t linear_tc_pair_qkv(const void* x, int64_t ldx, const void* w_perm, i
   rs.dhp = padded_head_dim(head_dim);
   rs.q_scale = q_scale;
   // the output tensor map is not used by this variant
-  if (row_partials != nullptr) {
-    NormArgs nm{};
-    nm.partials = const_cast<float*>(row_partials);
-    nm.n_parts = n_parts;
-    nm.inv_h = 1.0f / (float)K;
-    nm.eps = eps;
-    return launch<BN, 5, __nv_bfloat16, 0, false, true, 2>(tx, tw, tx, bias_perm, (int)M, (int)N, (int)K, status, s, rs, nm);
-  }
   return launch<BN, 5, __nv_bfloat16, 0, false, true>(tx, tw, tx, bias_perm, (int)M, (int)N, (int)K, status, s, rs);
-}
-
-// Residual update x += a w^T + bias that also prepares the RMSNorm of the new x: xg = bf16(x * gain) and
-// the per-row partial sums of squares (row_partials [M, norm_parts(N)]).
-int norm_parts(int64_t N) { return 2 * (int)((N + 255) / 256); }
-
-cudaError_t linear_tc_pair_residual_norm(const void* a, int64_t lda, const void* w, int64_t ldw, const void* bias,
-                                         float* x, int64_t ldo, int64_t M, int64_t N, int64_t K, const void* gain,
-                                         void* xg, float* row_partials, int* status, cudaStream_t s) {
-  constexpr int BN = 256;
-  CUtensorMap ta, tw, to;
-  if (!make_map(&ta, a, M, K, lda, BM, 2) || !make_map(&tw, w, N, K, ldw, BN / 2, 2) || !make_map(&to, x, M, N, ldo, 32, 4))
-    return cudaErrorInvalidValue;
-  if ((ldo % 4) || (N % 8) || ((uintptr_t)x & 15) || ((uintptr_t)xg & 15) || ((uintptr_t)gain & 7)) return cudaErrorInvalidValue;
-  NormArgs nm{};
-  nm.partials = row_partials;
-  nm.n_parts = norm_parts(N);
-  nm.xg = static_cast<__nv_bfloat16*>(xg);
-  nm.gain = static_cast<const __nv_bfloat16*>(gain);
-  return launch<BN, 5, float, 0, true, false, 1>(ta, tw, to, bias, (int)M, (int)N, (int)K, status, s, RopeSplitArgs{}, nm, x,
-                                                 ldo);
-}
-
-// y = act(RMSNorm(x) w^T + bias) from the prepared xg = bf16(x * gain) and the row partials: bf16 out.
-cudaError_t linear_tc_pair_normed(const void* xg, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
-                                  int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, const float* row_partials,
-                                  int n_parts, float eps, int* status, cudaStream_t s) {
-  constexpr int BN = 256;
-  CUtensorMap tx, tw, to;
-  if (!make_map(&tx, xg, M, K, ldx, BM, 2) || !make_map(&tw, w, N, K, ldw, BN / 2, 2) || !make_map(&to, out, M, N, ldo, 32, 2))
-    return cudaErrorInvalidValue;
-  NormArgs nm{};
-  nm.partials = const_cast<float*>(row_partials);
-  nm.n_parts = n_parts;
-  nm.inv_h = 1.0f / (float)K;
-  nm.eps = eps;
-  const RopeSplitArgs rs{};
-  if (flags & EPD_LINEAR_GELU_TANH)
-    return launch<BN, 5, __nv_bfloat16, 1, false, false, 2>(tx, tw, to, bias, (int)M, (int)N, (int)K, status, s, rs, nm);
-  if (flags & EPD_LINEAR_GELU_ERF)
-    return launch<BN, 5, __nv_bfloat16, 2, false, false, 2>(tx, tw, to, bias, (int)M, (int)N, (int)K, status, s, rs, nm);
-  return launch<BN, 5, __nv_bfloat16, 0, false, false, 2>(tx, tw, to, bias, (int)M, (int)N, (int)K, status, s, rs, nm);
 }
 
 namespace {

@@ -295,35 +295,6 @@ static cudaError_t rmsnorm_t(const float* x, const T* gain, T* out, const int32_
     return launch_pdl(rmsnorm_kernel<T>, dim3(blocks), dim3(warps * 32), 0, s, x, gain, out, dst_row, rows, hidden, eps);
 }
 
-// x -> the form the norm-consuming linear kernel reads: xg = bf16(x * gain) and the row's sum of squares in
-// partials[row][0] (the other n_parts - 1 entries zero).  One warp per row.
-__global__ void __launch_bounds__(256)
-rmsnorm_prepare_kernel(const float* __restrict__ x, const __nv_bfloat16* __restrict__ gain, __nv_bfloat16* __restrict__ xg,
-                       float* __restrict__ partials, int n_parts, int64_t rows, int hidden) {
-  pdl_launch_dependents();
-  pdl_wait();
-  const int lane = threadIdx.x & 31;
-  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= rows) return;
-  const float* xr = x + row * hidden;
-  float ss = 0.0f;
-  for (int i = lane; i < hidden; i += 32) {
-    const float v = xr[i];
-    ss += v * v;
-    xg[row * hidden + i] = __float2bfloat16(v * __bfloat162float(gain[i]));
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-  for (int i = lane; i < n_parts; i += 32) partials[row * n_parts + i] = i == 0 ? ss : 0.0f;
-}
-
-cudaError_t rmsnorm_prepare(const float* x, const void* gain, void* xg, float* partials, int n_parts, int64_t T,
-                            int hidden, cudaStream_t s) {
-  if (T == 0) return cudaSuccess;
-  return launch_pdl(rmsnorm_prepare_kernel, dim3((unsigned)((T + 7) / 8)), dim3(256), 0, s, x, (const __nv_bfloat16*)gain,
-                    (__nv_bfloat16*)xg, partials, n_parts, T, hidden);
-}
-
 cudaError_t rmsnorm(int dtype, const void* x, const void* gain, void* out, const int32_t* dst_row, int64_t T,
                     int hidden, float eps, cudaStream_t s) {
   if (T == 0) return cudaSuccess;

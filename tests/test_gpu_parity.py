@@ -118,47 +118,6 @@ def test_linear_tensor_core_tiles(tile_n, M, N, K, ldpad, mode):
     assert rel_err(to_np(out), to_np(out_fma)) <= tol
 
 
-@pytest.mark.parametrize("M,N,K,K2,act", [
-    (784, 1152, 1152, 1152, "gelu_tanh"),   # the 0.6B-class out-projection feeding fc1-sized columns (here N2 = K2)
-    (300, 1160, 72, 1160, "none"),          # ragged M, N not a multiple of the 128-column half tiles
-    (1000, 264, 200, 264, "gelu_erf"),      # a tile and a fraction along N: the second half tile is mostly empty
-    (100, 512, 64, 512, "none"),            # fewer rows than one CTA's 128
-])
-def test_rmsnorm_folded_into_linears(M, N, K, K2, act):
-    """x += a w1^T + b1 with the RMSNorm preparation in its epilogue, then act(RMSNorm(x) w2^T + b2) from the
-    prepared operands: both against the oracle's linear, rmsnorm and gelu; row statistics exact to fp32."""
-    dtype = epd.DTYPE_BF16
-    a = rnd((M, K), 51, 1.0, dtype)
-    w1 = rnd((N, K), 52, K ** -0.5, dtype)
-    b1 = rnd((N,), 53, 0.5, dtype)
-    x0 = rnd((M, N), 54, 1.0, epd.DTYPE_F32)
-    gain = synth.normal(55, "g", (N,), 0.02, 1.0, dtype)
-    N2 = 328
-    w2 = rnd((N2, K2), 56, K2 ** -0.5, dtype)
-    b2 = rnd((N2,), 57, 0.5, dtype)
-    x = torch.from_numpy(x0.copy()).cuda()
-    xg, partials = epd.op_linear_residual_norm(dev(a, dtype), dev(w1, dtype), dev(b1, dtype), x, dev(gain, dtype))
-    x_ref = O.linear(a.astype(np.float64), w1.astype(np.float64), b1.astype(np.float64)) + x0.astype(np.float64)
-    assert rel_err(to_np(x), x_ref) <= 1e-5
-    xs = to_np(x)                                   # the kernel's own new x: what xg and the statistics derive from
-    assert rel_err(to_np(xg), xs * gain.astype(np.float64)[None, :]) <= TOL_BF16_STEP
-    assert partials.shape[1] == 2 * ((N + 255) // 256)
-    assert np.allclose(to_np(partials).sum(axis=1), (xs * xs).sum(axis=1), rtol=1e-5)
-    flags = {"none": 0, "gelu_tanh": epd.LINEAR_GELU_TANH, "gelu_erf": epd.LINEAR_GELU_ERF}[act]
-    eps = 1e-6
-    out = epd.op_linear_normed(xg, dev(w2, dtype), dev(b2, dtype), partials, eps, flags)
-    ref = O.linear(O.rmsnorm(xs, gain.astype(np.float64), eps), w2.astype(np.float64), b2.astype(np.float64))
-    if act == "gelu_tanh":
-        ref = O.gelu(ref, O.ACT_GELU_TANH)
-    if act == "gelu_erf":
-        ref = O.gelu(ref, O.ACT_GELU_ERF)
-    assert rel_err(to_np(out), ref) <= TOL_BF16_STEP
-    # bit-reproducible
-    x2 = torch.from_numpy(x0.copy()).cuda()
-    xg2, partials2 = epd.op_linear_residual_norm(dev(a, dtype), dev(w1, dtype), dev(b1, dtype), x2, dev(gain, dtype))
-    assert torch.equal(x, x2) and torch.equal(xg, xg2) and torch.equal(partials, partials2)
-
-
 @pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
 @pytest.mark.parametrize("T,h", [(1, 8), (37, 256), (100, 1152), (9, 3200), (5, 30)])
 def test_rmsnorm(dtype, T, h):
