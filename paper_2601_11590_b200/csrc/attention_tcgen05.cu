@@ -385,15 +385,17 @@ __device__ __forceinline__ int merging_warpgroup(int fw, int n_kv) { return ((n_
 __device__ __forceinline__ int next_first_warpgroup(int fw, int n_kv) { return merging_warpgroup(fw, n_kv) ^ 1; }
 
 // Order in which the two issuing threads walk an item's key tiles: 0, 2, 1, 4, 3, 6, 5, ... for items of
-// at most 32 key tiles, 0, 1, 2, ... for longer ones.
+// at most 32 key tiles (and rings of four tiles), 0, 1, 2, ... otherwise.
 // The warpgroup that takes tile 0 is the one that did not merge the previous item; giving it its first
 // tiles one step early lets it work through three of them while the other warpgroup is still merging
 // (with the plain order 0, 1, 2, ... it stalls after one, behind the first product the merging
 // warpgroup is not ready for).  Each warpgroup still sees its own tiles in ascending order.  Measured:
 // 8 x 784 tokens 378 -> 393 TFLOP/s, 16 x 1024 tokens 456 -> 471; a 16384-token segment, where item
-// boundaries are rare, lost 1 % in that order and keeps the plain one.
-__device__ __forceinline__ int issue_order(int i, int n_kv) {
-  if (i == 0 || n_kv > 32) return i;
+// boundaries are rare, lost 1 % in that order and keeps the plain one.  It needs K and V rings of four
+// tiles: with three (head width 128) taking tile 2 before tile 1 leaves the loaders no slack (16 x 1024
+// tokens, 25 heads x 128: 788 -> 655 TFLOP/s), so those keep the plain order too.
+__device__ __forceinline__ int issue_order(int i, int n_kv, bool deep_rings) {
+  if (i == 0 || n_kv > 32 || !deep_rings) return i;
   const int j = (i & 1) ? i + 1 : i - 1;
   return j < n_kv ? j : i;
 }
@@ -515,7 +517,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         const uint64_t dq_main = smem_desc(sq, 16, 1024, 2);
         const uint64_t dq_tail = smem_desc(sq + P::kMainBoxes * P::kQMain, 16, 256, 6);
         for (int i = 0; i < it.n_kv; ++i) {
-          const int j = issue_order(i, it.n_kv);
+          const int j = issue_order(i, it.n_kv, P::KS >= 4 && P::VS >= 4);
           const uint32_t kt = kc + j;                   // the tile's number in the K ring
           const int w = (j & 1) ^ fw;
           const int ks = kt % P::KS;
@@ -561,7 +563,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
         const Item it = decode_item<BKV>(segs, heads, item);
         for (int i = 0; i < it.n_kv; ++i) {
-          const int j = issue_order(i, it.n_kv);
+          const int j = issue_order(i, it.n_kv, P::KS >= 4 && P::VS >= 4);
           const uint32_t vt = vc + j;                   // the tile's number in the V ring
           const int w = (j & 1) ^ fw;
           const int vs = vt % P::VS;
