@@ -164,6 +164,12 @@ def run_reference(args):
 
 # ----------------------------------------------------------------------------- replicas (N > 1)
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the linear kernel, mean over the linear launches of one
+# encode, from ncu captures of every linear shape of the workload (profiles/linear_pair_dram_traffic_cfg1_shapes.txt).
+# Only for the workload whose shapes were captured; None elsewhere, and to be reset to None when that kernel changes.
+LINEAR_DRAM_BYTES_PER_LAUNCH = {"cfg1_vit06b_b8_448": 58.26e6}
+
+
 def rank_env():
     """(world size, rank, local rank) as torch.distributed.run exports them; (1, 0, 0) when run alone."""
     return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")),
@@ -324,7 +330,7 @@ def run_cuda(args):
         "peak_source": f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
         "flops_per_launch": flops["linear"] / max(lin_launches, 1),
         "avg_launch_ms": lin_ms / max(lin_launches, 1), "launches_per_step": lin_launches,
-        "traffic": None,
+        "traffic": LINEAR_DRAM_BYTES_PER_LAUNCH.get(args.workload),
         "attention": {"achieved": flops["attention"] / (att_ms * 1e-3) / 1e12 if att_ms > 0 else 0.0,
                       "unit": "TFLOP/s", "ms_per_step": att_ms},
         "whole_step": {"achieved": flops["total"] / (ms_step * 1e-3) / 1e12, "unit": "TFLOP/s",
