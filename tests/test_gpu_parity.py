@@ -473,6 +473,30 @@ def test_block_diagonal_isolation_on_gpu():
     enc.close()
 
 
+def test_one_encoder_alternating_small_and_large_batches():
+    """The same encoder serves batches of at most 128 tokens (separate rotary kernel, single-CTA linear kernel)
+    and larger ones (rotary embedding in the QKV epilogue, which relies on padding columns written once at
+    create) in turn: every call matches the oracle, and a repeated batch gives the same bits as before."""
+    cfg = _small_bf16()
+    w = synth.make_weights(cfg, seed=31)
+    batches = [[(1, 8, 8)], [(1, 20, 24), (1, 6, 6)], [(1, 4, 4), (1, 6, 8)], [(1, 30, 14)], [(1, 8, 8)],
+               [(1, 20, 24), (1, 6, 6)]]
+    enc = epd.Encoder(cfg, w, max_tokens=600, max_images=4, max_grid=32)
+    seen = {}
+    for i, grids in enumerate(batches):
+        patches = synth.make_patches(cfg, grids, seed=40 + len(grids) + grids[0][1])
+        feats, cu_rows = enc.encode(dev(patches, cfg.dtype), grids)
+        torch.cuda.synchronize()
+        assert enc.last_status() == epd.EPD_OK
+        ref = O.encode(cfg, w, patches, grids)
+        assert rel_err(to_np(feats), ref) <= TOL_BF16_FINAL, (i, grids)
+        key = tuple(grids)
+        if key in seen:
+            assert torch.equal(seen[key], feats), (i, grids)
+        seen[key] = feats.clone()
+    enc.close()
+
+
 def test_run_to_run_determinism():
     cfg = _small_bf16()
     grids = [(1, 16, 16), (1, 10, 30)]
