@@ -337,6 +337,31 @@ int epd_feature_cache_stats(const epd_feature_cache_t* cache, int64_t* hits, int
                             int64_t* entries);
 
 /* ------------------------------------------------------------------------------------------
+ * Sharing the GPU with another stage (Section 3.5 "Physical Co-location"; Section 3.2 asynchronous
+ * prefetch)
+ * ---------------------------------------------------------------------------------------- */
+
+/* SM budget: the persistent kernels of this library (linear layers, attention) launch at most n_sms CTAs
+ * (0 = every SM, the default), leaving the other SMs to kernels of a co-located stage on another stream or
+ * in another process.  Process-wide; applies to launches made after the call.  Results do not depend on
+ * it (the same tiles are computed, by fewer CTAs).  The short non-persistent kernels (RMSNorm, patchify,
+ * layout) are not limited. */
+int epd_set_sm_limit(int32_t n_sms);
+int32_t epd_get_sm_limit(void);
+
+/* Enqueues a one-thread kernel that stores `value` to *flag (device memory, or host memory mapped into the
+ * device's address space) with system-scope release semantics once everything enqueued on the stream
+ * before it has completed: a consumer that polls the flag, or waits on it with a stream memory
+ * operation, may then read the features written by a preceding epd_encode* call. */
+int epd_signal_ready(uint32_t* flag, uint32_t value, void* stream);
+
+/* Memory-bound stand-in for a Decode step, for co-location measurements only: n_ctas persistent CTAs
+ * stream `bytes` of device memory `passes` times with 16-byte loads; cta_sums (device uint64 [n_ctas],
+ * zeroed by the caller) receives checksums so the loads cannot be elided. */
+int epd_op_stream_read(const void* data, int64_t bytes, int32_t passes, int32_t n_ctas, uint64_t* cta_sums,
+                       void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * Allocation-free variant (the paper has no counterpart: this is a convenience of this library)
  * ---------------------------------------------------------------------------------------- */
 

@@ -30,7 +30,7 @@ EXPORTED_SYMBOLS = [
     "epd_padded_head_dim", "epd_op_attention", "epd_op_merge", "epd_op_rope_attention_static",
     "epd_static_scratch_bytes", "epd_last_cuda_error", "epd_encode_frames", "epd_op_patchify",
     "epd_op_qkv_prepare", "epd_op_rope_table", "epd_op_qkv_pad_init", "epd_op_qkv_rope",
-    "epd_op_content_hash", "epd_feature_cache_create", "epd_feature_cache_destroy",
+    "epd_set_sm_limit", "epd_get_sm_limit", "epd_signal_ready", "epd_op_stream_read", "epd_op_content_hash", "epd_feature_cache_create", "epd_feature_cache_destroy",
     "epd_feature_cache_lookup", "epd_feature_cache_insert", "epd_feature_cache_stats",
 ]
 
@@ -100,6 +100,14 @@ def load_library() -> ctypes.CDLL:
     lib.epd_op_qkv_pad_init.argtypes = [vp, vp, vp, i64, i32, vp]
     lib.epd_op_qkv_rope.restype = ctypes.c_int
     lib.epd_op_qkv_rope.argtypes = [vp, i64, vp, vp, vp, vp, vp, i32, vp, vp, vp, i64, i32, i32, ctypes.c_float, vp]
+    lib.epd_set_sm_limit.restype = ctypes.c_int
+    lib.epd_set_sm_limit.argtypes = [i32]
+    lib.epd_get_sm_limit.restype = i32
+    lib.epd_get_sm_limit.argtypes = []
+    lib.epd_signal_ready.restype = ctypes.c_int
+    lib.epd_signal_ready.argtypes = [vp, ctypes.c_uint32, vp]
+    lib.epd_op_stream_read.restype = ctypes.c_int
+    lib.epd_op_stream_read.argtypes = [vp, i64, i32, i32, vp, vp]
     lib.epd_op_content_hash.restype = ctypes.c_int
     lib.epd_op_content_hash.argtypes = [vp, vp, i32, vp, vp]
     lib.epd_feature_cache_create.restype = ctypes.c_int
@@ -525,6 +533,25 @@ def op_qkv_rope(x, w, bias, pos_row, pos_col, heads, head_dim, theta, q_scale, t
                                table_rows, _ptr(q), _ptr(k), _ptr(v), T, heads, head_dim, q_scale, sp),
            "epd_op_qkv_rope")
     return q, k, v
+
+
+def set_sm_limit(n_sms: int) -> None:
+    """At most n_sms CTAs for the persistent kernels (0 = every SM)."""
+    _check(load_library().epd_set_sm_limit(n_sms), "epd_set_sm_limit")
+
+
+def get_sm_limit() -> int:
+    return int(load_library().epd_get_sm_limit())
+
+
+def signal_ready(flag, value: int, stream=None) -> None:
+    """Stream-ordered store of `value` to flag[0] (int32 device tensor)."""
+    _check(load_library().epd_signal_ready(_ptr(flag), value, _stream_ptr(stream)), "epd_signal_ready")
+
+
+def op_stream_read(data, passes: int, n_ctas: int, sums, stream=None) -> None:
+    _check(load_library().epd_op_stream_read(_ptr(data), data.numel() * data.element_size(), passes, n_ctas,
+                                             _ptr(sums), _stream_ptr(stream)), "epd_op_stream_read")
 
 
 def op_content_hash(data_dev, item_off, stream=None) -> np.ndarray:

@@ -932,7 +932,8 @@ cudaError_t launch(const Maps& maps, const SegList& segs, int n_items, void* out
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  const int grid = n_items < sm_count() ? n_items : sm_count();
+  const int sms = limited_sms(sm_count());
+  const int grid = n_items < sms ? n_items : sms;
   return launch_pdl(kern, dim3(grid), dim3(kThreads), P::kDynamic, s, maps, segs, n_items, (__nv_bfloat16*)out, T, heads, dh,
                     status);
 }

@@ -59,6 +59,15 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
   return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
+// ---- SM budget ---------------------------------------------------------------------------------
+// Upper bound on the CTAs of the persistent kernels (linear, attention): 0 = every SM.  Set through
+// epd_set_sm_limit() by a process that shares the GPU with another stage (co-location).
+int sm_limit();
+inline int limited_sms(int device_sms) {
+  const int lim = sm_limit();
+  return (lim > 0 && lim < device_sms) ? lim : device_sms;
+}
+
 // ---- plain-FMA kernels (kernels_fma.cu) -----------------------------------------------------
 cudaError_t linear_fma(int dtype, const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias,
                        void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, cudaStream_t s);

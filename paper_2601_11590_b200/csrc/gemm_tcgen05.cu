@@ -436,7 +436,8 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
     configured = true;
   }
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-  const int grid = tiles < sm_count() ? tiles : sm_count();
+  const int sms_avail = limited_sms(sm_count());
+  const int grid = tiles < sms_avail ? tiles : sms_avail;
   return launch_pdl(kern, dim3(grid), dim3(kThreads), L::kDynamic, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K, status);
 }
 
@@ -469,7 +470,7 @@ cudaError_t launch_bn(const CUtensorMap& tx, const CUtensorMap& tw, const CUtens
 int pick_bn(int M, int N) {
   const int cands[3] = {256, 192, 128};
   const double eff[3] = {1.0, 0.88, 0.65};
-  const int sms = sm_count();
+  const int sms = limited_sms(sm_count());
   const int m_tiles = (M + BM - 1) / BM;
   int best = 256;
   double best_cost = 1e300;

@@ -594,7 +594,8 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
     }
     max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
   }
-  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  const int avail = limited_sms(2 * max_pairs) / 2 > 0 ? limited_sms(2 * max_pairs) / 2 : 1;   // pairs within the SM budget
+  const int pairs = tiles < avail ? tiles : avail;
   return launch_pdl(kern, dim3(2 * pairs), dim3(kThreads), smem_bytes, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K,
                     status, rs);
 }

@@ -6,6 +6,8 @@
   python -m paper_2601_11590_b200.opbench rmsnorm --T 6272 --hidden 1152
   python -m paper_2601_11590_b200.opbench hash --items 64 --item-bytes 4816896
   python -m paper_2601_11590_b200.opbench qkv --T 6272 --heads 16 --dh 72        (projection + rotary + split, fused)
+  python -m paper_2601_11590_b200.opbench colocate --sm-limit 112 --standin-ctas 72   (encoder on an SM budget next to a
+                                                                      memory-bound Decode stand-in on a second stream)
 
 Each call goes through the C ABI (epd_op_*), is timed with CUDA events on the launching stream
 after warm-up, and prints one JSON line: average device time, algorithmic FLOP/s or bytes/s.
@@ -64,9 +66,62 @@ def time_op(torch, fn, iters: int, warmup: int, flush: bool) -> float:
     return total / iters
 
 
+def colocate(args, torch):
+    """The default benchmark encode on an SM budget, a memory-bound stand-in for a Decode step on the other
+    SMs, each alone and both at once on two streams: the mutual slowdown of co-locating the two stages."""
+    import synth
+    cfg, grids = synth.WORKLOADS["cfg1_vit06b_b8_448"]
+    w = synth.make_weights(cfg, seed=0)
+    T = synth.num_tokens(grids)
+    enc = epd.Encoder(cfg, w, max_tokens=T, max_images=len(grids), max_grid=max(max(g[1], g[2]) for g in grids))
+    patches = epd.to_device(synth.make_patches(cfg, grids, seed=0), cfg.dtype)
+    n_bytes = int(args.standin_gb * (1 << 30)) // 16 * 16
+    data = torch.randint(0, 255, (n_bytes,), dtype=torch.uint8, device="cuda")
+    sums = torch.zeros(4096, dtype=torch.int64, device="cuda")
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def run(encoder: bool, standin: bool, passes: int):
+        torch.cuda.synchronize()
+        ea0, ea1, eb0, eb1 = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+        if standin:
+            eb0.record(sb)
+            epd.op_stream_read(data, passes, args.standin_ctas, sums, stream=sb)
+            eb1.record(sb)
+        if encoder:
+            ea0.record(sa)
+            with torch.cuda.stream(sa):
+                for _ in range(args.encodes):
+                    enc.encode(patches, grids, stream=sa)
+            ea1.record(sa)
+        torch.cuda.synchronize()
+        return (ea0.elapsed_time(ea1) / args.encodes if encoder else None,
+                n_bytes * passes / (eb0.elapsed_time(eb1) * 1e-3) / 1e9 if standin else None)
+
+    res = {"op": "colocate", "workload": "cfg1_vit06b_b8_448", "encodes": args.encodes, "standin_gb": args.standin_gb,
+           "standin_ctas": args.standin_ctas}
+    epd.set_sm_limit(0)
+    run(True, False, 1)
+    res["encode_ms_all_sms"] = run(True, False, 1)[0]
+    epd.set_sm_limit(args.sm_limit)
+    res["sm_limit"] = args.sm_limit
+    run(True, False, 1)
+    res["encode_ms_alone"] = run(True, False, 1)[0]
+    run(False, True, 1)
+    res["standin_gbs_alone"] = run(False, True, 4)[1]
+    # size the stand-in to last about as long as the encodes
+    passes = max(1, int(res["encode_ms_alone"] * args.encodes * 1e-3 * res["standin_gbs_alone"] * 1e9 / n_bytes))
+    both = run(True, True, passes)
+    res.update(encode_ms_together=both[0], standin_gbs_together=both[1], standin_passes=passes)
+    res["encode_slowdown"] = both[0] / res["encode_ms_alone"]
+    res["standin_slowdown"] = res["standin_gbs_alone"] / both[1]
+    epd.set_sm_limit(0)
+    enc.close()
+    print(json.dumps(res))
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "attention", "rope", "rmsnorm", "merge", "hash", "qkv"])
+    ap.add_argument("op", choices=["linear", "attention", "rope", "rmsnorm", "merge", "hash", "qkv", "colocate"])
     ap.add_argument("--M", type=int, default=6272)
     ap.add_argument("--N", type=int, default=1152)
     ap.add_argument("--K", type=int, default=1152)
@@ -77,6 +132,10 @@ def main():
     ap.add_argument("--heads", type=int, default=16)
     ap.add_argument("--dh", type=int, default=72)
     ap.add_argument("--seglens", default="784x8")
+    ap.add_argument("--sm-limit", type=int, default=112)
+    ap.add_argument("--standin-ctas", type=int, default=72)
+    ap.add_argument("--standin-gb", type=float, default=2.0)
+    ap.add_argument("--encodes", type=int, default=10)
     ap.add_argument("--items", type=int, default=64)
     ap.add_argument("--item-bytes", type=int, default=4816896)
     ap.add_argument("--iters", type=int, default=20)
@@ -94,6 +153,10 @@ def main():
     g = torch.Generator(device="cuda").manual_seed(0)
     rnd = lambda *shape, std=1.0, dtype=bf: (torch.randn(*shape, generator=g, device="cuda") * std).to(dtype)
     res = {"op": args.op}
+
+    if args.op == "colocate":
+        colocate(args, torch)
+        return
 
     if args.op == "linear":
         M, N, K = args.M, args.N, args.K

@@ -497,6 +497,41 @@ def test_one_encoder_alternating_small_and_large_batches():
     enc.close()
 
 
+def test_sm_limit_ready_flag_and_stand_in():
+    """Co-location helpers: an SM budget leaves the features bit-identical; the ready flag is written after
+    the encode on its stream; the memory-bound stand-in's checksums match a host restatement."""
+    cfg = _small_bf16()
+    grids = [(1, 20, 24), (1, 12, 12)]
+    enc, w, patches, feats, _, _ = _run_stage(cfg, grids, seed=9, with_taps=False)
+    first = feats.clone()
+    p = dev(patches, cfg.dtype)
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    try:
+        for limit in (40, 7, 0):
+            epd.set_sm_limit(limit)
+            assert epd.get_sm_limit() == limit
+            again, _ = enc.encode(p, grids)
+            epd.signal_ready(flag, 100 + limit)
+            torch.cuda.synchronize()
+            assert int(flag.item()) == 100 + limit
+            assert torch.equal(first, again), limit
+    finally:
+        epd.set_sm_limit(0)
+    enc.close()
+    rng = np.random.default_rng(3)
+    words = rng.integers(0, 2 ** 32, size=(4096 + 3) * 4, dtype=np.uint64)          # a ragged split over 5 CTAs
+    data = torch.from_numpy(words.astype(np.uint32).view(np.int32)).cuda()
+    sums = torch.zeros(5, dtype=torch.int64, device="cuda")
+    passes = 3
+    epd.op_stream_read(data, passes, 5, sums)
+    torch.cuda.synchronize()
+    v = words.reshape(-1, 4)
+    per_vec = ((v[:, 0] ^ v[:, 1]) + (v[:, 2] ^ v[:, 3])).astype(np.uint64)
+    want = (int(per_vec.sum()) * passes + sum(range(passes)) * len(per_vec)) % (1 << 64)
+    got = int(sums.cpu().numpy().view(np.uint64).sum(dtype=np.uint64))
+    assert got == want
+
+
 def test_run_to_run_determinism():
     cfg = _small_bf16()
     grids = [(1, 16, 16), (1, 10, 30)]
