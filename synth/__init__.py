@@ -76,6 +76,16 @@ VIT_6B = EncoderConfig(
     proj_kind=PROJ_MLP, proj_hidden=12800, out_dim=8192)
 
 
+# A 0.7B-class encoder with the hand-off width the paper's E-P prefetching table prints (d = 3584, patch 14
+# with the 2x2 merge: 280x280 -> [100, 3584]).  The paper gives no internal widths: 32 layers of 16 heads x 80
+# with a 4x MLP are this repository's choice (0.63 G parameters in the blocks).
+VIT_07B = EncoderConfig(
+    name="vit-0.7b-bf16", dtype=DTYPE_BF16, in_channels=3, patch=14, temporal_patch=1,
+    hidden=1280, layers=32, heads=16, head_dim=80, mlp=5120, act=ACT_GELU_TANH,
+    eps=1e-6, rope_theta=10000.0, merge=2, final_norm=1,
+    proj_kind=PROJ_MLP, proj_hidden=5120, out_dim=3584)
+
+
 def tiny_variant(dtype: int = DTYPE_FP32, head_dim: int = 8, heads: int = 2, layers: int = 2,
                  mlp: int = 24, patch: int = 2, temporal_patch: int = 1, act: int = ACT_GELU_TANH,
                  proj_kind: int = PROJ_LINEAR, out_dim: int = 12) -> EncoderConfig:
@@ -219,6 +229,12 @@ def grid_long_sequences(patch: int = 16) -> List[Tuple[int, int, int]]:
     return [(1, 2048 // patch, 2048 // patch), (16 // 2, 448 // patch, 448 // patch)]
 
 
+def grid_prefetch_table() -> List[Tuple[int, int, int]]:
+    """The image sizes of the paper's E-P prefetching table, snapped to multiples of 28 pixels (patch 14):
+    280x280, 560x560, 720x1280, 1080x1920 and 4096x3112 -> 100, 400, 1196, 2691 and 16206 merged tokens."""
+    return [(1, 20, 20), (1, 40, 40), (1, 52, 92), (1, 78, 138), (1, 292, 222)]
+
+
 WORKLOADS = {
     # name: (config, grid list)
     "cfg0_tiny_fp32": (TINY_FP32, grid_batch_fixed(2, 224, 224, 14)),
@@ -226,6 +242,8 @@ WORKLOADS = {
     "cfg2_vit06b_var32": (VIT_06B, grid_variable_resolution(32, 16, 0)),
     "cfg3_vit06b_long": (VIT_06B_VIDEO, grid_long_sequences(16)),
     "cfg4_vit6b_b16_448": (VIT_6B, grid_batch_fixed(16, 448, 448, 14)),
+    # beyond the five benchmark configurations: the hand-off shapes the paper prints
+    "cfg5_vit07b_table42": (VIT_07B, grid_prefetch_table()),
 }
 
 

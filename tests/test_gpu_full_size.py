@@ -159,3 +159,19 @@ def test_cfg4_6b_widths_block_on_sampled_rows():
                  O.ACT_GELU_ERF)
     assert rel_err(to_np(ph), ref) <= 4e-3
     enc.close()
+
+
+def test_cfg5_prefetch_table_shapes_block_on_sampled_rows():
+    """The image sizes of the paper's E-P prefetching table on a 0.7B-class encoder (head width 80: no padding
+    column; a 292 x 222 patch grid: the rotary table does not fit shared memory and is read from global
+    memory), one layer: feature row counts as printed in the paper, the block on sampled rows of the smallest,
+    a middle and the 64824-token image."""
+    cfg0, grids = synth.WORKLOADS["cfg5_vit07b_table42"]
+    cfg = cfg0.with_layers(1)
+    w = synth.make_weights(cfg, seed=8)
+    enc, patches, feats, cu_rows, taps = _encode(cfg, grids, w, seed=8, taps=True)
+    assert np.diff(cu_rows).tolist() == [100, 400, 1196, 2691, 16206]       # the paper's [n, 3584] row counts
+    assert feats.shape == (20593, 3584) and torch.isfinite(feats.float()).all()
+    errs = _check_blocks_on_rows(cfg, w, grids, taps, images=[0, 2, 4], per_image=12, seed=9)
+    print("cfg5 block", errs)
+    enc.close()
