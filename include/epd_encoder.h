@@ -152,6 +152,22 @@ int epd_encode_host(epd_encoder_t* enc, const void* host_patches, const int32_t*
                     int64_t* out_rows, int32_t* out_cu_rows, void* stream);
 
 /*
+ * Pipelined form of epd_encode_host for a loop of requests: the host-to-device copy of the patches, the
+ * encode and the device-to-host copy of the features of one call run on three streams (the copies on two
+ * streams the encoder creates on first use, the encode on `stream`), with two staging slots in the
+ * workspace, so that the copies of neighbouring calls overlap the encodes: H2D(i+1) and D2H(i-1) run during
+ * encode(i).  Ordering is by events only; the call does not block the host.
+ *   host_patches of a call must stay unchanged until its copy has run, host_features are valid once work
+ *   enqueued after epd_encode_host_join(enc, stream) on `stream` runs (e.g. after joining and synchronising
+ *   the stream), or after a device-wide synchronisation.  Both should be page-locked.
+ * epd_encode_host_join makes `stream` wait for the feature copies of all earlier calls (no host wait).
+ */
+int epd_encode_host_async(epd_encoder_t* enc, const void* host_patches, const int32_t* grid_thw, int32_t n_images,
+                          void* host_features, int64_t features_capacity_rows, int64_t* out_rows,
+                          int32_t* out_cu_rows, void* stream);
+int epd_encode_host_join(epd_encoder_t* enc, void* stream);
+
+/*
  * The same stage fed with raw pixels: the step immediately in front of Eq. 1's E.  `frames` is a
  * device buffer of uint8 pixels holding the items back to back, item i as [t*Tp, C, h*P, w*P]
  * (frame, channel, y, x; t, h, w from grid_thw, Tp = temporal_patch, P = patch, C = in_channels <= 4).

@@ -23,6 +23,7 @@ ATTENTION_FORCE_FMA = 1
 
 EXPORTED_SYMBOLS = [
     "epd_encoder_workspace_bytes", "epd_encoder_create", "epd_encode", "epd_encode_host",
+    "epd_encode_host_async", "epd_encode_host_join",
     "epd_encoder_last_status", "epd_encoder_last_launch_count", "epd_encoder_uses_tensor_cores",
     "epd_encoder_destroy", "epd_strerror", "epd_debug_bookkeeping", "epd_debug_set_taps",
     "epd_debug_run_block", "epd_debug_profile", "epd_debug_profile_classes",
@@ -85,6 +86,10 @@ def load_library() -> ctypes.CDLL:
     lib.epd_encode.argtypes = [vp, vp, i64, i32p, i32, vp, i64, i64p, i32p, vp]
     lib.epd_encode_host.restype = ctypes.c_int
     lib.epd_encode_host.argtypes = [vp, vp, i32p, i32, vp, i64, i64p, i32p, vp]
+    lib.epd_encode_host_async.restype = ctypes.c_int
+    lib.epd_encode_host_async.argtypes = [vp, vp, i32p, i32, vp, i64, i64p, i32p, vp]
+    lib.epd_encode_host_join.restype = ctypes.c_int
+    lib.epd_encode_host_join.argtypes = [vp, vp]
     lib.epd_encoder_last_status.restype = ctypes.c_int
     lib.epd_encoder_last_status.argtypes = [vp]
     f32p = ctypes.POINTER(ctypes.c_float)
@@ -359,6 +364,21 @@ class Encoder:
                                         cu_rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
                                         _stream_ptr(stream)), "epd_encode_host")
         return rows.value, cu_rows
+
+    def encode_host_async(self, host_patches, grid_thw, host_features, stream=None):
+        """Pipelined encode_host: copies on the encoder's own streams; call host_join() before reading."""
+        g, gp = _i32_array(grid_thw)
+        n = g.size // 3
+        rows = ctypes.c_int64(0)
+        cu_rows = np.zeros(n + 1, dtype=np.int32)
+        _check(self.lib.epd_encode_host_async(self._h, _ptr(host_patches), gp, n, _ptr(host_features),
+                                              int(host_features.shape[0]), ctypes.byref(rows),
+                                              cu_rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                              _stream_ptr(stream)), "epd_encode_host_async")
+        return rows.value, cu_rows
+
+    def host_join(self, stream=None) -> None:
+        _check(self.lib.epd_encode_host_join(self._h, _stream_ptr(stream)), "epd_encode_host_join")
 
     def last_status(self) -> int:
         return int(self.lib.epd_encoder_last_status(self._h))

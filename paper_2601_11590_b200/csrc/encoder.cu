@@ -22,6 +22,7 @@ struct Layout {
   size_t x, a, qkv, qh, kh, vh, u, merged, proj_hidden, stage_patches, stage_features, pix_patches;
   size_t grid, cu, cu_out, item_off, pos_row, pos_col, merge_slot, merge_idx, rope, status, aux, total;
   size_t qkv_perm_w, qkv_perm_b;   // per layer: QKV weight / bias with q and k rows in rotation-pair order
+  size_t stage_patches2, stage_features2;   // second staging buffers of the pipelined host entry point
 };
 
 // The QKV projection can apply the rotary embedding and the head split in its epilogue.
@@ -65,6 +66,8 @@ Layout make_layout(const epd_config_t& c) {
   L.proj_hidden = take(c.proj_kind == EPD_PROJ_MLP ? Tm * (size_t)c.proj_hidden * es : 0);
   L.stage_patches = take(T * ((K + 7) / 8 * 8) * es);
   L.stage_features = take(Tm * (size_t)c.out_dim * es);
+  L.stage_patches2 = take(T * ((K + 7) / 8 * 8) * es);
+  L.stage_features2 = take(Tm * (size_t)c.out_dim * es);
   L.pix_patches = take(T * ((K + 7) / 8 * 8) * es);   // patch vectors built from raw frames
   L.grid = take((size_t)c.max_images * 3 * 4);
   L.cu = take(((size_t)c.max_images + 1) * 4);
@@ -111,6 +114,12 @@ struct epd_encoder {
   size_t prof_used = 0;
   bool use_tc = false;
   bool fused_rope = false;         // QKV epilogue does rotary + split (batches of more than 128 tokens)
+  // pipelined host entry point: copy streams of the library's own, double-buffered staging, and per slot
+  // the events "patches on the device", "encode finished", "features on the host"
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  cudaEvent_t h2d_done[2] = {nullptr, nullptr}, compute_done[2] = {nullptr, nullptr}, d2h_done[2] = {nullptr, nullptr};
+  bool compute_valid[2] = {false, false}, d2h_valid[2] = {false, false};
+  uint64_t host_calls = 0;
 
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -486,6 +495,69 @@ int epd_encode_host(epd_encoder_t* enc, const void* host_patches, const int32_t*
   return EPD_OK;
 }
 
+int epd_encode_host_async(epd_encoder_t* enc, const void* host_patches, const int32_t* grid_thw, int32_t n_images,
+                          void* host_features, int64_t features_capacity_rows, int64_t* out_rows,
+                          int32_t* out_cu_rows, void* stream) {
+  if (!enc) return EPD_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const epd_config_t& c = enc->cfg;
+  const size_t es = c.dtype == EPD_DTYPE_F32 ? 4 : 2;
+  if (n_images < 0 || (n_images > 0 && !grid_thw)) return EPD_EINVAL;
+  int64_t T = 0;
+  for (int i = 0; i < n_images; ++i) {
+    const int64_t t = grid_thw[3 * i], h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
+    if (t < 1 || h < 1 || w < 1) return EPD_EINVAL;
+    if (t > c.max_tokens || t * h > c.max_tokens || t * h * w > c.max_tokens) return EPD_ECAPACITY;
+    T += t * h * w;
+    if (T > c.max_tokens) return EPD_ECAPACITY;
+  }
+  if (T > 0 && (!host_patches || !host_features)) return EPD_EINVAL;
+  // lazily: two copy streams and six events
+  if (!enc->h2d_stream) {
+    EPD_CUDA(cudaStreamCreateWithFlags(&enc->h2d_stream, cudaStreamNonBlocking));
+    EPD_CUDA(cudaStreamCreateWithFlags(&enc->d2h_stream, cudaStreamNonBlocking));
+    for (int b = 0; b < 2; ++b) {
+      EPD_CUDA(cudaEventCreateWithFlags(&enc->h2d_done[b], cudaEventDisableTiming));
+      EPD_CUDA(cudaEventCreateWithFlags(&enc->compute_done[b], cudaEventDisableTiming));
+      EPD_CUDA(cudaEventCreateWithFlags(&enc->d2h_done[b], cudaEventDisableTiming));
+    }
+  }
+  const int b = (int)(enc->host_calls++ & 1);
+  void* dp = enc->at<void>(b ? enc->lay.stage_patches2 : enc->lay.stage_patches);
+  void* df = enc->at<void>(b ? enc->lay.stage_features2 : enc->lay.stage_features);
+  const int64_t ld = c.dtype == EPD_DTYPE_BF16 ? (enc->patch_dim + 7) / 8 * 8 : enc->patch_dim;
+  // patches -> staging slot b, once the encode that last read this slot (two calls ago) has finished
+  if (enc->compute_valid[b]) EPD_CUDA(cudaStreamWaitEvent(enc->h2d_stream, enc->compute_done[b], 0));
+  if (T > 0)
+    EPD_CUDA(cudaMemcpy2DAsync(dp, (size_t)ld * es, host_patches, (size_t)enc->patch_dim * es,
+                               (size_t)enc->patch_dim * es, (size_t)T, cudaMemcpyHostToDevice, enc->h2d_stream));
+  EPD_CUDA(cudaEventRecord(enc->h2d_done[b], enc->h2d_stream));
+  // the encode, on the caller's stream: after its patches have arrived and after the features this slot held
+  // two calls ago have left for the host
+  EPD_CUDA(cudaStreamWaitEvent(s, enc->h2d_done[b], 0));
+  if (enc->d2h_valid[b]) EPD_CUDA(cudaStreamWaitEvent(s, enc->d2h_done[b], 0));
+  int64_t rows = 0;
+  int rc = encode_device(enc, dp, ld, grid_thw, n_images, df, features_capacity_rows, &rows, out_cu_rows, s);
+  if (rc) return rc;
+  if (out_rows) *out_rows = rows;
+  EPD_CUDA(cudaEventRecord(enc->compute_done[b], s));
+  enc->compute_valid[b] = true;
+  // features -> host, behind the encode, while the caller's stream goes on with the next call
+  EPD_CUDA(cudaStreamWaitEvent(enc->d2h_stream, enc->compute_done[b], 0));
+  if (rows > 0)
+    EPD_CUDA(cudaMemcpyAsync(host_features, df, (size_t)rows * c.out_dim * es, cudaMemcpyDeviceToHost, enc->d2h_stream));
+  EPD_CUDA(cudaEventRecord(enc->d2h_done[b], enc->d2h_stream));
+  enc->d2h_valid[b] = true;
+  return EPD_OK;
+}
+
+int epd_encode_host_join(epd_encoder_t* enc, void* stream) {
+  if (!enc) return EPD_EINVAL;
+  for (int b = 0; b < 2; ++b)
+    if (enc->d2h_valid[b]) EPD_CUDA(cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), enc->d2h_done[b], 0));
+  return EPD_OK;
+}
+
 int epd_encode_frames(epd_encoder_t* enc, const void* frames, const int32_t* grid_thw, int32_t n_images,
                       const float* mean, const float* inv_std, void* features, int64_t features_capacity_rows,
                       int64_t* out_rows, int32_t* out_cu_rows, void* stream) {
@@ -548,6 +620,13 @@ int epd_encoder_destroy(epd_encoder_t* enc) {
   cudaDeviceSynchronize();
   if (enc->staged) cudaEventDestroy(enc->staged);
   if (enc->staged_off) cudaEventDestroy(enc->staged_off);
+  for (int b = 0; b < 2; ++b) {
+    if (enc->h2d_done[b]) cudaEventDestroy(enc->h2d_done[b]);
+    if (enc->compute_done[b]) cudaEventDestroy(enc->compute_done[b]);
+    if (enc->d2h_done[b]) cudaEventDestroy(enc->d2h_done[b]);
+  }
+  if (enc->h2d_stream) cudaStreamDestroy(enc->h2d_stream);
+  if (enc->d2h_stream) cudaStreamDestroy(enc->d2h_stream);
   if (enc->pinned_off) cudaFreeHost(enc->pinned_off);
   for (cudaEvent_t ev : enc->prof_events) cudaEventDestroy(ev);
   if (enc->pinned) cudaFreeHost(enc->pinned);

@@ -573,6 +573,36 @@ def test_host_buffer_entry_point_with_patch_length_not_a_multiple_of_8():
     enc.close()
 
 
+def test_pipelined_host_entry_point_over_a_stream_of_requests():
+    """Seven requests of different batches through epd_encode_host_async, each with host buffers of its own:
+    after one join and a synchronisation of the stream every request's features equal those of the device entry
+    point bit for bit (two staging slots are reused several times; the copies run on the encoder's streams)."""
+    cfg = _small_bf16()
+    w = synth.make_weights(cfg, seed=33)
+    batches = [[(1, 16, 16), (1, 6, 10)], [(1, 8, 8)], [(1, 20, 24)], [(1, 16, 16), (1, 6, 10)], [(1, 4, 4), (1, 30, 14)],
+               [(1, 8, 8)], [(1, 20, 24)]]
+    enc = epd.Encoder(cfg, w, max_tokens=600, max_images=4, max_grid=32)
+    want, hps, hfs = [], [], []
+    for i, grids in enumerate(batches):
+        patches = synth.make_patches(cfg, grids, seed=60 + i)
+        feats, _ = enc.encode(dev(patches, cfg.dtype), grids)
+        want.append(feats.cpu().clone())
+        hps.append(dev(patches, cfg.dtype).cpu().pin_memory())
+        hfs.append(torch.zeros((feats.shape[0], cfg.out_dim), dtype=feats.dtype).pin_memory())
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for grids, hp, hf in zip(batches, hps, hfs):
+            rows, _ = enc.encode_host_async(hp, grids, hf, stream=stream)
+            assert rows == hf.shape[0]
+        enc.host_join(stream=stream)
+    stream.synchronize()                                 # only the caller's stream: the join covers the copies
+    for i, (hf, ref) in enumerate(zip(hfs, want)):
+        assert torch.equal(hf, ref), i
+    assert enc.last_status() == epd.EPD_OK
+    enc.close()
+
+
 # ----------------------------------------------------------------------------- edge cases / errors
 
 def test_empty_and_invalid_batches():
