@@ -220,6 +220,16 @@ int epd_debug_set_taps(epd_encoder_t* enc, void* const* taps);
 int epd_debug_run_block(epd_encoder_t* enc, int32_t layer, void* x, const int32_t* grid_thw,
                         int32_t n_images, void* stream);
 
+/* A repeated request - same grid list, same patch and feature buffers, same SM budget - replays the launch
+ * sequence captured as a CUDA graph on its previous occurrence (up to 8 graphs are kept, oldest dropped):
+ * one graph launch instead of ~190 kernel launches, which matters for small batches, whose latency is
+ * otherwise bound by the host's launch rate.  Needs a capturable stream (not the legacy default stream) that
+ * is not itself being captured; otherwise, and with taps or profiling on, the kernels are launched one by
+ * one.  epd_debug_use_graphs(enc, 0) switches the mechanism off; epd_debug_graph_count returns how many graphs
+ * the encoder holds. */
+int epd_debug_use_graphs(epd_encoder_t* enc, int32_t enable);
+int32_t epd_debug_graph_count(const epd_encoder_t* enc);
+
 /* Per-step timing of the next encodes: with enable != 0 every launch of epd_encode() is bracketed
  * by CUDA events on the launching stream (this costs a few microseconds per launch, so it is
  * meant for a separate measuring pass).  epd_debug_profile_read() synchronises on the last event

@@ -23,7 +23,7 @@ ATTENTION_FORCE_FMA = 1
 
 EXPORTED_SYMBOLS = [
     "epd_encoder_workspace_bytes", "epd_encoder_create", "epd_encode", "epd_encode_host",
-    "epd_encode_host_async", "epd_encode_host_join",
+    "epd_encode_host_async", "epd_encode_host_join", "epd_debug_use_graphs", "epd_debug_graph_count",
     "epd_encoder_last_status", "epd_encoder_last_launch_count", "epd_encoder_uses_tensor_cores",
     "epd_encoder_destroy", "epd_strerror", "epd_debug_bookkeeping", "epd_debug_set_taps",
     "epd_debug_run_block", "epd_debug_profile", "epd_debug_profile_classes",
@@ -90,6 +90,10 @@ def load_library() -> ctypes.CDLL:
     lib.epd_encode_host_async.argtypes = [vp, vp, i32p, i32, vp, i64, i64p, i32p, vp]
     lib.epd_encode_host_join.restype = ctypes.c_int
     lib.epd_encode_host_join.argtypes = [vp, vp]
+    lib.epd_debug_use_graphs.restype = ctypes.c_int
+    lib.epd_debug_use_graphs.argtypes = [vp, i32]
+    lib.epd_debug_graph_count.restype = i32
+    lib.epd_debug_graph_count.argtypes = [vp]
     lib.epd_encoder_last_status.restype = ctypes.c_int
     lib.epd_encoder_last_status.argtypes = [vp]
     f32p = ctypes.POINTER(ctypes.c_float)
@@ -379,6 +383,12 @@ class Encoder:
 
     def host_join(self, stream=None) -> None:
         _check(self.lib.epd_encode_host_join(self._h, _stream_ptr(stream)), "epd_encode_host_join")
+
+    def use_graphs(self, enable: bool) -> None:
+        _check(self.lib.epd_debug_use_graphs(self._h, 1 if enable else 0), "epd_debug_use_graphs")
+
+    def graph_count(self) -> int:
+        return int(self.lib.epd_debug_graph_count(self._h))
 
     def last_status(self) -> int:
         return int(self.lib.epd_encoder_last_status(self._h))

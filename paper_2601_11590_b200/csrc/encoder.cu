@@ -114,6 +114,15 @@ struct epd_encoder {
   size_t prof_used = 0;
   bool use_tc = false;
   bool fused_rope = false;         // QKV epilogue does rotary + split (batches of more than 128 tokens)
+  // Launch sequences captured as CUDA graphs, one per (batch geometry, buffers): a repeated request is one
+  // graph launch instead of ~190 kernel launches (the host needs ~11 us per launch, which bounds the latency
+  // of small batches).
+  struct GraphEntry {
+    const void* patches; int64_t ld; void* features; int sm_limit; std::vector<int32_t> grid;
+    cudaGraphExec_t exec; int64_t launches;
+  };
+  std::vector<GraphEntry> graphs;
+  bool use_graphs = true;
   // pipelined host entry point: copy streams of the library's own, double-buffered staging, and per slot
   // the events "patches on the device", "encode finished", "features on the host"
   cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
@@ -177,8 +186,9 @@ int linear_dispatch(epd_encoder* enc, int dtype, const void* x, int64_t ldx, con
 // Validates the grids, fills host outputs and (if the batch differs from the last one) stages
 // the integer layout on the device.
 int prepare_batch(epd_encoder* enc, const int32_t* grid_thw, int32_t n, int64_t capacity_rows, int64_t* out_rows,
-                  int32_t* out_cu_rows, int64_t* T_out, cudaStream_t s) {
+                  int32_t* out_cu_rows, int64_t* T_out, cudaStream_t s, bool* unchanged = nullptr) {
   const epd_config_t& c = enc->cfg;
+  if (unchanged) *unchanged = false;
   if (n < 0 || (n > 0 && !grid_thw)) return EPD_EINVAL;
   if (n > c.max_images) return EPD_ECAPACITY;
   int64_t T = 0, Tm = 0;
@@ -202,7 +212,10 @@ int prepare_batch(epd_encoder* enc, const int32_t* grid_thw, int32_t n, int64_t 
 
   const bool same = enc->last_T == T && (int)enc->last_grid.size() == 3 * n &&
                     std::memcmp(enc->last_grid.data(), grid_thw, 3 * n * sizeof(int32_t)) == 0;
-  if (same) return EPD_OK;
+  if (same) {
+    if (unchanged) *unchanged = true;
+    return EPD_OK;
+  }
   // The pinned staging buffer may still be the source of the previous batch's copy.
   if (enc->staged_valid) EPD_CUDA(cudaEventSynchronize(enc->staged));
   int32_t* pg = enc->pinned;
@@ -290,6 +303,9 @@ int finish_profile(epd_encoder* enc, cudaStream_t s) {
   return mark(enc, KC_END, s);
 }
 
+int launch_sequence(epd_encoder* enc, const void* patches, int64_t patches_ld, int32_t n, void* features, int64_t T,
+                    cudaStream_t s);
+
 int encode_device(epd_encoder* enc, const void* patches, int64_t patches_ld, const int32_t* grid_thw, int32_t n,
                   void* features, int64_t cap_rows, int64_t* out_rows, int32_t* out_cu_rows, cudaStream_t s) {
   const epd_config_t& c = enc->cfg;
@@ -299,13 +315,66 @@ int encode_device(epd_encoder* enc, const void* patches, int64_t patches_ld, con
   enc->launches = 0;
   enc->prof_used = 0;
   int64_t T = 0;
-  int rc = prepare_batch(enc, grid_thw, n, cap_rows, out_rows, out_cu_rows, &T, s);
+  bool unchanged = false;
+  int rc = prepare_batch(enc, grid_thw, n, cap_rows, out_rows, out_cu_rows, &T, s, &unchanged);
   if (rc) return rc;
   if (T == 0) return EPD_OK;
   if (!patches || !features) return EPD_EINVAL;
   if (((uintptr_t)patches & 15) || ((uintptr_t)features & 15)) return EPD_EINVAL;
   if (patches_ld < enc->patch_dim) return EPD_EINVAL;
   if (dt == EPD_DTYPE_BF16 && (patches_ld % 8)) return EPD_EINVAL;
+
+  // A repeated request (same grids, same buffers) replays its captured launch sequence.  Capturing needs the
+  // integer layout already on the device (no copies inside the capture), a stream that can be captured, and
+  // no debugging hooks.
+  if (enc->use_graphs && unchanged && s != nullptr && !enc->profile && enc->taps.empty()) {
+    const int lim = sm_limit();
+    for (const epd_encoder::GraphEntry& g : enc->graphs) {
+      if (g.patches == patches && g.ld == patches_ld && g.features == features && g.sm_limit == lim &&
+          (int)g.grid.size() == 3 * n && std::memcmp(g.grid.data(), grid_thw, 3 * n * sizeof(int32_t)) == 0) {
+        enc->launches = g.launches;
+        EPD_CUDA(cudaGraphLaunch(g.exec, s));
+        return EPD_OK;
+      }
+    }
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone &&
+        cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+      rc = launch_sequence(enc, patches, patches_ld, n, features, T, s);
+      cudaGraph_t graph = nullptr;
+      const cudaError_t e_end = cudaStreamEndCapture(s, &graph);
+      cudaGraphExec_t exec = nullptr;
+      if (rc == EPD_OK && e_end == cudaSuccess && graph != nullptr &&
+          cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+        cudaGraphDestroy(graph);
+        if (enc->graphs.size() >= 8) {
+          cudaGraphExecDestroy(enc->graphs.front().exec);
+          enc->graphs.erase(enc->graphs.begin());
+        }
+        enc->graphs.push_back({patches, patches_ld, features, lim, std::vector<int32_t>(grid_thw, grid_thw + 3 * n), exec,
+                               enc->launches});
+        EPD_CUDA(cudaGraphLaunch(exec, s));
+        return EPD_OK;
+      }
+      // capture did not work out: plain launches from now on
+      if (graph) cudaGraphDestroy(graph);
+      (void)cudaGetLastError();
+      enc->use_graphs = false;
+      enc->launches = 0;
+    } else {
+      (void)cudaGetLastError();
+    }
+  }
+  return launch_sequence(enc, patches, patches_ld, n, features, T, s);
+}
+
+// The kernels of one encode, patch embedding to projector, on stream s.
+int launch_sequence(epd_encoder* enc, const void* patches, int64_t patches_ld, int32_t n, void* features, int64_t T,
+                    cudaStream_t s) {
+  const epd_config_t& c = enc->cfg;
+  const int dt = c.dtype;
+  const int h = c.hidden;
+  int rc;
   const int64_t Tm = T / 4;
   float* x = enc->at<float>(enc->lay.x);
 
@@ -620,6 +689,7 @@ int epd_encoder_destroy(epd_encoder_t* enc) {
   cudaDeviceSynchronize();
   if (enc->staged) cudaEventDestroy(enc->staged);
   if (enc->staged_off) cudaEventDestroy(enc->staged_off);
+  for (epd_encoder::GraphEntry& g : enc->graphs) cudaGraphExecDestroy(g.exec);
   for (int b = 0; b < 2; ++b) {
     if (enc->h2d_done[b]) cudaEventDestroy(enc->h2d_done[b]);
     if (enc->compute_done[b]) cudaEventDestroy(enc->compute_done[b]);
@@ -681,6 +751,14 @@ int epd_debug_run_block(epd_encoder_t* enc, int32_t layer, void* x, const int32_
   if ((rc = run_block(enc, layer, static_cast<float*>(x), T, n_images, s))) return rc;
   return finish_profile(enc, s);
 }
+
+int epd_debug_use_graphs(epd_encoder_t* enc, int32_t enable) {
+  if (!enc) return EPD_EINVAL;
+  enc->use_graphs = enable != 0;
+  return EPD_OK;
+}
+
+int32_t epd_debug_graph_count(const epd_encoder_t* enc) { return enc ? (int32_t)enc->graphs.size() : 0; }
 
 int epd_debug_profile(epd_encoder_t* enc, int32_t enable) {
   if (!enc) return EPD_EINVAL;

@@ -603,6 +603,60 @@ def test_pipelined_host_entry_point_over_a_stream_of_requests():
     enc.close()
 
 
+def test_repeated_requests_replay_a_captured_graph():
+    """On a capturable stream the second identical request captures its launch sequence and later ones replay
+    it: same bits as the plain launches, one graph per (batch, buffers); other batches in between, a changed
+    SM budget and switching the mechanism off all keep the results identical."""
+    cfg = _small_bf16()
+    w = synth.make_weights(cfg, seed=35)
+    ga, gb = [(1, 20, 24), (1, 6, 6)], [(1, 8, 8)]
+    pa = dev(synth.make_patches(cfg, ga, seed=70), cfg.dtype)
+    pb = dev(synth.make_patches(cfg, gb, seed=71), cfg.dtype)
+    enc = epd.Encoder(cfg, w, max_tokens=600, max_images=4, max_grid=32)
+    ref_a = enc.encode(pa, ga)[0].clone()                     # default stream: plain launches
+    ref_b = enc.encode(pb, gb)[0].clone()
+    torch.cuda.synchronize()
+    assert enc.graph_count() == 0
+    stream = torch.cuda.Stream()
+    fa = torch.empty_like(ref_a)
+    fb = torch.empty_like(ref_b)
+    with torch.cuda.stream(stream):
+        for i in range(4):                                    # a, a (capture), a (replay), a (replay)
+            fa.zero_()
+            enc.encode(pa, ga, features=fa, stream=stream)
+            stream.synchronize()
+            assert torch.equal(fa, ref_a), i
+        assert enc.graph_count() == 1 and enc.last_launch_count() == 7 * cfg.layers + 4
+        for i in range(3):                                    # alternate with another batch: layouts restaged
+            fb.zero_()
+            enc.encode(pb, gb, features=fb, stream=stream)
+            fa.zero_()
+            enc.encode(pa, ga, features=fa, stream=stream)
+            stream.synchronize()
+            assert torch.equal(fb, ref_b) and torch.equal(fa, ref_a), i
+        for _ in range(2):
+            fb.zero_()
+            enc.encode(pb, gb, features=fb, stream=stream)    # b, b: the second one captures
+        stream.synchronize()
+        assert torch.equal(fb, ref_b) and enc.graph_count() == 2
+        try:
+            epd.set_sm_limit(24)                              # another budget: another graph
+            for _ in range(3):
+                fa.zero_()
+                enc.encode(pa, ga, features=fa, stream=stream)
+            stream.synchronize()
+            assert torch.equal(fa, ref_a) and enc.graph_count() == 3
+        finally:
+            epd.set_sm_limit(0)
+        enc.use_graphs(False)
+        fa.zero_()
+        enc.encode(pa, ga, features=fa, stream=stream)
+        stream.synchronize()
+        assert torch.equal(fa, ref_a) and enc.graph_count() == 3
+    assert enc.last_status() == epd.EPD_OK
+    enc.close()
+
+
 # ----------------------------------------------------------------------------- edge cases / errors
 
 def test_empty_and_invalid_batches():
