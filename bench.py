@@ -170,6 +170,15 @@ def run_reference(args):
 LINEAR_DRAM_BYTES_PER_LAUNCH = {"cfg1_vit06b_b8_448": 58.26e6}
 
 
+def weight_bytes(cfg) -> float:
+    """Bytes of the encoder's weight matrices (the part a step streams from HBM)."""
+    es = 2 if cfg.dtype == synth.DTYPE_BF16 else 4
+    h, m = cfg.hidden, cfg.mlp
+    per_layer = 3 * h * h + h * h + 2 * h * m
+    proj = 4 * h * cfg.proj_hidden + cfg.proj_hidden * cfg.out_dim if cfg.proj_kind == synth.PROJ_MLP else 4 * h * cfg.out_dim
+    return es * float(cfg.layers * per_layer + cfg.patch_dim * h + proj)
+
+
 def rank_env():
     """(world size, rank, local rank) as torch.distributed.run exports them; (1, 0, 0) when run alone."""
     return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")),
@@ -355,7 +364,8 @@ def run_cuda(args):
         "vs_baseline": None, "dtype": "bf16" if cfg.dtype == synth.DTYPE_BF16 else "f32", "data": "synthetic",
         "config": {"workload": args.workload, "encoder": cfg.name, "images_per_gpu": len(grids),
                    "tokens_per_gpu": T, "merged_tokens_per_gpu": Tm, "out_dim": cfg.out_dim,
-                   "l2": "weights (0.9 GB) and activations exceed the 126 MB L2; no flush between steps",
+                   "l2": f"weights ({weight_bytes(cfg) / 1e9:.1f} GB) and activations exceed the 126 MB L2; "
+                         "no flush between steps",
                    "parallelism": f"replicas x{world}", "tflop_per_step": flops["total"] / 1e12},
         "images_per_s": world * len(grids) * args.steps / (ms_total * 1e-3),
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / args.steps,
