@@ -112,6 +112,10 @@ size_t epd_encoder_workspace_bytes(const epd_config_t* cfg);
  * Build an encoder.  `workspace` is device memory of at least epd_encoder_workspace_bytes(cfg)
  * bytes, 256-byte aligned, owned by the caller and reserved for this encoder until destroy.
  * Synchronous: builds the rotary table on the device and returns after it is ready.
+ * Weights are borrowed (they must stay valid and unchanged until destroy) with one exception: for bf16
+ * configurations whose head_dim is a multiple of 8 the encoder keeps, inside the workspace, its own copy
+ * of every layer's QKV weight and bias with the q and k rows reordered for the rotary epilogue; changing
+ * those weights afterwards needs a new encoder.
  * Errors: EPD_EINVAL (bad config / NULL / alignment), EPD_ENOMEM (workspace too small),
  * EPD_EUNSUPPORTED, EPD_ECUDA.
  */
