@@ -657,6 +657,44 @@ def test_repeated_requests_replay_a_captured_graph():
     enc.close()
 
 
+@pytest.mark.parametrize("which", ["dh72", "dh128", "dh80"])
+def test_random_batches_repeat_bit_identically(which):
+    """Random item lists (1-6 items, stills and clips, grids of 2..64 patches a side) on two-layer encoders of
+    the three head widths: every batch, encoded four more times on a side stream (plain, captured, replayed),
+    gives the bits of its first encode and leaves the status word clean."""
+    import dataclasses
+    base = {"dh72": synth.VIT_06B, "dh128": synth.VIT_6B, "dh80": synth.VIT_07B}[which]
+    cfg = dataclasses.replace(base, layers=2, name=which)
+    w = synth.make_weights(cfg, seed=1)
+    enc = epd.Encoder(cfg, w, max_tokens=12000, max_images=8, max_grid=64)
+    rng = np.random.default_rng({"dh72": 5, "dh128": 6, "dh80": 7}[which])
+    side = torch.cuda.Stream()
+    K = cfg.patch_dim
+    ld = (K + 7) // 8 * 8
+    done = 0
+    while done < 8:
+        n = int(rng.integers(1, 7))
+        grids = [(int(rng.integers(1, 3)), 2 * int(rng.integers(1, 33)), 2 * int(rng.integers(1, 33))) for _ in range(n)]
+        T = synth.num_tokens(grids)
+        if T > 12000:
+            continue
+        done += 1
+        p = torch.zeros((T, ld), dtype=torch.bfloat16, device="cuda")
+        p[:, :K] = epd.to_device(synth.normal(100 + done, "p", (T, K), 1.0, 0.0, cfg.dtype), cfg.dtype)
+        ref = enc.encode(p, grids)[0].clone()
+        torch.cuda.synchronize()
+        assert enc.last_status() == epd.EPD_OK and torch.isfinite(ref.float()).all()
+        out = torch.empty_like(ref)
+        with torch.cuda.stream(side):
+            for rep in range(4):
+                out.zero_()
+                enc.encode(p, grids, features=out, stream=side)
+                side.synchronize()
+                assert torch.equal(out, ref), (grids, rep)
+        assert enc.last_status() == epd.EPD_OK
+    enc.close()
+
+
 # ----------------------------------------------------------------------------- edge cases / errors
 
 def test_empty_and_invalid_batches():
