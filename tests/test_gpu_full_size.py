@@ -175,3 +175,21 @@ def test_cfg5_prefetch_table_shapes_block_on_sampled_rows():
     errs = _check_blocks_on_rows(cfg, w, grids, taps, images=[0, 2, 4], per_image=12, seed=9)
     print("cfg5 block", errs)
     enc.close()
+
+
+def test_cfg4_6b_widths_eight_layers_one_image_end_to_end():
+    """The 6B-class widths on the benchmark's 16-image batch, eight of the 45 layers: image 5's features against
+    the oracle's encode of image 5 alone (error growth over depth at these widths; the per-block figure is
+    ~2.5e-3)."""
+    cfg0, grids = synth.WORKLOADS["cfg4_vit6b_b16_448"]
+    cfg = cfg0.with_layers(8)
+    w = synth.make_weights(cfg, seed=11)
+    enc, patches, feats, cu_rows, _ = _encode(cfg, grids, w, seed=11)
+    bk = O.bookkeeping(grids)
+    i = 5
+    a, b = int(bk["cu_seqlens"][i]), int(bk["cu_seqlens"][i + 1])
+    ref = O.encode(cfg, w, patches[a:b], [grids[i]])
+    e = rel_err(to_np(feats[cu_rows[i]:cu_rows[i + 1]]), ref)
+    print("cfg4 8 layers image 5 final", e)
+    assert e <= TOL_FINAL, e
+    enc.close()
