@@ -137,8 +137,11 @@ int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, vo
  *   out_rows     HOST, optional: total feature rows written (T/4).
  *   out_cu_rows  HOST [n_images+1], optional: prefix sums of per-item feature rows.
  *   stream       cudaStream_t (NULL = legacy default stream).
- * Validation happens on the host before anything is launched; host outputs are filled
- * synchronously (they depend on grid_thw only).  n_images == 0 is valid and launches nothing.
+ * Every argument is validated on the host before anything is enqueued (no copy, no kernel): a call that
+ * returns EPD_EINVAL or EPD_ECAPACITY has touched neither the stream nor the workspace, and
+ * epd_encoder_last_launch_count() is 0 after it.  Host outputs are filled synchronously (they depend on
+ * grid_thw only).  n_images == 0 is valid and launches nothing.  The same holds for the host-buffer and
+ * raw-frame forms below.
  * Errors: EPD_EINVAL, EPD_ECAPACITY, EPD_ECUDA.
  */
 int epd_encode(epd_encoder_t* enc, const void* patches, int64_t patches_ld, const int32_t* grid_thw,
@@ -185,8 +188,28 @@ int epd_encode_frames(epd_encoder_t* enc, const void* frames, const int32_t* gri
                       const float* mean, const float* inv_std, void* features, int64_t features_capacity_rows,
                       int64_t* out_rows, int32_t* out_cu_rows, void* stream);
 
-/* Reads the encoder's device status word (synchronises the device): EPD_OK or the first
- * device-side error (EPD_ETIMEOUT), then clears it. */
+/*
+ * epd_encode_frames() behind a feature cache (Section 3.2: features are stored under a hash of the input, so a
+ * repeated input is not encoded again).  The items' content keys are computed on the device
+ * (epd_op_content_hash over each item's frame bytes, whose size must be a multiple of 8) and read back -- the
+ * one point where this call waits for the stream; items whose key (with the same row count) is cached are
+ * copied from the cache to their rows of `features`; the others are encoded as one batch, the first occurrence
+ * of every distinct key only, copied to their rows and inserted into the cache (an item larger than the whole
+ * pool is returned but not cached).  `features` ends up exactly as epd_encode_frames() would leave it.
+ *   out_keys  HOST [n_images], optional: the content keys.
+ *   out_hit   HOST [n_images], optional: 1 where the item came from the cache.
+ * The cache must be used with this one stream (see epd_feature_cache_insert).
+ */
+typedef struct epd_feature_cache epd_feature_cache_t;
+int epd_encode_frames_cached(epd_encoder_t* enc, epd_feature_cache_t* cache, const void* frames,
+                             const int32_t* grid_thw, int32_t n_images, const float* mean, const float* inv_std,
+                             void* features, int64_t features_capacity_rows, int64_t* out_rows, int32_t* out_cu_rows,
+                             uint64_t* out_keys, uint8_t* out_hit, void* stream);
+
+/* Reads the encoder's device status word: EPD_OK or the first device-side error (EPD_ETIMEOUT), then clears
+ * it.  Blocks the calling host thread until the encoder's own most recent work has finished (an event recorded
+ * behind its last launch) and reads the word on a non-blocking stream of the encoder's; it does not
+ * synchronise the device, so other streams -- a co-located stage -- keep running. */
 int epd_encoder_last_status(epd_encoder_t* enc);
 
 /* Number of kernels the last epd_encode() call launched. */
@@ -233,6 +256,14 @@ int epd_debug_run_block(epd_encoder_t* enc, int32_t layer, void* x, const int32_
  * the encoder holds. */
 int epd_debug_use_graphs(epd_encoder_t* enc, int32_t enable);
 int32_t epd_debug_graph_count(const epd_encoder_t* enc);
+
+/* Cycle limit of every bounded device-side wait of kernels launched after the call (process-wide); cycles <= 0
+ * restores the default (about 2 s).  A wait that exceeds the limit gives up: the kernel records EPD_ETIMEOUT in
+ * the encoder's status word, lets what it has in flight complete, frees its tensor memory and returns; its
+ * output is then undefined and epd_encoder_last_status() reports the code.  A test hook: a limit of a few
+ * thousand cycles makes ordinary waits (a first tile still on its way from memory) expire, which exercises that
+ * path without anything being made to hang or fault. */
+int epd_debug_set_wait_limit(int64_t cycles);
 
 /* Per-step timing of the next encodes: with enable != 0 every launch of epd_encode() is bracketed
  * by CUDA events on the launching stream (this costs a few microseconds per launch, so it is
@@ -349,8 +380,6 @@ int epd_op_merge(int32_t dtype, const void* y, const int32_t* merge_idx, void* o
 int epd_op_content_hash(const void* data, const int64_t* item_offsets, int32_t n_items, uint64_t* hashes,
                         void* stream);
 
-typedef struct epd_feature_cache epd_feature_cache_t;
-
 /* A cache of feature matrices by key inside `pool` (device memory, 256-byte aligned, owned by the
  * caller and reserved for the cache until destroy).  row_bytes = out_dim * sizeof(element).  The index
  * lives on the host; entries are evicted first-in-first-out when the pool wraps.  Not thread-safe. */
@@ -360,8 +389,11 @@ int epd_feature_cache_destroy(epd_feature_cache_t* cache);
  * the stream), 1 on a miss (no entry with this key and row count), < 0 on error. */
 int epd_feature_cache_lookup(epd_feature_cache_t* cache, uint64_t key, int64_t rows, void* dst, void* stream);
 /* Enqueues the copy of `rows` feature rows from src (device) into the pool and records them under
- * key; evicts the oldest entries if room is needed.  EPD_ECAPACITY if they can never fit.  The copy is
- * stream-ordered: a lookup on the same stream afterwards sees the data. */
+ * key; evicts the oldest entries if room is needed.  A key that is already cached with the same row count is
+ * left as it is; with another row count the old entry is dropped and the new one stored.  EPD_ECAPACITY if the
+ * rows can never fit.  The copies are ordered by the stream only: use ONE stream for all lookups and inserts of a
+ * cache (an eviction lets a later insert overwrite pool bytes that a lookup's copy on another stream may still
+ * be reading). */
 int epd_feature_cache_insert(epd_feature_cache_t* cache, uint64_t key, int64_t rows, const void* src, void* stream);
 int epd_feature_cache_stats(const epd_feature_cache_t* cache, int64_t* hits, int64_t* misses, int64_t* evictions,
                             int64_t* entries);
@@ -410,8 +442,11 @@ int epd_op_stream_read(const void* data, int64_t bytes, int32_t passes, int32_t 
  *     256 bytes) must not exceed epd_static_scratch_bytes() (16 MiB); larger batches return
  *     EPD_ECAPACITY and launch nothing.
  *   - Every GPU that loads the library holds the array until the process exits.
- *   - The first call on a device looks up the array's device address; make that first call
- *     outside any stream capture.
+ *   - The first call on a device looks up the array's device address (which may make the CUDA runtime load
+ *     the library's device code on that GPU: the moment the 16 MiB are backed); make that first call
+ *     outside any stream capture and outside latency-critical code.
+ *   - heads <= 65535.  A bounded device-side wait that expires inside the attention kernel leaves `out`
+ *     undefined; this entry point has no status word, such an expiry is not reported.
  *   - All calls on a device share the array: calls whose kernels can overlap on the GPU
  *     (different streams without ordering) race.  Nothing has to be cleared between calls: every
  *     element that is read, padding included, is rewritten first by the same call.

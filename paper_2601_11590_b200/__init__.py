@@ -33,6 +33,7 @@ EXPORTED_SYMBOLS = [
     "epd_op_qkv_prepare", "epd_op_rope_table", "epd_op_qkv_pad_init", "epd_op_qkv_rope",
     "epd_set_sm_limit", "epd_get_sm_limit", "epd_signal_ready", "epd_op_stream_read", "epd_op_content_hash", "epd_feature_cache_create", "epd_feature_cache_destroy",
     "epd_feature_cache_lookup", "epd_feature_cache_insert", "epd_feature_cache_stats",
+    "epd_encode_frames_cached", "epd_debug_set_wait_limit",
 ]
 
 
@@ -99,6 +100,11 @@ def load_library() -> ctypes.CDLL:
     f32p = ctypes.POINTER(ctypes.c_float)
     lib.epd_encode_frames.restype = ctypes.c_int
     lib.epd_encode_frames.argtypes = [vp, vp, i32p, i32, f32p, f32p, vp, i64, i64p, i32p, vp]
+    lib.epd_encode_frames_cached.restype = ctypes.c_int
+    lib.epd_encode_frames_cached.argtypes = [vp, vp, vp, i32p, i32, f32p, f32p, vp, i64, i64p, i32p,
+                                             ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint8), vp]
+    lib.epd_debug_set_wait_limit.restype = ctypes.c_int
+    lib.epd_debug_set_wait_limit.argtypes = [i64]
     lib.epd_op_patchify.restype = ctypes.c_int
     lib.epd_op_patchify.argtypes = [i32, vp, vp, vp, vp, i32, i64, vp, i64, i32, i32, i32, f32p, f32p, vp]
     lib.epd_op_qkv_prepare.restype = ctypes.c_int
@@ -328,34 +334,28 @@ class Encoder:
                                           _stream_ptr(stream)), "epd_encode_frames")
         return features[: rows.value], cu_rows
 
-    def encode_frames_cached(self, cache: "FeatureCache", frames, item_off, grid_thw, mean, std, stream=None):
-        """encode_frames with a feature cache in front: items whose content key is cached are not
-        encoded again.  Returns (list of per-item feature tensors, keys uint64 [n], hit mask)."""
+    def encode_frames_cached(self, cache: "FeatureCache", frames, grid_thw, mean, std, features=None, stream=None):
+        """encode_frames with a feature cache in front (epd_encode_frames_cached): items whose content key is
+        cached are not encoded again.  Returns (list of per-item feature tensors, keys uint64 [n], hit mask)."""
         torch = _torch()
-        g = np.asarray(grid_thw, dtype=np.int32).reshape(-1, 3)
-        n = g.shape[0]
-        off = np.asarray(item_off, dtype=np.int64)
-        keys = op_content_hash(frames, off, stream)
-        rows = [int(t) * int(h) * int(w) // 4 for t, h, w in g]
-        out = [cache.lookup(int(keys[i]), rows[i], stream) for i in range(n)]
-        hit = np.array([o is not None for o in out], dtype=bool)
-        # one encode per distinct missing key
-        todo = {}
-        for i in range(n):
-            if not hit[i]:
-                todo.setdefault(int(keys[i]), i)
-        if todo:
-            idx = list(todo.values())
-            sub = torch.cat([frames[int(off[i]):int(off[i + 1])] for i in idx])
-            feats, cu = self.encode_frames(sub, g[idx], mean, std, stream=stream)
-            for j, i in enumerate(idx):
-                f = feats[int(cu[j]):int(cu[j + 1])].contiguous()
-                cache.insert(int(keys[i]), f, stream)
-                todo[int(keys[i])] = f
-            for i in range(n):
-                if not hit[i]:
-                    out[i] = todo[int(keys[i])]
-        return out, keys, hit
+        g, gp = _i32_array(grid_thw)
+        n = g.size // 3
+        T = int(sum(int(g[3 * i]) * int(g[3 * i + 1]) * int(g[3 * i + 2]) for i in range(n)))
+        if features is None:
+            features = torch.empty((max(T // 4, 1), self.cfg.out_dim), dtype=torch_dtype(self.dtype),
+                                   device=self.device)
+        rows = ctypes.c_int64(0)
+        cu_rows = np.zeros(n + 1, dtype=np.int32)
+        keys = np.zeros(n, dtype=np.uint64)
+        hit = np.zeros(n, dtype=np.uint8)
+        m = (ctypes.c_float * len(mean))(*[float(v) for v in mean])
+        istd = (ctypes.c_float * len(std))(*[1.0 / float(v) for v in std])
+        _check(self.lib.epd_encode_frames_cached(
+            self._h, cache._h, _ptr(frames), gp, n, m, istd, _ptr(features), int(features.shape[0]),
+            ctypes.byref(rows), cu_rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+            keys.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64)), hit.ctypes.data_as(ctypes.POINTER(ctypes.c_uint8)),
+            _stream_ptr(stream)), "epd_encode_frames_cached")
+        return [features[int(cu_rows[i]):int(cu_rows[i + 1])] for i in range(n)], keys, hit.astype(bool)
 
     def encode_host(self, host_patches, grid_thw, host_features, stream=None):
         """host_patches / host_features: CPU tensors (pinned for asynchronous copies)."""
@@ -532,20 +532,9 @@ def op_patchify(dtype, frames_dev, item_off, grid_thw, cu_seqlens, in_channels, 
     return out
 
 
-def qkv_pair_order(heads: int, head_dim: int) -> np.ndarray:
-    """Index map of epd_op_qkv_prepare for one of q / k: element j of the prepared order is element
-    order[j] of the natural one (argument marshalling for tests: no arithmetic of the method)."""
-    nf = head_dim // 4
-    j = np.arange(head_dim)
-    p = j // 2
-    hf, f = p // nf, p % nf
-    inside = hf * (head_dim // 2) + f + (j % 2) * nf
-    return (np.arange(heads)[:, None] * head_dim + inside[None, :]).reshape(-1)
-
-
 def op_qkv_rope(x, w, bias, pos_row, pos_col, heads, head_dim, theta, q_scale, table_rows, stream=None):
     """Fused QKV projection + rotary + head split (bf16).  Returns q, k, v [heads, T, padded]; q and k in
-    the prepared (pair) order of qkv_pair_order()."""
+    the prepared (pair) order epd_op_qkv_prepare documents."""
     torch = _torch()
     lib = load_library()
     T, h = x.shape[0], heads * head_dim
@@ -563,6 +552,11 @@ def op_qkv_rope(x, w, bias, pos_row, pos_col, heads, head_dim, theta, q_scale, t
                                table_rows, _ptr(q), _ptr(k), _ptr(v), T, heads, head_dim, q_scale, sp),
            "epd_op_qkv_rope")
     return q, k, v
+
+
+def set_wait_limit(cycles: int) -> None:
+    """Cycle limit of the kernels' bounded waits (test hook); 0 restores the default."""
+    _check(load_library().epd_debug_set_wait_limit(int(cycles)), "epd_debug_set_wait_limit")
 
 
 def set_sm_limit(n_sms: int) -> None:

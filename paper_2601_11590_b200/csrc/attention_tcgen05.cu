@@ -43,80 +43,21 @@
 // 32-byte-swizzled boxes of 16 columns, so that one MMA covers all 80 output columns (an MMA costs
 // max(45, N/2) clocks whatever its width, so few wide ones beat many narrow ones).
 // Every mbarrier wait is bounded: on expiry the kernel records EPD_ETIMEOUT and drains.
-#include <cuda.h>
-
 #include <algorithm>
-#include <mutex>
 #include <vector>
 
-#include "common.cuh"
+#include "tcgen05_common.cuh"
 
 namespace epd {
 namespace {
 
+using namespace tc;
+
 constexpr int BQ = 128;          // query rows per work item
 constexpr int kThreads = 384;    // warps 0..3: loaders and MMA issuers; warps 4..11: two softmax warpgroups
 constexpr int kMaxSegs = 128;    // segments one launch can describe
-constexpr long long kWaitCycles = 4000000000LL;
 constexpr int kFmaExpEvery = 0;            // 1 in this many exponentials is computed with FMAs (even; 0 = none)
 constexpr float kRescaleThreshold = 8.0f;  // log2 of the largest P value tolerated before rescaling
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false (and raises *abort_flag) if the phase did not complete in time or
-// another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  int spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 255) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycles) {
-        *abort_flag = 1;
-        return false;
-      }
-    }
-  }
-  return true;
-}
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(smem_u32(bar)), "r"(x), "r"(y)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
-               "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem] . B[smem]
 __device__ __forceinline__ void umma_ss(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
@@ -138,12 +79,6 @@ __device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64
       ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// mbarrier arrives once all tcgen05.mma issued so far by this thread have completed.
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-
 #define EPD_R8(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), \
     "=r"(r[o + 6]), "=r"(r[o + 7])
 #define EPD_W8(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]),       \
@@ -168,7 +103,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : EPD_R16(r, 0) : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+__device__ __forceinline__ void tmem_ld32p(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -214,7 +149,7 @@ __device__ __forceinline__ void tmem_st64(uint32_t taddr, const uint32_t* r) {
 template <int N>
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t* r) {
   if constexpr (N >= 64) { tmem_ld64(taddr, r); tmem_ld_cols<N - 64>(taddr + 64, r + 64); }
-  else if constexpr (N >= 32) { tmem_ld32(taddr, r); tmem_ld_cols<N - 32>(taddr + 32, r + 32); }
+  else if constexpr (N >= 32) { tmem_ld32p(taddr, r); tmem_ld_cols<N - 32>(taddr + 32, r + 32); }
   else if constexpr (N >= 16) { tmem_ld16(taddr, r); tmem_ld_cols<N - 16>(taddr + 16, r + 16); }
   else if constexpr (N >= 8) { tmem_ld8(taddr, r); tmem_ld_cols<N - 8>(taddr + 8, r + 8); }
 }
@@ -225,8 +160,6 @@ __device__ __forceinline__ void tmem_st_cols(uint32_t taddr, const uint32_t* r) 
   else if constexpr (N >= 16) { tmem_st16(taddr, r); tmem_st_cols<N - 16>(taddr + 16, r + 16); }
   else if constexpr (N >= 8) { tmem_st8(taddr, r); tmem_st_cols<N - 8>(taddr + 8, r + 8); }
 }
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float r;
@@ -298,8 +231,8 @@ struct Plan {
   static constexpr int kMl = kV + VS * kKStride;       // (m, l) of both warpgroups, by item parity: float2[2][2][128]
   static constexpr int kBar = kMl + 4 * BQ * 8;
   // q_full[2] q_empty[2] k_full[KS] k_empty[KS] v_full[VS] v_empty[VS] s_full[2] s_free[2] p_full[2] p_free[2]
-  // o_done[2] o_free[2] ml_pub[2]
-  static constexpr int kNumBars = 4 + 2 * KS + 2 * VS + 14;
+  // o_done[2] o_free[2] ml_pub[2] drain[2]
+  static constexpr int kNumBars = 4 + 2 * KS + 2 * VS + 16;
   static constexpr int kTotal = kBar + kNumBars * 8 + 32;
   static constexpr int kDynamic = kTotal + 1024;       // slack to align the tiles to 1024 bytes
   static_assert(kQBytes % 1024 == 0, "Q buffers keep the rings 1024-byte aligned");
@@ -406,7 +339,8 @@ __device__ __forceinline__ int issue_order(int i, int n_kv, bool deep_rings) {
 template <int DHP, bool ONES>
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ SegList segs, int n_items,
-                    __nv_bfloat16* __restrict__ out, int T, int heads, int dh, int* __restrict__ status) {
+                    __nv_bfloat16* __restrict__ out, int T, int heads, int dh, int* __restrict__ status,
+                    long long wait_limit) {
   using P = Plan<DHP>;
   constexpr int BKV = P::BKV;
   pdl_launch_dependents();
@@ -426,8 +360,11 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
   uint64_t* o_done = p_free + 2;              // [2]  warpgroup w's P V products of the item complete: O_w final
   uint64_t* o_free = o_done + 2;              // [2]  O_w read out by the merging warpgroup (4 warp arrivals)
   uint64_t* ml_pub = o_free + 2;              // [2]  warpgroup w published its (m, l) of the item (4 warp arrivals)
+  uint64_t* drain = ml_pub + 2;               // [2]  after an abort: the MMAs of issuing thread 0 / 1 have completed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + P::kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const WaitCtx wc{abort_flag, 0u, wait_limit};
+  uint32_t q_loads = 0, kv_loads = 0;         // loads issued by this thread (warp 0: Q and K tiles, warp 3: V tiles)
   float2* ml_all = reinterpret_cast<float2*>(smem + P::kMl);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -459,7 +396,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         const Item it = decode_item<BKV>(segs, heads, item);
         const int row_base = it.head * T;
         const int qb = n & 1;
-        if (!mbar_wait(&q_empty[qb], ((n >> 1) & 1) ^ 1, abort_flag)) break;
+        if (!mbar_wait(&q_empty[qb], ((n >> 1) & 1) ^ 1, wc)) break;
         {
           uint8_t* dst = smem + P::kQ + qb * P::kQBytes;
           mbar_expect_tx(&q_full[qb], P::kQBytes);
@@ -468,16 +405,18 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
             tma_load_2d(dst + b * P::kQMain, &maps.q_main, b * 64, row_base + it.q0, &q_full[qb]);
           if (P::kTail)
             tma_load_2d(dst + P::kMainBoxes * P::kQMain, &maps.q_tail, P::kMainBoxes * 64, row_base + it.q0, &q_full[qb]);
+          ++q_loads;
         }
         for (int j = 0; j < it.n_kv; ++j, ++kc) {
           const int row = row_base + it.seg_beg + j * BKV;
           const int ks = kc % P::KS;
-          if (!mbar_wait(&k_empty[ks], ((kc / P::KS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(&k_empty[ks], ((kc / P::KS) & 1) ^ 1, wc)) { ok = false; break; }
           uint8_t* dk = smem + P::kK + ks * P::kKStride;
           mbar_expect_tx(&k_full[ks], P::kKBytes);
 #pragma unroll
           for (int b = 0; b < P::kMainBoxes; ++b) tma_load_2d(dk + b * P::kKMain, &maps.k_main, b * 64, row, &k_full[ks]);
           if (P::kTail) tma_load_2d(dk + P::kMainBoxes * P::kKMain, &maps.k_tail, P::kMainBoxes * 64, row, &k_full[ks]);
+          ++kv_loads;
         }
       }
     }
@@ -493,12 +432,13 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         for (int j = 0; j < it.n_kv; ++j, ++vc) {
           const int row = row_base + it.seg_beg + j * BKV;
           const int vs = vc % P::VS;
-          if (!mbar_wait(&v_empty[vs], ((vc / P::VS) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(&v_empty[vs], ((vc / P::VS) & 1) ^ 1, wc)) { ok = false; break; }
           uint8_t* dv = smem + P::kV + vs * P::kKStride;
           mbar_expect_tx(&v_full[vs], P::kKBytes);
 #pragma unroll
           for (int b = 0; b < P::kVBoxes; ++b)
             tma_load_2d(dv + b * P::kVBox, &maps.v, b * (P::kV32 ? 16 : 64), row, &v_full[vs]);
+          ++kv_loads;
         }
       }
     }
@@ -512,7 +452,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
         const Item it = decode_item<BKV>(segs, heads, item);
         const int qb = n & 1;
-        if (!mbar_wait(&q_full[qb], (n >> 1) & 1, abort_flag)) break;
+        if (!mbar_wait(&q_full[qb], (n >> 1) & 1, wc)) break;
         const uint32_t sq = smem_u32(smem + P::kQ + qb * P::kQBytes);
         const uint64_t dq_main = smem_desc(sq, 16, 1024, 2);
         const uint64_t dq_tail = smem_desc(sq + P::kMainBoxes * P::kQMain, 16, 256, 6);
@@ -521,10 +461,10 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           const uint32_t kt = kc + j;                   // the tile's number in the K ring
           const int w = (j & 1) ^ fw;
           const int ks = kt % P::KS;
-          if (!mbar_wait(&k_full[ks], (kt / P::KS) & 1, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(&k_full[ks], (kt / P::KS) & 1, wc)) { ok = false; break; }
           uint32_t& sc = w ? sc1 : sc0;
           // the warpgroup must have copied its previous score tile out of S_w
-          if (sc > 0 && !mbar_wait(&s_free[w], (sc - 1) & 1, abort_flag)) { ok = false; break; }
+          if (sc > 0 && !mbar_wait(&s_free[w], (sc - 1) & 1, wc)) { ok = false; break; }
           ++sc;
           tc_fence_after();
           const uint32_t sk = smem_u32(smem + P::kK + ks * P::kKStride);
@@ -569,13 +509,13 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           const int vs = vt % P::VS;
           uint32_t& pc = w ? pc1 : pc0;
           // V arrives long before P: take that wait first so that only P's is on the critical path
-          if (!mbar_wait(&v_full[vs], (vt / P::VS) & 1, abort_flag)) { ok = false; break; }
-          if (!mbar_wait(&p_full[w], pc & 1, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(&v_full[vs], (vt / P::VS) & 1, wc)) { ok = false; break; }
+          if (!mbar_wait(&p_full[w], pc & 1, wc)) { ok = false; break; }
           ++pc;
           if (j < 2) {
             // the warpgroup's accumulator of its previous item must have been read out before it is overwritten
             uint32_t& items = w ? items1 : items0;
-            if (items > 0 && !mbar_wait(&o_free[w], (items - 1) & 1, abort_flag)) { ok = false; break; }
+            if (items > 0 && !mbar_wait(&o_free[w], (items - 1) & 1, wc)) { ok = false; break; }
             ++items;
           }
           tc_fence_after();
@@ -626,7 +566,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
       // the tcgen05.st of this tile's P, so the two TMEM round trips overlap.
       auto load_scores = [&](int j) -> bool {
         const int kv_valid = min(BKV, it.seg_len - j * BKV);
-        if (!mbar_wait(&s_full[w], tc & 1, abort_flag)) return false;
+        if (!mbar_wait(&s_full[w], tc & 1, wc)) return false;
         tc_fence_after();
         if (kv_valid == BKV) {
           tmem_ld_cols<BKV>(tmem_s, s);
@@ -714,7 +654,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         }
         if (!ONES) l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
         // P_w and O_w are free once this warpgroup's previous P V has completed
-        if (tc > 0 && !mbar_wait(&p_free[w], (tc - 1) & 1, abort_flag)) { ok = false; break; }
+        if (tc > 0 && !mbar_wait(&p_free[w], (tc - 1) & 1, wc)) { ok = false; break; }
         ++tc;
         tc_fence_after();
         if (__any_sync(0xffffffffu, grow)) {
@@ -749,7 +689,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         // not overtake the reader of this warpgroup's previous publication: that reader has finished once
         // O_w of this warpgroup's previous item with key tiles was read out (with two or more key tiles
         // in this item that is already known through the P V products).
-        if (my_pubs > 0 && my_items >= 2 && !mbar_wait(&o_free[w], (my_items - 2) & 1, abort_flag)) { ok = false; break; }
+        if (my_pubs > 0 && my_items >= 2 && !mbar_wait(&o_free[w], (my_items - 2) & 1, wc)) { ok = false; break; }
         ml_all[(n & 1) * 2 * BQ + w * BQ + r] = make_float2(m, l);
         __syncwarp();
         if (lane == 0) mbar_arrive(&ml_pub[w]);
@@ -763,8 +703,8 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
       // accumulator back, so that the other warpgroup's next item is not held up by this merge
       constexpr bool kEarly = DHP + 32 <= BKV;
       if (has_other) {
-        if (!mbar_wait(&ml_pub[w ^ 1], other_pubs & 1, abort_flag)) { ok = false; break; }
-        if (!mbar_wait(&o_done[w ^ 1], (other_items - 1) & 1, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(&ml_pub[w ^ 1], other_pubs & 1, wc)) { ok = false; break; }
+        if (!mbar_wait(&o_done[w ^ 1], (other_items - 1) & 1, wc)) { ok = false; break; }
         tc_fence_after();
         ml_b = ml_all[(n & 1) * 2 * BQ + (w ^ 1) * BQ + r];
         if constexpr (kEarly) {
@@ -785,7 +725,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
             if (i == (dh & 7)) ml_b.y = __uint_as_float(t1[i]);
         }
       }
-      if (!mbar_wait(&o_done[w], (my_items - 1) & 1, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(&o_done[w], (my_items - 1) & 1, wc)) { ok = false; break; }
       tc_fence_after();
       const int token = it.q0 + r;
       const bool row_ok = token < it.seg_beg + it.seg_len;
@@ -866,7 +806,19 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
   tc_fence_before();
   __syncthreads();
   if (*abort_flag) {
+    // A wait expired.  Every role has left its loop, so nothing new is issued.  What was issued completes by
+    // itself: each loader waits for its last load of every ring slot, each issuing thread for its last MMA (a
+    // commit arrives only after all earlier MMAs); the softmax warps write their rows with ordinary stores.  A
+    // fixed pause on top, then shared and tensor memory are released.
     if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, 0, kStatusTimeout);
+    if (lane == 0) {
+      if (warp == 0) { drain_ring(q_full, 2, q_loads); drain_ring(k_full, P::KS, kv_loads); }
+      if (warp == 3) drain_ring(v_full, P::VS, kv_loads);
+      if (warp == 1 || warp == 2) {
+        umma_commit(&drain[warp - 1]);
+        mbar_wait_drain(&drain[warp - 1], 0);
+      }
+    }
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
   }
@@ -879,46 +831,10 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  });
-  return fn;
-}
-
 // Map over a bf16 matrix [rows, dhp] (row pitch dhp*2 bytes): box = box_rows rows x box_cols columns.
 bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int dhp, int box_cols, int box_rows,
               CUtensorMapSwizzle swz) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)dhp, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)dhp * 2};
-  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
+  return make_tensor_map_2d(tm, base, rows, dhp, (int64_t)dhp * 2, box_rows, box_cols, 2, swz);
 }
 
 template <int DHP, bool ONES>
@@ -926,16 +842,15 @@ cudaError_t launch(const Maps& maps, const SegList& segs, int n_items, void* out
                    int* status, cudaStream_t s) {
   using P = Plan<DHP>;
   auto kern = attention_tc_kernel<DHP, ONES>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P::kDynamic);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  const int sms = limited_sms(sm_count());
+  static PerDeviceOnce configured;
+  cudaError_t e = once_per_device(configured, [&] {
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P::kDynamic);
+  });
+  if (e != cudaSuccess) return e;
+  const int sms = limited_sms(device_sm_count());
   const int grid = n_items < sms ? n_items : sms;
   return launch_pdl(kern, dim3(grid), dim3(kThreads), P::kDynamic, s, maps, segs, n_items, (__nv_bfloat16*)out, T, heads, dh,
-                    status);
+                    status, wait_limit_cycles());
 }
 
 bool attention_tc_supported(const void* q, const void* k, const void* v, const void* out, int64_t T, int heads,
@@ -945,7 +860,7 @@ bool attention_tc_supported(const void* q, const void* k, const void* v, const v
   if (head_dim % 8) return false;
   if (((uintptr_t)q & 15) || ((uintptr_t)k & 15) || ((uintptr_t)v & 15) || ((uintptr_t)out & 15)) return false;
   if ((int64_t)heads * T > (1 << 30) || heads > 65535) return false;
-  return encode_tiled_fn() != nullptr;
+  return tensor_maps_available();
 }
 
 cudaError_t attention_tc(const void* q, const void* k, const void* v, const int32_t* host_cu_seqlens, int n_seg,

@@ -23,6 +23,7 @@ struct Layout {
   size_t grid, cu, cu_out, item_off, pos_row, pos_col, merge_slot, merge_idx, rope, status, aux, total;
   size_t qkv_perm_w, qkv_perm_b;   // per layer: QKV weight / bias with q and k rows in rotation-pair order
   size_t stage_patches2, stage_features2;   // second staging buffers of the pipelined host entry point
+  size_t keys;                              // content keys of a batch's items (cached encode)
 };
 
 // The QKV projection can apply the rotary embedding and the head split in its epilogue.
@@ -73,6 +74,7 @@ Layout make_layout(const epd_config_t& c) {
   L.cu = take(((size_t)c.max_images + 1) * 4);
   L.cu_out = take(((size_t)c.max_images + 1) * 4);
   L.item_off = take(((size_t)c.max_images + 1) * 8);
+  L.keys = take((size_t)c.max_images * 8);
   L.pos_row = take(T * 4);
   L.pos_col = take(T * 4);
   L.merge_slot = take(T * 4);
@@ -97,10 +99,15 @@ struct epd_encoder {
   uint8_t* ws = nullptr;
   int32_t* pinned = nullptr;       // [3*max_images | max_images+1 | max_images+1]
   int64_t* pinned_off = nullptr;   // [max_images+1] byte offsets of the items' frames
+  uint64_t* pinned_keys = nullptr; // [max_images] content keys read back by the cached encode
   cudaEvent_t staged_off = nullptr;
   bool staged_off_valid = false;
   cudaEvent_t staged = nullptr;    // recorded after the layout copy of the last batch
   bool staged_valid = false;
+  cudaEvent_t last_launch = nullptr;   // recorded behind the encoder's most recent work on the caller's stream
+  bool last_launch_valid = false;
+  cudaStream_t aux_stream = nullptr;   // non-blocking stream of the encoder's own: reads the status word
+  int32_t* pinned_status = nullptr;
   std::vector<int32_t> last_grid;  // grids of the batch whose layout is on the device
   std::vector<int32_t> host_cu;
   int64_t last_T = -1;
@@ -183,33 +190,61 @@ int linear_dispatch(epd_encoder* enc, int dtype, const void* x, int64_t ldx, con
   return EPD_OK;
 }
 
-// Validates the grids, fills host outputs and (if the batch differs from the last one) stages
-// the integer layout on the device.
-int prepare_batch(epd_encoder* enc, const int32_t* grid_thw, int32_t n, int64_t capacity_rows, int64_t* out_rows,
-                  int32_t* out_cu_rows, int64_t* T_out, cudaStream_t s, bool* unchanged = nullptr) {
+// Integer facts of a batch that follow from the grid list alone.
+struct BatchShape {
+  int64_t T = 0, Tm = 0;
+  std::vector<int32_t> cu, cuo;    // prefix sums of tokens / merged tokens per item
+};
+
+// Host-only validation of a grid list against the encoder's capacities; nothing is enqueued.
+int validate_grids(const epd_encoder* enc, const int32_t* grid_thw, int32_t n, int64_t capacity_rows, BatchShape* bs) {
   const epd_config_t& c = enc->cfg;
-  if (unchanged) *unchanged = false;
   if (n < 0 || (n > 0 && !grid_thw)) return EPD_EINVAL;
   if (n > c.max_images) return EPD_ECAPACITY;
-  int64_t T = 0, Tm = 0;
-  std::vector<int32_t> cu(n + 1, 0), cuo(n + 1, 0);
+  bs->T = bs->Tm = 0;
+  bs->cu.assign(n + 1, 0);
+  bs->cuo.assign(n + 1, 0);
   for (int i = 0; i < n; ++i) {
     const int64_t t = grid_thw[3 * i], h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
     if (t < 1 || h < 1 || w < 1 || (h & 1) || (w & 1)) return EPD_EINVAL;
     if (h > c.max_grid || w > c.max_grid) return EPD_ECAPACITY;
     if (t > c.max_tokens || t * h > c.max_tokens || t * h * w > c.max_tokens) return EPD_ECAPACITY;
-    T += t * h * w;
-    Tm += t * (h / 2) * (w / 2);
-    if (T > c.max_tokens) return EPD_ECAPACITY;
-    cu[i + 1] = (int32_t)T;
-    cuo[i + 1] = (int32_t)Tm;
+    bs->T += t * h * w;
+    bs->Tm += t * (h / 2) * (w / 2);
+    if (bs->T > c.max_tokens) return EPD_ECAPACITY;
+    bs->cu[i + 1] = (int32_t)bs->T;
+    bs->cuo[i + 1] = (int32_t)bs->Tm;
   }
-  if (capacity_rows >= 0 && Tm > capacity_rows) return EPD_ECAPACITY;
-  if (out_rows) *out_rows = Tm;
-  if (out_cu_rows) std::memcpy(out_cu_rows, cuo.data(), (n + 1) * sizeof(int32_t));
-  *T_out = T;
-  if (n == 0) return EPD_OK;
+  if (capacity_rows >= 0 && bs->Tm > capacity_rows) return EPD_ECAPACITY;
+  return EPD_OK;
+}
 
+// Validation of everything an encode of device buffers needs, before anything is enqueued.
+int validate_encode(const epd_encoder* enc, const void* patches, int64_t patches_ld, const int32_t* grid_thw,
+                    int32_t n, const void* features, int64_t cap_rows, BatchShape* bs) {
+  if (cap_rows < 0) return EPD_EINVAL;
+  const int rc = validate_grids(enc, grid_thw, n, cap_rows, bs);
+  if (rc) return rc;
+  if (bs->T == 0) return EPD_OK;
+  if (!patches || !features) return EPD_EINVAL;
+  if (((uintptr_t)patches & 15) || ((uintptr_t)features & 15)) return EPD_EINVAL;
+  if (patches_ld < enc->patch_dim) return EPD_EINVAL;
+  if (enc->cfg.dtype == EPD_DTYPE_BF16 && (patches_ld % 8)) return EPD_EINVAL;
+  return EPD_OK;
+}
+
+void fill_host_outputs(const BatchShape& bs, int32_t n, int64_t* out_rows, int32_t* out_cu_rows) {
+  if (out_rows) *out_rows = bs.Tm;
+  if (out_cu_rows) std::memcpy(out_cu_rows, bs.cuo.data(), (n + 1) * sizeof(int32_t));
+}
+
+// Stages the integer layout of a validated batch on the device, unless it is the layout already there.
+int stage_layout(epd_encoder* enc, const int32_t* grid_thw, int32_t n, const BatchShape& bs, cudaStream_t s,
+                 bool* unchanged = nullptr) {
+  const epd_config_t& c = enc->cfg;
+  if (unchanged) *unchanged = false;
+  if (n == 0) return EPD_OK;
+  const int64_t T = bs.T;
   const bool same = enc->last_T == T && (int)enc->last_grid.size() == 3 * n &&
                     std::memcmp(enc->last_grid.data(), grid_thw, 3 * n * sizeof(int32_t)) == 0;
   if (same) {
@@ -222,8 +257,8 @@ int prepare_batch(epd_encoder* enc, const int32_t* grid_thw, int32_t n, int64_t 
   int32_t* pcu = pg + 3 * (size_t)c.max_images;
   int32_t* pcuo = pcu + c.max_images + 1;
   std::memcpy(pg, grid_thw, 3 * n * sizeof(int32_t));
-  std::memcpy(pcu, cu.data(), (n + 1) * sizeof(int32_t));
-  std::memcpy(pcuo, cuo.data(), (n + 1) * sizeof(int32_t));
+  std::memcpy(pcu, bs.cu.data(), (n + 1) * sizeof(int32_t));
+  std::memcpy(pcuo, bs.cuo.data(), (n + 1) * sizeof(int32_t));
   EPD_CUDA(cudaMemcpyAsync(enc->at<int32_t>(enc->lay.grid), pg, 3 * n * sizeof(int32_t), cudaMemcpyHostToDevice, s));
   EPD_CUDA(cudaMemcpyAsync(enc->at<int32_t>(enc->lay.cu), pcu, (n + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, s));
   EPD_CUDA(cudaMemcpyAsync(enc->at<int32_t>(enc->lay.cu_out), pcuo, (n + 1) * sizeof(int32_t),
@@ -236,8 +271,19 @@ int prepare_batch(epd_encoder* enc, const int32_t* grid_thw, int32_t n, int64_t 
                         enc->at<int32_t>(enc->lay.pos_col), enc->at<int32_t>(enc->lay.merge_slot),
                         enc->at<int32_t>(enc->lay.merge_idx), s));
   enc->last_grid.assign(grid_thw, grid_thw + 3 * n);
-  enc->host_cu = cu;
+  enc->host_cu = bs.cu;
   enc->last_T = T;
+  return EPD_OK;
+}
+
+// Marks the end of the encoder's work on stream s for epd_encoder_last_status (not while s is being captured:
+// an event recorded into a capture cannot be waited for).
+int note_last_launch(epd_encoder* enc, cudaStream_t s) {
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  if (cudaStreamIsCapturing(s, &cap) != cudaSuccess) { (void)cudaGetLastError(); return EPD_OK; }
+  if (cap != cudaStreamCaptureStatusNone) return EPD_OK;
+  EPD_CUDA(cudaEventRecord(enc->last_launch, s));
+  enc->last_launch_valid = true;
   return EPD_OK;
 }
 
@@ -306,24 +352,29 @@ int finish_profile(epd_encoder* enc, cudaStream_t s) {
 int launch_sequence(epd_encoder* enc, const void* patches, int64_t patches_ld, int32_t n, void* features, int64_t T,
                     cudaStream_t s);
 
+// Encode of device buffers.  `bs` is the batch as validate_encode() left it: nothing here can fail validation.
+int encode_validated(epd_encoder* enc, const void* patches, int64_t patches_ld, const int32_t* grid_thw, int32_t n,
+                     void* features, const BatchShape& bs, cudaStream_t s);
+
 int encode_device(epd_encoder* enc, const void* patches, int64_t patches_ld, const int32_t* grid_thw, int32_t n,
                   void* features, int64_t cap_rows, int64_t* out_rows, int32_t* out_cu_rows, cudaStream_t s) {
-  const epd_config_t& c = enc->cfg;
-  const int dt = c.dtype;
-  const int h = c.hidden;
-  if (cap_rows < 0) return EPD_EINVAL;
   enc->launches = 0;
   enc->prof_used = 0;
-  int64_t T = 0;
-  bool unchanged = false;
-  int rc = prepare_batch(enc, grid_thw, n, cap_rows, out_rows, out_cu_rows, &T, s, &unchanged);
+  BatchShape bs;
+  const int rc = validate_encode(enc, patches, patches_ld, grid_thw, n, features, cap_rows, &bs);
   if (rc) return rc;
-  if (T == 0) return EPD_OK;
-  if (!patches || !features) return EPD_EINVAL;
-  if (((uintptr_t)patches & 15) || ((uintptr_t)features & 15)) return EPD_EINVAL;
-  if (patches_ld < enc->patch_dim) return EPD_EINVAL;
-  if (dt == EPD_DTYPE_BF16 && (patches_ld % 8)) return EPD_EINVAL;
+  fill_host_outputs(bs, n, out_rows, out_cu_rows);
+  if (bs.T == 0) return EPD_OK;
+  return encode_validated(enc, patches, patches_ld, grid_thw, n, features, bs, s);
+}
 
+int encode_validated(epd_encoder* enc, const void* patches, int64_t patches_ld, const int32_t* grid_thw, int32_t n,
+                     void* features, const BatchShape& bs, cudaStream_t s) {
+  const int64_t T = bs.T;
+  bool unchanged = false;
+  int rc = stage_layout(enc, grid_thw, n, bs, s, &unchanged);
+  if (rc) return rc;
+  rc = [&]() -> int {
   // A repeated request (same grids, same buffers) replays its captured launch sequence.  Capturing needs the
   // integer layout already on the device (no copies inside the capture), a stream that can be captured, and
   // no debugging hooks.
@@ -366,6 +417,9 @@ int encode_device(epd_encoder* enc, const void* patches, int64_t patches_ld, con
     }
   }
   return launch_sequence(enc, patches, patches_ld, n, features, T, s);
+  }();
+  if (rc) return rc;
+  return note_last_launch(enc, s);
 }
 
 // The kernels of one encode, patch embedding to projector, on stream s.
@@ -420,6 +474,60 @@ int launch_sequence(epd_encoder* enc, const void* patches, int64_t patches_ld, i
       return rc;
   }
   return finish_profile(enc, s);
+}
+
+// Bytes of one item's raw frames: [t*Tp, C, h*P, w*P] uint8.
+int64_t item_frame_bytes(const epd_config_t& c, const int32_t* thw) {
+  return (int64_t)thw[0] * c.temporal_patch * c.in_channels * ((int64_t)thw[1] * c.patch) * ((int64_t)thw[2] * c.patch);
+}
+
+// Pixels of a validated batch -> patch vectors -> the stage.  item_off[i] is the byte offset of item i's frames
+// inside `frames` (HOST array of n entries; the items need not be adjacent).
+int encode_frames_at(epd_encoder* enc, const void* frames, const int64_t* item_off, const int32_t* grid_thw, int32_t n,
+                     const float* mean, const float* inv_std, void* features, const BatchShape& bs, cudaStream_t s) {
+  const epd_config_t& c = enc->cfg;
+  const int64_t ld = (enc->patch_dim + 7) / 8 * 8;
+  if (enc->staged_off_valid) EPD_CUDA(cudaEventSynchronize(enc->staged_off));
+  for (int i = 0; i < n; ++i) enc->pinned_off[i] = item_off[i];
+  enc->pinned_off[n] = 0;
+  enc->launches = 0;
+  // the integer layout (grid, cu_seqlens) must be on the device before the patch kernel reads it
+  int rc = stage_layout(enc, grid_thw, n, bs, s);
+  if (rc) return rc;
+  const int64_t launches_layout = enc->launches;
+  EPD_CUDA(cudaMemcpyAsync(enc->at<int64_t>(enc->lay.item_off), enc->pinned_off, ((size_t)n + 1) * sizeof(int64_t),
+                           cudaMemcpyHostToDevice, s));
+  EPD_CUDA(cudaEventRecord(enc->staged_off, s));
+  enc->staged_off_valid = true;
+  EPD_CUDA(patchify(c.dtype, static_cast<const uint8_t*>(frames), enc->at<int64_t>(enc->lay.item_off),
+                    enc->at<int32_t>(enc->lay.grid), enc->at<int32_t>(enc->lay.cu), n, bs.T,
+                    enc->at<void>(enc->lay.pix_patches), ld, c.in_channels, c.patch, c.temporal_patch, mean, inv_std, s));
+  enc->launches = 0;
+  rc = encode_validated(enc, enc->at<void>(enc->lay.pix_patches), ld, grid_thw, n, features, bs, s);
+  enc->launches += launches_layout + 1;
+  return rc;
+}
+
+// Frees everything the encoder object owns on the host side (events, streams, pinned buffers) and the object.
+void release_host_side(epd_encoder* enc) {
+  if (enc->staged) cudaEventDestroy(enc->staged);
+  if (enc->staged_off) cudaEventDestroy(enc->staged_off);
+  if (enc->last_launch) cudaEventDestroy(enc->last_launch);
+  for (epd_encoder::GraphEntry& g : enc->graphs) cudaGraphExecDestroy(g.exec);
+  for (int b = 0; b < 2; ++b) {
+    if (enc->h2d_done[b]) cudaEventDestroy(enc->h2d_done[b]);
+    if (enc->compute_done[b]) cudaEventDestroy(enc->compute_done[b]);
+    if (enc->d2h_done[b]) cudaEventDestroy(enc->d2h_done[b]);
+  }
+  if (enc->h2d_stream) cudaStreamDestroy(enc->h2d_stream);
+  if (enc->d2h_stream) cudaStreamDestroy(enc->d2h_stream);
+  if (enc->aux_stream) cudaStreamDestroy(enc->aux_stream);
+  if (enc->pinned_off) cudaFreeHost(enc->pinned_off);
+  if (enc->pinned_status) cudaFreeHost(enc->pinned_status);
+  if (enc->pinned_keys) cudaFreeHost(enc->pinned_keys);
+  for (cudaEvent_t ev : enc->prof_events) cudaEventDestroy(ev);
+  if (enc->pinned) cudaFreeHost(enc->pinned);
+  delete enc;
 }
 
 }  // namespace
@@ -486,12 +594,13 @@ int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, vo
   }
   if (cudaEventCreateWithFlags(&e->staged, cudaEventDisableTiming) != cudaSuccess ||
       cudaEventCreateWithFlags(&e->staged_off, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&e->last_launch, cudaEventDisableTiming) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&e->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaMallocHost(reinterpret_cast<void**>(&e->pinned_status), 64) != cudaSuccess ||
+      cudaMallocHost(reinterpret_cast<void**>(&e->pinned_keys), (size_t)cfg->max_images * sizeof(uint64_t)) != cudaSuccess ||
       cudaMallocHost(reinterpret_cast<void**>(&e->pinned_off), ((size_t)cfg->max_images + 1) * sizeof(int64_t)) !=
           cudaSuccess) {
-    if (e->staged) cudaEventDestroy(e->staged);
-    if (e->staged_off) cudaEventDestroy(e->staged_off);
-    cudaFreeHost(e->pinned);
-    delete e;
+    release_host_side(e);
     return EPD_ECUDA;
   }
   cudaError_t err = cudaMemset(e->ws + lay.status, 0, 256);
@@ -512,11 +621,7 @@ int epd_encoder_create(const epd_config_t* cfg, const epd_weights_t* weights, vo
   }
   if (err == cudaSuccess) err = cudaDeviceSynchronize();
   if (err != cudaSuccess) {
-    cudaEventDestroy(e->staged);
-    cudaEventDestroy(e->staged_off);
-    cudaFreeHost(e->pinned_off);
-    cudaFreeHost(e->pinned);
-    delete e;
+    release_host_side(e);
     return EPD_ECUDA;
   }
   *out = e;
@@ -538,30 +643,26 @@ int epd_encode_host(epd_encoder_t* enc, const void* host_patches, const int32_t*
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const epd_config_t& c = enc->cfg;
   const size_t es = c.dtype == EPD_DTYPE_F32 ? 4 : 2;
-  if (n_images < 0 || (n_images > 0 && !grid_thw)) return EPD_EINVAL;
-  int64_t T = 0;
-  for (int i = 0; i < n_images; ++i) {
-    const int64_t t = grid_thw[3 * i], h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
-    if (t < 1 || h < 1 || w < 1) return EPD_EINVAL;
-    if (t > c.max_tokens || t * h > c.max_tokens || t * h * w > c.max_tokens) return EPD_ECAPACITY;
-    T += t * h * w;
-    if (T > c.max_tokens) return EPD_ECAPACITY;
-  }
-  if (T > 0 && (!host_patches || !host_features)) return EPD_EINVAL;
+  enc->launches = 0;
+  enc->prof_used = 0;
   void* dp = enc->at<void>(enc->lay.stage_patches);
   void* df = enc->at<void>(enc->lay.stage_features);
   // the staged copy gets a leading dimension the tensor-core path accepts (a multiple of 8 elements)
   const int64_t ld = c.dtype == EPD_DTYPE_BF16 ? (enc->patch_dim + 7) / 8 * 8 : enc->patch_dim;
-  if (T > 0)
-    EPD_CUDA(cudaMemcpy2DAsync(dp, (size_t)ld * es, host_patches, (size_t)enc->patch_dim * es,
-                               (size_t)enc->patch_dim * es, (size_t)T, cudaMemcpyHostToDevice, s));
-  int64_t rows = 0;
-  int rc = encode_device(enc, dp, ld, grid_thw, n_images, df, features_capacity_rows, &rows, out_cu_rows, s);
+  // everything is validated before the first copy is enqueued
+  if (features_capacity_rows < 0) return EPD_EINVAL;
+  BatchShape bs;
+  int rc = validate_grids(enc, grid_thw, n_images, features_capacity_rows, &bs);
   if (rc) return rc;
-  if (out_rows) *out_rows = rows;
-  if (rows > 0)
-    EPD_CUDA(cudaMemcpyAsync(host_features, df, (size_t)rows * c.out_dim * es, cudaMemcpyDeviceToHost, s));
-  return EPD_OK;
+  if (bs.T > 0 && (!host_patches || !host_features)) return EPD_EINVAL;
+  fill_host_outputs(bs, n_images, out_rows, out_cu_rows);
+  if (bs.T == 0) return EPD_OK;
+  EPD_CUDA(cudaMemcpy2DAsync(dp, (size_t)ld * es, host_patches, (size_t)enc->patch_dim * es,
+                             (size_t)enc->patch_dim * es, (size_t)bs.T, cudaMemcpyHostToDevice, s));
+  rc = encode_validated(enc, dp, ld, grid_thw, n_images, df, bs, s);
+  if (rc) return rc;
+  EPD_CUDA(cudaMemcpyAsync(host_features, df, (size_t)bs.Tm * c.out_dim * es, cudaMemcpyDeviceToHost, s));
+  return note_last_launch(enc, s);
 }
 
 int epd_encode_host_async(epd_encoder_t* enc, const void* host_patches, const int32_t* grid_thw, int32_t n_images,
@@ -571,16 +672,16 @@ int epd_encode_host_async(epd_encoder_t* enc, const void* host_patches, const in
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const epd_config_t& c = enc->cfg;
   const size_t es = c.dtype == EPD_DTYPE_F32 ? 4 : 2;
-  if (n_images < 0 || (n_images > 0 && !grid_thw)) return EPD_EINVAL;
-  int64_t T = 0;
-  for (int i = 0; i < n_images; ++i) {
-    const int64_t t = grid_thw[3 * i], h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
-    if (t < 1 || h < 1 || w < 1) return EPD_EINVAL;
-    if (t > c.max_tokens || t * h > c.max_tokens || t * h * w > c.max_tokens) return EPD_ECAPACITY;
-    T += t * h * w;
-    if (T > c.max_tokens) return EPD_ECAPACITY;
-  }
-  if (T > 0 && (!host_patches || !host_features)) return EPD_EINVAL;
+  enc->launches = 0;
+  enc->prof_used = 0;
+  // everything is validated before the first copy is enqueued
+  if (features_capacity_rows < 0) return EPD_EINVAL;
+  BatchShape bs;
+  int rc = validate_grids(enc, grid_thw, n_images, features_capacity_rows, &bs);
+  if (rc) return rc;
+  if (bs.T > 0 && (!host_patches || !host_features)) return EPD_EINVAL;
+  fill_host_outputs(bs, n_images, out_rows, out_cu_rows);
+  if (bs.T == 0) return EPD_OK;
   // lazily: two copy streams and six events
   if (!enc->h2d_stream) {
     EPD_CUDA(cudaStreamCreateWithFlags(&enc->h2d_stream, cudaStreamNonBlocking));
@@ -597,24 +698,20 @@ int epd_encode_host_async(epd_encoder_t* enc, const void* host_patches, const in
   const int64_t ld = c.dtype == EPD_DTYPE_BF16 ? (enc->patch_dim + 7) / 8 * 8 : enc->patch_dim;
   // patches -> staging slot b, once the encode that last read this slot (two calls ago) has finished
   if (enc->compute_valid[b]) EPD_CUDA(cudaStreamWaitEvent(enc->h2d_stream, enc->compute_done[b], 0));
-  if (T > 0)
-    EPD_CUDA(cudaMemcpy2DAsync(dp, (size_t)ld * es, host_patches, (size_t)enc->patch_dim * es,
-                               (size_t)enc->patch_dim * es, (size_t)T, cudaMemcpyHostToDevice, enc->h2d_stream));
+  EPD_CUDA(cudaMemcpy2DAsync(dp, (size_t)ld * es, host_patches, (size_t)enc->patch_dim * es,
+                             (size_t)enc->patch_dim * es, (size_t)bs.T, cudaMemcpyHostToDevice, enc->h2d_stream));
   EPD_CUDA(cudaEventRecord(enc->h2d_done[b], enc->h2d_stream));
   // the encode, on the caller's stream: after its patches have arrived and after the features this slot held
   // two calls ago have left for the host
   EPD_CUDA(cudaStreamWaitEvent(s, enc->h2d_done[b], 0));
   if (enc->d2h_valid[b]) EPD_CUDA(cudaStreamWaitEvent(s, enc->d2h_done[b], 0));
-  int64_t rows = 0;
-  int rc = encode_device(enc, dp, ld, grid_thw, n_images, df, features_capacity_rows, &rows, out_cu_rows, s);
+  rc = encode_validated(enc, dp, ld, grid_thw, n_images, df, bs, s);
   if (rc) return rc;
-  if (out_rows) *out_rows = rows;
   EPD_CUDA(cudaEventRecord(enc->compute_done[b], s));
   enc->compute_valid[b] = true;
   // features -> host, behind the encode, while the caller's stream goes on with the next call
   EPD_CUDA(cudaStreamWaitEvent(enc->d2h_stream, enc->compute_done[b], 0));
-  if (rows > 0)
-    EPD_CUDA(cudaMemcpyAsync(host_features, df, (size_t)rows * c.out_dim * es, cudaMemcpyDeviceToHost, enc->d2h_stream));
+  EPD_CUDA(cudaMemcpyAsync(host_features, df, (size_t)bs.Tm * c.out_dim * es, cudaMemcpyDeviceToHost, enc->d2h_stream));
   EPD_CUDA(cudaEventRecord(enc->d2h_done[b], enc->d2h_stream));
   enc->d2h_valid[b] = true;
   return EPD_OK;
@@ -632,51 +729,130 @@ int epd_encode_frames(epd_encoder_t* enc, const void* frames, const int32_t* gri
                       int64_t* out_rows, int32_t* out_cu_rows, void* stream) {
   if (!enc) return EPD_EINVAL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const epd_config_t& c = enc->cfg;
-  if (n_images < 0 || (n_images > 0 && (!grid_thw || !frames || !mean || !inv_std))) return EPD_EINVAL;
-  if (c.in_channels > 4) return EPD_EUNSUPPORTED;
-  if (n_images > c.max_images) return EPD_ECAPACITY;
-  // byte offset of every item's frames in the packed buffer
-  if (enc->staged_off_valid) EPD_CUDA(cudaEventSynchronize(enc->staged_off));
-  int64_t off = 0, T = 0;
-  for (int i = 0; i < n_images; ++i) {
-    const int64_t t = grid_thw[3 * i], h = grid_thw[3 * i + 1], w = grid_thw[3 * i + 2];
-    if (t < 1 || h < 1 || w < 1) return EPD_EINVAL;
-    if (t > c.max_tokens || t * h > c.max_tokens || t * h * w > c.max_tokens) return EPD_ECAPACITY;
-    T += t * h * w;
-    if (T > c.max_tokens) return EPD_ECAPACITY;
-    enc->pinned_off[i] = off;
-    off += t * c.temporal_patch * c.in_channels * (h * c.patch) * (w * c.patch);
-  }
-  enc->pinned_off[n_images] = off;
-  // the integer layout (grid, cu_seqlens) must be on the device before the patch kernel reads it
   enc->launches = 0;
   enc->prof_used = 0;
-  int64_t T2 = 0;
-  int rc = prepare_batch(enc, grid_thw, n_images, features_capacity_rows, out_rows, out_cu_rows, &T2, s);
+  // everything is validated before anything is enqueued
+  if (enc->cfg.in_channels > 4) return EPD_EUNSUPPORTED;
+  BatchShape bs;
+  int rc = validate_encode(enc, enc->at<void>(enc->lay.pix_patches), (enc->patch_dim + 7) / 8 * 8, grid_thw, n_images,
+                           features, features_capacity_rows, &bs);
   if (rc) return rc;
-  if (T2 == 0) return EPD_OK;
-  const int64_t launches_layout = enc->launches;
+  if (bs.T > 0 && (!frames || !mean || !inv_std)) return EPD_EINVAL;
+  fill_host_outputs(bs, n_images, out_rows, out_cu_rows);
+  if (bs.T == 0) return EPD_OK;
+  std::vector<int64_t> off(n_images);
+  int64_t at = 0;
+  for (int i = 0; i < n_images; ++i) {
+    off[i] = at;
+    at += item_frame_bytes(enc->cfg, grid_thw + 3 * i);
+  }
+  return encode_frames_at(enc, frames, off.data(), grid_thw, n_images, mean, inv_std, features, bs, s);
+}
+
+int epd_encode_frames_cached(epd_encoder_t* enc, epd_feature_cache_t* cache, const void* frames,
+                             const int32_t* grid_thw, int32_t n_images, const float* mean, const float* inv_std,
+                             void* features, int64_t features_capacity_rows, int64_t* out_rows, int32_t* out_cu_rows,
+                             uint64_t* out_keys, uint8_t* out_hit, void* stream) {
+  if (!enc || !cache) return EPD_EINVAL;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const epd_config_t& c = enc->cfg;
+  const size_t row_bytes = (size_t)c.out_dim * (c.dtype == EPD_DTYPE_F32 ? 4 : 2);
+  enc->launches = 0;
+  enc->prof_used = 0;
+  if (c.in_channels > 4) return EPD_EUNSUPPORTED;
+  BatchShape bs;
+  int rc = validate_encode(enc, enc->at<void>(enc->lay.pix_patches), (enc->patch_dim + 7) / 8 * 8, grid_thw, n_images,
+                           features, features_capacity_rows, &bs);
+  if (rc) return rc;
+  if (bs.T > 0 && (!frames || !mean || !inv_std)) return EPD_EINVAL;
+  fill_host_outputs(bs, n_images, out_rows, out_cu_rows);
+  if (bs.T == 0) return EPD_OK;
+  // content keys of all items: hashed on the device, read back (the one host wait of this call)
+  if (enc->staged_off_valid) EPD_CUDA(cudaEventSynchronize(enc->staged_off));
+  std::vector<int64_t> off(n_images + 1);
+  off[0] = 0;
+  for (int i = 0; i < n_images; ++i) off[i + 1] = off[i] + item_frame_bytes(c, grid_thw + 3 * i);
+  for (int i = 0; i <= n_images; ++i) {
+    if (off[i] % 8) return EPD_EUNSUPPORTED;   // the hash reads 8-byte words
+    enc->pinned_off[i] = off[i];
+  }
   EPD_CUDA(cudaMemcpyAsync(enc->at<int64_t>(enc->lay.item_off), enc->pinned_off, ((size_t)n_images + 1) * sizeof(int64_t),
                            cudaMemcpyHostToDevice, s));
   EPD_CUDA(cudaEventRecord(enc->staged_off, s));
   enc->staged_off_valid = true;
-  const int64_t ld = (enc->patch_dim + 7) / 8 * 8;
-  EPD_CUDA(patchify(c.dtype, static_cast<const uint8_t*>(frames), enc->at<int64_t>(enc->lay.item_off),
-                    enc->at<int32_t>(enc->lay.grid), enc->at<int32_t>(enc->lay.cu), n_images, T2,
-                    enc->at<void>(enc->lay.pix_patches), ld, c.in_channels, c.patch, c.temporal_patch, mean, inv_std, s));
-  rc = encode_device(enc, enc->at<void>(enc->lay.pix_patches), ld, grid_thw, n_images, features, features_capacity_rows,
-                     out_rows, out_cu_rows, s);
-  enc->launches += launches_layout + 1;
-  return rc;
+  EPD_CUDA(content_hash(frames, enc->at<int64_t>(enc->lay.item_off), n_images, enc->at<uint64_t>(enc->lay.keys), s));
+  EPD_CUDA(cudaMemcpyAsync(enc->pinned_keys, enc->at<uint64_t>(enc->lay.keys), (size_t)n_images * sizeof(uint64_t),
+                           cudaMemcpyDeviceToHost, s));
+  EPD_CUDA(cudaStreamSynchronize(s));
+  const int64_t hash_launches = 2;
+  // hits are copied from the cache straight to their rows; the first occurrence of every missing key is encoded
+  std::vector<int> todo;               // items to encode
+  std::vector<int> source(n_images, -1);   // for a missing item: position in `todo` of the item that carries its key
+  for (int i = 0; i < n_images; ++i) {
+    const uint64_t key = enc->pinned_keys[i];
+    const int64_t rows = bs.cuo[i + 1] - bs.cuo[i];
+    if (out_keys) out_keys[i] = key;
+    const int st = epd_feature_cache_lookup(cache, key, rows, static_cast<uint8_t*>(features) + (size_t)bs.cuo[i] * row_bytes,
+                                            stream);
+    if (st < 0) return st;
+    if (out_hit) out_hit[i] = st == EPD_OK ? 1 : 0;
+    if (st == EPD_OK) continue;
+    for (size_t k = 0; k < todo.size() && source[i] < 0; ++k)
+      if (enc->pinned_keys[todo[k]] == key && std::memcmp(grid_thw + 3 * todo[k], grid_thw + 3 * i, 12) == 0)
+        source[i] = (int)k;
+    if (source[i] < 0) {
+      source[i] = (int)todo.size();
+      todo.push_back(i);
+    }
+  }
+  int64_t launches = hash_launches;
+  if (!todo.empty()) {
+    const int m = (int)todo.size();
+    std::vector<int32_t> g(3 * m);
+    std::vector<int64_t> sub_off(m);
+    for (int k = 0; k < m; ++k) {
+      std::memcpy(&g[3 * k], grid_thw + 3 * todo[k], 12);
+      sub_off[k] = off[todo[k]];
+    }
+    BatchShape sub;
+    if ((rc = validate_grids(enc, g.data(), m, -1, &sub))) return rc;
+    // the missing items are encoded as a batch of their own into the staging buffer of the workspace
+    uint8_t* scratch = enc->at<uint8_t>(enc->lay.stage_features);
+    rc = encode_frames_at(enc, frames, sub_off.data(), g.data(), m, mean, inv_std, scratch, sub, s);
+    if (rc) return rc;
+    launches += enc->launches;
+    for (int i = 0; i < n_images; ++i) {
+      if (source[i] < 0) continue;
+      const int k = source[i];
+      const size_t bytes = (size_t)(sub.cuo[k + 1] - sub.cuo[k]) * row_bytes;
+      if (bytes)
+        EPD_CUDA(cudaMemcpyAsync(static_cast<uint8_t*>(features) + (size_t)bs.cuo[i] * row_bytes,
+                                 scratch + (size_t)sub.cuo[k] * row_bytes, bytes, cudaMemcpyDeviceToDevice, s));
+    }
+    for (int k = 0; k < m; ++k) {
+      rc = epd_feature_cache_insert(cache, enc->pinned_keys[todo[k]], sub.cuo[k + 1] - sub.cuo[k],
+                                    scratch + (size_t)sub.cuo[k] * row_bytes, stream);
+      if (rc == EPD_ECAPACITY) rc = EPD_OK;      // an item larger than the whole pool is simply not cached
+      if (rc) return rc;
+    }
+  }
+  enc->launches = launches;
+  return note_last_launch(enc, s);
 }
 
 int epd_encoder_last_status(epd_encoder_t* enc) {
   if (!enc) return EPD_EINVAL;
-  int32_t st = 0;
-  EPD_CUDA(cudaDeviceSynchronize());
-  EPD_CUDA(cudaMemcpy(&st, enc->ws + enc->lay.status, sizeof(st), cudaMemcpyDeviceToHost));
-  if (st != 0) EPD_CUDA(cudaMemset(enc->ws + enc->lay.status, 0, sizeof(st)));
+  // wait for the encoder's own most recent work only (an event behind its last launch), and read the word on
+  // a non-blocking stream of the encoder's: other streams and processes sharing the GPU are not stalled
+  if (enc->last_launch_valid) EPD_CUDA(cudaStreamWaitEvent(enc->aux_stream, enc->last_launch, 0));
+  EPD_CUDA(cudaMemcpyAsync(enc->pinned_status, enc->ws + enc->lay.status, sizeof(int32_t), cudaMemcpyDeviceToHost,
+                           enc->aux_stream));
+  EPD_CUDA(cudaStreamSynchronize(enc->aux_stream));
+  const int32_t st = *enc->pinned_status;
+  if (st != 0) {
+    EPD_CUDA(cudaMemsetAsync(enc->ws + enc->lay.status, 0, sizeof(int32_t), enc->aux_stream));
+    EPD_CUDA(cudaStreamSynchronize(enc->aux_stream));
+  }
   return st;
 }
 
@@ -686,21 +862,14 @@ int epd_encoder_uses_tensor_cores(const epd_encoder_t* enc) { return enc && enc-
 
 int epd_encoder_destroy(epd_encoder_t* enc) {
   if (!enc) return EPD_OK;
-  cudaDeviceSynchronize();
-  if (enc->staged) cudaEventDestroy(enc->staged);
-  if (enc->staged_off) cudaEventDestroy(enc->staged_off);
-  for (epd_encoder::GraphEntry& g : enc->graphs) cudaGraphExecDestroy(g.exec);
-  for (int b = 0; b < 2; ++b) {
-    if (enc->h2d_done[b]) cudaEventDestroy(enc->h2d_done[b]);
-    if (enc->compute_done[b]) cudaEventDestroy(enc->compute_done[b]);
-    if (enc->d2h_done[b]) cudaEventDestroy(enc->d2h_done[b]);
-  }
-  if (enc->h2d_stream) cudaStreamDestroy(enc->h2d_stream);
-  if (enc->d2h_stream) cudaStreamDestroy(enc->d2h_stream);
-  if (enc->pinned_off) cudaFreeHost(enc->pinned_off);
-  for (cudaEvent_t ev : enc->prof_events) cudaEventDestroy(ev);
-  if (enc->pinned) cudaFreeHost(enc->pinned);
-  delete enc;
+  // the encoder's work must be over before its buffers go away: its last launch on the caller's stream, and
+  // the copies on its own streams
+  if (enc->last_launch_valid) cudaEventSynchronize(enc->last_launch);
+  for (int b = 0; b < 2; ++b)
+    if (enc->d2h_valid[b]) cudaEventSynchronize(enc->d2h_done[b]);
+  if (enc->h2d_stream) cudaStreamSynchronize(enc->h2d_stream);
+  if (enc->aux_stream) cudaStreamSynchronize(enc->aux_stream);
+  release_host_side(enc);
   return EPD_OK;
 }
 
@@ -722,7 +891,7 @@ const char* epd_strerror(int status) {
 int epd_debug_bookkeeping(epd_encoder_t* enc, int32_t* cu_seqlens, int32_t* pos_row, int32_t* pos_col,
                           int32_t* merge_idx) {
   if (!enc || enc->last_T < 0) return EPD_EINVAL;
-  EPD_CUDA(cudaDeviceSynchronize());
+  if (enc->last_launch_valid) EPD_CUDA(cudaEventSynchronize(enc->last_launch));
   const size_t n = enc->last_grid.size() / 3, T = (size_t)enc->last_T;
   if (cu_seqlens) EPD_CUDA(cudaMemcpy(cu_seqlens, enc->ws + enc->lay.cu, (n + 1) * 4, cudaMemcpyDeviceToHost));
   if (pos_row) EPD_CUDA(cudaMemcpy(pos_row, enc->ws + enc->lay.pos_row, T * 4, cudaMemcpyDeviceToHost));
@@ -745,11 +914,15 @@ int epd_debug_run_block(epd_encoder_t* enc, int32_t layer, void* x, const int32_
   int64_t T = 0;
   enc->launches = 0;
   enc->prof_used = 0;
-  int rc = prepare_batch(enc, grid_thw, n_images, -1, nullptr, nullptr, &T, s);
+  BatchShape bs;
+  int rc = validate_grids(enc, grid_thw, n_images, -1, &bs);
   if (rc) return rc;
+  T = bs.T;
   if (T == 0) return EPD_OK;
+  if ((rc = stage_layout(enc, grid_thw, n_images, bs, s))) return rc;
   if ((rc = run_block(enc, layer, static_cast<float*>(x), T, n_images, s))) return rc;
-  return finish_profile(enc, s);
+  if ((rc = finish_profile(enc, s))) return rc;
+  return note_last_launch(enc, s);
 }
 
 int epd_debug_use_graphs(epd_encoder_t* enc, int32_t enable) {

@@ -163,7 +163,15 @@ int epd_feature_cache_lookup(epd_feature_cache_t* c, uint64_t key, int64_t rows,
 
 int epd_feature_cache_insert(epd_feature_cache_t* c, uint64_t key, int64_t rows, const void* src, void* stream) {
   if (!c || rows < 0 || (rows > 0 && !src)) return EPD_EINVAL;
-  if (c->index.count(key)) return EPD_OK;            // already cached
+  auto found = c->index.find(key);
+  if (found != c->index.end()) {
+    if (c->fifo[found->second].rows == rows) return EPD_OK;    // already cached
+    // same key, other row count: the old entry could never be hit again (lookups require the row count to
+    // match), so it is dropped and the new one stored
+    c->fifo.erase(c->fifo.begin() + (long)found->second);
+    c->evictions++;
+    c->reindex();
+  }
   const size_t bytes = ((size_t)rows * c->row_bytes + 255) / 256 * 256;
   if (bytes > c->pool_bytes) return EPD_ECAPACITY;
   // ring allocation: continue at head, wrap to 0 when the tail of the pool is too short, evict oldest

@@ -12,99 +12,18 @@
 // Both operands are K-major (row-major [rows, K]), so one shared-memory descriptor form serves both.
 // Ragged M, N and K are handled by TMA: zero fill on loads, clipping on stores.
 // Every mbarrier wait is bounded: on expiry the kernel records EPD_ETIMEOUT and drains.
-#include <cuda.h>
-
-#include <mutex>
-
-#include "common.cuh"
+#include "tcgen05_common.cuh"
 
 namespace epd {
 namespace {
+
+using namespace tc;
 
 constexpr int BM = 128;
 constexpr int BK = 64;          // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int kEpiWarps = 4;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
-constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
-
-// ---------------------------------------------------------------------------------------------
-// PTX wrappers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false (and raises *abort_flag) if the phase did not complete in time or
-// another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  int spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 255) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycles) {
-        *abort_flag = 1;
-        return false;
-      }
-    }
-  }
-  return true;
-}
-
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(smem_u32(bar)), "r"(x), "r"(y)
-      : "memory");
-}
-
-// TMA tensor store / reduce-add of one staged box, tracked by the issuing thread's bulk group.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, int x, int y, const void* smem_src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, int x, int y, const void* smem_src) {
-  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void bulk_wait_read() {
-  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
-               "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // D[tmem] (+)= A[smem] . B[smem]^T, bf16 inputs, fp32 accumulation, issued by one thread.
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
@@ -116,49 +35,9 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint
       ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// mbarrier arrives once all tcgen05.mma issued so far by this thread have completed.
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-
-// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives row (lane base + i).
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled
-// (the layout a TMA box of 64 bf16 columns produces): 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);  // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                       // leading byte offset (unused for swizzled K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;             // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;                       // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                       // 128-byte swizzle
-  return d;
-}
-
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = BN.
 __host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-
-__device__ __forceinline__ float gelu_tanh_fast(float x) {
-  const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-  float t;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
-  return 0.5f * x * (1.0f + t);
 }
 
 template <int BN, int STAGES>
@@ -171,8 +50,9 @@ struct SmemLayout {
   static constexpr int kOutBufBytes = 32 * 128;
   static constexpr int kOutOffset = STAGES * kStageBytes;
   static constexpr int kBarOffset = kOutOffset + kEpiWarps * kOutBufs * kOutBufBytes;
-  // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], tmem base, abort flag, bias[kEpiWarps][BN]
-  static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 4) * 8 + 16;
+  // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain, (spare), tmem base, abort flag,
+  // bias[kEpiWarps][BN]
+  static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 6) * 8 + 16;
   static constexpr int kTotal = kBiasOffset + kEpiWarps * BN * 4;
   static_assert(kTotal + 1024 <= 232448, "exceeds the shared memory of one CTA");
   static constexpr int kDynamic = kTotal + 1024;  // slack to align the ring to 1024 bytes
@@ -185,7 +65,7 @@ template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                  const __grid_constant__ CUtensorMap tm_out, const __nv_bfloat16* __restrict__ bias, int M, int N,
-                 int K, int* __restrict__ status) {
+                 int K, int* __restrict__ status, long long wait_limit) {
   using L = SmemLayout<BN, STAGES>;
   static_assert(L::kDynamic > 116 * 1024, "one CTA per SM is assumed by the TMEM allocation");
   static_assert(BN % 16 == 0 && BN >= 32 && BN <= 256, "UMMA N");
@@ -199,8 +79,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
   uint64_t* empty = full + STAGES;
   uint64_t* tmem_full = empty + STAGES;
   uint64_t* tmem_empty = tmem_full + 2;
-  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  uint64_t* drain_bar = tmem_empty + 2;    // after an abort: the issuing thread's MMAs have completed
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(drain_bar + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
+  const WaitCtx wc{abort_flag, 0u, wait_limit};
+  uint32_t loads_issued = 0;               // stage loads issued by the producer thread
   float* bias_s = reinterpret_cast<float*>(smem + L::kBiasOffset);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -211,6 +94,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], kEpiWarps); }
+    mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -228,19 +112,20 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_x) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
+      prefetch_map(&tm_x);
+      prefetch_map(&tm_w);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(&empty[stage], phase ^ 1, wc)) { ok = false; break; }
           uint8_t* sa = smem + stage * L::kStageBytes;
           mbar_expect_tx(&full[stage], L::kStageBytes);
           tma_load_2d(sa, &tm_x, kb * BK, m0, &full[stage]);
           tma_load_2d(sa + L::kABytes, &tm_w, kb * BK, n0, &full[stage]);
+          ++loads_issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }
@@ -256,11 +141,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        if (!mbar_wait(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) break;
+        if (!mbar_wait(&tmem_empty[acc], acc_phase ^ 1, wc)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kAccStride;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(&full[stage], phase, wc)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint64_t da = smem_desc_k_sw128(sa), db = smem_desc_k_sw128(sa + L::kABytes);
@@ -287,14 +172,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     int obuf = 0;
     int acc = 0;
     uint32_t acc_phase = 0;
-    if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_out) : "memory");
+    if (lane == 0) prefetch_map(&tm_out);
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
       const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
       __syncwarp();
       for (int i = lane; i < BN; i += 32)
         bs[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
       __syncwarp();
-      if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) break;
+      if (!mbar_wait(&tmem_full[acc], acc_phase, wc)) break;
       tc_fence_after();
       const int row0 = m0 + q * 32;
       const uint32_t taddr = tmem_base + acc * kAccStride + ((uint32_t)(q * 32) << 16);
@@ -365,9 +250,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
   tc_fence_before();
   __syncthreads();
   if (*abort_flag) {
-    // a wait expired: report it and give loads still in flight time to land before the CTA's
-    // shared memory is released
+    // A wait expired.  Every role has left its loop (the barrier above), so nothing new is issued.  What was
+    // issued completes by itself: the producer waits for its last load of every stage, the issuing thread for
+    // its last MMA (a commit arrives only after all earlier MMAs), the epilogue warps have waited for their
+    // stores; a fixed pause on top, then shared and tensor memory are released.
     if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, 0, kStatusTimeout);
+    if (warp == 0 && lane == 0) drain_ring(full, STAGES, loads_issued);
+    if (warp == 1 && lane == 0) {
+      umma_commit(drain_bar);
+      mbar_wait_drain(drain_bar, 0);
+    }
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
   }
@@ -380,48 +272,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  });
-  return fn;
-}
-
 // Tensor map of a row-major matrix [rows, cols] with leading dimension ld (elements of elem_bytes),
 // box = box_rows x (128 bytes of columns), 128-byte swizzle.
 bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows,
               int elem_bytes) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * elem_bytes};
-  cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(tm, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
-            const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
+  return make_tensor_map_2d(tm, base, rows, cols, ld * elem_bytes, box_rows, 128 / elem_bytes, elem_bytes,
+                            CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM>
@@ -429,16 +285,16 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
                    int K, int* status, cudaStream_t s) {
   using L = SmemLayout<BN, STAGES>;
   auto kern = linear_tc_kernel<BN, STAGES, OutT, ACT, ACCUM>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static PerDeviceOnce configured;
+  cudaError_t e = once_per_device(configured, [&] {
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+  });
+  if (e != cudaSuccess) return e;
   const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
-  const int sms_avail = limited_sms(sm_count());
+  const int sms_avail = limited_sms(device_sm_count());
   const int grid = tiles < sms_avail ? tiles : sms_avail;
-  return launch_pdl(kern, dim3(grid), dim3(kThreads), L::kDynamic, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K, status);
+  return launch_pdl(kern, dim3(grid), dim3(kThreads), L::kDynamic, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K, status,
+                    wait_limit_cycles());
 }
 
 template <int BN, int STAGES>
@@ -470,7 +326,7 @@ cudaError_t launch_bn(const CUtensorMap& tx, const CUtensorMap& tw, const CUtens
 int pick_bn(int M, int N) {
   const int cands[3] = {256, 192, 128};
   const double eff[3] = {1.0, 0.88, 0.65};
-  const int sms = limited_sms(sm_count());
+  const int sms = limited_sms(device_sm_count());
   const int m_tiles = (M + BM - 1) / BM;
   int best = 256;
   double best_cost = 1e300;
@@ -493,7 +349,7 @@ bool linear_tc_supported(const void* x, int64_t ldx, const void* w, int64_t ldw,
   if (M < 1 || N < 8 || K < 8 || (N % 8) || M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return false;
   if (((uintptr_t)x & 15) || ((uintptr_t)w & 15) || ((uintptr_t)out & 15)) return false;
   if ((ldx % 8) || (ldw % 8) || (ldo % (out_f32 ? 4 : 8))) return false;
-  return encode_tiled_fn() != nullptr;
+  return tensor_maps_available();
 }
 
 cudaError_t linear_tc(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out, int64_t ldo,

@@ -29,23 +29,19 @@
 // and k share it.
 // Every mbarrier wait is bounded: on expiry the CTA records EPD_ETIMEOUT and drains; the two cluster
 // barriers (start, end) are reached by both CTAs on every path.
-#include <cuda.h>
-
-#include <mutex>
-
-#include "common.cuh"
+#include "tcgen05_common.cuh"
 
 namespace epd {
 namespace {
+
+using namespace tc;
 
 constexpr int BM = 128;         // rows of x per CTA (256 per pair)
 constexpr int BK = 64;          // 64 bf16 = 128 bytes = one swizzle row
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
-constexpr long long kWaitCycles = 4000000000LL;  // ~2 s at 2 GHz
 constexpr int kMaxDynamicSmem = 232448;           // 227 KB: the most one CTA can have
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ uint32_t cluster_rank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -61,44 +57,12 @@ __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
 // Arrive on a barrier given by its cluster-window address (own CTA's or the peer's).  Relaxed: the
 // arrival only says "my tcgen05.ld of this accumulator have completed" (tcgen05.wait::ld has returned),
 // no memory written by this thread is handed over; a release here would also wait for the thread's
 // output stores still in flight to L2 (measured ~2000 clocks per tile).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  int spins = 0;
-  while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 255) == 0) {
-      if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycles) {
-        *abort_flag = 1;
-        return false;
-      }
-    }
-  }
-  return true;
 }
 // Tensor load into this CTA's shared memory whose completion bytes are counted on a barrier that may
 // live in the other CTA of the pair (given by its cluster-window address).
@@ -109,18 +73,6 @@ __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorM
       ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(bar_cluster_addr), "r"(x), "r"(y)
       : "memory");
 }
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, int x, int y, const void* smem_src) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* tm, int x, int y, const void* smem_src) {
-  asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
                "r"(cols) : "memory");
@@ -131,8 +83,6 @@ __device__ __forceinline__ void tmem_relinquish_pair() {
 __device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t cols) {
   asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
 }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
 // D[tmem, both CTAs] (+)= A[smem, 128 rows per CTA] . B[smem, half the columns per CTA]^T; issued by
 // one thread of the leader CTA.
@@ -154,40 +104,9 @@ __device__ __forceinline__ void umma_commit_both(uint64_t* bar) {
       : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// K-major tile whose rows are 128 bytes, 128-byte swizzled: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr & 0x3FFFF) >> 4);
-  d |= (uint64_t)1 << 16;
-  d |= (uint64_t)(1024 >> 4) << 32;
-  d |= (uint64_t)1 << 46;
-  d |= (uint64_t)2 << 61;
-  return d;
-}
 // bf16 x bf16 -> fp32, both operands K-major, M = 256 over the pair, N = BN.
 __host__ __device__ constexpr uint32_t instr_desc_pair(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-}
-
-__device__ __forceinline__ float gelu_tanh_fast(float x) {
-  const float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-  float t;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
-  return 0.5f * x * (1.0f + t);
 }
 
 // Destination of the QKV variant's epilogue.
@@ -209,8 +128,9 @@ struct PairLayout {
   static constexpr int kOutBufBytes = 32 * 128;         // one staging buffer per epilogue warp
   static constexpr int kOutOffset = STAGES * kStageBytes;
   static constexpr int kBarOffset = kOutOffset + kEpiWarps * kOutBufBytes;
-  // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], tmem base, abort flag, bias[kEpiWarps][BN/2]
-  static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 4) * 8 + 16;
+  // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain, (spare), tmem base, abort flag,
+  // bias[kEpiWarps][BN/2]
+  static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 6) * 8 + 16;
   static constexpr int kTotal = kBiasOffset + kEpiWarps * (BN / 2) * 4;
   static constexpr int kDynamic = kTotal + 1024;
   static_assert(kDynamic <= 232448, "exceeds the shared memory of one CTA");
@@ -224,7 +144,7 @@ template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_out, const __nv_bfloat16* __restrict__ bias, int M, int N,
-                   int K, int* __restrict__ status, const RopeSplitArgs rs) {
+                   int K, int* __restrict__ status, long long wait_limit, const RopeSplitArgs rs) {
   static_assert(!ROPE || (sizeof(OutT) == 2 && ACT == 0 && !ACCUM), "the QKV variant writes bf16, no activation");
   using L = PairLayout<BN, STAGES>;
   static_assert(BN == 256 || BN == 128, "tile width");
@@ -238,12 +158,16 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   uint64_t* empty = full + STAGES;                                      // one set per CTA
   uint64_t* tmem_full = empty + STAGES;                                 // one set per CTA
   uint64_t* tmem_empty = tmem_full + 2;                                 // used in the leader only
-  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+  uint64_t* drain_bar = tmem_empty + 2;     // one per CTA; after an abort: the pair's MMAs have completed
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(drain_bar + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_base_slot + 1);
+  uint32_t loads_issued = 0;                // stage loads issued by this CTA's producer thread
   float* bias_s = reinterpret_cast<float*>(smem + L::kBiasOffset);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();          // 0 = leader
+  // a wait that expires raises the abort flag of both CTAs of the pair
+  const WaitCtx wc{abort_flag, map_to_rank(smem_u32(const_cast<int*>(abort_flag)), rank ^ 1u), wait_limit};
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int m_tiles = (M + 2 * BM - 1) / (2 * BM), n_tiles = (N + BN - 1) / BN;
   const int num_tiles = m_tiles * n_tiles;
@@ -252,6 +176,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tmem_full[a], 1); mbar_init(&tmem_empty[a], 2 * kEpiWarps); }
+    mbar_init(drain_bar, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -270,8 +195,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_x) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
+      prefetch_map(&tm_x);
+      prefetch_map(&tm_w);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -279,13 +204,14 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;        // this CTA's rows of x
         const int n0 = (tile / m_tiles) * BN + (int)rank * (BN / 2);       // this CTA's half of the w tile
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(&empty[stage], phase ^ 1, abort_flag)) { ok = false; break; }
+          if (!mbar_wait<true>(&empty[stage], phase ^ 1, wc)) { ok = false; break; }
           uint8_t* sa = smem + stage * L::kStageBytes;
           // the leader's barrier counts the bytes of both CTAs
           if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
           const uint32_t bar = map_to_rank(smem_u32(&full[stage]), 0);
           tma_load_2d_pair(sa, &tm_x, kb * BK, m0, bar);
           tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BK, n0, bar);
+          ++loads_issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }
@@ -301,11 +227,11 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
-        if (!mbar_wait(&tmem_empty[acc], acc_phase ^ 1, abort_flag)) break;
+        if (!mbar_wait<true>(&tmem_empty[acc], acc_phase ^ 1, wc)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kAccStride;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(&full[stage], phase, abort_flag)) { ok = false; break; }
+          if (!mbar_wait<true>(&full[stage], phase, wc)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint64_t da = smem_desc_k_sw128(sa), db = smem_desc_k_sw128(sa + L::kABytes);
@@ -332,7 +258,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     const uint32_t tmem_empty_leader0 = map_to_rank(smem_u32(&tmem_empty[0]), 0);
     int acc = 0;
     uint32_t acc_phase = 0;
-    if (!ROPE && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_out) : "memory");
+    if (!ROPE && lane == 0) prefetch_map(&tm_out);
     const float2* rope_tab = rs.table;
     if constexpr (ROPE) {
       if (rs.table_in_smem > 0) {
@@ -352,7 +278,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       for (int i = lane; i < BN / 2; i += 32)
         bs[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
       __syncwarp();
-      if (!mbar_wait(&tmem_full[acc], acc_phase, abort_flag)) break;
+      if (!mbar_wait<true>(&tmem_full[acc], acc_phase, wc)) break;
       tc_fence_after();
       const int row0 = m0 + q * 32;
       const uint32_t taddr = tmem_base + acc * kAccStride + half * (BN / 2) + ((uint32_t)(q * 32) << 16);
@@ -451,7 +377,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           if (lane == 0) mbar_arrive_cluster(tmem_empty_leader0 + acc * 8);
         }
         // the staging buffer is free once the bulk store issued from it has read it
-        if (!ROPE && lane == 0) bulk_wait_read_all();
+        if (!ROPE && lane == 0) bulk_wait_read<0>();
         __syncwarp();
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -501,7 +427,18 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   tc_fence_before();
   __syncthreads();
   if (*abort_flag) {
+    // A wait expired (here or in the other CTA of the pair).  Every role of this CTA has left its loop, so
+    // nothing new is issued.  What was issued completes by itself: the leader's producer waits for the last
+    // load of every stage (its barriers count the bytes of both CTAs), the leader's issuing thread commits
+    // to the drain barrier of both CTAs (a commit arrives only after all earlier MMAs) and each CTA waits for
+    // it, the epilogue warps have waited for their stores; a fixed pause on top, then the cluster barrier, after
+    // which shared and tensor memory are released.
     if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, 0, kStatusTimeout);
+    if (warp == 0 && lane == 0 && rank == 0) drain_ring<true>(full, STAGES, loads_issued);
+    if (warp == 1 && lane == 0) {
+      if (rank == 0) umma_commit_both(drain_bar);
+      mbar_wait_drain<true>(drain_bar, 0);
+    }
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
   }
@@ -515,48 +452,12 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
 // ---------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  });
-  return fn;
-}
-
 // Tensor map of a row-major matrix [rows, cols] with leading dimension ld (elements of elem_bytes),
 // box = box_rows x (128 bytes of columns), 128-byte swizzle.
 bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows,
               int elem_bytes) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)ld * elem_bytes};
-  cuuint32_t box[2] = {(cuuint32_t)(128 / elem_bytes), (cuuint32_t)box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(tm, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
-            const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-    if (n <= 0) n = 148;
-  }
-  return n;
+  return make_tensor_map_2d(tm, base, rows, cols, ld * elem_bytes, box_rows, 128 / elem_bytes, elem_bytes,
+                            CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
 template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE = false>
@@ -564,20 +465,23 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
                    int K, int* status, cudaStream_t s, const RopeSplitArgs& rs = RopeSplitArgs{}) {
   using L = PairLayout<BN, STAGES>;
   auto kern = linear_pair_kernel<BN, STAGES, OutT, ACT, ACCUM, ROPE>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         ROPE ? kMaxDynamicSmem : L::kDynamic);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  static PerDeviceOnce configured;
+  cudaError_t e = once_per_device(configured, [&] {
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ROPE ? kMaxDynamicSmem : L::kDynamic);
+  });
+  if (e != cudaSuccess) return e;
   const size_t smem_bytes = L::kDynamic + (ROPE ? (size_t)rs.table_in_smem * sizeof(float2) : 0);
   const int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
-  // pairs that can be resident at once (SMs pair up inside a GPC, so this can be below SMs / 2)
-  static int max_pairs = 0;
-  if (max_pairs == 0) {
+  // pairs that can be resident at once on this device (SMs pair up inside a GPC, so this can be below SMs / 2)
+  static PerDeviceInt resident;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  const int slot = dev >= 0 && dev < 64 ? dev : 0;
+  int max_pairs = resident.v[slot].load(std::memory_order_relaxed);
+  if (max_pairs == 0 || slot != dev) {
+    const int sms = device_sm_count();
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(sm_count() / 2 * 2);
+    cfg.gridDim = dim3(sms / 2 * 2);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = L::kDynamic;
     cudaLaunchAttribute attr;
@@ -590,14 +494,15 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n <= 0) {
       (void)cudaGetLastError();
-      n = sm_count() / 2;
+      n = sms / 2;
     }
-    max_pairs = n < sm_count() / 2 ? n : sm_count() / 2;
+    max_pairs = n < sms / 2 ? n : sms / 2;
+    if (slot == dev) resident.v[slot].store(max_pairs, std::memory_order_relaxed);
   }
   const int avail = limited_sms(2 * max_pairs) / 2 > 0 ? limited_sms(2 * max_pairs) / 2 : 1;   // pairs within the SM budget
   const int pairs = tiles < avail ? tiles : avail;
   return launch_pdl(kern, dim3(2 * pairs), dim3(kThreads), smem_bytes, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K,
-                    status, rs);
+                    status, wait_limit_cycles(), rs);
 }
 
 template <int BN, int STAGES>

@@ -51,7 +51,9 @@ int epd_op_rope_attention_static(int32_t dtype, const void* qkv, const int32_t* 
                                  int64_t T, int32_t heads, int32_t head_dim, float theta, void* stream) {
   using namespace epd;
   if (dtype != EPD_DTYPE_F32 && dtype != EPD_DTYPE_BF16) return EPD_EINVAL;
-  if (T < 0 || n_seg < 0 || heads < 1 || head_dim < 4 || head_dim % 4 || head_dim > kMaxHeadDim) return EPD_EINVAL;
+  if (T < 0 || T > (1 << 30) || n_seg < 0 || heads < 1 || heads > 65535 || head_dim < 4 || head_dim % 4 ||
+      head_dim > kMaxHeadDim)
+    return EPD_EINVAL;   // also keeps the size arithmetic below far from overflow
   if (T == 0 || n_seg == 0) return EPD_OK;
   if (!qkv || !pos_row || !pos_col || !cu_seqlens || !host_cu_seqlens || !out) return EPD_EINVAL;
   if (host_cu_seqlens[0] != 0 || host_cu_seqlens[n_seg] != T) return EPD_EINVAL;

@@ -138,13 +138,39 @@ def normal(seed: int, tensor_id: str, shape: Sequence[int], std: float, mean: fl
 
 # ----------------------------------------------------------------------------- weights / inputs
 
-def make_weights(cfg: EncoderConfig, seed: int = 0, qkv_scale: float = 1.0) -> Dict:
+def make_layer_weights(cfg: EncoderConfig, l: int, seed: int = 0, qkv_scale: float = 1.0) -> Dict:
+    """Parameters of block l (each tensor has its own random stream, so blocks can be drawn one at a time)."""
+    h, m, d = cfg.hidden, cfg.mlp, cfg.dtype
+    p = f"layer{l}."
+
+    def mat(tid, shape, scale=1.0):
+        return normal(seed, p + tid, shape, 0.02 * scale, 0.0, d)
+
+    def gain(tid, n):
+        return normal(seed, p + tid, (n,), 0.02, 1.0, d)
+
+    return {
+        "norm1_w": gain("norm1_w", h),
+        "qkv_w": mat("qkv_w", (3 * h, h), qkv_scale),
+        "qkv_b": mat("qkv_b", (3 * h,)),
+        "out_w": mat("out_w", (h, h)),
+        "out_b": mat("out_b", (h,)),
+        "norm2_w": gain("norm2_w", h),
+        "fc1_w": mat("fc1_w", (m, h)),
+        "fc1_b": mat("fc1_b", (m,)),
+        "fc2_w": mat("fc2_w", (h, m)),
+        "fc2_b": mat("fc2_b", (h,)),
+    }
+
+
+def make_weights(cfg: EncoderConfig, seed: int = 0, qkv_scale: float = 1.0, with_layers: bool = True) -> Dict:
     """All encoder parameters as float32 arrays ([out, in] row-major matrices).
 
     qkv_scale > 1 multiplies W_qkv so attention logits become sharply peaked (a stress case
     for the online-softmax rescaling; not one of the benchmark configurations).
+    with_layers=False leaves "layers" empty (the caller draws the blocks with make_layer_weights).
     """
-    h, K, m = cfg.hidden, cfg.patch_dim, cfg.mlp
+    h, K = cfg.hidden, cfg.patch_dim
     d = cfg.dtype
 
     def mat(tid, shape, scale=1.0):
@@ -154,20 +180,8 @@ def make_weights(cfg: EncoderConfig, seed: int = 0, qkv_scale: float = 1.0) -> D
         return normal(seed, tid, (n,), 0.02, 1.0, d)
 
     w = {"patch_w": mat("patch_w", (h, K)), "patch_b": mat("patch_b", (h,)), "layers": []}
-    for l in range(cfg.layers):
-        p = f"layer{l}."
-        w["layers"].append({
-            "norm1_w": gain(p + "norm1_w", h),
-            "qkv_w": mat(p + "qkv_w", (3 * h, h), qkv_scale),
-            "qkv_b": mat(p + "qkv_b", (3 * h,)),
-            "out_w": mat(p + "out_w", (h, h)),
-            "out_b": mat(p + "out_b", (h,)),
-            "norm2_w": gain(p + "norm2_w", h),
-            "fc1_w": mat(p + "fc1_w", (m, h)),
-            "fc1_b": mat(p + "fc1_b", (m,)),
-            "fc2_w": mat(p + "fc2_w", (h, m)),
-            "fc2_b": mat(p + "fc2_b", (h,)),
-        })
+    if with_layers:
+        w["layers"] = [make_layer_weights(cfg, l, seed, qkv_scale) for l in range(cfg.layers)]
     w["final_norm_w"] = gain("final_norm_w", h)
     D4 = cfg.merge * cfg.merge * h
     if cfg.proj_kind == PROJ_LINEAR:

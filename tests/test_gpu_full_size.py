@@ -17,18 +17,12 @@ import torch
 import synth
 import paper_2601_11590_b200 as epd
 from oracle import encoder_oracle as O
+from tests.metrics import assert_parity, rel_err, worst_row_err
 
 pytestmark = pytest.mark.gpu
 
 TOL_BLOCK = 1e-2
 TOL_FINAL = 3e-2
-
-
-def rel_err(got, ref):
-    got = np.asarray(got, dtype=np.float64)
-    ref = np.asarray(ref, dtype=np.float64)
-    assert got.shape == ref.shape, (got.shape, ref.shape)
-    return float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300))
 
 
 def to_np(t):
@@ -82,8 +76,7 @@ def _check_blocks_on_rows(cfg, w, grids, taps, images, per_image, seed):
         x_in = to_np(taps[l])
         want = O.block_rows(cfg, w["layers"][l], x_in, bk, rows)
         got = to_np(taps[l + 1][torch.from_numpy(rows).cuda()])
-        errs.append(rel_err(got, want))
-    assert all(e <= TOL_BLOCK for e in errs), errs
+        errs.append(assert_parity(got, want, TOL_BLOCK, f"block {l}"))
     return errs
 
 
@@ -99,9 +92,8 @@ def test_cfg1_full_batch_one_image_end_to_end():
     a, b = int(bk["cu_seqlens"][i]), int(bk["cu_seqlens"][i + 1])
     ref = O.encode(cfg, w, patches[a:b], [grids[i]])
     got = to_np(feats[cu_rows[i]:cu_rows[i + 1]])
-    e = rel_err(got, ref)
-    print("cfg1 image 3 final", e)
-    assert e <= TOL_FINAL, e
+    e = assert_parity(got, ref, TOL_FINAL, "cfg1 image 3")
+    print("cfg1 image 3 final", e, "worst row", worst_row_err(got, ref))
     assert torch.isfinite(feats.float()).all()
     enc.close()
 
@@ -157,7 +149,7 @@ def test_cfg4_6b_widths_block_on_sampled_rows():
                   cfg.proj_hidden, 4 * cfg.hidden, epd.LINEAR_GELU_ERF)
     ref = O.gelu(O.linear(x.astype(np.float64), w["proj_w1"].astype(np.float64), w["proj_b1"].astype(np.float64)),
                  O.ACT_GELU_ERF)
-    assert rel_err(to_np(ph), ref) <= 4e-3
+    assert_parity(to_np(ph), ref, 4e-3)
     enc.close()
 
 
@@ -189,7 +181,110 @@ def test_cfg4_6b_widths_eight_layers_one_image_end_to_end():
     i = 5
     a, b = int(bk["cu_seqlens"][i]), int(bk["cu_seqlens"][i + 1])
     ref = O.encode(cfg, w, patches[a:b], [grids[i]])
-    e = rel_err(to_np(feats[cu_rows[i]:cu_rows[i + 1]]), ref)
+    e = assert_parity(to_np(feats[cu_rows[i]:cu_rows[i + 1]]), ref, TOL_FINAL, "cfg4 8 layers image 5")
     print("cfg4 8 layers image 5 final", e)
-    assert e <= TOL_FINAL, e
     enc.close()
+
+
+# ----------------------------------------------------------------------------- full batch, full depth
+
+def _full_depth_one_item(workload, item, seed):
+    """The whole batch of a benchmark configuration through every layer on the GPU; the features of one
+    item against the oracle's encode of that item alone (exact: attention is block-diagonal and every
+    other step is row-wise).  Returns (Frobenius ratio, worst-row ratio)."""
+    cfg, grids = synth.WORKLOADS[workload]
+    w = synth.make_weights(cfg, seed=seed)
+    enc, patches, feats, cu_rows, _ = _encode(cfg, grids, w, seed=seed)
+    bk = O.bookkeeping(grids)
+    assert np.array_equal(cu_rows, bk["cu_out"])
+    assert feats.shape == (synth.num_tokens(grids) // 4, cfg.out_dim) and torch.isfinite(feats.float()).all()
+    a, b = int(bk["cu_seqlens"][item]), int(bk["cu_seqlens"][item + 1])
+    got = to_np(feats[cu_rows[item]:cu_rows[item + 1]])
+    enc.close()
+    del enc, feats
+    torch.cuda.empty_cache()
+    ref = O.encode(cfg, w, patches[a:b], [grids[item]])
+    e = assert_parity(got, ref, TOL_FINAL, f"{workload} item {item}")
+    wr = worst_row_err(got, ref)
+    print(workload, "layers", cfg.layers, "item", item, "tokens", b - a, "final", e, "worst row", wr)
+    return e, wr
+
+
+def test_cfg2_full_batch_full_depth_smallest_image():
+    """32 variable-resolution images, all 27 layers: the smallest image of the batch."""
+    _, grids = synth.WORKLOADS["cfg2_vit06b_var32"]
+    lens = [t * h * w for t, h, w in grids]
+    _full_depth_one_item("cfg2_vit06b_var32", int(np.argmin(lens)), seed=0)
+
+
+def test_cfg3_full_batch_full_depth_clip():
+    """The 16384-token image + the 8-frame clip, all 27 layers: the 6272-token clip (attention over all
+    of its frames)."""
+    _full_depth_one_item("cfg3_vit06b_long", 1, seed=0)
+
+
+def test_cfg4_full_batch_full_depth_one_image():
+    """The 6B-class encoder, 16 images, all 45 layers (11.6 GB of weights): image 11."""
+    _full_depth_one_item("cfg4_vit6b_b16_448", 11, seed=0)
+
+
+# ----------------------------------------------------------------------------- one batch split over replicas
+
+def _device_weights(cfg, w):
+    """The weight dictionary with every array already on the GPU in the encoder's element type (so that several
+    encoders can borrow the same tensors)."""
+    conv = lambda a: None if a is None else epd.to_device(a, cfg.dtype)
+    out = {k: conv(v) for k, v in w.items() if k != "layers"}
+    out["layers"] = [{k: conv(v) for k, v in lw.items()} for lw in w["layers"]]
+    return out
+
+
+def test_cfg2_batch_split_over_replicas_by_item_cost():
+    """The 32 variable-resolution images dealt to 2, 3 and 8 replicas by the cost model (least-loaded first,
+    costliest item first); every replica encodes its share with an encoder of its own (here: one after the
+    other on the one GPU), and its rows go where the whole batch's layout puts them.  An item's features do
+    not depend on what else is in the batch, so the reassembled buffer equals the whole-batch encode bit for
+    bit; one item is also compared with the oracle."""
+    from paper_2601_11590_b200 import replicas
+    cfg, grids = synth.WORKLOADS["cfg2_vit06b_var32"]
+    w = synth.make_weights(cfg, seed=0)
+    wd = _device_weights(cfg, w)
+    T, K = synth.num_tokens(grids), cfg.patch_dim
+    patches = synth.make_patches(cfg, grids, seed=0)
+    p_all = epd.to_device(patches, cfg.dtype)
+    bk = O.bookkeeping(grids)
+    cu = bk["cu_seqlens"]
+    max_grid = max(max(g[1], g[2]) for g in grids)
+
+    enc = epd.Encoder(cfg, wd, max_tokens=T, max_images=len(grids), max_grid=max_grid)
+    whole, cu_rows = enc.encode(p_all, grids)
+    torch.cuda.synchronize()
+    assert enc.last_status() == epd.EPD_OK
+    whole = whole.clone()
+    enc.close()
+    ranges = replicas.feature_row_ranges(grids)
+    assert [r[0] for r in ranges] == cu_rows[:-1].tolist()
+
+    for world in (2, 3, 8):
+        shares = replicas.assign_items(grids, world, cfg.hidden, cfg.mlp)
+        assert sorted(i for s in shares for i in s) == list(range(len(grids)))
+        out = torch.full_like(whole, float("nan"))
+        for items in shares:
+            if not items:
+                continue
+            g = [grids[i] for i in items]
+            p = torch.cat([p_all[int(cu[i]):int(cu[i + 1])] for i in items])
+            e = epd.Encoder(cfg, wd, max_tokens=synth.num_tokens(g), max_images=len(g), max_grid=max_grid)
+            f, cr = e.encode(p, g)
+            torch.cuda.synchronize()
+            assert e.last_status() == epd.EPD_OK
+            for j, i in enumerate(items):
+                out[ranges[i][0]:ranges[i][1]] = f[int(cr[j]):int(cr[j + 1])]
+            e.close()
+        assert torch.equal(out.view(torch.int16), whole.view(torch.int16)), world
+
+    lens = np.diff(cu)
+    i = int(np.argsort(lens)[1])                      # the second smallest image
+    ref = O.encode(cfg, w, patches[int(cu[i]):int(cu[i + 1])], [grids[i]])
+    e = assert_parity(to_np(whole[ranges[i][0]:ranges[i][1]]), ref, TOL_FINAL, f"cfg2 item {i}")
+    print("cfg2 split: item", i, "tokens", int(lens[i]), "final", e)

@@ -30,6 +30,7 @@ def test_two_gloo_ranks_reduce_to_the_slowest_rank_and_rank0_prints():
     assert d["world"] == 2 and d["ms_max"] == 20.0          # rank r reported 10 (r + 1) ms
     assert d["distinct_batches"] == 2                       # every replica drew its own batch
     assert abs(d["value"] - 2 * 512 / 20e-3) < 1e-6         # all ranks' tokens over the slowest rank's time
+    assert d["split_covers_batch_once"] is True             # --split: the ranks' shares partition the one batch
 
 
 def test_reference_arm_under_two_ranks_prints_one_line():

@@ -5,7 +5,8 @@ owns the GPU's memory, or they cannot tolerate the synchronisation an allocation
 its q/k/v intermediates in a fixed array inside the library.  Here it is called twice in a row through
 the C ABI -- the second batch smaller than the first, so anything the first call left in the shared
 array would show up if it were read -- and each result is compared with epd_op_rope_split() +
-epd_op_attention() on caller-provided buffers.  This file sorts last so that a stop-at-first-failure
+epd_op_attention() on caller-provided buffers, and with the CPU oracle's rotary embedding + block-diagonal
+attention on the same inputs.  This file sorts last so that a stop-at-first-failure
 run has already executed every other test.
 """
 import numpy as np
@@ -14,6 +15,8 @@ import torch
 
 import synth
 import paper_2601_11590_b200 as epd
+from oracle import encoder_oracle as O
+from tests.metrics import assert_parity
 
 pytestmark = pytest.mark.gpu
 
@@ -29,6 +32,18 @@ def _case(dtype, heads, dh, seglens, seed):
     pr = torch.from_numpy(rng.integers(0, 64, T).astype(np.int32)).cuda()
     pc = torch.from_numpy(rng.integers(0, 64, T).astype(np.int32)).cuda()
     return qkv, pr, pc, cu, T, h
+
+
+def _oracle(qkv, pr, pc, cu, heads, dh, theta):
+    """Rotary embedding of q and k at the tokens' (row, column) positions, then softmax(q k^T / sqrt(dh)) v
+    inside each segment, in float64 from the same input numbers."""
+    x = qkv.float().cpu().numpy().astype(np.float64)
+    T, h = x.shape[0], heads * dh
+    pos_r, pos_c = pr.cpu().numpy(), pc.cpu().numpy()
+    q = O.rope_2d(x[:, :h].reshape(T, heads, dh), pos_r, pos_c, theta)
+    k = O.rope_2d(x[:, h:2 * h].reshape(T, heads, dh), pos_r, pos_c, theta)
+    v = x[:, 2 * h:].reshape(T, heads, dh)
+    return O.attention_block_diagonal(q, k, v, cu).reshape(T, h)
 
 
 @pytest.mark.parametrize("dtype", [epd.DTYPE_BF16, epd.DTYPE_F32])
@@ -49,6 +64,9 @@ def test_static_scratch_entry_point_matches_ordinary_entry_points_twice(dtype):
         err = np.linalg.norm(a - b) / np.linalg.norm(b)
         assert np.isfinite(a).all()
         assert err <= (TOL if dtype == epd.DTYPE_BF16 else 1e-6), err
+        # against the oracle: two rounded steps in bf16 (rotated q, k stored as bf16, then the attention output)
+        assert_parity(a, _oracle(qkv, pr, pc, cu, heads, dh, theta), 2 * TOL if dtype == epd.DTYPE_BF16 else 1e-5,
+                      "static entry point against the oracle")
 
 
 def test_static_scratch_rejects_oversized_batches():
