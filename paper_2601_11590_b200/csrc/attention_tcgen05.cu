@@ -566,7 +566,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
       // the tcgen05.st of this tile's P, so the two TMEM round trips overlap.
       auto load_scores = [&](int j) -> bool {
         const int kv_valid = min(BKV, it.seg_len - j * BKV);
-        if (!mbar_wait(&s_full[w], tc & 1, wc)) return false;
+        if (!mbar_wait_warp(&s_full[w], tc & 1, wc)) return false;
         tc_fence_after();
         if (kv_valid == BKV) {
           tmem_ld_cols<BKV>(tmem_s, s);
@@ -654,7 +654,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         }
         if (!ONES) l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
         // P_w and O_w are free once this warpgroup's previous P V has completed
-        if (tc > 0 && !mbar_wait(&p_free[w], (tc - 1) & 1, wc)) { ok = false; break; }
+        if (tc > 0 && !mbar_wait_warp(&p_free[w], (tc - 1) & 1, wc)) { ok = false; break; }
         ++tc;
         tc_fence_after();
         if (__any_sync(0xffffffffu, grow)) {
@@ -689,7 +689,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
         // not overtake the reader of this warpgroup's previous publication: that reader has finished once
         // O_w of this warpgroup's previous item with key tiles was read out (with two or more key tiles
         // in this item that is already known through the P V products).
-        if (my_pubs > 0 && my_items >= 2 && !mbar_wait(&o_free[w], (my_items - 2) & 1, wc)) { ok = false; break; }
+        if (my_pubs > 0 && my_items >= 2 && !mbar_wait_warp(&o_free[w], (my_items - 2) & 1, wc)) { ok = false; break; }
         ml_all[(n & 1) * 2 * BQ + w * BQ + r] = make_float2(m, l);
         __syncwarp();
         if (lane == 0) mbar_arrive(&ml_pub[w]);
@@ -703,8 +703,8 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
       // accumulator back, so that the other warpgroup's next item is not held up by this merge
       constexpr bool kEarly = DHP + 32 <= BKV;
       if (has_other) {
-        if (!mbar_wait(&ml_pub[w ^ 1], other_pubs & 1, wc)) { ok = false; break; }
-        if (!mbar_wait(&o_done[w ^ 1], (other_items - 1) & 1, wc)) { ok = false; break; }
+        if (!mbar_wait_warp(&ml_pub[w ^ 1], other_pubs & 1, wc)) { ok = false; break; }
+        if (!mbar_wait_warp(&o_done[w ^ 1], (other_items - 1) & 1, wc)) { ok = false; break; }
         tc_fence_after();
         ml_b = ml_all[(n & 1) * 2 * BQ + (w ^ 1) * BQ + r];
         if constexpr (kEarly) {
@@ -725,7 +725,7 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
             if (i == (dh & 7)) ml_b.y = __uint_as_float(t1[i]);
         }
       }
-      if (!mbar_wait(&o_done[w], (my_items - 1) & 1, wc)) { ok = false; break; }
+      if (!mbar_wait_warp(&o_done[w], (my_items - 1) & 1, wc)) { ok = false; break; }
       tc_fence_after();
       const int token = it.q0 + r;
       const bool row_ok = token < it.seg_beg + it.seg_len;

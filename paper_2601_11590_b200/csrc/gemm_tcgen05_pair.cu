@@ -278,7 +278,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       for (int i = lane; i < BN / 2; i += 32)
         bs[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
       __syncwarp();
-      if (!mbar_wait<true>(&tmem_full[acc], acc_phase, wc)) break;
+      if (!mbar_wait_warp<true>(&tmem_full[acc], acc_phase, wc)) break;
       tc_fence_after();
       const int row0 = m0 + q * 32;
       const uint32_t taddr = tmem_base + acc * kAccStride + half * (BN / 2) + ((uint32_t)(q * 32) << 16);

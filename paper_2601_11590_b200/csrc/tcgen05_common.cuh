@@ -100,13 +100,15 @@ __device__ __forceinline__ void raise_abort(const WaitCtx& wc) {
 }
 
 // Bounded wait.  Returns false if the phase did not complete within the limit (the abort flag is raised, in the
-// peer CTA too) or another role has already given up.  A short limit (a test's) is checked on every poll, the
-// ordinary one every 256 polls.
+// peer CTA too) or another role has already given up.  The ordinary limit is checked every 256 polls.  A short
+// limit (a test's) is checked on every poll, and once more when the phase has completed: a poll may itself
+// suspend the thread for longer than such a limit, and the wait must count as expired all the same.
 template <bool kCluster = false>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
   if (mbar_try_wait<kCluster>(bar, parity)) return true;
   const long long t0 = clock64();
-  const int mask = wc.limit < (1LL << 22) ? 0 : 255;
+  const bool short_limit = wc.limit < (1LL << 22);
+  const int mask = short_limit ? 0 : 255;
   int spins = 0;
   while (!mbar_try_wait<kCluster>(bar, parity)) {
     if ((++spins & mask) == 0) {
@@ -117,7 +119,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
       }
     }
   }
+  if (short_limit && clock64() - t0 > wc.limit) {
+    raise_abort(wc);
+    return false;
+  }
   return true;
+}
+// The same wait made by all 32 lanes of a warp, with one outcome for the whole warp (false if any lane gave up):
+// what follows such a wait is warp-synchronous (tcgen05.ld / st with .sync.aligned), so the lanes must not part.
+template <bool kCluster = false>
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, const WaitCtx& wc) {
+  return __all_sync(0xffffffffu, mbar_wait<kCluster>(bar, parity, wc));
 }
 // Wait used while draining after an abort: its own fixed limit, indifferent to the abort flag.
 template <bool kCluster = false>

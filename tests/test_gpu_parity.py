@@ -723,22 +723,75 @@ def test_empty_and_invalid_batches():
     out, cu_rows = enc.encode(None, [], features=feats)
     assert out.shape[0] == 0 and cu_rows.tolist() == [0]
     p = dev(synth.make_patches(cfg, [(1, 2, 2)]), cfg.dtype)
+    enc.encode(p, [(1, 2, 2)], features=feats)
+    assert enc.last_launch_count() > 0
     for bad in ([(1, 3, 2)], [(0, 2, 2)], [(1, 2, -2)]):
         with pytest.raises(epd.EpdError) as ei:
             enc.encode(p, bad, features=feats)
-        assert ei.value.status == epd.EPD_EINVAL
+        assert ei.value.status == epd.EPD_EINVAL and enc.last_launch_count() == 0
     for too_big in ([(1, 2, 2)] * 3, [(1, 10, 2)], [(1, 8, 8), (1, 2, 2)]):
         with pytest.raises(epd.EpdError) as ei:
             enc.encode(p, too_big, features=feats)
-        assert ei.value.status == epd.EPD_ECAPACITY
+        assert ei.value.status == epd.EPD_ECAPACITY and enc.last_launch_count() == 0
     with pytest.raises(epd.EpdError) as ei:   # feature buffer too small
         enc.encode(dev(synth.make_patches(cfg, [(1, 8, 8)]), cfg.dtype), [(1, 8, 8)], features=feats[:8])
-    assert ei.value.status == epd.EPD_ECAPACITY
+    assert ei.value.status == epd.EPD_ECAPACITY and enc.last_launch_count() == 0
+    # a rejected call enqueues nothing: not on the device entry point (a NULL / misaligned buffer is found before
+    # the layout is staged), not on the host-buffer and raw-frame entry points (odd grid found before the copy)
+    grids_new = [(1, 4, 4)]                      # a layout the device does not hold yet
+    with pytest.raises(epd.EpdError) as ei:
+        enc.encode(None, grids_new, features=feats)
+    assert ei.value.status == epd.EPD_EINVAL and enc.last_launch_count() == 0
+    with pytest.raises(epd.EpdError) as ei:
+        raw = torch.zeros(16 * cfg.patch_dim + 4, device="cuda")
+        enc.encode(raw[1:1 + 16 * cfg.patch_dim].view(16, cfg.patch_dim), grids_new, features=feats)   # 4-byte aligned only
+    assert ei.value.status == epd.EPD_EINVAL and enc.last_launch_count() == 0
+    hp = torch.zeros((64, cfg.patch_dim)).pin_memory()
+    hf = torch.zeros((16, cfg.out_dim)).pin_memory()
+    for call in (enc.encode_host, enc.encode_host_async):
+        with pytest.raises(epd.EpdError) as ei:
+            call(hp, [(1, 3, 2)], hf)
+        assert ei.value.status == epd.EPD_EINVAL and enc.last_launch_count() == 0
+    with pytest.raises(epd.EpdError) as ei:
+        enc.encode_frames(torch.zeros(64, dtype=torch.uint8, device="cuda"), [(1, 3, 2)], synth.PIXEL_MEAN, synth.PIXEL_STD,
+                          features=feats)
+    assert ei.value.status == epd.EPD_EINVAL and enc.last_launch_count() == 0
     # the encoder still works afterwards, at its maximum size
     grids = [(1, 8, 8)]
     out, _ = enc.encode(dev(synth.make_patches(cfg, grids), cfg.dtype), grids, features=feats)
     ref = O.encode(cfg, w, synth.make_patches(cfg, grids), grids)
     assert_parity(to_np(out), ref, TOL_F32)
+    enc.close()
+
+
+def test_expired_wait_is_reported_and_the_encoder_recovers():
+    """The bounded device-side waits, made to run out: with a limit of a thousand cycles the ordinary wait of an
+    epilogue warp for its first accumulator (tiles still on their way from memory) counts as expired; the kernels
+    record the timeout, let what they have in flight complete, free their tensor memory and return.  The status
+    call reports EPD_ETIMEOUT once; with the limit restored, the next encode is bit-identical to the one before."""
+    cfg = _small_bf16()
+    grids = [(1, 16, 16), (1, 8, 12)]
+    T = synth.num_tokens(grids)
+    w = synth.make_weights(cfg, seed=40)
+    enc = epd.Encoder(cfg, w, max_tokens=T, max_images=len(grids), max_grid=16)
+    p = dev(synth.make_patches(cfg, grids, seed=40), cfg.dtype)
+    ref, _ = enc.encode(p, grids)
+    ref = ref.clone()
+    torch.cuda.synchronize()
+    assert enc.last_status() == epd.EPD_OK
+    epd.set_wait_limit(1000)
+    try:
+        enc.encode(p, grids)
+        torch.cuda.synchronize()
+        st = enc.last_status()
+    finally:
+        epd.set_wait_limit(0)
+    assert st == epd.EPD_ETIMEOUT
+    assert enc.last_status() == epd.EPD_OK          # reading the status cleared it
+    again, _ = enc.encode(p, grids)
+    torch.cuda.synchronize()
+    assert enc.last_status() == epd.EPD_OK
+    assert torch.equal(again, ref)
     enc.close()
 
 
