@@ -340,7 +340,13 @@ int epd_op_qkv_rope(const void* x, int64_t ldx, const void* w_prepared, const vo
                     void* q, void* k, void* v, int64_t T, int32_t heads, int32_t head_dim, float q_scale,
                     void* stream);
 
-enum { EPD_ATTENTION_FORCE_FMA = 1 /* use the plain-FMA kernel even where the tensor-core kernel applies */ };
+enum {
+  EPD_ATTENTION_FORCE_FMA = 1,        /* use the plain-FMA kernel even where a tensor-core kernel applies */
+  EPD_ATTENTION_SPLIT_KEYS = 2,       /* force the tensor-core kernel that gives one query tile to both softmax
+                                         warpgroups (alternate key tiles, merged at the end) */
+  EPD_ATTENTION_TWO_QUERY_TILES = 4   /* force the tensor-core kernel with two query tiles per CTA sharing every
+                                         K / V tile; without either flag the faster one for the shape is chosen */
+};
 
 /* Block-diagonal bidirectional attention.  q, k, v [heads, T, head_dim_padded] per dtype as written
  * by epd_op_rope_split(): q already multiplied by log2(e)/sqrt(head_dim), pad columns zero except

@@ -20,6 +20,8 @@ EPD_OK, EPD_EINVAL, EPD_ENOMEM, EPD_ECUDA, EPD_ECAPACITY, EPD_EUNSUPPORTED, EPD_
 DTYPE_F32, DTYPE_BF16 = 0, 1
 LINEAR_GELU_TANH, LINEAR_GELU_ERF, LINEAR_ACCUMULATE, LINEAR_OUT_F32, LINEAR_FORCE_FMA = 1, 2, 4, 8, 16
 ATTENTION_FORCE_FMA = 1
+ATTENTION_SPLIT_KEYS = 2
+ATTENTION_TWO_QUERY_TILES = 4
 
 EXPORTED_SYMBOLS = [
     "epd_encoder_workspace_bytes", "epd_encoder_create", "epd_encode", "epd_encode_host",

@@ -1,0 +1,743 @@
+// Block-diagonal bidirectional flash attention on the 5th-generation tensor cores: two query tiles per CTA.
+//
+// Persistent kernel, one CTA per SM.  A work item is one (segment, head, 256 query rows): two tiles of 128
+// query rows that walk the segment's keys / values together, so every K and V tile brought into shared
+// memory serves both.  Each query tile w has its own softmax warpgroup (one thread per query row), its own
+// issuing thread, two score buffers S_w[0], S_w[1] and an output accumulator O_w in tensor memory, its own
+// running max and row sum; there is nothing to merge at the end of an item.  The keys are walked in steps of
+// 64; step t of query tile w uses score buffer t mod 2:
+//   S_w[b] = Q_w K_t^T     tcgen05.mma, both operands K-major in shared memory, fp32 scores in TMEM
+//   online softmax         warpgroup w reads its S row into registers (tcgen05.ld), takes the row maximum,
+//                          P = exp2(S - m) as bf16 pairs, written back over the first half of the same buffer
+//                          (tcgen05.st).  q arrives scaled by log2(e)/sqrt(head_dim): base-2 exponentials suffice
+//   O_w += P_w V_t         one tcgen05.mma per 16 keys with P as the TMEM operand, V read MN-major from shared
+//                          memory
+// Each query tile has two issuing threads: one issues  P_w V_t  as soon as P is written, the other issues
+// Q_w K_(t+2)^T  into the buffer P was read from as soon as that product is complete.  (Issuing a product, a
+// commit or a barrier wait each costs a thread 60 to 100 clocks, and a step needs nine products, four commits
+// and four waits per query tile: one thread per query tile was measured to take ~1600 clocks per step and was
+// the kernel's bound.)  While the softmax warpgroup works on one buffer, the score product for the other one is
+// already complete or under way: the tensor-pipe round trip is off the warpgroup's critical path, which is then
+// load - max - exponentials - store.  The unit that bounds the kernel at head width 72 is the exponential unit (16 results per clock per
+// SM: 1024 clocks for the 2 x 128 x 64 scores of a step against 810 clocks of products).
+// The running max only advances (and O_w is rescaled in TMEM) when it grows by more than 2^8; until then the
+// stale max serves P, the row sum and O_w alike, which leaves the result unchanged.  A rescale first waits for
+// the previous step's P V (the only product that may still be adding to O_w: the one before it is complete
+// once the scores of the current step are).  Where head_dim is below the padded width, column head_dim of V
+// holds 1.0 and column head_dim of O_w is the row sum of P, summed by the tensor core from the same bf16
+// values as the numerator.
+// A segment whose length is not a multiple of 256 ends with an item whose second query tile is partly or
+// wholly beyond the segment: rows beyond it are computed and not stored; a wholly empty second tile is
+// skipped (its issuing thread only hands the K / V slots back, its warpgroup idles for that item).
+// TMEM (512 columns): S_0[0] | S_0[1] | S_1[0] | S_1[1] | O_0 | O_1, 64 columns per score buffer and the
+// padded head width per accumulator.
+// Warp roles: warp 0 TMA producer of Q (per tile, NQ buffers) and the K ring, warp 3 TMA producer of the V
+// ring, warps 1 / 2 the P V products of query tile 0 / 1 (warp 1 also allocates tensor memory), warps 4 / 5
+// their score products, warps 6, 7 idle, warps 8..11 and 12..15 the softmax warpgroups of query tile 0 and 1
+// (also epilogue).  The softmax warps raise their register allowance at the expense of warps 0..7 (setmaxnreg).
+// head_dim 72 is stored padded to 80.  Q and K tiles: columns 0..63 form a 128-byte-swizzled box, columns
+// 64..79 a 32-byte-swizzled box, each contraction step its own MMA.  V tiles: five 32-byte-swizzled boxes of 16
+// columns, so that one MMA covers all 80 output columns.
+// Every mbarrier wait is bounded: on expiry the kernel records EPD_ETIMEOUT and drains.  No load is a
+// multicast load.
+#include <algorithm>
+#include <vector>
+
+#include "tcgen05_common.cuh"
+
+namespace epd {
+namespace {
+
+using namespace tc;
+
+constexpr int BQ = 128;          // query rows per tile; an item has two tiles
+constexpr int BKV = 64;          // keys per step
+constexpr int kThreads = 512;    // warps 0..7: loaders and issuing threads; warps 8..15: two softmax warpgroups
+constexpr int kRegsLow = 64, kRegsHigh = 192;   // 256 x 64 + 256 x 192 = 512 x 128
+constexpr int kMaxSegs = 128;    // segments one launch can describe
+constexpr float kRescaleThreshold = 8.0f;  // log2 of the largest P value tolerated before rescaling
+
+// D[tmem] (+)= A[smem] . B[smem]
+__device__ __forceinline__ void umma_ss(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] . B[smem]
+__device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                        uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+#define EPD_R8(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), \
+    "=r"(r[o + 6]), "=r"(r[o + 7])
+#define EPD_W8(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]),       \
+    "r"(r[o + 6]), "r"(r[o + 7])
+#define EPD_R16(r, o) EPD_R8(r, o), EPD_R8(r, o + 8)
+#define EPD_W16(r, o) EPD_W8(r, o), EPD_W8(r, o + 8)
+#define EPD_R32(r, o) EPD_R16(r, o), EPD_R16(r, o + 16)
+#define EPD_W32(r, o) EPD_W16(r, o), EPD_W16(r, o + 16)
+#define EPD_R64(r, o) EPD_R32(r, o), EPD_R32(r, o + 32)
+#define EPD_W64(r, o) EPD_W32(r, o), EPD_W32(r, o + 32)
+
+// tcgen05.ld / tcgen05.st, shape 32x32b: thread i of the warp owns TMEM lane (base + i) and moves N
+// consecutive 32-bit columns.
+__device__ __forceinline__ void ld8(uint32_t taddr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : EPD_R8(r, 0) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : EPD_R16(r, 0) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : EPD_R32(r, 0) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void ld64(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
+      : EPD_R64(r, 0) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void st8(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), EPD_W8(r, 0) : "memory");
+}
+__device__ __forceinline__ void st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), EPD_W16(r, 0) : "memory");
+}
+__device__ __forceinline__ void st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), EPD_W32(r, 0) : "memory");
+}
+__device__ __forceinline__ void st64(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x64.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, "
+      "%33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, "
+      "%49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63, %64};"
+      ::"r"(taddr), EPD_W64(r, 0) : "memory");
+}
+// N columns (a multiple of 8) with as few instructions as possible.
+template <int N>
+__device__ __forceinline__ void ld_cols(uint32_t taddr, uint32_t* r) {
+  if constexpr (N >= 64) { ld64(taddr, r); ld_cols<N - 64>(taddr + 64, r + 64); }
+  else if constexpr (N >= 32) { ld32(taddr, r); ld_cols<N - 32>(taddr + 32, r + 32); }
+  else if constexpr (N >= 16) { ld16(taddr, r); ld_cols<N - 16>(taddr + 16, r + 16); }
+  else if constexpr (N >= 8) { ld8(taddr, r); ld_cols<N - 8>(taddr + 8, r + 8); }
+}
+template <int N>
+__device__ __forceinline__ void st_cols(uint32_t taddr, const uint32_t* r) {
+  if constexpr (N >= 64) { st64(taddr, r); st_cols<N - 64>(taddr + 64, r + 64); }
+  else if constexpr (N >= 32) { st32(taddr, r); st_cols<N - 32>(taddr + 32, r + 32); }
+  else if constexpr (N >= 16) { st16(taddr, r); st_cols<N - 16>(taddr + 16, r + 16); }
+  else if constexpr (N >= 8) { st8(taddr, r); st_cols<N - 8>(taddr + 8, r + 8); }
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+template <int N> __device__ __forceinline__ void regs_dec() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N> __device__ __forceinline__ void regs_inc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+// Shared-memory matrix descriptor.  layout: 2 = 128-byte swizzle, 6 = 32-byte swizzle.
+// K-major operand: sbo = distance between 8-row groups.  MN-major operand: lbo = distance between
+// swizzle-wide column groups, sbo = distance between 8-row (contraction) groups.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)(lbo_bytes >> 4) << 16;
+  d |= (uint64_t)(sbo_bytes >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)layout << 61;
+  return d;
+}
+// bf16 x bf16 -> fp32, M = 128; b_mn = 1 when the B operand is MN-major (V: head_dim contiguous).
+__host__ __device__ constexpr uint32_t instr_desc(int n, int b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(128 >> 4) << 24);
+}
+
+// Shared-memory and tensor-memory plan for a padded head width DHP (64, 80 or 128).
+template <int DHP>
+struct Plan {
+  // score buffers S_w[b] at column (2 w + b) * BKV
+  static constexpr int kO0 = 4 * BKV, kO1 = kO0 + DHP;
+  static_assert(kO1 + DHP <= 512, "tensor memory plan does not fit");
+  static constexpr int kMainBoxes = DHP / 64;          // Q, K: 128-byte-swizzled boxes of 64 columns
+  static constexpr int kTail = DHP % 64;               // Q, K: 0 or 16 columns, 32-byte swizzle
+  static_assert(kTail == 0 || kTail == 16, "padded head width must be 64*a or 64*a + 16");
+  static constexpr bool kV32 = kTail != 0;             // V as 32-byte-swizzled boxes of 16 columns
+  static constexpr int kQMain = BQ * 128;              // bytes of a main box of a Q tile
+  static constexpr int kQTile = BQ * DHP * 2;          // bytes of a Q tile
+  static constexpr int kKMain = BKV * 128;             // bytes of a main box of a K tile
+  static constexpr int kKTile = BKV * DHP * 2;         // bytes of a K or V tile
+  static_assert(kQTile % 1024 == 0 && kKTile % 1024 == 0, "tiles keep the 1024-byte alignment of the swizzled boxes");
+  static constexpr int kVBox = kV32 ? BKV * 32 : BKV * 128;
+  static constexpr int kVBoxes = kV32 ? DHP / 16 : DHP / 64;
+  static_assert(kVBox * kVBoxes == kKTile, "V tile");
+  static constexpr int NQ = DHP == 128 ? 1 : 2;        // buffers per query tile
+  static constexpr int KS = DHP == 128 ? 4 : DHP == 80 ? 6 : 8;   // K ring depth
+  static constexpr int VS = DHP == 128 ? 5 : DHP == 80 ? 6 : 8;   // V ring depth
+  static constexpr int kQ = 0;                         // [tile w][buffer b]
+  static constexpr int kK = 2 * NQ * kQTile;
+  static constexpr int kV = kK + KS * kKTile;
+  static constexpr int kBar = kV + VS * kKTile;
+  // q_full[2][NQ] q_empty[2][NQ] k_full[KS] k_empty[KS] v_full[VS] v_empty[VS] s_full[2][2] p_full[2][2]
+  // pv_done[2][2] o_done[2] o_free[2] drain[4]
+  static constexpr int kNumBars = 4 * NQ + 2 * KS + 2 * VS + 20;
+  static constexpr int kTotal = kBar + kNumBars * 8 + 32;
+  static constexpr int kDynamic = kTotal + 1024;       // slack to align the tiles to 1024 bytes
+  static_assert(kDynamic > 116 * 1024, "one CTA per SM is assumed by the TMEM allocation");
+  static_assert(kDynamic <= 232448, "exceeds the shared memory of one CTA");
+};
+
+struct Maps {
+  CUtensorMap q_main, q_tail, k_main, k_tail, v;   // q boxes are BQ rows high, k and v boxes BKV rows
+};
+
+// Segments of one launch, longest first (host-sorted).
+struct SegList {
+  int n;
+  int beg[kMaxSegs];
+  int len[kMaxSegs];
+};
+
+struct Item {
+  int head, seg_beg, seg_len, q0, n_kv;
+  bool two;     // the second query tile holds rows of the segment
+};
+
+// Item i -> (segment, head, 256-row query block): segments in list order, then head, then query block, so
+// that neighbouring items (which run at the same time on different SMs) share K and V in L2.
+__device__ __forceinline__ Item decode_item(const SegList& segs, int heads, int i) {
+  Item it{0, 0, 0, 0, 0, false};
+  for (int s = 0; s < segs.n; ++s) {
+    const int qb = (segs.len[s] + 2 * BQ - 1) / (2 * BQ);
+    const int cnt = qb * heads;
+    if (i < cnt) {
+      it.head = i / qb;
+      it.seg_beg = segs.beg[s];
+      it.seg_len = segs.len[s];
+      it.q0 = it.seg_beg + (i - it.head * qb) * 2 * BQ;
+      it.n_kv = (it.seg_len + BKV - 1) / BKV;
+      it.two = it.q0 + BQ < it.seg_beg + it.seg_len;
+      return it;
+    }
+    i -= cnt;
+  }
+  return it;
+}
+
+// ONES: head_dim < DHP and column head_dim of every V row holds 1.0, so column head_dim of O_w is the row sum
+// of P_w and the softmax threads need not add it up.
+template <int DHP, bool ONES>
+__global__ void __launch_bounds__(kThreads, 1)
+attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__ SegList segs, int n_items,
+                      __nv_bfloat16* __restrict__ out, int T, int heads, int dh, int* __restrict__ status,
+                      long long wait_limit) {
+  using P = Plan<DHP>;
+  constexpr int NQ = P::NQ;
+  pdl_launch_dependents();
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + P::kBar);
+  uint64_t* q_full = bars;                    // [2][NQ]  Q tile w, buffer b loaded
+  uint64_t* q_empty = q_full + 2 * NQ;        // [2][NQ]  its last score product is complete
+  uint64_t* k_full = q_empty + 2 * NQ;        // [KS]
+  uint64_t* k_empty = k_full + P::KS;         // [KS]  both issuing threads are done with the slot (2 arrivals)
+  uint64_t* v_full = k_empty + P::KS;         // [VS]
+  uint64_t* v_empty = v_full + P::VS;         // [VS]  (2 arrivals)
+  uint64_t* s_full = v_empty + P::VS;         // [2][2]  S_w[b] complete
+  uint64_t* p_full = s_full + 4;              // [2][2]  P written over S_w[b] (4 warp arrivals)
+  uint64_t* pv_done = p_full + 4;             // [2][2]  the P_w V product that read P from S_w[b] is complete
+  uint64_t* o_done = pv_done + 4;             // [2]  the item's last P_w V is complete: O_w final
+  uint64_t* o_free = o_done + 2;              // [2]  O_w read out by its warpgroup (4 warp arrivals)
+  uint64_t* drain = o_free + 2;               // [4]  after an abort: the products of an issuing thread have completed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + P::kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const WaitCtx wc{abort_flag, 0u, wait_limit};
+  uint32_t q_loads0 = 0, q_loads1 = 0, kv_loads = 0;   // loads issued by this thread (warp 0: Q and K tiles, warp 3: V tiles)
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < P::kNumBars; ++i) mbar_init(&bars[i], 1);
+    for (int i = 0; i < P::KS; ++i) mbar_init(&k_empty[i], 2);
+    for (int i = 0; i < P::VS; ++i) mbar_init(&v_empty[i], 2);
+    for (int i = 0; i < 4; ++i) mbar_init(&p_full[i], 4);
+    for (int w = 0; w < 2; ++w) mbar_init(&o_free[w], 4);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();   // nothing above touches global memory
+  if (warp < 8) regs_dec<kRegsLow>();
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- TMA producer of Q and K
+    if (lane == 0) {
+      uint32_t kc = 0, n = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
+        const Item it = decode_item(segs, heads, item);
+        const int row_base = it.head * T;
+        const int qb = n % NQ;
+        const uint32_t qphase = (n / NQ) & 1;
+        // both query tiles are loaded even when the second holds no row of the segment: the barrier
+        // counters then advance the same way for every item
+        for (int w = 0; w < 2 && ok; ++w) {
+          if (!mbar_wait(&q_empty[w * NQ + qb], qphase ^ 1, wc)) { ok = false; break; }
+          uint8_t* dst = smem + P::kQ + (w * NQ + qb) * P::kQTile;
+          uint64_t* full = &q_full[w * NQ + qb];
+          const int row = row_base + it.q0 + w * BQ;
+          mbar_expect_tx(full, P::kQTile);
+#pragma unroll
+          for (int b = 0; b < P::kMainBoxes; ++b) tma_load_2d(dst + b * P::kQMain, &maps.q_main, b * 64, row, full);
+          if (P::kTail) tma_load_2d(dst + P::kMainBoxes * P::kQMain, &maps.q_tail, P::kMainBoxes * 64, row, full);
+          if (w == 0) ++q_loads0; else ++q_loads1;
+        }
+        if (!ok) break;
+        for (int j = 0; j < it.n_kv; ++j, ++kc) {
+          const int row = row_base + it.seg_beg + j * BKV;
+          const int ks = kc % P::KS;
+          if (!mbar_wait(&k_empty[ks], ((kc / P::KS) & 1) ^ 1, wc)) { ok = false; break; }
+          uint8_t* dk = smem + P::kK + ks * P::kKTile;
+          mbar_expect_tx(&k_full[ks], P::kKTile);
+#pragma unroll
+          for (int b = 0; b < P::kMainBoxes; ++b) tma_load_2d(dk + b * P::kKMain, &maps.k_main, b * 64, row, &k_full[ks]);
+          if (P::kTail) tma_load_2d(dk + P::kMainBoxes * P::kKMain, &maps.k_tail, P::kMainBoxes * 64, row, &k_full[ks]);
+          ++kv_loads;
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 3) {
+    // ---------------------------------------------------------------- TMA producer of V
+    if (lane == 0) {
+      uint32_t vc = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const Item it = decode_item(segs, heads, item);
+        const int row_base = it.head * T;
+        for (int j = 0; j < it.n_kv; ++j, ++vc) {
+          const int row = row_base + it.seg_beg + j * BKV;
+          const int vs = vc % P::VS;
+          if (!mbar_wait(&v_empty[vs], ((vc / P::VS) & 1) ^ 1, wc)) { ok = false; break; }
+          uint8_t* dv = smem + P::kV + vs * P::kKTile;
+          mbar_expect_tx(&v_full[vs], P::kKTile);
+#pragma unroll
+          for (int b = 0; b < P::kVBoxes; ++b)
+            tma_load_2d(dv + b * P::kVBox, &maps.v, b * (P::kV32 ? 16 : 64), row, &v_full[vs]);
+          ++kv_loads;
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1 || warp == 2) {
+    // ---------------------------------------------------------------- P V products of query tile w
+    if (lane == 0) {
+      const int w = warp - 1;
+      uint32_t vc = 0;                 // V tiles seen (all of them, also in skipped items)
+      uint32_t c = 0;                  // steps of this query tile so far: step c uses score buffer c & 1
+      uint32_t items_w = 0;            // items in which this query tile took part
+      constexpr uint32_t idesc_pv = instr_desc(DHP, 1);
+      constexpr uint32_t kVStep = P::kV32 ? 512 / 16 : 2048 / 16;   // 16 keys further down the V tile, 16-byte units
+      const uint32_t tmem_o = tmem_base + (w ? P::kO1 : P::kO0);
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const Item it = decode_item(segs, heads, item);
+        if (w == 1 && !it.two) {
+          // nothing to compute for this query tile: hand every V slot back, each only once it has been filled
+          // (so that an arrival can never be counted for a later use of the slot)
+          for (int j = 0; j < it.n_kv; ++j, ++vc) {
+            if (!mbar_wait(&v_full[vc % P::VS], (vc / P::VS) & 1, wc)) { ok = false; break; }
+            mbar_arrive(&v_empty[vc % P::VS]);
+          }
+          continue;
+        }
+        for (int t = 0; t < it.n_kv; ++t, ++vc, ++c) {
+          const int vs = vc % P::VS;
+          if (!mbar_wait(&v_full[vs], (vc / P::VS) & 1, wc)) { ok = false; break; }
+          if (t == 0) {
+            // the accumulator of the query tile's previous item must have been read out
+            if (items_w > 0 && !mbar_wait(&o_free[w], (items_w - 1) & 1, wc)) { ok = false; break; }
+            ++items_w;
+          }
+          // P of this step is in tensor memory
+          if (!mbar_wait(&p_full[2 * w + (c & 1)], (c >> 1) & 1, wc)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sv = smem_u32(smem + P::kV + vs * P::kKTile);
+          // MN-major V: boxes (16 or 64 columns wide) are kVBox apart, 8-row groups 256 / 1024 bytes apart
+          const uint64_t dv = P::kV32 ? smem_desc(sv, P::kVBox, 256, 6) : smem_desc(sv, P::kVBox, 1024, 2);
+          const uint32_t tmem_p = tmem_base + (2 * w + (c & 1)) * BKV;
+          const int kv_valid = min(BKV, it.seg_len - t * BKV);
+          const int steps = (kv_valid + 15) >> 4;
+          if (steps == BKV / 16) {
+#pragma unroll
+            for (int s = 0; s < BKV / 16; ++s)       // 16 bf16 of P = 8 columns
+              umma_ts(tmem_o, tmem_p + s * 8, dv + s * kVStep, idesc_pv, (t | s) != 0 ? 1u : 0u);
+          } else {
+            for (int s = 0; s < steps; ++s)
+              umma_ts(tmem_o, tmem_p + s * 8, dv + s * kVStep, idesc_pv, (t | s) != 0 ? 1u : 0u);
+          }
+          umma_commit(&pv_done[2 * w + (c & 1)]);    // frees the score buffer, orders rescales
+          umma_commit(&v_empty[vs]);
+          if (t == it.n_kv - 1) umma_commit(&o_done[w]);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 4 || warp == 5) {
+    // ---------------------------------------------------------------- score products of query tile w
+    if (lane == 0) {
+      const int w = warp - 4;
+      uint32_t kc = 0, n = 0;          // K tiles / items seen (all of them, also in skipped items)
+      uint32_t g = 0;                  // score tiles of this query tile so far: tile g goes to buffer g & 1
+      bool ok = true;
+      for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
+        const Item it = decode_item(segs, heads, item);
+        const int qb = n % NQ;
+        const uint32_t qphase = (n / NQ) & 1;
+        if (!mbar_wait(&q_full[w * NQ + qb], qphase, wc)) break;
+        if (w == 1 && !it.two) {
+          // nothing to compute for this query tile: hand the Q buffer and every K slot back, each only once it
+          // has been filled
+          mbar_arrive(&q_empty[w * NQ + qb]);
+          for (int j = 0; j < it.n_kv; ++j, ++kc) {
+            if (!mbar_wait(&k_full[kc % P::KS], (kc / P::KS) & 1, wc)) { ok = false; break; }
+            mbar_arrive(&k_empty[kc % P::KS]);
+          }
+          continue;
+        }
+        const uint32_t sq = smem_u32(smem + P::kQ + (w * NQ + qb) * P::kQTile);
+        const uint64_t dq_main = smem_desc(sq, 16, 1024, 2);
+        const uint64_t dq_tail = smem_desc(sq + P::kMainBoxes * P::kQMain, 16, 256, 6);
+        for (int t = 0; t < it.n_kv; ++t, ++kc, ++g) {
+          const int ks = kc % P::KS;
+          if (!mbar_wait(&k_full[ks], (kc / P::KS) & 1, wc)) { ok = false; break; }
+          // the buffer's previous content (P of the step two before) must have been consumed by its P V product.
+          // One barrier per buffer: the buffer's next product cannot complete before these scores exist, so the
+          // barrier is at most one phase past the one waited for and the parity is unambiguous.
+          if (g >= 2 && !mbar_wait(&pv_done[2 * w + (g & 1)], ((g >> 1) - 1) & 1, wc)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sk = smem_u32(smem + P::kK + ks * P::kKTile);
+          const uint64_t dk_main = smem_desc(sk, 16, 1024, 2);
+          const uint64_t dk_tail = smem_desc(sk + P::kMainBoxes * P::kKMain, 16, 256, 6);
+          const uint32_t tmem_s = tmem_base + (2 * w + (g & 1)) * BKV;
+          const int kv_valid = min(BKV, it.seg_len - t * BKV);
+          const uint32_t idesc = kv_valid == BKV ? instr_desc(BKV, 0) : instr_desc((kv_valid + 15) & ~15, 0);
+          // descriptor addresses count 16-byte units: one 16-element step inside a swizzled row is +2
+#pragma unroll
+          for (int b = 0; b < P::kMainBoxes; ++b) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              umma_ss(tmem_s, dq_main + (b * P::kQMain / 16 + 2 * k), dk_main + (b * P::kKMain / 16 + 2 * k), idesc,
+                      (b | k) != 0);
+          }
+          if (P::kTail) umma_ss(tmem_s, dq_tail, dk_tail, idesc, 1);
+          umma_commit(&s_full[2 * w + (g & 1)]);
+          umma_commit(&k_empty[ks]);
+          if (t == it.n_kv - 1) umma_commit(&q_empty[w * NQ + qb]);   // the query tile's last score product
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp >= 8) {
+    // ---------------------------------------------------------------- softmax / rescale / epilogue
+    regs_inc<kRegsHigh>();
+    const int w = (warp - 8) >> 2;                      // query tile of this warpgroup
+    const int qr = warp & 3;                            // TMEM lane quarter this warp may access
+    const int r = qr * 32 + lane;                       // query row inside the tile
+    const uint32_t lane_off = (uint32_t)(qr * 32) << 16;
+    const uint32_t tmem_s0 = tmem_base + 2 * w * BKV + lane_off;   // S_w[0]; S_w[1] is BKV columns further
+    const uint32_t tmem_o = tmem_base + (w ? P::kO1 : P::kO0) + lane_off;
+    uint32_t c = 0, oc = 0;                             // steps / items processed by this warpgroup
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+      const Item it = decode_item(segs, heads, item);
+      if (w == 1 && !it.two) continue;                  // no row of the segment in this query tile
+      float m = -INFINITY, l = 0.0f;
+      uint32_t s[BKV > DHP ? BKV : DHP];
+      for (int t = 0; t < it.n_kv; ++t, ++c) {
+        const int kv_valid = min(BKV, it.seg_len - t * BKV);
+        const uint32_t tmem_s = tmem_s0 + (c & 1) * BKV;   // P lives in the buffer's first BKV / 2 columns
+        if (!mbar_wait_warp(&s_full[2 * w + (c & 1)], (c >> 1) & 1, wc)) { ok = false; break; }
+        tc_fence_after();
+        if (kv_valid == BKV) {
+          ld_cols<BKV>(tmem_s, s);
+        } else {
+#pragma unroll
+          for (int q = 0; q < BKV / 16; ++q)
+            if (q * 16 < kv_valid) ld16(tmem_s + q * 16, s + q * 16);
+        }
+        tmem_ld_wait();
+
+        float mx[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) mx[i] = -INFINITY;
+        if (kv_valid == BKV) {
+#pragma unroll
+          for (int i = 0; i < BKV / 2; ++i)
+            mx[i & 3] = max3(mx[i & 3], __uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
+        } else {
+#pragma unroll
+          for (int i = 0; i < BKV; ++i)
+            if (i < kv_valid) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(s[i]));
+        }
+        const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+        // advance the running max only when it would grow by more than the threshold
+        float scale = 1.0f;
+        bool grow = false;
+        if (t == 0) {
+          m = m_tile;
+        } else if (m_tile - m > kRescaleThreshold) {
+          scale = ex2(m - m_tile);
+          m = m_tile;
+          l *= scale;
+          grow = true;
+        }
+        if (__any_sync(0xffffffffu, grow)) {
+          // O_w must be quiescent: the product of step t-2 is complete (these scores were issued behind it); the
+          // product of step t-1 is the only one that may still be adding to it
+          if (!mbar_wait_warp(&pv_done[2 * w + ((c - 1) & 1)], ((c - 1) >> 1) & 1, wc)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int q = 0; q < DHP / 16; ++q) {
+            uint32_t o[16];
+            ld16(tmem_o + q * 16, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * scale);
+            st16(tmem_o + q * 16, o);
+          }
+        }
+        // P = exp2(S - m) as bf16 pairs, in place
+        const float neg_m = -m;
+        float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        if (kv_valid == BKV) {
+#pragma unroll
+          for (int i = 0; i < BKV / 2; ++i) {
+            const float p0 = ex2(__uint_as_float(s[2 * i]) + neg_m);
+            const float p1 = ex2(__uint_as_float(s[2 * i + 1]) + neg_m);
+            if (!ONES) sum[i & 3] += p0 + p1;
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+            s[i] = *reinterpret_cast<uint32_t*>(&b2);
+          }
+          st_cols<BKV / 2>(tmem_s, s);
+        } else {
+#pragma unroll
+          for (int i = 0; i < BKV / 2; ++i) {
+            const float p0 = 2 * i < kv_valid ? ex2(__uint_as_float(s[2 * i]) + neg_m) : 0.0f;
+            const float p1 = 2 * i + 1 < kv_valid ? ex2(__uint_as_float(s[2 * i + 1]) + neg_m) : 0.0f;
+            if (!ONES) sum[i & 3] += p0 + p1;
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+            s[i] = *reinterpret_cast<uint32_t*>(&b2);
+          }
+#pragma unroll
+          for (int q = 0; q < BKV / 16; ++q)
+            if (q * 16 < kv_valid) st8(tmem_s + q * 8, s + q * 8);
+        }
+        if (!ONES) l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full[2 * w + (c & 1)]);
+      }
+      if (!ok) break;
+      // ---- epilogue: O_w / l -> out
+      if (!mbar_wait_warp(&o_done[w], oc & 1, wc)) { ok = false; break; }
+      ++oc;
+      tc_fence_after();
+      const int token = it.q0 + w * BQ + r;
+      const bool row_ok = token < it.seg_beg + it.seg_len;
+      __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + it.head * dh;
+      // the whole accumulator row goes into the (dead) score registers, then the accumulator is handed back
+      ld_cols<DHP>(tmem_o, s);
+      tmem_ld_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&o_free[w]);
+      if (ONES) l = __uint_as_float(s[DHP - 8]);       // head_dim = DHP - 8: the row sum sits in column head_dim
+      const float inv = 1.0f / l;
+      if (row_ok) {
+#pragma unroll
+        for (int g = 0; g < DHP / 8; ++g) {
+          if (g * 8 < dh) {                              // head_dim is a multiple of 8
+            uint32_t pk[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(s[8 * g + 2 * e]) * inv,
+                                                        __uint_as_float(s[8 * g + 2 * e + 1]) * inv);
+              pk[e] = *reinterpret_cast<uint32_t*>(&b2);
+            }
+            *reinterpret_cast<uint4*>(orow + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // A wait expired.  Every role has left its loop, so nothing new is issued.  What was issued completes by
+    // itself: each loader waits for its last load of every ring slot, each issuing thread for its last product
+    // (a commit arrives only after all earlier products); the softmax warps write their rows with ordinary
+    // stores.  A fixed pause on top, then shared and tensor memory are released.
+    if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, 0, kStatusTimeout);
+    if (lane == 0) {
+      if (warp == 0) {
+        drain_ring(q_full, NQ, q_loads0);
+        drain_ring(q_full + NQ, NQ, q_loads1);
+        drain_ring(k_full, P::KS, kv_loads);
+      }
+      if (warp == 3) drain_ring(v_full, P::VS, kv_loads);
+      if (warp == 1 || warp == 2 || warp == 4 || warp == 5) {
+        const int d = warp < 3 ? warp - 1 : warp - 2;
+        umma_commit(&drain[d]);
+        mbar_wait_drain(&drain[d], 0);
+      }
+    }
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+
+// Map over a bf16 matrix [rows, dhp] (row pitch dhp*2 bytes): box = box_rows rows x box_cols columns.
+bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int dhp, int box_rows, int box_cols,
+              CUtensorMapSwizzle swz) {
+  return make_tensor_map_2d(tm, base, rows, dhp, (int64_t)dhp * 2, box_rows, box_cols, 2, swz);
+}
+
+template <int DHP, bool ONES>
+cudaError_t launch(const Maps& maps, const SegList& segs, int n_items, void* out, int T, int heads, int dh,
+                   int* status, cudaStream_t s) {
+  using P = Plan<DHP>;
+  auto kern = attention_pair_kernel<DHP, ONES>;
+  static PerDeviceOnce configured;
+  cudaError_t e = once_per_device(configured, [&] {
+    return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, P::kDynamic);
+  });
+  if (e != cudaSuccess) return e;
+  const int sms = limited_sms(device_sm_count());
+  const int grid = n_items < sms ? n_items : sms;
+  return launch_pdl(kern, dim3(grid), dim3(kThreads), P::kDynamic, s, maps, segs, n_items, (__nv_bfloat16*)out, T, heads, dh,
+                    status, wait_limit_cycles());
+}
+
+}  // namespace
+
+bool attention_pair_supported(const void* q, const void* k, const void* v, const void* out, int64_t T, int heads,
+                              int head_dim) {
+  const int dhp = padded_head_dim(head_dim);
+  if (dhp != 64 && dhp != 80 && dhp != 128) return false;
+  if (head_dim % 8) return false;
+  if (dhp != head_dim && dhp - head_dim != 8) return false;   // the row-sum column is read at padded width - 8
+  if (((uintptr_t)q & 15) || ((uintptr_t)k & 15) || ((uintptr_t)v & 15) || ((uintptr_t)out & 15)) return false;
+  if ((int64_t)heads * T > (1 << 30) || heads > 65535) return false;
+  return tensor_maps_available();
+}
+
+cudaError_t attention_pair(const void* q, const void* k, const void* v, const int32_t* host_cu_seqlens, int n_seg,
+                           void* out, int64_t T, int heads, int head_dim, int* status, cudaStream_t s) {
+  const int dhp = padded_head_dim(head_dim);
+  if (n_seg <= 0) return cudaSuccess;
+  const int64_t rows = (int64_t)heads * T;
+  Maps maps;
+  if (!make_map(&maps.q_main, q, rows, dhp, BQ, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&maps.q_tail, q, rows, dhp, BQ, 16, CU_TENSOR_MAP_SWIZZLE_32B) ||
+      !make_map(&maps.k_main, k, rows, dhp, BKV, 64, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_map(&maps.k_tail, k, rows, dhp, BKV, 16, CU_TENSOR_MAP_SWIZZLE_32B))
+    return cudaErrorInvalidValue;
+  if (dhp % 64 ? !make_map(&maps.v, v, rows, dhp, BKV, 16, CU_TENSOR_MAP_SWIZZLE_32B)
+               : !make_map(&maps.v, v, rows, dhp, BKV, 64, CU_TENSOR_MAP_SWIZZLE_128B))
+    return cudaErrorInvalidValue;
+  // longest segments first: items are dealt round-robin, so the long ones spread evenly and the
+  // short ones fill the tail
+  std::vector<int> order(n_seg);
+  for (int i = 0; i < n_seg; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+    return host_cu_seqlens[a + 1] - host_cu_seqlens[a] > host_cu_seqlens[b + 1] - host_cu_seqlens[b];
+  });
+  for (int first = 0; first < n_seg; first += kMaxSegs) {
+    SegList segs;
+    segs.n = n_seg - first < kMaxSegs ? n_seg - first : kMaxSegs;
+    int n_items = 0;
+    for (int i = 0; i < segs.n; ++i) {
+      const int sg = order[first + i];
+      segs.beg[i] = host_cu_seqlens[sg];
+      segs.len[i] = host_cu_seqlens[sg + 1] - host_cu_seqlens[sg];
+      n_items += (segs.len[i] + 2 * BQ - 1) / (2 * BQ) * heads;
+    }
+    for (int i = segs.n; i < kMaxSegs; ++i) segs.beg[i] = segs.len[i] = 0;
+    cudaError_t e;
+    switch (dhp) {
+#define EPD_ATT(D)                                                                                          \
+  e = head_dim < D ? launch<D, true>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s)          \
+                   : launch<D, false>(maps, segs, n_items, out, (int)T, heads, head_dim, status, s)
+      case 64: EPD_ATT(64); break;
+      case 80: EPD_ATT(80); break;
+      case 128: EPD_ATT(128); break;
+#undef EPD_ATT
+      default: return cudaErrorInvalidValue;
+    }
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace epd

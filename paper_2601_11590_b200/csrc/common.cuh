@@ -33,6 +33,11 @@ __device__ __forceinline__ float gelu_tanh_f(float x) {
 }
 __device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f)); }
 
+// Internal flag of the linear kernels (above the public EPD_LINEAR_* bits): the weight matrix is not written by
+// any kernel that may still be running when this one starts (an encoder's own weights), so its first tiles may
+// be fetched before the wait for the previous kernel.
+constexpr int kLinearStaticWeights = 1 << 20;
+
 // ---- programmatic dependent launch ---------------------------------------------------------------
 // The kernels of one encode run back to back on one stream.  Launched with the programmatic-stream-
 // serialization attribute, a kernel's CTAs may become resident as soon as every CTA of the previous
@@ -94,6 +99,12 @@ cudaError_t token_layout(const int32_t* grid_thw, const int32_t* cu_seqlens, con
                          cudaStream_t s);
 
 
+// Attention with two query tiles per CTA sharing every K / V tile (attention_pair_tcgen05.cu).
+bool attention_pair_supported(const void* q, const void* k, const void* v, const void* out, int64_t T, int heads,
+                              int head_dim);
+cudaError_t attention_pair(const void* q, const void* k, const void* v, const int32_t* host_cu_seqlens, int n_seg,
+                           void* out, int64_t T, int heads, int head_dim, int* status, cudaStream_t s);
+
 // ---- tensor-core kernels (gemm_tcgen05.cu) ---------------------------------------------------
 // bf16 x bf16 -> fp32 linear layer on tcgen05; `status` (device int, may be NULL) receives
 // EPD_ETIMEOUT if a bounded wait expires.  forced_bn: 0 = choose the tile width automatically.
@@ -109,11 +120,11 @@ cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ld
 
 // QKV projection whose epilogue applies the rotary embedding and writes head-major q, k, v (the
 // padding columns are left as the caller initialised them with qkv_pad_init).  w_perm / bias_perm come
-// from qkv_permute (pair order inside each head of q and k).
+// from qkv_permute (pair order inside each head of q and k).  static_w: see kLinearStaticWeights.
 cudaError_t linear_tc_pair_qkv(const void* x, int64_t ldx, const void* w_perm, int64_t ldw, const void* bias_perm,
                                void* q, void* k, void* v, const int32_t* pos_row, const int32_t* pos_col,
                                const float2* table, int table_rows, int64_t M, int heads, int head_dim, float q_scale,
-                               int* status, cudaStream_t s);
+                               int static_w, int* status, cudaStream_t s);
 cudaError_t qkv_permute(const void* w, int64_t ldw, const void* bias, void* w_out, void* bias_out, int heads,
                         int head_dim, cudaStream_t s);
 cudaError_t qkv_pad_init(void* q, void* k, void* v, int64_t rows, int head_dim, cudaStream_t s);

@@ -183,7 +183,8 @@ int linear_dispatch(epd_encoder* enc, int dtype, const void* x, int64_t ldx, con
     int* status = enc ? enc->at<int>(enc->lay.status) : nullptr;
     const int forced_bn = (flags >> EPD_LINEAR_TILE_N_SHIFT) & 0x1FF;
     if (forced_bn != 0 && forced_bn != 128 && forced_bn != 192 && forced_bn != 256) return EPD_EINVAL;
-    EPD_CUDA(linear_tc(x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, forced_bn, status, s));
+    EPD_CUDA(linear_tc(x, ldx, w, ldw, bias, out, ldo, M, N, K, enc ? (flags | kLinearStaticWeights) : flags, forced_bn,
+                       status, s));
     return EPD_OK;
   }
   EPD_CUDA(linear_fma(dtype, x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, s));
@@ -317,7 +318,7 @@ int run_block(epd_encoder* enc, int l, float* x, int64_t T, int n_seg, cudaStrea
                                 enc->ws + enc->lay.qkv_perm_b + (size_t)l * align_up(3 * hh * 2, 256),
                                 enc->at<void>(enc->lay.qh), enc->at<void>(enc->lay.kh), enc->at<void>(enc->lay.vh),
                                 enc->at<int32_t>(enc->lay.pos_row), enc->at<int32_t>(enc->lay.pos_col),
-                                enc->at<float2>(enc->lay.rope), c.max_grid, T, c.heads, c.head_dim, q_scale,
+                                enc->at<float2>(enc->lay.rope), c.max_grid, T, c.heads, c.head_dim, q_scale, 1,
                                 enc->at<int>(enc->lay.status), s));
   } else {
     if ((rc = linear_dispatch(enc, dt, a, h, enc->qkv_w[l], h, enc->qkv_b[l], qkv, 3 * h, T, 3 * h, h, 0, s)))
@@ -1033,7 +1034,7 @@ int epd_op_qkv_rope(const void* x, int64_t ldx, const void* w_prepared, const vo
   if (((uintptr_t)x | (uintptr_t)w_prepared | (uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)table) & 15)
     return EPD_EINVAL;
   EPD_CUDA(linear_tc_pair_qkv(x, ldx, w_prepared, h, bias_prepared, q, k, v, pos_row, pos_col,
-                              reinterpret_cast<const float2*>(table), table_rows, T, heads, head_dim, q_scale, nullptr,
+                              reinterpret_cast<const float2*>(table), table_rows, T, heads, head_dim, q_scale, 0, nullptr,
                               static_cast<cudaStream_t>(stream)));
   return EPD_OK;
 }

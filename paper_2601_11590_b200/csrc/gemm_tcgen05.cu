@@ -193,7 +193,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
           for (int j = 0; j < 32; ++j) {
             float t = __uint_as_float(pk[j]) + bs[c * CC + j];
             if (ACT == 1) t = gelu_tanh_fast(t);
-            if (ACT == 2) t = gelu_erf_f(t);
+            if (ACT == 2) t = gelu_erf_fast(t);
             pk[j] = __float_as_uint(t);
           }
         } else {
@@ -208,7 +208,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
             float t0 = __uint_as_float(src[jj]) + bs[c * CC + 2 * j];
             float t1 = __uint_as_float(src[jj + 1]) + bs[c * CC + 2 * j + 1];
             if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); }
-            if (ACT == 2) { t0 = gelu_erf_f(t0); t1 = gelu_erf_f(t1); }
+            if (ACT == 2) { t0 = gelu_erf_fast(t0); t1 = gelu_erf_fast(t1); }
             __nv_bfloat162 b = __floats2bfloat162_rn(t0, t1);
             pk[j] = *reinterpret_cast<uint32_t*>(&b);
           }

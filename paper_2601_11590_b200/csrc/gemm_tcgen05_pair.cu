@@ -144,7 +144,7 @@ template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_out, const __nv_bfloat16* __restrict__ bias, int M, int N,
-                   int K, int* __restrict__ status, long long wait_limit, const RopeSplitArgs rs) {
+                   int K, int* __restrict__ status, long long wait_limit, int static_w, const RopeSplitArgs rs) {
   static_assert(!ROPE || (sizeof(OutT) == 2 && ACT == 0 && !ACCUM), "the QKV variant writes bf16, no activation");
   using L = PairLayout<BN, STAGES>;
   static_assert(BN == 256 || BN == 128, "tile width");
@@ -190,7 +190,21 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   cluster_sync();                                 // both CTAs' barriers exist before either signals the other
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_slot;
-  pdl_wait();   // nothing above touches global memory
+  // The weight tiles of the first stages do not depend on the previous kernel (static_w): the producer fetches
+  // them before the wait below, so they arrive while the previous kernel is still finishing; the x tiles follow
+  // after the wait, into the same stages, counted on the same barrier phase.
+  int early = 0;
+  if (static_w && warp == 0 && lane == 0 && pair < num_tiles) {
+    prefetch_map(&tm_w);
+    const int n0 = (pair / m_tiles) * BN + (int)rank * (BN / 2);
+    early = k_blocks < STAGES ? k_blocks : STAGES;
+    for (int kb = 0; kb < early; ++kb) {
+      if (rank == 0) mbar_expect_tx(&full[kb], 2 * L::kStageBytes);
+      tma_load_2d_pair(smem + kb * L::kStageBytes + L::kABytes, &tm_w, kb * BK, n0, map_to_rank(smem_u32(&full[kb]), 0));
+    }
+    loads_issued = early;     // for the drain after an abort: these stages have loads in flight
+  }
+  pdl_wait();   // nothing above touches global memory that an earlier kernel of the stream writes
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
@@ -200,17 +214,22 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      loads_issued = 0;
       for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
         const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;        // this CTA's rows of x
         const int n0 = (tile / m_tiles) * BN + (int)rank * (BN / 2);       // this CTA's half of the w tile
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait<true>(&empty[stage], phase ^ 1, wc)) { ok = false; break; }
           uint8_t* sa = smem + stage * L::kStageBytes;
-          // the leader's barrier counts the bytes of both CTAs
-          if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
           const uint32_t bar = map_to_rank(smem_u32(&full[stage]), 0);
+          if (early > 0) {
+            --early;                                  // this stage's bytes are expected and its w tile is on its way
+          } else {
+            // the leader's barrier counts the bytes of both CTAs
+            if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
+            tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BK, n0, bar);
+          }
           tma_load_2d_pair(sa, &tm_x, kb * BK, m0, bar);
-          tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BK, n0, bar);
           ++loads_issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -307,7 +326,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             for (int e = 0; e < 4; ++e) {
               float t = __uint_as_float(pk[4 * j4 + e]) + bb[e];
               if (ACT == 1) t = gelu_tanh_fast(t);
-              if (ACT == 2) t = gelu_erf_f(t);
+              if (ACT == 2) t = gelu_erf_fast(t);
               pk[4 * j4 + e] = __float_as_uint(t);
             }
           }
@@ -363,7 +382,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
               float t0 = __uint_as_float(src[jj]) + bv.x, t1 = __uint_as_float(src[jj + 1]) + bv.y;
               float t2 = __uint_as_float(src[jj + 2]) + bv.z, t3 = __uint_as_float(src[jj + 3]) + bv.w;
               if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); t2 = gelu_tanh_fast(t2); t3 = gelu_tanh_fast(t3); }
-              if (ACT == 2) { t0 = gelu_erf_f(t0); t1 = gelu_erf_f(t1); t2 = gelu_erf_f(t2); t3 = gelu_erf_f(t3); }
+              if (ACT == 2) { t0 = gelu_erf_fast(t0); t1 = gelu_erf_fast(t1); t2 = gelu_erf_fast(t2); t3 = gelu_erf_fast(t3); }
               __nv_bfloat162 b0 = __floats2bfloat162_rn(t0, t1), b1 = __floats2bfloat162_rn(t2, t3);
               pk[2 * j2] = *reinterpret_cast<uint32_t*>(&b0);
               pk[2 * j2 + 1] = *reinterpret_cast<uint32_t*>(&b1);
@@ -462,7 +481,7 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int
 
 template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE = false>
 cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& to, const void* bias, int M, int N,
-                   int K, int* status, cudaStream_t s, const RopeSplitArgs& rs = RopeSplitArgs{}) {
+                   int K, int* status, cudaStream_t s, int static_w, const RopeSplitArgs& rs = RopeSplitArgs{}) {
   using L = PairLayout<BN, STAGES>;
   auto kern = linear_pair_kernel<BN, STAGES, OutT, ACT, ACCUM, ROPE>;
   static PerDeviceOnce configured;
@@ -502,7 +521,7 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
   const int avail = limited_sms(2 * max_pairs) / 2 > 0 ? limited_sms(2 * max_pairs) / 2 : 1;   // pairs within the SM budget
   const int pairs = tiles < avail ? tiles : avail;
   return launch_pdl(kern, dim3(2 * pairs), dim3(kThreads), smem_bytes, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K,
-                    status, wait_limit_cycles(), rs);
+                    status, wait_limit_cycles(), static_w, rs);
 }
 
 template <int BN, int STAGES>
@@ -511,7 +530,8 @@ cudaError_t launch_bn(const CUtensorMap& tx, const CUtensorMap& tw, const CUtens
   const int act = (flags & EPD_LINEAR_GELU_TANH) ? 1 : (flags & EPD_LINEAR_GELU_ERF) ? 2 : 0;
   const bool accum = flags & EPD_LINEAR_ACCUMULATE;
   const bool out_f32 = accum || (flags & EPD_LINEAR_OUT_F32);
-#define EPD_TC(OUT, A, C) return launch<BN, STAGES, OUT, A, C>(tx, tw, to, bias, M, N, K, status, s)
+#define EPD_TC(OUT, A, C) \
+  return launch<BN, STAGES, OUT, A, C>(tx, tw, to, bias, M, N, K, status, s, (flags & kLinearStaticWeights) ? 1 : 0)
   if (accum) {
     if (act == 0) EPD_TC(float, 0, true);
     if (act == 1) EPD_TC(float, 1, true);
@@ -548,7 +568,7 @@ cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ld
 cudaError_t linear_tc_pair_qkv(const void* x, int64_t ldx, const void* w_perm, int64_t ldw, const void* bias_perm,
                                void* q, void* k, void* v, const int32_t* pos_row, const int32_t* pos_col,
                                const float2* table, int table_rows, int64_t M, int heads, int head_dim, float q_scale,
-                               int* status, cudaStream_t s) {
+                               int static_w, int* status, cudaStream_t s) {
   constexpr int BN = 256;
   const int64_t hdim = (int64_t)heads * head_dim, N = 3 * hdim, K = hdim;
   if (head_dim % 8 || !table) return cudaErrorInvalidValue;
@@ -569,7 +589,7 @@ cudaError_t linear_tc_pair_qkv(const void* x, int64_t ldx, const void* w_perm, i
   rs.dhp = padded_head_dim(head_dim);
   rs.q_scale = q_scale;
   // the output tensor map is not used by this variant
-  return launch<BN, 5, __nv_bfloat16, 0, false, true>(tx, tw, tx, bias_perm, (int)M, (int)N, (int)K, status, s, rs);
+  return launch<BN, 5, __nv_bfloat16, 0, false, true>(tx, tw, tx, bias_perm, (int)M, (int)N, (int)K, status, s, static_w, rs);
 }
 
 namespace {

@@ -142,6 +142,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--no-flush", action="store_true")
     ap.add_argument("--fma", action="store_true", help="force the plain-FMA kernel")
+    ap.add_argument("--two-query-tiles", action="store_true",
+                    help="attention: force the kernel with two query tiles per CTA")
+    ap.add_argument("--split-keys", action="store_true",
+                    help="attention: the kernel with one query tile per CTA and key tiles split between the warpgroups")
     args = ap.parse_args()
 
     import torch
@@ -185,13 +189,14 @@ def main():
         lib = epd.load_library()
         out = torch.empty((T, args.heads * args.dh), dtype=bf, device="cuda")
         hcu, hp = epd._i32_array(cu)
-        flags = epd.ATTENTION_FORCE_FMA if args.fma else 0
+        flags = epd.ATTENTION_FORCE_FMA if args.fma else epd.ATTENTION_SPLIT_KEYS if args.split_keys else \
+            epd.ATTENTION_TWO_QUERY_TILES if args.two_query_tiles else 0
 
         def fn():
             epd._check(lib.epd_op_attention(dt, epd._ptr(q), epd._ptr(k), epd._ptr(v), epd._ptr(cu_dev), hp,
                                             hcu.size - 1, epd._ptr(out), T, args.heads, args.dh, flags,
                                             epd._stream_ptr(None)), "epd_op_attention")
-        res.update(heads=args.heads, dh=args.dh, T=T, n_seg=len(seg),
+        res.update(heads=args.heads, dh=args.dh, T=T, n_seg=len(seg), split_keys=bool(args.split_keys),
                    flops=4.0 * args.heads * args.dh * float(sum(s * s for s in seg)),
                    bytes=2.0 * args.heads * T * (3 * dhp + args.dh))
     elif args.op == "rope":

@@ -249,12 +249,20 @@ def test_attention(dtype, heads, dh, seglens):
     (2, 72, [100, 1300, 128, 129, 4]),   # ragged tails on both the query and the key side
     (3, 64, [2000]),                     # 16 key tiles
     (2, 128, [700, 260]),
+    (2, 72, [256, 257, 255, 512, 384]),  # query blocks of 256 rows: exactly full, one row over, one row short
+    (1, 80, [1000, 130]),                # head width 80: no padding column, row sums in registers
+    (3, 128, [1024, 1024]),              # the 6B-class encoder's images
+    (2, 56, [300]),                      # padded width 64 with a ones column
+    (148, 72, [300]),                    # more items than SMs: several items per CTA, second tile partly empty
 ])
 def test_attention_tensor_core_long_segments(heads, dh, seglens):
     got, ref = _attention_case(epd.DTYPE_BF16, heads, dh, seglens, 40)
     assert_parity(got, ref, TOL_BF16_STEP)
     fma, _ = _attention_case(epd.DTYPE_BF16, heads, dh, seglens, 40, flags=epd.ATTENTION_FORCE_FMA)
     assert_parity(got, fma, TOL_BF16_STEP)
+    for forced in (epd.ATTENTION_SPLIT_KEYS, epd.ATTENTION_TWO_QUERY_TILES):      # both tensor-core kernels
+        other, _ = _attention_case(epd.DTYPE_BF16, heads, dh, seglens, 40, flags=forced)
+        assert_parity(other, ref, TOL_BF16_STEP)
 
 
 def test_attention_more_segments_than_one_launch_describes():
@@ -265,11 +273,14 @@ def test_attention_more_segments_than_one_launch_describes():
     seglens[7], seglens[100] = 300, 129
     got, ref = _attention_case(epd.DTYPE_BF16, 2, 72, seglens, 50)
     assert_parity(got, ref, TOL_BF16_STEP)
+    two, _ = _attention_case(epd.DTYPE_BF16, 2, 72, seglens, 50, flags=epd.ATTENTION_TWO_QUERY_TILES)
+    assert_parity(two, ref, TOL_BF16_STEP)
     fma, _ = _attention_case(epd.DTYPE_BF16, 2, 72, seglens, 50, flags=epd.ATTENTION_FORCE_FMA)
     assert_parity(got, fma, TOL_BF16_STEP)
 
 
-def test_attention_rescale_path():
+@pytest.mark.parametrize("kernel", ["split_keys", "two_query_tiles"])
+def test_attention_rescale_path(kernel):
     """Keys ordered so that the running maximum keeps growing from tile to tile by far more than the
     rescale threshold: every key tile forces a rescale of the accumulated output."""
     dtype, heads, dh, T = epd.DTYPE_BF16, 1, 64, 1024
@@ -282,7 +293,8 @@ def test_attention_rescale_path():
     v = np.zeros((heads, T, dhp), np.float32)
     v[:, :, :dh] = synth.round_to_bf16(rng.standard_normal((heads, T, dh)).astype(np.float32))
     cu = np.array([0, T], np.int32)
-    out = epd.op_attention(dtype, dev(q, dtype), dev(k, dtype), dev(v, dtype), torch.from_numpy(cu).cuda(), cu, dh)
+    flags = epd.ATTENTION_SPLIT_KEYS if kernel == "split_keys" else epd.ATTENTION_TWO_QUERY_TILES
+    out = epd.op_attention(dtype, dev(q, dtype), dev(k, dtype), dev(v, dtype), torch.from_numpy(cu).cuda(), cu, dh, flags)
     # the kernel's q carries log2(e)/sqrt(dh); hand the oracle the unscaled q it implies
     q_eff = q[:, :, :dh].astype(np.float64) * np.log(2.0) * np.sqrt(dh)
     ref = O.attention_block_diagonal(q_eff.transpose(1, 0, 2), k[:, :, :dh].astype(np.float64).transpose(1, 0, 2),
@@ -295,6 +307,10 @@ def test_attention_peaked_logits(dtype):
     """Logit standard deviation ~ 50: exercises the running-max rescaling of the online softmax."""
     got, ref = _attention_case(dtype, 2, 72, [300, 520], 20, logit_scale=2.5)
     assert_parity(got, ref, (1e-4 if dtype == epd.DTYPE_F32 else 1e-2))
+    if dtype == epd.DTYPE_BF16:
+        for forced in (epd.ATTENTION_SPLIT_KEYS, epd.ATTENTION_TWO_QUERY_TILES):
+            got, ref = _attention_case(dtype, 2, 72, [300, 520], 20, logit_scale=2.5, flags=forced)
+            assert_parity(got, ref, 1e-2)
 
 
 @pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
