@@ -48,6 +48,7 @@ typedef enum {
 enum { EPD_DTYPE_F32 = 0, EPD_DTYPE_BF16 = 1 };
 enum { EPD_ACT_GELU_TANH = 0, EPD_ACT_GELU_ERF = 1 };
 enum { EPD_PROJ_LINEAR = 0, EPD_PROJ_MLP = 1 };
+enum { EPD_FRAMES_U8 = 0, EPD_FRAMES_BF16 = 1 };   /* element type of raw frames; both on the 0..255 scale */
 
 /* Static description of the encoder E of Eq. 1. */
 typedef struct {
@@ -176,8 +177,10 @@ int epd_encode_host_join(epd_encoder_t* enc, void* stream);
 
 /*
  * The same stage fed with raw pixels: the step immediately in front of Eq. 1's E.  `frames` is a
- * device buffer of uint8 pixels holding the items back to back, item i as [t*Tp, C, h*P, w*P]
- * (frame, channel, y, x; t, h, w from grid_thw, Tp = temporal_patch, P = patch, C = in_channels <= 4).
+ * device buffer holding the items back to back, item i as [t*Tp, C, h*P, w*P]
+ * (frame, channel, y, x; t, h, w from grid_thw, Tp = temporal_patch, P = patch, C = in_channels <= 4), elements
+ * uint8 (epd_encode_frames, and frame_format EPD_FRAMES_U8) or bfloat16 on the same 0..255 scale
+ * (EPD_FRAMES_BF16, e.g. the output of a resize that keeps fractions).
  * Pixel v of channel c becomes (v/255 - mean[c]) * inv_std[c] (mean, inv_std: HOST arrays of C floats)
  * and token (frame f, row r, column c) gathers its patch in element order (channel, temporal, y, x)
  * -- the patch matrix epd_encode() takes -- in a buffer inside the workspace; then the stage runs as
@@ -187,6 +190,9 @@ int epd_encode_host_join(epd_encoder_t* enc, void* stream);
 int epd_encode_frames(epd_encoder_t* enc, const void* frames, const int32_t* grid_thw, int32_t n_images,
                       const float* mean, const float* inv_std, void* features, int64_t features_capacity_rows,
                       int64_t* out_rows, int32_t* out_cu_rows, void* stream);
+int epd_encode_frames_fmt(epd_encoder_t* enc, const void* frames, int32_t frame_format, const int32_t* grid_thw,
+                          int32_t n_images, const float* mean, const float* inv_std, void* features,
+                          int64_t features_capacity_rows, int64_t* out_rows, int32_t* out_cu_rows, void* stream);
 
 /*
  * epd_encode_frames() behind a feature cache (Section 3.2: features are stored under a hash of the input, so a
@@ -360,13 +366,18 @@ int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v,
                      int32_t head_dim, int32_t flags, void* stream);
 
 /* Pixels -> patch vectors (the front end of epd_encode_frames()).  frames: device uint8 as described
- * there; item_offsets: device int64 [n_images+1] byte offsets of the items inside frames; grid_thw:
- * device int32 [n_images, 3]; cu_seqlens: device int32 [n_images+1]; patches: device [T, ld] per
- * dtype, ld >= C*Tp*P*P (columns beyond are zeroed); mean, inv_std: HOST arrays of in_channels floats. */
+ * there (epd_op_patchify) or in the given frame_format (epd_op_patchify_fmt); item_offsets: device int64
+ * [n_images+1] BYTE offsets of the items inside frames; grid_thw: device int32 [n_images, 3]; cu_seqlens: device
+ * int32 [n_images+1]; patches: device [T, ld] per dtype, ld >= C*Tp*P*P (columns beyond are zeroed); mean,
+ * inv_std: HOST arrays of in_channels floats. */
 int epd_op_patchify(int32_t dtype, const void* frames, const int64_t* item_offsets, const int32_t* grid_thw,
                     const int32_t* cu_seqlens, int32_t n_images, int64_t T, void* patches, int64_t ld,
                     int32_t in_channels, int32_t patch, int32_t temporal_patch, const float* mean, const float* inv_std,
                     void* stream);
+int epd_op_patchify_fmt(int32_t dtype, int32_t frame_format, const void* frames, const int64_t* item_offsets,
+                        const int32_t* grid_thw, const int32_t* cu_seqlens, int32_t n_images, int64_t T, void* patches,
+                        int64_t ld, int32_t in_channels, int32_t patch, int32_t temporal_patch, const float* mean,
+                        const float* inv_std, void* stream);
 
 /* out[o, q*hidden:(q+1)*hidden] = y[merge_idx[o*4+q], :], y [T, hidden], out [T/4, 4*hidden] per dtype. */
 int epd_op_merge(int32_t dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm,

@@ -32,6 +32,11 @@ intermediate rounding:
       (dy,dx) = (0,0),(0,1),(1,0),(1,1)
   O10 projector: linear, or linear-GELU-linear, producing the [n, d] hand-off features.
 
+  Q   (variant, Section 3.5's operator mix at lower precision: not part of the bf16 path) a linear layer with
+      8-bit floating-point operands: rows of x and rows of w are scaled to the E4M3 range, rounded to E4M3
+      (4 exponent bits, bias 7, 3 mantissa bits, largest finite value 448, no infinities), multiplied exactly and
+      rescaled: quantize_e4m3_rows, linear_e4m3.
+
 Parity pins (tests/test_oracle_*.py): pure-Python brute force on tiny inputs, PyTorch CPU
 float64 library routines for each step, closed forms and invariants, and the merged-row
 counts the paper prints.  The numerical values of the features themselves are
@@ -166,6 +171,67 @@ def gelu(x: np.ndarray, act: int) -> np.ndarray:
 def linear(x: np.ndarray, w: np.ndarray, b: Optional[np.ndarray]) -> np.ndarray:
     """y = x @ w^T + b with w stored [out, in]."""
     y = x @ w.T
+    if b is not None:
+        y = y + b
+    return y
+
+
+# ----------------------------------------------------------------------------- Q  8-bit floating-point variant
+
+E4M3_MAX = 448.0
+
+
+def round_to_e4m3(v: np.ndarray) -> np.ndarray:
+    """Nearest E4M3 value (ties to the even mantissa), saturating at +-448; the result is returned as float64.
+
+    E4M3: sign, 4 exponent bits with bias 7, 3 mantissa bits.  Normal values 2^e (1 + k/8), e = -6..8 (the top
+    binade stops at 448 = 2^8 * 1.75: its last code is NaN); subnormals k * 2^-9, k = 0..7.  So the spacing of
+    representable values around |v| is 2^(e-3) with e = max(floor(log2 |v|), -6).
+    """
+    v = np.asarray(v, dtype=np.float64)
+    a = np.abs(v)
+    e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.maximum(e, -6.0)
+    quantum = np.exp2(e - 3.0)
+    q = np.rint(a / quantum) * quantum          # rint: round half to even; a / quantum is exact (power of two)
+    q = np.minimum(q, E4M3_MAX)
+    return np.sign(v) * q
+
+
+def e4m3_bits(q: np.ndarray) -> np.ndarray:
+    """The byte codes of values that are exactly representable in E4M3."""
+    q = np.asarray(q, dtype=np.float64)
+    a = np.abs(q)
+    sign = (np.signbit(q)).astype(np.uint8) << 7
+    e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    normal = a >= 2.0 ** -6
+    exp_field = np.where(normal, e + 7, 0).astype(np.int64)
+    mant = np.where(normal, a / np.exp2(e) * 8 - 8, a * 2.0 ** 9)
+    assert np.all(mant == np.rint(mant)), "not an E4M3 value"
+    return (sign | (exp_field.astype(np.uint8) << 3) | mant.astype(np.uint8)).astype(np.uint8)
+
+
+def quantize_e4m3_rows(x: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Per-row scaling to the E4M3 range and rounding: returns (q, scale) with x[i, :] ~ q[i, :] * scale[i].
+
+    scale[i] = max_j |x[i, j]| / 448 (1 for an all-zero row), q[i, j] = round_to_e4m3(x[i, j] / scale[i]).
+    The scale and the quotient decide which 8-bit code an element gets, so they are evaluated in float32
+    arithmetic (one correctly rounded division each), the precision the CUDA path takes these decisions in;
+    the rounding to E4M3 itself is exact.
+    """
+    x32 = np.ascontiguousarray(x, dtype=np.float32)
+    amax = np.max(np.abs(x32), axis=1)
+    scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    t = (x32 / scale[:, None]).astype(np.float32)
+    return round_to_e4m3(t), scale.astype(np.float64)
+
+
+def linear_e4m3(x: np.ndarray, w: np.ndarray, b: Optional[np.ndarray]) -> np.ndarray:
+    """y = (q_x @ q_w^T) * (s_x s_w^T) + b: both operands quantised row by row (a row of w is one output
+    feature), the products and sums exact (float64), the two scales applied to the sum."""
+    qx, sx = quantize_e4m3_rows(x)
+    qw, sw = quantize_e4m3_rows(w)
+    y = (qx @ qw.T) * sx[:, None] * sw[None, :]
     if b is not None:
         y = y + b
     return y

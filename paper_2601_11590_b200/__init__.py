@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libepd_encoder.so")
 EPD_OK, EPD_EINVAL, EPD_ENOMEM, EPD_ECUDA, EPD_ECAPACITY, EPD_EUNSUPPORTED, EPD_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 DTYPE_F32, DTYPE_BF16 = 0, 1
 LINEAR_GELU_TANH, LINEAR_GELU_ERF, LINEAR_ACCUMULATE, LINEAR_OUT_F32, LINEAR_FORCE_FMA = 1, 2, 4, 8, 16
+FRAMES_U8, FRAMES_BF16 = 0, 1
 ATTENTION_FORCE_FMA = 1
 ATTENTION_SPLIT_KEYS = 2
 ATTENTION_TWO_QUERY_TILES = 4
@@ -35,7 +36,7 @@ EXPORTED_SYMBOLS = [
     "epd_op_qkv_prepare", "epd_op_rope_table", "epd_op_qkv_pad_init", "epd_op_qkv_rope",
     "epd_set_sm_limit", "epd_get_sm_limit", "epd_signal_ready", "epd_op_stream_read", "epd_op_content_hash", "epd_feature_cache_create", "epd_feature_cache_destroy",
     "epd_feature_cache_lookup", "epd_feature_cache_insert", "epd_feature_cache_stats",
-    "epd_encode_frames_cached", "epd_debug_set_wait_limit",
+    "epd_encode_frames_cached", "epd_debug_set_wait_limit", "epd_encode_frames_fmt", "epd_op_patchify_fmt",
 ]
 
 
@@ -109,6 +110,10 @@ def load_library() -> ctypes.CDLL:
     lib.epd_debug_set_wait_limit.argtypes = [i64]
     lib.epd_op_patchify.restype = ctypes.c_int
     lib.epd_op_patchify.argtypes = [i32, vp, vp, vp, vp, i32, i64, vp, i64, i32, i32, i32, f32p, f32p, vp]
+    lib.epd_op_patchify_fmt.restype = ctypes.c_int
+    lib.epd_op_patchify_fmt.argtypes = [i32, i32, vp, vp, vp, vp, i32, i64, vp, i64, i32, i32, i32, f32p, f32p, vp]
+    lib.epd_encode_frames_fmt.restype = ctypes.c_int
+    lib.epd_encode_frames_fmt.argtypes = [vp, vp, i32, i32p, i32, f32p, f32p, vp, i64, i64p, i32p, vp]
     lib.epd_op_qkv_prepare.restype = ctypes.c_int
     lib.epd_op_qkv_prepare.argtypes = [vp, i64, vp, vp, vp, i32, i32, vp]
     lib.epd_op_rope_table.restype = ctypes.c_int
@@ -318,8 +323,9 @@ class Encoder:
         return features[: rows.value], cu_rows
 
     def encode_frames(self, frames, grid_thw, mean, std, features=None, stream=None):
-        """frames: device uint8 tensor, the items' [t*Tp, C, H, W] frames back to back (flattened)."""
+        """frames: device uint8 or bfloat16 tensor, the items' [t*Tp, C, H, W] frames back to back (flattened)."""
         torch = _torch()
+        fmt = FRAMES_BF16 if frames.dtype == torch.bfloat16 else FRAMES_U8
         g, gp = _i32_array(grid_thw)
         n = g.size // 3
         T = int(sum(int(g[3 * i]) * int(g[3 * i + 1]) * int(g[3 * i + 2]) for i in range(n)))
@@ -330,10 +336,10 @@ class Encoder:
         cu_rows = np.zeros(n + 1, dtype=np.int32)
         m = (ctypes.c_float * len(mean))(*[float(v) for v in mean])
         istd = (ctypes.c_float * len(std))(*[1.0 / float(v) for v in std])
-        _check(self.lib.epd_encode_frames(self._h, _ptr(frames), gp, n, m, istd, _ptr(features),
-                                          int(features.shape[0]), ctypes.byref(rows),
-                                          cu_rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
-                                          _stream_ptr(stream)), "epd_encode_frames")
+        _check(self.lib.epd_encode_frames_fmt(self._h, _ptr(frames), fmt, gp, n, m, istd, _ptr(features),
+                                              int(features.shape[0]), ctypes.byref(rows),
+                                              cu_rows.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                                              _stream_ptr(stream)), "epd_encode_frames_fmt")
         return features[: rows.value], cu_rows
 
     def encode_frames_cached(self, cache: "FeatureCache", frames, grid_thw, mean, std, features=None, stream=None):
@@ -504,10 +510,15 @@ def op_merge(dtype, y, merge_idx, stream=None):
     return out
 
 
-def pack_frames(frames: Sequence[np.ndarray]):
-    """List of uint8 [t*Tp, C, H, W] arrays -> one flat device tensor (items back to back) and the
-    int64 byte offsets of the items."""
+def pack_frames(frames: Sequence[np.ndarray], bf16: bool = False):
+    """List of [t*Tp, C, H, W] arrays -> one flat device tensor (items back to back; uint8, or bfloat16 for
+    float-valued frames) and the int64 BYTE offsets of the items."""
     torch = _torch()
+    if bf16:
+        flat = np.concatenate([np.ascontiguousarray(f, dtype=np.float32).reshape(-1) for f in frames]) if frames \
+            else np.zeros(0, np.float32)
+        off = np.concatenate([[0], np.cumsum([2 * f.size for f in frames])]).astype(np.int64)
+        return torch.from_numpy(flat).cuda().to(torch.bfloat16), off
     flat = np.concatenate([np.ascontiguousarray(f, dtype=np.uint8).reshape(-1) for f in frames]) if frames \
         else np.zeros(0, np.uint8)
     off = np.concatenate([[0], np.cumsum([f.size for f in frames])]).astype(np.int64)
@@ -529,8 +540,10 @@ def op_patchify(dtype, frames_dev, item_off, grid_thw, cu_seqlens, in_channels, 
     off_d = torch.from_numpy(np.asarray(item_off, dtype=np.int64)).cuda()
     g_d = torch.from_numpy(g.copy()).cuda()
     cu_d = torch.from_numpy(np.asarray(cu_seqlens, dtype=np.int32)).cuda()
-    _check(lib.epd_op_patchify(dtype, _ptr(frames_dev), _ptr(off_d), _ptr(g_d), _ptr(cu_d), n, T, _ptr(out), ld,
-                               in_channels, patch, temporal_patch, m, istd, _stream_ptr(stream)), "epd_op_patchify")
+    fmt = FRAMES_BF16 if frames_dev.dtype == torch.bfloat16 else FRAMES_U8
+    _check(lib.epd_op_patchify_fmt(dtype, fmt, _ptr(frames_dev), _ptr(off_d), _ptr(g_d), _ptr(cu_d), n, T, _ptr(out),
+                                   ld, in_channels, patch, temporal_patch, m, istd, _stream_ptr(stream)),
+           "epd_op_patchify_fmt")
     return out
 
 

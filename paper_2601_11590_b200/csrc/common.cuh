@@ -88,7 +88,7 @@ cudaError_t attention_fma(int dtype, const void* q, const void* k, const void* v
 cudaError_t attention_any(int dtype, const void* q, const void* k, const void* v, const int32_t* cu_seqlens,
                           const int32_t* host_cu_seqlens, int n_seg, void* out, int64_t T, int heads, int head_dim,
                           int flags, int* status, cudaStream_t s);
-cudaError_t patchify(int dtype, const uint8_t* frames, const int64_t* item_off, const int32_t* grid_thw,
+cudaError_t patchify(int dtype, int frame_format, const void* frames, const int64_t* item_off, const int32_t* grid_thw,
                      const int32_t* cu_seqlens, int n_images, int64_t T, void* patches, int64_t ld, int C, int P, int Tp,
                      const float* mean, const float* inv_std, cudaStream_t s);
 cudaError_t content_hash(const void* data, const int64_t* item_off, int n_items, uint64_t* hashes, cudaStream_t s);

@@ -477,14 +477,16 @@ int launch_sequence(epd_encoder* enc, const void* patches, int64_t patches_ld, i
   return finish_profile(enc, s);
 }
 
-// Bytes of one item's raw frames: [t*Tp, C, h*P, w*P] uint8.
-int64_t item_frame_bytes(const epd_config_t& c, const int32_t* thw) {
-  return (int64_t)thw[0] * c.temporal_patch * c.in_channels * ((int64_t)thw[1] * c.patch) * ((int64_t)thw[2] * c.patch);
+// Bytes of one item's raw frames: [t*Tp, C, h*P, w*P] pixels of 1 (uint8) or 2 (bf16) bytes.
+int64_t item_frame_bytes(const epd_config_t& c, const int32_t* thw, int frame_format = EPD_FRAMES_U8) {
+  return (int64_t)thw[0] * c.temporal_patch * c.in_channels * ((int64_t)thw[1] * c.patch) * ((int64_t)thw[2] * c.patch) *
+         (frame_format == EPD_FRAMES_BF16 ? 2 : 1);
 }
 
 // Pixels of a validated batch -> patch vectors -> the stage.  item_off[i] is the byte offset of item i's frames
 // inside `frames` (HOST array of n entries; the items need not be adjacent).
-int encode_frames_at(epd_encoder* enc, const void* frames, const int64_t* item_off, const int32_t* grid_thw, int32_t n,
+int encode_frames_at(epd_encoder* enc, const void* frames, int frame_format, const int64_t* item_off,
+                     const int32_t* grid_thw, int32_t n,
                      const float* mean, const float* inv_std, void* features, const BatchShape& bs, cudaStream_t s) {
   const epd_config_t& c = enc->cfg;
   const int64_t ld = (enc->patch_dim + 7) / 8 * 8;
@@ -500,7 +502,7 @@ int encode_frames_at(epd_encoder* enc, const void* frames, const int64_t* item_o
                            cudaMemcpyHostToDevice, s));
   EPD_CUDA(cudaEventRecord(enc->staged_off, s));
   enc->staged_off_valid = true;
-  EPD_CUDA(patchify(c.dtype, static_cast<const uint8_t*>(frames), enc->at<int64_t>(enc->lay.item_off),
+  EPD_CUDA(patchify(c.dtype, frame_format, frames, enc->at<int64_t>(enc->lay.item_off),
                     enc->at<int32_t>(enc->lay.grid), enc->at<int32_t>(enc->lay.cu), n, bs.T,
                     enc->at<void>(enc->lay.pix_patches), ld, c.in_channels, c.patch, c.temporal_patch, mean, inv_std, s));
   enc->launches = 0;
@@ -725,29 +727,38 @@ int epd_encode_host_join(epd_encoder_t* enc, void* stream) {
   return EPD_OK;
 }
 
-int epd_encode_frames(epd_encoder_t* enc, const void* frames, const int32_t* grid_thw, int32_t n_images,
-                      const float* mean, const float* inv_std, void* features, int64_t features_capacity_rows,
-                      int64_t* out_rows, int32_t* out_cu_rows, void* stream) {
+int epd_encode_frames_fmt(epd_encoder_t* enc, const void* frames, int32_t frame_format, const int32_t* grid_thw,
+                          int32_t n_images, const float* mean, const float* inv_std, void* features,
+                          int64_t features_capacity_rows, int64_t* out_rows, int32_t* out_cu_rows, void* stream) {
   if (!enc) return EPD_EINVAL;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   enc->launches = 0;
   enc->prof_used = 0;
   // everything is validated before anything is enqueued
+  if (frame_format != EPD_FRAMES_U8 && frame_format != EPD_FRAMES_BF16) return EPD_EINVAL;
   if (enc->cfg.in_channels > 4) return EPD_EUNSUPPORTED;
   BatchShape bs;
   int rc = validate_encode(enc, enc->at<void>(enc->lay.pix_patches), (enc->patch_dim + 7) / 8 * 8, grid_thw, n_images,
                            features, features_capacity_rows, &bs);
   if (rc) return rc;
   if (bs.T > 0 && (!frames || !mean || !inv_std)) return EPD_EINVAL;
+  if (frame_format == EPD_FRAMES_BF16 && ((uintptr_t)frames & 1)) return EPD_EINVAL;
   fill_host_outputs(bs, n_images, out_rows, out_cu_rows);
   if (bs.T == 0) return EPD_OK;
   std::vector<int64_t> off(n_images);
   int64_t at = 0;
   for (int i = 0; i < n_images; ++i) {
     off[i] = at;
-    at += item_frame_bytes(enc->cfg, grid_thw + 3 * i);
+    at += item_frame_bytes(enc->cfg, grid_thw + 3 * i, frame_format);
   }
-  return encode_frames_at(enc, frames, off.data(), grid_thw, n_images, mean, inv_std, features, bs, s);
+  return encode_frames_at(enc, frames, frame_format, off.data(), grid_thw, n_images, mean, inv_std, features, bs, s);
+}
+
+int epd_encode_frames(epd_encoder_t* enc, const void* frames, const int32_t* grid_thw, int32_t n_images,
+                      const float* mean, const float* inv_std, void* features, int64_t features_capacity_rows,
+                      int64_t* out_rows, int32_t* out_cu_rows, void* stream) {
+  return epd_encode_frames_fmt(enc, frames, EPD_FRAMES_U8, grid_thw, n_images, mean, inv_std, features,
+                               features_capacity_rows, out_rows, out_cu_rows, stream);
 }
 
 int epd_encode_frames_cached(epd_encoder_t* enc, epd_feature_cache_t* cache, const void* frames,
@@ -819,7 +830,7 @@ int epd_encode_frames_cached(epd_encoder_t* enc, epd_feature_cache_t* cache, con
     if ((rc = validate_grids(enc, g.data(), m, -1, &sub))) return rc;
     // the missing items are encoded as a batch of their own into the staging buffer of the workspace
     uint8_t* scratch = enc->at<uint8_t>(enc->lay.stage_features);
-    rc = encode_frames_at(enc, frames, sub_off.data(), g.data(), m, mean, inv_std, scratch, sub, s);
+    rc = encode_frames_at(enc, frames, EPD_FRAMES_U8, sub_off.data(), g.data(), m, mean, inv_std, scratch, sub, s);
     if (rc) return rc;
     launches += enc->launches;
     for (int i = 0; i < n_images; ++i) {
@@ -1054,18 +1065,27 @@ int epd_op_attention(int32_t dtype, const void* q, const void* k, const void* v,
   return EPD_OK;
 }
 
-int epd_op_patchify(int32_t dtype, const void* frames, const int64_t* item_offsets, const int32_t* grid_thw,
-                    const int32_t* cu_seqlens, int32_t n_images, int64_t T, void* patches, int64_t ld,
-                    int32_t in_channels, int32_t patch, int32_t temporal_patch, const float* mean, const float* inv_std,
-                    void* stream) {
+int epd_op_patchify_fmt(int32_t dtype, int32_t frame_format, const void* frames, const int64_t* item_offsets,
+                        const int32_t* grid_thw, const int32_t* cu_seqlens, int32_t n_images, int64_t T, void* patches,
+                        int64_t ld, int32_t in_channels, int32_t patch, int32_t temporal_patch, const float* mean,
+                        const float* inv_std, void* stream) {
   if (dtype != EPD_DTYPE_F32 && dtype != EPD_DTYPE_BF16) return EPD_EINVAL;
+  if (frame_format != EPD_FRAMES_U8 && frame_format != EPD_FRAMES_BF16) return EPD_EINVAL;
   if (n_images < 0 || T < 0 || in_channels < 1 || in_channels > 4 || patch < 1 || temporal_patch < 1) return EPD_EINVAL;
   if (T == 0 || n_images == 0) return EPD_OK;
   if (!frames || !item_offsets || !grid_thw || !cu_seqlens || !patches || !mean || !inv_std) return EPD_EINVAL;
   if (ld < (int64_t)in_channels * temporal_patch * patch * patch) return EPD_EINVAL;
-  EPD_CUDA(patchify(dtype, static_cast<const uint8_t*>(frames), item_offsets, grid_thw, cu_seqlens, n_images, T, patches,
-                    ld, in_channels, patch, temporal_patch, mean, inv_std, static_cast<cudaStream_t>(stream)));
+  EPD_CUDA(patchify(dtype, frame_format, frames, item_offsets, grid_thw, cu_seqlens, n_images, T, patches, ld, in_channels,
+                    patch, temporal_patch, mean, inv_std, static_cast<cudaStream_t>(stream)));
   return EPD_OK;
+}
+
+int epd_op_patchify(int32_t dtype, const void* frames, const int64_t* item_offsets, const int32_t* grid_thw,
+                    const int32_t* cu_seqlens, int32_t n_images, int64_t T, void* patches, int64_t ld,
+                    int32_t in_channels, int32_t patch, int32_t temporal_patch, const float* mean, const float* inv_std,
+                    void* stream) {
+  return epd_op_patchify_fmt(dtype, EPD_FRAMES_U8, frames, item_offsets, grid_thw, cu_seqlens, n_images, T, patches, ld,
+                             in_channels, patch, temporal_patch, mean, inv_std, stream);
 }
 
 int epd_op_merge(int32_t dtype, const void* y, const int32_t* merge_idx, void* out, int64_t Tm, int32_t hidden,

@@ -47,22 +47,31 @@ cudaError_t token_layout(const int32_t* grid_thw, const int32_t* cu_seqlens, con
 }
 
 // =============================================================================================
-// Pixels -> patch vectors: token j = (item, frame f, row r, column c) gathers, from the item's uint8
-// frames [t*Tp, C, h*P, w*P], the window rows r*P.., columns c*P.. of frames f*Tp.. in element order
-// (channel, temporal, y, x); value = (pixel/255 - mean[channel]) * inv_std[channel].
-// One block per token, one thread per (channel, temporal, y) pixel row: P contiguous bytes in, P
-// contiguous elements out.  Bytes per token: K read + K*sizeof(T) written.
+// Pixels -> patch vectors: token j = (item, frame f, row r, column c) gathers, from the item's frames
+// [t*Tp, C, h*P, w*P] (uint8, or bf16 on the same 0..255 scale), the window rows r*P.., columns c*P.. of frames
+// f*Tp.. in element order (channel, temporal, y, x); value = (pixel/255 - mean[channel]) * inv_std[channel].
+// One thread per 8 consecutive elements of a token's patch vector: they are 8 consecutive pixels of one image
+// row when P is a multiple of 8 (one 8-byte / 16-byte load), otherwise they are gathered one by one; either way
+// the thread writes them with 16-byte stores, and neighbouring threads write neighbouring pieces of the same
+// row of the patch matrix.  Bytes per token: K * sizeof(pixel) read + K * sizeof(T) written: HBM bound.
 // =============================================================================================
 struct PixelNorm {
   float mean[4], inv_std[4];
 };
 
-template <typename T>
+__device__ __forceinline__ float pixel_value(uint8_t v) { return (float)v; }
+__device__ __forceinline__ float pixel_value(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T, typename PixT>
 __global__ void __launch_bounds__(256)
-patchify_kernel(const uint8_t* __restrict__ frames, const int64_t* __restrict__ item_off,
-                const int32_t* __restrict__ grid_thw, const int32_t* __restrict__ cu, int n, T* __restrict__ patches,
-                int64_t ld, int C, int P, int Tp, PixelNorm norm) {
-  const int64_t j = blockIdx.x;
+patchify_kernel(const PixT* __restrict__ frames, const int64_t* __restrict__ item_off,
+                const int32_t* __restrict__ grid_thw, const int32_t* __restrict__ cu, int n, int64_t T_tokens,
+                T* __restrict__ patches, int64_t ld, int C, int P, int Tp, PixelNorm norm) {
+  const int pieces = (int)((ld + 7) / 8);                       // 8-element pieces per patch-matrix row
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v >= T_tokens * pieces) return;
+  const int64_t j = v / pieces;
+  const int k0 = (int)(v - j * pieces) * 8;
   int lo = 0, hi = n;  // largest i with cu[i] <= j
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
@@ -75,23 +84,63 @@ patchify_kernel(const uint8_t* __restrict__ frames, const int64_t* __restrict__ 
   const int rem = local - f * h * w;
   const int r = rem / w, c = rem - r * w;
   const int64_t H = (int64_t)h * P, W = (int64_t)w * P;
-  const uint8_t* base = frames + item_off[i];
-  T* out = patches + j * ld;
-  const int rows = C * Tp * P;
-  for (int e = threadIdx.x; e < rows; e += blockDim.x) {
-    const int y = e % P;
-    const int tp = (e / P) % Tp;
-    const int ch = e / (P * Tp);
-    const uint8_t* src = base + (((int64_t)(f * Tp + tp) * C + ch) * H + (int64_t)r * P + y) * W + (int64_t)c * P;
+  const int K = C * Tp * P * P;
+  // item_off counts bytes
+  const PixT* base = reinterpret_cast<const PixT*>(reinterpret_cast<const uint8_t*>(frames) + item_off[i]);
+  float val[8];
+  auto source = [&](int k) -> const PixT* {
+    const int x = k % P, y = (k / P) % P, tp = (k / (P * P)) % Tp, ch = k / (P * P * Tp);
+    return base + (((int64_t)(f * Tp + tp) * C + ch) * H + (int64_t)r * P + y) * W + (int64_t)c * P + x;
+  };
+  if (k0 + 8 <= K && P % 8 == 0) {
+    // 8 pixels of one image row, one channel
+    const PixT* src = source(k0);
+    const int ch = k0 / (P * P * Tp);
     const float m = norm.mean[ch], is = norm.inv_std[ch];
-    T* dst = out + (int64_t)e * P;
-    for (int x = 0; x < P; ++x) dst[x] = from_float<T>(((float)src[x] * (1.0f / 255.0f) - m) * is);
+    PixT px[8];
+    if ((reinterpret_cast<uintptr_t>(src) & (8 * sizeof(PixT) - 1)) == 0) {
+      if constexpr (sizeof(PixT) == 1) *reinterpret_cast<uint2*>(px) = *reinterpret_cast<const uint2*>(src);
+      else *reinterpret_cast<uint4*>(px) = *reinterpret_cast<const uint4*>(src);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) px[e] = src[e];
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) val[e] = (pixel_value(px[e]) * (1.0f / 255.0f) - m) * is;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int k = k0 + e;
+      if (k < K) {
+        const int ch = k / (P * P * Tp);
+        val[e] = (pixel_value(*source(k)) * (1.0f / 255.0f) - norm.mean[ch]) * norm.inv_std[ch];
+      } else {
+        val[e] = 0.0f;   // padding columns of the row (leading dimension > K) are zeroed so that they are never garbage
+      }
+    }
   }
-  // padding columns of the row (leading dimension > K) are zeroed so that they are never garbage
-  for (int e = rows * P + threadIdx.x; e < ld; e += blockDim.x) out[e] = from_float<T>(0.0f);
+  T* out = patches + j * ld + k0;
+  if (k0 + 8 <= ld && (reinterpret_cast<uintptr_t>(out) & 15) == 0) {
+    if constexpr (sizeof(T) == 2) {
+      uint32_t pk[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(val[2 * e], val[2 * e + 1]);
+        pk[e] = *reinterpret_cast<uint32_t*>(&b2);
+      }
+      *reinterpret_cast<uint4*>(out) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    } else {
+      reinterpret_cast<float4*>(out)[0] = make_float4(val[0], val[1], val[2], val[3]);
+      reinterpret_cast<float4*>(out)[1] = make_float4(val[4], val[5], val[6], val[7]);
+    }
+  } else {
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+      if (k0 + e < ld) out[e] = from_float<T>(val[e]);
+  }
 }
 
-cudaError_t patchify(int dtype, const uint8_t* frames, const int64_t* item_off, const int32_t* grid_thw,
+cudaError_t patchify(int dtype, int frame_format, const void* frames, const int64_t* item_off, const int32_t* grid_thw,
                      const int32_t* cu_seqlens, int n_images, int64_t T, void* patches, int64_t ld, int C, int P, int Tp,
                      const float* mean, const float* inv_std, cudaStream_t s) {
   if (T == 0) return cudaSuccess;
@@ -100,12 +149,17 @@ cudaError_t patchify(int dtype, const uint8_t* frames, const int64_t* item_off, 
     norm.mean[c] = c < C ? mean[c] : 0.0f;
     norm.inv_std[c] = c < C ? inv_std[c] : 1.0f;
   }
-  if (dtype == EPD_DTYPE_F32)
-    patchify_kernel<float><<<(unsigned)T, 128, 0, s>>>(frames, item_off, grid_thw, cu_seqlens, n_images, (float*)patches,
-                                                       ld, C, P, Tp, norm);
-  else
-    patchify_kernel<__nv_bfloat16><<<(unsigned)T, 128, 0, s>>>(frames, item_off, grid_thw, cu_seqlens, n_images,
-                                                               (__nv_bfloat16*)patches, ld, C, P, Tp, norm);
+  const int64_t vectors = T * ((ld + 7) / 8);
+  const unsigned blocks = (unsigned)((vectors + 255) / 256);
+#define EPD_PATCHIFY(OUT, PIX)                                                                                   \
+  patchify_kernel<OUT, PIX><<<blocks, 256, 0, s>>>(static_cast<const PIX*>(frames), item_off, grid_thw, cu_seqlens, \
+                                                   n_images, T, static_cast<OUT*>(patches), ld, C, P, Tp, norm)
+  if (frame_format == EPD_FRAMES_U8) {
+    if (dtype == EPD_DTYPE_F32) EPD_PATCHIFY(float, uint8_t); else EPD_PATCHIFY(__nv_bfloat16, uint8_t);
+  } else {
+    if (dtype == EPD_DTYPE_F32) EPD_PATCHIFY(float, __nv_bfloat16); else EPD_PATCHIFY(__nv_bfloat16, __nv_bfloat16);
+  }
+#undef EPD_PATCHIFY
   return cudaGetLastError();
 }
 

@@ -121,7 +121,10 @@ def colocate(args, torch):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["linear", "attention", "rope", "rmsnorm", "merge", "hash", "qkv", "colocate"])
+    ap.add_argument("op", choices=["linear", "attention", "rope", "rmsnorm", "merge", "hash", "qkv", "colocate", "patchify"])
+    ap.add_argument("--image", default="448x448", help="patchify: HxW of every image")
+    ap.add_argument("--patch", type=int, default=16)
+    ap.add_argument("--bf16-frames", action="store_true")
     ap.add_argument("--M", type=int, default=6272)
     ap.add_argument("--N", type=int, default=1152)
     ap.add_argument("--K", type=int, default=1152)
@@ -214,6 +217,31 @@ def main():
                                              epd._ptr(v), T, heads, dh, 10000.0, 0.17, epd._stream_ptr(None)),
                        "epd_op_rope_split")
         res.update(T=T, heads=heads, dh=dh, bytes=2.0 * T * 3 * h + 2.0 * 3 * heads * T * dhp + 8.0 * T)
+    elif args.op == "patchify":
+        H, W = (int(v) for v in args.image.split("x"))
+        P, n = args.patch, args.items
+        hh, ww = H // P, W // P
+        T, K = n * hh * ww, 3 * P * P
+        ld = (K + 7) // 8 * 8
+        pix = torch.randint(0, 256, (n * 3 * hh * P * ww * P,), generator=g, device="cuda", dtype=torch.uint8)
+        es = 1
+        if args.bf16_frames:
+            pix, es = pix.to(bf), 2
+        item_bytes = 3 * hh * P * ww * P * es
+        off = torch.arange(n + 1, device="cuda", dtype=torch.int64) * item_bytes
+        grid = torch.tensor([[1, hh, ww]] * n, device="cuda", dtype=torch.int32)
+        cu = torch.arange(n + 1, device="cuda", dtype=torch.int32) * (hh * ww)
+        out = torch.empty((T, ld), dtype=bf, device="cuda")
+        import ctypes
+        mean = (ctypes.c_float * 3)(0.5, 0.5, 0.5)
+        istd = (ctypes.c_float * 3)(2.0, 2.0, 2.0)
+        lib = epd.load_library()
+
+        def fn():
+            epd._check(lib.epd_op_patchify_fmt(dt, epd.FRAMES_BF16 if args.bf16_frames else epd.FRAMES_U8, epd._ptr(pix),
+                                               epd._ptr(off), epd._ptr(grid), epd._ptr(cu), n, T, epd._ptr(out), ld, 3, P, 1,
+                                               mean, istd, epd._stream_ptr(None)), "epd_op_patchify_fmt")
+        res.update(items=n, image=args.image, patch=P, T=T, K=K, bytes=float(T) * K * (es + 2))
     elif args.op == "rmsnorm":
         T, h = args.T, args.hidden
         x = rnd(T, h, dtype=torch.float32)

@@ -324,16 +324,22 @@ def test_merge(dtype):
 
 
 @pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
-@pytest.mark.parametrize("P,Tp,grids,ldpad", [(16, 1, [(1, 4, 6), (1, 2, 2)], 0), (14, 1, [(1, 2, 4)], 4),
+@pytest.mark.parametrize("P,Tp,grids,ldpad", [(16, 1, [(1, 4, 6), (1, 2, 2)], 0), (14, 1, [(1, 2, 4)], 4), (8, 1, [(1, 2, 6)], 3),
                                               (16, 2, [(3, 2, 4), (1, 6, 2)], 0), (2, 2, [(2, 2, 2)], 8)])
-def test_patchify(dtype, P, Tp, grids, ldpad):
-    """Raw uint8 frames -> patch vectors against the oracle (one rounding to the element type)."""
+@pytest.mark.parametrize("pixels", ["u8", "bf16"])
+def test_patchify(dtype, P, Tp, grids, ldpad, pixels):
+    """Raw frames (uint8, or bf16 values with fractions on the same 0..255 scale) -> patch vectors against the
+    oracle (one rounding to the element type)."""
     cfg = synth.tiny_variant(patch=P, temporal_patch=Tp)
     frames = synth.make_frames(cfg, grids, seed=21)
+    if pixels == "bf16":
+        rng = np.random.default_rng(3)
+        frames = [synth.round_to_bf16((f.astype(np.float32) + rng.random(f.shape, dtype=np.float32)) * 0.97)
+                  for f in frames]
     mean, std = (0.48, 0.46, 0.41), (0.27, 0.26, 0.28)
     ref = O.patchify(frames, grids, P, Tp, mean, std)
     bk = O.bookkeeping(grids)
-    fd, off = epd.pack_frames(frames)
+    fd, off = epd.pack_frames(frames, bf16=pixels == "bf16")
     K = cfg.patch_dim
     got = epd.op_patchify(dtype, fd, off, grids, bk["cu_seqlens"], cfg.in_channels, P, Tp, mean, std, ld=K + ldpad)
     g = to_np(got)
@@ -361,6 +367,11 @@ def test_stage_from_raw_frames():
     again, _ = enc.encode_frames(fd, grids, synth.PIXEL_MEAN, synth.PIXEL_STD)
     torch.cuda.synchronize()
     assert torch.equal(feats, again)
+    # the same pixels handed over as bfloat16 (0..255 is exact in it): the same features, bit for bit
+    fb, _ = epd.pack_frames([f.astype(np.float32) for f in frames], bf16=True)
+    from_bf16, _ = enc.encode_frames(fb, grids, synth.PIXEL_MEAN, synth.PIXEL_STD)
+    torch.cuda.synchronize()
+    assert torch.equal(feats, from_bf16)
     enc.close()
 
 

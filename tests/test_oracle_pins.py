@@ -481,3 +481,71 @@ def test_content_hash_against_vectorised_restatement_and_properties():
     assert O.content_hash(data + bytes(8)) != h           # trailing zeros matter
     with pytest.raises(ValueError):
         O.content_hash(b"abc")
+
+
+# ----------------------------------------------------------------------------- 8-bit floating-point variant
+
+def test_round_to_e4m3_hand_computed_values():
+    """Values worked out by hand from the format's definition (sign, 4 exponent bits with bias 7, 3 mantissa
+    bits, largest finite value 448, subnormal step 2^-9, ties to the even mantissa, saturation)."""
+    cases = [
+        (0.3, 0.3125),        # binade [0.25, 0.5): step 2^-5; 0.3 / 2^-5 = 9.6 -> 10
+        (17.0, 16.0),         # binade [16, 32): step 2; 8.5 -> 8 (tie to even)
+        (19.0, 20.0),         # 9.5 -> 10 (tie to even)
+        (21.0, 20.0),         # 10.5 -> 10
+        (448.0, 448.0), (449.0, 448.0), (1e6, 448.0), (-500.0, -448.0),     # saturation
+        (464.0, 448.0),       # would round to 480, which the format does not have
+        (2.0 ** -9, 2.0 ** -9), (0.001, 2.0 ** -9), (0.0009, 0.0),          # subnormals: step 2^-9
+        (1.5 * 2.0 ** -9, 2.0 ** -8),                                        # tie between 1 and 2 steps -> 2 (even)
+        (2.0 ** -6, 2.0 ** -6), (0.0, 0.0), (-1.0625, -1.0), (1.0625 + 1e-9, 1.125),
+    ]
+    for v, want in cases:
+        assert float(O.round_to_e4m3(np.array([v]))[0]) == want, (v, want)
+    # every one of the 2 x 127 finite codes maps to itself, and the codes come back
+    codes = np.array([c for c in range(256) if (c & 0x7F) != 0x7F], dtype=np.uint8)
+    sign = np.where(codes & 0x80, -1.0, 1.0)
+    ef, mf = ((codes >> 3) & 0xF).astype(np.float64), (codes & 7).astype(np.float64)
+    vals = sign * np.where(ef > 0, np.exp2(ef - 7) * (1 + mf / 8), mf * 2.0 ** -9)
+    assert np.array_equal(O.round_to_e4m3(vals), vals)
+    nonzero = vals != 0
+    assert np.array_equal(O.e4m3_bits(vals[nonzero]), codes[nonzero])
+    assert np.max(np.abs(vals)) == 448.0
+
+
+def test_round_to_e4m3_agrees_with_the_library_conversion():
+    """Inside the finite range PyTorch's CPU conversion to float8_e4m3fn is the same rounding."""
+    torch = pytest.importorskip("torch")
+    if not hasattr(torch, "float8_e4m3fn"):
+        pytest.skip("no float8 in this torch")
+    rng = np.random.default_rng(0)
+    v = np.concatenate([rng.standard_normal(20000) * 30, rng.standard_normal(20000) * 0.01,
+                        rng.uniform(-440, 440, 20000)]).astype(np.float32)
+    lib = torch.from_numpy(v).to(torch.float8_e4m3fn).to(torch.float32).numpy().astype(np.float64)
+    assert np.array_equal(O.round_to_e4m3(v), lib)
+
+
+def test_quantize_rows_and_linear_e4m3_properties():
+    rng = np.random.default_rng(1)
+    x = rng.standard_normal((7, 40)) * np.array([1e-3, 1, 5, 100, 0.2, 3, 1])[:, None]
+    x[4, :] = 0.0
+    q, s = O.quantize_e4m3_rows(x)
+    assert s[4] == 1.0 and np.all(q[4] == 0)
+    amax = np.max(np.abs(x.astype(np.float32)), axis=1)
+    for i in (0, 1, 2, 3, 5, 6):
+        assert np.max(np.abs(q[i])) == 448.0                         # the largest element of a row lands on 448
+        assert abs(s[i] * 448.0 / amax[i] - 1) < 1e-6
+    # relative error of an element at most half a step of its binade: 2^-4 of the value (normal range)
+    big = np.abs(q) >= 2.0 ** -6
+    rel = np.abs(q * s[:, None] - x)[big] / np.abs(x)[big]
+    assert rel.max() <= 2.0 ** -4 + 1e-6
+    # values that are already E4M3 multiples of the row scale pass through exactly: linear_e4m3 == plain product
+    xs = O.round_to_e4m3(rng.uniform(-448, 448, (5, 16)))
+    ws = O.round_to_e4m3(rng.uniform(-448, 448, (3, 16)))
+    xs[:, 0], ws[:, 0] = 448.0, -448.0                               # every row's scale becomes exactly 1
+    b = rng.standard_normal(3)
+    assert np.allclose(O.linear_e4m3(xs, ws, b), xs @ ws.T + b, rtol=0, atol=1e-9)
+    # scale invariance: scaling a row of x by a power of two scales its outputs by the same factor, exactly
+    x2 = x.copy(); x2[1] *= 8.0
+    w = rng.standard_normal((6, 40))
+    y, y2 = O.linear_e4m3(x, w, None), O.linear_e4m3(x2, w, None)
+    assert np.array_equal(y2[1], 8.0 * y[1]) and np.array_equal(y2[0], y[0])
