@@ -302,6 +302,23 @@ enum {
 int epd_op_linear(int32_t dtype, const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias,
                   void* out, int64_t ldo, int64_t M, int64_t N, int64_t K, int32_t flags, void* stream);
 
+/* The same layer with 8-bit floating-point operands, a variant beside the bf16 path (Section 3.5 names the
+ * operator mix of the stages; the paper states no precision).  Format E4M3: 4 exponent bits with bias 7, 3
+ * mantissa bits, largest finite value 448, no infinities.
+ * epd_op_quantize_e4m3: x bf16 [M, K] (leading dimension ldx, a multiple of 8) -> q bytes [M, ldq] (ldq a multiple
+ *   of 16, padding bytes zeroed) and scale float [M]:  scale[i] = max_j |x[i,j]| / 448 (1 for an all-zero row),
+ *   q[i,j] = the E4M3 value nearest to x[i,j] / scale[i] (ties to even, saturating); both divisions are IEEE float
+ *   divisions.  Used for activations (one scale per token) and, once, for weights (one scale per output feature).
+ * epd_op_linear_e4m3: out[M,N] = act((xq . wq^T) * x_scale * w_scale^T + bias), xq [M, K] and wq [N, K] byte codes,
+ *   products exact and summed in float on the tensor cores (tcgen05.mma kind::f8f6f4); bias bf16 or NULL; out bf16,
+ *   or float with EPD_LINEAR_OUT_F32; the GELU flags apply; EPD_LINEAR_ACCUMULATE is not offered.  All pointers
+ *   device, 16-byte aligned; N a multiple of 8. */
+int epd_op_quantize_e4m3(const void* x, int64_t ldx, void* q, int64_t ldq, float* scale, int64_t M, int64_t K,
+                         void* stream);
+int epd_op_linear_e4m3(const void* xq, int64_t ldx, const float* x_scale, const void* wq, int64_t ldw,
+                       const float* w_scale, const void* bias, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                       int32_t flags, void* stream);
+
 /* out[j,:] = x[j,:] / sqrt(mean(x[j,:]^2) + eps) * gain, x float [T, hidden], out per dtype.
  * If dst_row != NULL (device int32 [T]) row j is written at element offset dst_row[j]*hidden
  * instead of j*hidden (used to fuse the 2x2 merge into the final norm). */

@@ -195,7 +195,7 @@ def round_to_e4m3(v: np.ndarray) -> np.ndarray:
     quantum = np.exp2(e - 3.0)
     q = np.rint(a / quantum) * quantum          # rint: round half to even; a / quantum is exact (power of two)
     q = np.minimum(q, E4M3_MAX)
-    return np.sign(v) * q
+    return np.copysign(q, v)                    # the sign survives, for zeros too (the format has a negative zero)
 
 
 def e4m3_bits(q: np.ndarray) -> np.ndarray:

@@ -37,6 +37,7 @@ EXPORTED_SYMBOLS = [
     "epd_set_sm_limit", "epd_get_sm_limit", "epd_signal_ready", "epd_op_stream_read", "epd_op_content_hash", "epd_feature_cache_create", "epd_feature_cache_destroy",
     "epd_feature_cache_lookup", "epd_feature_cache_insert", "epd_feature_cache_stats",
     "epd_encode_frames_cached", "epd_debug_set_wait_limit", "epd_encode_frames_fmt", "epd_op_patchify_fmt",
+    "epd_op_quantize_e4m3", "epd_op_linear_e4m3",
 ]
 
 
@@ -110,6 +111,10 @@ def load_library() -> ctypes.CDLL:
     lib.epd_debug_set_wait_limit.argtypes = [i64]
     lib.epd_op_patchify.restype = ctypes.c_int
     lib.epd_op_patchify.argtypes = [i32, vp, vp, vp, vp, i32, i64, vp, i64, i32, i32, i32, f32p, f32p, vp]
+    lib.epd_op_quantize_e4m3.restype = ctypes.c_int
+    lib.epd_op_quantize_e4m3.argtypes = [vp, i64, vp, i64, vp, i64, i64, vp]
+    lib.epd_op_linear_e4m3.restype = ctypes.c_int
+    lib.epd_op_linear_e4m3.argtypes = [vp, i64, vp, vp, i64, vp, vp, vp, i64, i64, i64, i64, i32, vp]
     lib.epd_op_patchify_fmt.restype = ctypes.c_int
     lib.epd_op_patchify_fmt.argtypes = [i32, i32, vp, vp, vp, vp, i32, i64, vp, i64, i32, i32, i32, f32p, f32p, vp]
     lib.epd_encode_frames_fmt.restype = ctypes.c_int
@@ -464,6 +469,28 @@ def op_linear(dtype, x, w, bias, out, M, N, K, flags=0, ldx=None, ldw=None, ldo=
                              ldw if ldw is not None else w.stride(0), _ptr(bias), _ptr(out),
                              ldo if ldo is not None else out.stride(0), M, N, K, flags, _stream_ptr(stream)),
            "epd_op_linear")
+    return out
+
+
+def op_quantize_e4m3(x, stream=None):
+    """bf16 [M, K] -> (E4M3 byte codes [M, ldq] with ldq = K rounded up to 16, float scales [M])."""
+    torch = _torch()
+    lib = load_library()
+    M, K = x.shape
+    ldq = (K + 15) // 16 * 16
+    q = torch.empty((M, ldq), dtype=torch.uint8, device=x.device)
+    scale = torch.empty(M, dtype=torch.float32, device=x.device)
+    _check(lib.epd_op_quantize_e4m3(_ptr(x), x.stride(0), _ptr(q), ldq, _ptr(scale), M, K, _stream_ptr(stream)),
+           "epd_op_quantize_e4m3")
+    return q, scale
+
+
+def op_linear_e4m3(xq, x_scale, wq, w_scale, bias, out, K, flags=0, stream=None):
+    lib = load_library()
+    M, N = xq.shape[0], wq.shape[0]
+    _check(lib.epd_op_linear_e4m3(_ptr(xq), xq.stride(0), _ptr(x_scale), _ptr(wq), wq.stride(0), _ptr(w_scale),
+                                  _ptr(bias), _ptr(out), out.stride(0), M, N, K, flags, _stream_ptr(stream)),
+           "epd_op_linear_e4m3")
     return out
 
 

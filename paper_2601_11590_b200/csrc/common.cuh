@@ -105,6 +105,9 @@ bool attention_pair_supported(const void* q, const void* k, const void* v, const
 cudaError_t attention_pair(const void* q, const void* k, const void* v, const int32_t* host_cu_seqlens, int n_seg,
                            void* out, int64_t T, int heads, int head_dim, int* status, cudaStream_t s);
 
+// True if the driver offers the tensor-map encoder the tensor-core kernels need.
+bool tensor_core_path_available();
+
 // ---- tensor-core kernels (gemm_tcgen05.cu) ---------------------------------------------------
 // bf16 x bf16 -> fp32 linear layer on tcgen05; `status` (device int, may be NULL) receives
 // EPD_ETIMEOUT if a bounded wait expires.  forced_bn: 0 = choose the tile width automatically.
@@ -117,6 +120,13 @@ cudaError_t linear_tc(const void* x, int64_t ldx, const void* w, int64_t ldw, co
 cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
                            int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, int* status, cudaStream_t s);
 
+
+// 8-bit floating-point (E4M3) variant: row quantiser (kernels_fma.cu) and the layer itself (gemm_tcgen05_pair.cu).
+cudaError_t quantize_rows_e4m3(const void* x, int64_t ldx, void* q, int64_t ldq, float* scale, int64_t M, int64_t K,
+                               cudaStream_t s);
+cudaError_t linear_tc_pair_e4m3(const void* xq, int64_t ldx, const float* row_scale, const void* wq, int64_t ldw,
+                                const float* col_scale, const void* bias, void* out, int64_t ldo, int64_t M, int64_t N,
+                                int64_t K, int flags, int* status, cudaStream_t s);
 
 // QKV projection whose epilogue applies the rotary embedding and writes head-major q, k, v (the
 // padding columns are left as the caller initialised them with qkv_pad_init).  w_perm / bias_perm come

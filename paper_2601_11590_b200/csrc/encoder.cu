@@ -996,6 +996,33 @@ int epd_op_rmsnorm(int32_t dtype, const void* x, const void* gain, void* out, co
   return EPD_OK;
 }
 
+int epd_op_quantize_e4m3(const void* x, int64_t ldx, void* q, int64_t ldq, float* scale, int64_t M, int64_t K,
+                         void* stream) {
+  if (M < 0 || K < 1 || ldx < K || ldq < K) return EPD_EINVAL;
+  if (M == 0) return EPD_OK;
+  if (!x || !q || !scale) return EPD_EINVAL;
+  if (((uintptr_t)x & 15) || ((uintptr_t)q & 15) || (ldx % 8) || (ldq % 16)) return EPD_EINVAL;
+  EPD_CUDA(quantize_rows_e4m3(x, ldx, q, ldq, scale, M, K, static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
+int epd_op_linear_e4m3(const void* xq, int64_t ldx, const float* x_scale, const void* wq, int64_t ldw,
+                       const float* w_scale, const void* bias, void* out, int64_t ldo, int64_t M, int64_t N, int64_t K,
+                       int32_t flags, void* stream) {
+  if (M < 0 || N < 0 || K < 1 || ldx < K || ldw < K || ldo < N) return EPD_EINVAL;
+  if (flags & (EPD_LINEAR_ACCUMULATE | EPD_LINEAR_FORCE_FMA)) return EPD_EUNSUPPORTED;
+  if (M == 0 || N == 0) return EPD_OK;
+  if (!xq || !wq || !x_scale || !w_scale || !out) return EPD_EINVAL;
+  const bool out_f32 = flags & EPD_LINEAR_OUT_F32;
+  if (((uintptr_t)xq | (uintptr_t)wq | (uintptr_t)out) & 15) return EPD_EINVAL;
+  if ((ldx % 16) || (ldw % 16) || (ldo % (out_f32 ? 4 : 8)) || (N % 8) || M > (1 << 30) || N > (1 << 30) || K > (1 << 30))
+    return EPD_EUNSUPPORTED;
+  if (!tensor_core_path_available()) return EPD_EUNSUPPORTED;
+  EPD_CUDA(linear_tc_pair_e4m3(xq, ldx, x_scale, wq, ldw, w_scale, bias, out, ldo, M, N, K, flags, nullptr,
+                               static_cast<cudaStream_t>(stream)));
+  return EPD_OK;
+}
+
 int32_t epd_padded_head_dim(int32_t head_dim) { return padded_head_dim(head_dim); }
 
 int epd_op_rope_split(int32_t dtype, const void* qkv, const int32_t* pos_row, const int32_t* pos_col, void* q,

@@ -85,15 +85,26 @@ __device__ __forceinline__ void tmem_dealloc_pair(uint32_t addr, uint32_t cols) 
 }
 
 // D[tmem, both CTAs] (+)= A[smem, 128 rows per CTA] . B[smem, half the columns per CTA]^T; issued by
-// one thread of the leader CTA.
-__device__ __forceinline__ void umma_pair_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                               uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
-      : "memory");
+// one thread of the leader CTA.  FP8: 8-bit floating-point operands (kind::f8f6f4, 32 elements per instruction)
+// instead of 16-bit ones (kind::f16, 16 elements per instruction): 32 bytes of every row either way.
+template <bool FP8>
+__device__ __forceinline__ void umma_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                          uint32_t accumulate) {
+  if constexpr (FP8) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
 }
 // Once all MMAs issued so far by this thread have completed, arrive on the barrier at this offset in
 // both CTAs of the pair.
@@ -104,9 +115,10 @@ __device__ __forceinline__ void umma_commit_both(uint64_t* bar) {
       : "memory");
 }
 
-// bf16 x bf16 -> fp32, both operands K-major, M = 256 over the pair, N = BN.
-__host__ __device__ constexpr uint32_t instr_desc_pair(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+// Instruction descriptor: fp32 accumulation, both operands K-major, M = 256 over the pair, N = BN; operand format
+// bf16 (code 1 of kind::f16) or E4M3 (code 0 of kind::f8f6f4).
+__host__ __device__ constexpr uint32_t instr_desc_pair(int n, bool fp8) {
+  return (1u << 4) | (fp8 ? 0u : ((1u << 7) | (1u << 10))) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 
 // Destination of the QKV variant's epilogue.
@@ -131,7 +143,8 @@ struct PairLayout {
   // full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2], drain, (spare), tmem base, abort flag,
   // bias[kEpiWarps][BN/2]
   static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 6) * 8 + 16;
-  static constexpr int kTotal = kBiasOffset + kEpiWarps * (BN / 2) * 4;
+  static constexpr int kScaleOffset = kBiasOffset + kEpiWarps * (BN / 2) * 4;   // column scales of the 8-bit variant
+  static constexpr int kTotal = kScaleOffset + kEpiWarps * (BN / 2) * 4;
   static constexpr int kDynamic = kTotal + 1024;
   static_assert(kDynamic <= 232448, "exceeds the shared memory of one CTA");
   static_assert(kDynamic > 116 * 1024, "one CTA per SM is assumed by the TMEM allocation");
@@ -140,12 +153,16 @@ struct PairLayout {
 // ---------------------------------------------------------------------------------------------
 // Kernel
 // ---------------------------------------------------------------------------------------------
-template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE>
+template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE, bool FP8>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_out, const __nv_bfloat16* __restrict__ bias, int M, int N,
-                   int K, int* __restrict__ status, long long wait_limit, int static_w, const RopeSplitArgs rs) {
+                   int K, int* __restrict__ status, long long wait_limit, int static_w, const RopeSplitArgs rs,
+                   const float* __restrict__ row_scale, const float* __restrict__ col_scale) {
   static_assert(!ROPE || (sizeof(OutT) == 2 && ACT == 0 && !ACCUM), "the QKV variant writes bf16, no activation");
+  static_assert(!(ROPE && FP8), "the QKV variant takes bf16 operands");
+  // elements per contraction block (128 bytes of a row) and per MMA (32 bytes)
+  constexpr int BKE = FP8 ? 2 * BK : BK;
   using L = PairLayout<BN, STAGES>;
   static_assert(BN == 256 || BN == 128, "tile width");
   constexpr int kAccStride = BN;                 // TMEM columns between the two accumulators
@@ -171,7 +188,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
   const int m_tiles = (M + 2 * BM - 1) / (2 * BM), n_tiles = (N + BN - 1) / BN;
   const int num_tiles = m_tiles * n_tiles;
-  const int k_blocks = (K + BK - 1) / BK;
+  const int k_blocks = (K + BKE - 1) / BKE;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -200,7 +217,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     early = k_blocks < STAGES ? k_blocks : STAGES;
     for (int kb = 0; kb < early; ++kb) {
       if (rank == 0) mbar_expect_tx(&full[kb], 2 * L::kStageBytes);
-      tma_load_2d_pair(smem + kb * L::kStageBytes + L::kABytes, &tm_w, kb * BK, n0, map_to_rank(smem_u32(&full[kb]), 0));
+      tma_load_2d_pair(smem + kb * L::kStageBytes + L::kABytes, &tm_w, kb * BKE, n0, map_to_rank(smem_u32(&full[kb]), 0));
     }
     loads_issued = early;     // for the drain after an abort: these stages have loads in flight
   }
@@ -227,9 +244,9 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           } else {
             // the leader's barrier counts the bytes of both CTAs
             if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
-            tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BK, n0, bar);
+            tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BKE, n0, bar);
           }
-          tma_load_2d_pair(sa, &tm_x, kb * BK, m0, bar);
+          tma_load_2d_pair(sa, &tm_x, kb * BKE, m0, bar);
           ++loads_issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -239,7 +256,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader only)
     if (lane == 0 && rank == 0) {
-      constexpr uint32_t idesc = instr_desc_pair(BN);
+      constexpr uint32_t idesc = instr_desc_pair(BN, FP8);
       int stage = 0;
       uint32_t phase = 0;
       int acc = 0;
@@ -255,8 +272,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint64_t da = smem_desc_k_sw128(sa), db = smem_desc_k_sw128(sa + L::kABytes);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)   // 16 bf16 along K inside the swizzled row = 32 bytes = 2 descriptor units
-            umma_pair_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+          for (int k = 0; k < BK / 16; ++k)   // one MMA per 32 bytes along K inside the swizzled row = 2 descriptor units
+            umma_pair<FP8>(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
           umma_commit_both(&empty[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -273,6 +290,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     const int q = warp & 3;                          // TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;                // which half of the columns
     float* bs = bias_s + (warp - 2) * (BN / 2);
+    float* cs = reinterpret_cast<float*>(smem + L::kScaleOffset) + (warp - 2) * (BN / 2);
     uint8_t* sbuf = smem + L::kOutOffset + (warp - 2) * L::kOutBufBytes;
     const uint32_t tmem_empty_leader0 = map_to_rank(smem_u32(&tmem_empty[0]), 0);
     int acc = 0;
@@ -294,12 +312,16 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;
       const int n0 = (tile / m_tiles) * BN + half * (BN / 2);
       __syncwarp();
-      for (int i = lane; i < BN / 2; i += 32)
+      for (int i = lane; i < BN / 2; i += 32) {
         bs[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
+        if constexpr (FP8) cs[i] = n0 + i < N ? col_scale[n0 + i] : 0.0f;
+      }
       __syncwarp();
       if (!mbar_wait_warp<true>(&tmem_full[acc], acc_phase, wc)) break;
       tc_fence_after();
       const int row0 = m0 + q * 32;
+      float rscale = 1.0f;                              // 8-bit variant: this thread's row scale
+      if constexpr (FP8) rscale = row0 + lane < M ? row_scale[row0 + lane] : 0.0f;
       const uint32_t taddr = tmem_base + acc * kAccStride + half * (BN / 2) + ((uint32_t)(q * 32) << 16);
       // QKV variant: this thread's row positions, and (tensor, head, dim) of its first column
       int prow = 0, pcol = 0, rt = 0, rhead = 0, rd = 0;
@@ -324,7 +346,9 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
             const float bb[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              float t = __uint_as_float(pk[4 * j4 + e]) + bb[e];
+              float t = __uint_as_float(pk[4 * j4 + e]);
+              if constexpr (FP8) t *= rscale * cs[c * CC + 4 * j4 + e];
+              t += bb[e];
               if (ACT == 1) t = gelu_tanh_fast(t);
               if (ACT == 2) t = gelu_erf_fast(t);
               pk[4 * j4 + e] = __float_as_uint(t);
@@ -379,8 +403,13 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
               const uint32_t* src = j2 < 8 ? r0 : r1;
               const int jj = (4 * j2) & 31;
               const float4 bv = bs4[j2];
-              float t0 = __uint_as_float(src[jj]) + bv.x, t1 = __uint_as_float(src[jj + 1]) + bv.y;
-              float t2 = __uint_as_float(src[jj + 2]) + bv.z, t3 = __uint_as_float(src[jj + 3]) + bv.w;
+              float t0 = __uint_as_float(src[jj]), t1 = __uint_as_float(src[jj + 1]);
+              float t2 = __uint_as_float(src[jj + 2]), t3 = __uint_as_float(src[jj + 3]);
+              if constexpr (FP8) {
+                const float4 sv = *reinterpret_cast<const float4*>(cs + c * CC + 4 * j2);
+                t0 *= rscale * sv.x; t1 *= rscale * sv.y; t2 *= rscale * sv.z; t3 *= rscale * sv.w;
+              }
+              t0 += bv.x; t1 += bv.y; t2 += bv.z; t3 += bv.w;
               if (ACT == 1) { t0 = gelu_tanh_fast(t0); t1 = gelu_tanh_fast(t1); t2 = gelu_tanh_fast(t2); t3 = gelu_tanh_fast(t3); }
               if (ACT == 2) { t0 = gelu_erf_fast(t0); t1 = gelu_erf_fast(t1); t2 = gelu_erf_fast(t2); t3 = gelu_erf_fast(t3); }
               __nv_bfloat162 b0 = __floats2bfloat162_rn(t0, t1), b1 = __floats2bfloat162_rn(t2, t3);
@@ -479,11 +508,12 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int
                             CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
-template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE = false>
+template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE = false, bool FP8 = false>
 cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& to, const void* bias, int M, int N,
-                   int K, int* status, cudaStream_t s, int static_w, const RopeSplitArgs& rs = RopeSplitArgs{}) {
+                   int K, int* status, cudaStream_t s, int static_w, const RopeSplitArgs& rs = RopeSplitArgs{},
+                   const float* row_scale = nullptr, const float* col_scale = nullptr) {
   using L = PairLayout<BN, STAGES>;
-  auto kern = linear_pair_kernel<BN, STAGES, OutT, ACT, ACCUM, ROPE>;
+  auto kern = linear_pair_kernel<BN, STAGES, OutT, ACT, ACCUM, ROPE, FP8>;
   static PerDeviceOnce configured;
   cudaError_t e = once_per_device(configured, [&] {
     return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, ROPE ? kMaxDynamicSmem : L::kDynamic);
@@ -521,7 +551,7 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
   const int avail = limited_sms(2 * max_pairs) / 2 > 0 ? limited_sms(2 * max_pairs) / 2 : 1;   // pairs within the SM budget
   const int pairs = tiles < avail ? tiles : avail;
   return launch_pdl(kern, dim3(2 * pairs), dim3(kThreads), smem_bytes, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K,
-                    status, wait_limit_cycles(), static_w, rs);
+                    status, wait_limit_cycles(), static_w, rs, row_scale, col_scale);
 }
 
 template <int BN, int STAGES>
@@ -560,6 +590,33 @@ cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ld
       !make_map(&to, out, M, N, ldo, 32, out_f32 ? 4 : 2))
     return cudaErrorInvalidValue;
   return launch_bn<BN, 5>(tx, tw, to, bias, (int)M, (int)N, (int)K, flags, status, s);
+}
+
+// The same layer with 8-bit floating-point operands (E4M3): xq [M, K] and wq [N, K] hold byte codes, row_scale [M] and
+// col_scale [N] the factors they were divided by; out = act((xq . wq^T) * row_scale * col_scale^T + bias), bf16 or
+// (EPD_LINEAR_OUT_F32) float.  K a multiple of 16 bytes, leading dimensions too.
+cudaError_t linear_tc_pair_e4m3(const void* xq, int64_t ldx, const float* row_scale, const void* wq, int64_t ldw,
+                                const float* col_scale, const void* bias, void* out, int64_t ldo, int64_t M, int64_t N,
+                                int64_t K, int flags, int* status, cudaStream_t s) {
+  constexpr int BN = 256;
+  const bool out_f32 = flags & EPD_LINEAR_OUT_F32;
+  const int act = (flags & EPD_LINEAR_GELU_TANH) ? 1 : (flags & EPD_LINEAR_GELU_ERF) ? 2 : 0;
+  CUtensorMap tx, tw, to;
+  if (!make_map(&tx, xq, M, K, ldx, BM, 1) || !make_map(&tw, wq, N, K, ldw, BN / 2, 1) ||
+      !make_map(&to, out, M, N, ldo, 32, out_f32 ? 4 : 2))
+    return cudaErrorInvalidValue;
+#define EPD_F8(OUT, A) \
+  return launch<BN, 5, OUT, A, false, false, true>(tx, tw, to, bias, (int)M, (int)N, (int)K, status, s, 0, RopeSplitArgs{}, \
+                                                   row_scale, col_scale)
+  if (out_f32) {
+    if (act == 0) EPD_F8(float, 0);
+    if (act == 1) EPD_F8(float, 1);
+    EPD_F8(float, 2);
+  }
+  if (act == 0) EPD_F8(__nv_bfloat16, 0);
+  if (act == 1) EPD_F8(__nv_bfloat16, 1);
+  EPD_F8(__nv_bfloat16, 2);
+#undef EPD_F8
 }
 
 // QKV projection with the rotary embedding and the head split in its epilogue.  w and bias hold the q

@@ -164,6 +164,68 @@ cudaError_t patchify(int dtype, int frame_format, const void* frames, const int6
 }
 
 // =============================================================================================
+// Row-wise quantisation to 8-bit floating point (E4M3) for the 8-bit variant of the linear layer:
+//   scale[i] = max_j |x[i, j]| / 448 (1 for an all-zero row),  q[i, j] = e4m3(x[i, j] / scale[i])
+// with round-to-nearest-even and saturation.  One warp per row; the row is read twice (the second pass hits
+// L2), 16 bytes per load, 8 bytes per store.  Both divisions are IEEE float divisions: the quotient decides the
+// 8-bit code, so it is formed the same way wherever the codes are checked.
+// =============================================================================================
+__device__ __forceinline__ uint16_t e4m3x2(float lo, float hi) {
+  uint16_t d;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));   // first source -> upper byte
+  return d;
+}
+
+__global__ void __launch_bounds__(256)
+quantize_rows_e4m3_kernel(const __nv_bfloat16* __restrict__ x, int64_t ldx, uint8_t* __restrict__ q, int64_t ldq,
+                          float* __restrict__ scale, int64_t M, int K) {
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const __nv_bfloat16* xr = x + row * ldx;
+  const int vecs = K / 8;
+  float amax = 0.0f;
+  for (int v = lane; v < vecs; v += 32) {
+    const uint4 u = *reinterpret_cast<const uint4*>(xr + 8 * v);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(h[e]);
+      amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));
+    }
+  }
+  for (int k = vecs * 8 + lane; k < K; k += 32) amax = fmaxf(amax, fabsf(__bfloat162float(xr[k])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  const float sc = amax > 0.0f ? __fdiv_rn(amax, 448.0f) : 1.0f;
+  if (lane == 0) scale[row] = sc;
+  uint8_t* qr = q + row * ldq;
+  for (int v = lane; v < vecs; v += 32) {
+    const uint4 u = *reinterpret_cast<const uint4*>(xr + 8 * v);
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+    uint16_t c[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 f = __bfloat1622float2(h[e]);
+      c[e] = e4m3x2(__fdiv_rn(f.x, sc), __fdiv_rn(f.y, sc));
+    }
+    *reinterpret_cast<uint2*>(qr + 8 * v) = make_uint2((uint32_t)c[0] | ((uint32_t)c[1] << 16),
+                                                       (uint32_t)c[2] | ((uint32_t)c[3] << 16));
+  }
+  for (int k = vecs * 8 + lane; k < K; k += 32)
+    qr[k] = (uint8_t)(e4m3x2(__fdiv_rn(__bfloat162float(xr[k]), sc), 0.0f) & 0xFF);
+  for (int64_t k = K + lane; k < ldq; k += 32) qr[k] = 0;     // padding bytes of the row: zero codes
+}
+
+cudaError_t quantize_rows_e4m3(const void* x, int64_t ldx, void* q, int64_t ldq, float* scale, int64_t M, int64_t K,
+                               cudaStream_t s) {
+  if (M == 0) return cudaSuccess;
+  quantize_rows_e4m3_kernel<<<(unsigned)((M + 7) / 8), 256, 0, s>>>(static_cast<const __nv_bfloat16*>(x), ldx,
+                                                                  static_cast<uint8_t*>(q), ldq, scale, M, (int)K);
+  return cudaGetLastError();
+}
+
+// =============================================================================================
 // Linear layer with plain FMAs: out = act(x . w^T + bias), 64x64 tile, 4x4 outputs per thread.
 // =============================================================================================
 constexpr int kFmaTile = 64;

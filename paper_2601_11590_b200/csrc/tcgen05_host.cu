@@ -31,6 +31,7 @@ std::atomic<int> g_sm_count[64] = {};
 }  // namespace
 
 bool tensor_maps_available() { return encode_tiled_fn() != nullptr; }
+bool tensor_core_path_available() { return tensor_maps_available(); }
 
 bool make_tensor_map_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t pitch_bytes,
                         int box_rows, int box_cols, int elem_bytes, CUtensorMapSwizzle swizzle) {

@@ -129,6 +129,7 @@ def main():
     ap.add_argument("--N", type=int, default=1152)
     ap.add_argument("--K", type=int, default=1152)
     ap.add_argument("--mode", default="plain", choices=["plain", "gelu_tanh", "gelu_erf", "accum", "out_f32"])
+    ap.add_argument("--e4m3", action="store_true", help="linear: the 8-bit floating-point variant (operands quantised beforehand)")
     ap.add_argument("--tile-n", type=int, default=0)
     ap.add_argument("--T", type=int, default=6272)
     ap.add_argument("--hidden", type=int, default=1152)
@@ -176,6 +177,11 @@ def main():
         f32 = args.mode in ("accum", "out_f32")
         out = torch.zeros((M, N), dtype=torch.float32 if f32 else bf, device="cuda")
         fn = lambda: epd.op_linear(dt, x, w, b, out, M, N, K, flags)
+        if args.e4m3:
+            xq, xs = epd.op_quantize_e4m3(x)
+            wq, ws = epd.op_quantize_e4m3(w)
+            fn = lambda: epd.op_linear_e4m3(xq, xs, wq, ws, b, out, K, flags)
+            res.update(e4m3=True)
         res.update(M=M, N=N, K=K, mode=args.mode, tile_n=args.tile_n, flops=2.0 * M * N * K,
                    bytes=2.0 * (M * K + N * K) + (8.0 if args.mode == "accum" else 4.0 if f32 else 2.0) * M * N)
     elif args.op == "attention":

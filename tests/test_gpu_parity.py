@@ -112,6 +112,36 @@ def test_linear_tensor_core_tiles(tile_n, M, N, K, ldpad, mode):
     assert_parity(to_np(out), to_np(out_fma), tol)
 
 
+@pytest.mark.parametrize("M,N,K", [(300, 1080, 1152), (130, 288, 4304), (700, 520, 80)])
+def test_linear_e4m3_variant(M, N, K):
+    """The 8-bit floating-point variant of the linear layer: the row quantiser's codes and scales bit for bit
+    against the oracle (both take the rounding decisions from float32 quotients), then the layer on those codes
+    (products exact, float accumulation: 2e-5 with float output, one bf16 rounding otherwise).  The distance to
+    the unquantised layer is printed, not bounded: it is the format's error, not the kernel's."""
+    dtype = epd.DTYPE_BF16
+    x = rnd((M, K), 61, 1.0, dtype) * synth.round_to_bf16(np.exp2(np.arange(M) % 7 - 3).astype(np.float32))[:, None]
+    x[M // 2, :] = 0.0                                           # an all-zero row: scale 1, zero codes
+    w = rnd((N, K), 62, K ** -0.5, dtype)
+    b = rnd((N,), 63, 0.5, dtype)
+    xd, wd = dev(x, dtype), dev(w, dtype)
+    xq, xs = epd.op_quantize_e4m3(xd)
+    wq, ws = epd.op_quantize_e4m3(wd)
+    for arr, q, sc in ((x, xq, xs), (w, wq, ws)):
+        q_ref, s_ref = O.quantize_e4m3_rows(arr)
+        assert np.array_equal(sc.cpu().numpy(), s_ref.astype(np.float32))
+        assert np.array_equal(q.cpu().numpy()[:, :K], O.e4m3_bits(q_ref))
+        assert not q.cpu().numpy()[:, K:].any()
+    ref = O.linear_e4m3(x, w, b.astype(np.float64))
+    out32 = torch.zeros((M, N), dtype=torch.float32, device="cuda")
+    epd.op_linear_e4m3(xq, xs, wq, ws, dev(b, dtype), out32, K, epd.LINEAR_OUT_F32)
+    assert_parity(to_np(out32), ref, 2e-5)
+    out16 = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+    epd.op_linear_e4m3(xq, xs, wq, ws, dev(b, dtype), out16, K, epd.LINEAR_GELU_TANH)
+    assert_parity(to_np(out16), O.gelu(ref, O.ACT_GELU_TANH), TOL_BF16_STEP)
+    exact = O.linear(x.astype(np.float64), w.astype(np.float64), b.astype(np.float64))
+    print("e4m3 linear", (M, N, K), "distance to the unquantised layer", rel_err(ref, exact))
+
+
 @pytest.mark.parametrize("dtype", [epd.DTYPE_F32, epd.DTYPE_BF16])
 @pytest.mark.parametrize("T,h", [(1, 8), (37, 256), (100, 1152), (9, 3200), (5, 30)])
 def test_rmsnorm(dtype, T, h):

@@ -501,6 +501,9 @@ def test_round_to_e4m3_hand_computed_values():
     ]
     for v, want in cases:
         assert float(O.round_to_e4m3(np.array([v]))[0]) == want, (v, want)
+    # the sign of a zero survives (IEEE convention; the format has a negative zero, code 0x80)
+    z = O.round_to_e4m3(np.array([-0.0, -1e-9, 0.0]))
+    assert np.signbit(z).tolist() == [True, True, False] and O.e4m3_bits(z).tolist() == [0x80, 0x80, 0]
     # every one of the 2 x 127 finite codes maps to itself, and the codes come back
     codes = np.array([c for c in range(256) if (c & 0x7F) != 0x7F], dtype=np.uint8)
     sign = np.where(codes & 0x80, -1.0, 1.0)
