@@ -116,7 +116,11 @@ bool linear_tc_supported(const void* x, int64_t ldx, const void* w, int64_t ldw,
 cudaError_t linear_tc(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out, int64_t ldo,
                       int64_t M, int64_t N, int64_t K, int flags, int forced_bn, int* status, cudaStream_t s);
 
-// Same contract on CTA pairs (256 x 256 tiles, tcgen05.mma.cta_group::2); gemm_tcgen05_pair.cu.
+// Same contract on CTA pairs (256 x 256 tiles, tcgen05.mma.cta_group::2); gemm_tcgen05_pair.cu.  A large residual
+// update runs as linear_tc_pair_slices() consecutive launches over slices of K.
+int linear_tc_pair_slices(int64_t N, int64_t K, int flags);
+// Kernel launches linear_tc() makes for a shape.
+int linear_tc_launches(int64_t M, int64_t N, int64_t K, int flags, int forced_bn);
 cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
                            int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, int* status, cudaStream_t s);
 

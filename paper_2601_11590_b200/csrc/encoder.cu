@@ -185,6 +185,7 @@ int linear_dispatch(epd_encoder* enc, int dtype, const void* x, int64_t ldx, con
     if (forced_bn != 0 && forced_bn != 128 && forced_bn != 192 && forced_bn != 256) return EPD_EINVAL;
     EPD_CUDA(linear_tc(x, ldx, w, ldw, bias, out, ldo, M, N, K, enc ? (flags | kLinearStaticWeights) : flags, forced_bn,
                        status, s));
+    if (enc) enc->launches += linear_tc_launches(M, N, K, flags, forced_bn) - 1;   // the caller counted one
     return EPD_OK;
   }
   EPD_CUDA(linear_fma(dtype, x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, s));

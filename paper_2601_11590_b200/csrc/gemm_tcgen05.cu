@@ -352,6 +352,10 @@ bool linear_tc_supported(const void* x, int64_t ldx, const void* w, int64_t ldw,
   return tensor_maps_available();
 }
 
+int linear_tc_launches(int64_t M, int64_t N, int64_t K, int flags, int forced_bn) {
+  return (forced_bn == 0 && M > BM) ? linear_tc_pair_slices(N, K, flags) : 1;
+}
+
 cudaError_t linear_tc(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out, int64_t ldo,
                       int64_t M, int64_t N, int64_t K, int flags, int forced_bn, int* status, cudaStream_t s) {
   // Without a forced tile width, anything taller than one 128-row tile goes to the CTA-pair kernel.

@@ -64,14 +64,31 @@ __device__ __forceinline__ void cluster_sync() {
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// L2 eviction policies for the bulk copies: the operand a band of tiles keeps coming back to should stay in L2
+// (evict last), what streams past once (the other operand, the output) should leave first.
+__device__ __forceinline__ uint64_t policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
 // Tensor load into this CTA's shared memory whose completion bytes are counted on a barrier that may
 // live in the other CTA of the pair (given by its cluster-window address).
 __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* tm, int x, int y,
-                                                 uint32_t bar_cluster_addr) {
+                                                 uint32_t bar_cluster_addr, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(bar_cluster_addr), "r"(x), "r"(y), "l"(policy)
       : "memory");
+}
+__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* tm, int x, int y, const void* smem_src, uint64_t policy) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+               ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_result)),
@@ -132,6 +149,29 @@ struct RopeSplitArgs {
   float q_scale;
 };
 
+// Order in which the pairs walk the grid of output tiles.  The pairs resident at one time work on consecutive
+// tiles, so the order decides what they share in L2: with `by_rows`, the tile grid is cut into bands of `group` tile
+// rows, and inside a band the tiles are taken column by column (the band's rows of x stay in L2 while the whole of w
+// streams past once per band); otherwise into bands of `group` tile columns taken row by row (the band's rows of w
+// stay, x streams past once per band).  Row-major or column-major over the whole grid are the bands of full width.
+struct TileOrder {
+  int by_rows;
+  int group;
+};
+__device__ __forceinline__ void tile_coords(int tile, int m_tiles, int n_tiles, const TileOrder& o, int& mt, int& nt) {
+  if (o.by_rows) {
+    const int per = o.group * n_tiles, band = tile / per, r = tile - band * per;
+    const int first = band * o.group, rows = min(o.group, m_tiles - first);
+    nt = r / rows;
+    mt = first + (r - nt * rows);
+  } else {
+    const int per = o.group * m_tiles, band = tile / per, r = tile - band * per;
+    const int first = band * o.group, cols = min(o.group, n_tiles - first);
+    mt = r / cols;
+    nt = first + (r - mt * cols);
+  }
+}
+
 template <int BN, int STAGES>
 struct PairLayout {
   static constexpr int kABytes = BM * BK * 2;
@@ -157,8 +197,8 @@ template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE, boo
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w,
                    const __grid_constant__ CUtensorMap tm_out, const __nv_bfloat16* __restrict__ bias, int M, int N,
-                   int K, int* __restrict__ status, long long wait_limit, int static_w, const RopeSplitArgs rs,
-                   const float* __restrict__ row_scale, const float* __restrict__ col_scale) {
+                   int K, int* __restrict__ status, long long wait_limit, int static_w, const TileOrder order,
+                   const RopeSplitArgs rs, const float* __restrict__ row_scale, const float* __restrict__ col_scale) {
   static_assert(!ROPE || (sizeof(OutT) == 2 && ACT == 0 && !ACCUM), "the QKV variant writes bf16, no activation");
   static_assert(!(ROPE && FP8), "the QKV variant takes bf16 operands");
   // elements per contraction block (128 bytes of a row) and per MMA (32 bytes)
@@ -213,11 +253,15 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   int early = 0;
   if (static_w && warp == 0 && lane == 0 && pair < num_tiles) {
     prefetch_map(&tm_w);
-    const int n0 = (pair / m_tiles) * BN + (int)rank * (BN / 2);
+    int mt, nt;
+    tile_coords(pair, m_tiles, n_tiles, order, mt, nt);
+    const int n0 = nt * BN + (int)rank * (BN / 2);
+    const uint64_t pol_w = order.by_rows ? policy_evict_first() : policy_evict_last();
     early = k_blocks < STAGES ? k_blocks : STAGES;
     for (int kb = 0; kb < early; ++kb) {
       if (rank == 0) mbar_expect_tx(&full[kb], 2 * L::kStageBytes);
-      tma_load_2d_pair(smem + kb * L::kStageBytes + L::kABytes, &tm_w, kb * BKE, n0, map_to_rank(smem_u32(&full[kb]), 0));
+      tma_load_2d_pair(smem + kb * L::kStageBytes + L::kABytes, &tm_w, kb * BKE, n0, map_to_rank(smem_u32(&full[kb]), 0),
+                       pol_w);
     }
     loads_issued = early;     // for the drain after an abort: these stages have loads in flight
   }
@@ -232,9 +276,14 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       uint32_t phase = 0;
       bool ok = true;
       loads_issued = 0;
+      // the operand of the band stays in L2, the other one streams past
+      const uint64_t pol_x = order.by_rows ? policy_evict_last() : policy_evict_first();
+      const uint64_t pol_w = order.by_rows ? policy_evict_first() : policy_evict_last();
       for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
-        const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;        // this CTA's rows of x
-        const int n0 = (tile / m_tiles) * BN + (int)rank * (BN / 2);       // this CTA's half of the w tile
+        int mt, nt;
+        tile_coords(tile, m_tiles, n_tiles, order, mt, nt);
+        const int m0 = mt * (2 * BM) + (int)rank * BM;        // this CTA's rows of x
+        const int n0 = nt * BN + (int)rank * (BN / 2);       // this CTA's half of the w tile
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait<true>(&empty[stage], phase ^ 1, wc)) { ok = false; break; }
           uint8_t* sa = smem + stage * L::kStageBytes;
@@ -244,9 +293,9 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
           } else {
             // the leader's barrier counts the bytes of both CTAs
             if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
-            tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BKE, n0, bar);
+            tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BKE, n0, bar, pol_w);
           }
-          tma_load_2d_pair(sa, &tm_x, kb * BKE, m0, bar);
+          tma_load_2d_pair(sa, &tm_x, kb * BKE, m0, bar, pol_x);
           ++loads_issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -296,6 +345,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     int acc = 0;
     uint32_t acc_phase = 0;
     if (!ROPE && lane == 0) prefetch_map(&tm_out);
+    const uint64_t pol_out = policy_evict_first();   // the output is not read again by this kernel
     const float2* rope_tab = rs.table;
     if constexpr (ROPE) {
       if (rs.table_in_smem > 0) {
@@ -309,8 +359,10 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       }
     }
     for (int tile = pair; tile < num_tiles; tile += n_pairs) {
-      const int m0 = (tile % m_tiles) * (2 * BM) + (int)rank * BM;
-      const int n0 = (tile / m_tiles) * BN + half * (BN / 2);
+      int mt, nt;
+      tile_coords(tile, m_tiles, n_tiles, order, mt, nt);
+      const int m0 = mt * (2 * BM) + (int)rank * BM;
+      const int n0 = nt * BN + half * (BN / 2);
       __syncwarp();
       for (int i = lane; i < BN / 2; i += 32) {
         bs[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.0f;
@@ -460,7 +512,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         if (lane == 0) {
           if (row0 < M && n0 + c * CC < N) {
             if (ACCUM) tma_reduce_add_2d(&tm_out, n0 + c * CC, row0, sbuf);
-            else tma_store_2d(&tm_out, n0 + c * CC, row0, sbuf);
+            else tma_store_2d_hint(&tm_out, n0 + c * CC, row0, sbuf, pol_out);
           }
           bulk_commit();
         }
@@ -508,6 +560,24 @@ bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int
                             CU_TENSOR_MAP_SWIZZLE_128B);
 }
 
+// Tile order with the least modelled DRAM traffic.  The operand of a band (its rows of x, or its rows of w) is
+// read once per band and kept in L2 (evict-last loads) while the other operand streams past (evict-first); a band
+// may hold up to kL2Resident bytes.  Measured on the 6B-class fc1 shape (16384 x 12800 x 3200; operands 187 MB):
+// with the whole grid taken column by column x was read from DRAM again for every tile column, 3.2 GB per launch
+// at 1193 TFLOP/s; bands of 72 / 40 / 24 / 12 MB with the eviction hints: 1.8 / 0.48 / 1.1 / 1.9 GB, 1329 / 1453 /
+// 1431 / 1401 TFLOP/s.  (The 126 MB L2 is two halves; 40 MB is what a band can count on.)
+constexpr double kL2Resident = 40.0 * 1024 * 1024;
+TileOrder choose_order(int M, int N, int K, int elem_bytes) {
+  const int m_tiles = (M + 2 * BM - 1) / (2 * BM), n_tiles = (N + 255) / 256;
+  const double tile_bytes = 256.0 * K * elem_bytes, x_bytes = (double)M * K * elem_bytes, w_bytes = (double)N * K * elem_bytes;
+  const int cap = (int)(1.1 * kL2Resident / tile_bytes) > 1 ? (int)(1.1 * kL2Resident / tile_bytes) : 1;
+  // bands of equal height: as few as the cap allows
+  const int m_bands = (m_tiles + cap - 1) / cap, n_bands = (n_tiles + cap - 1) / cap;
+  const double by_rows = x_bytes + w_bytes * m_bands;     // x once, w once per band of tile rows
+  const double by_cols = w_bytes + x_bytes * n_bands;     // w once, x once per band of tile columns
+  return by_rows <= by_cols ? TileOrder{1, (m_tiles + m_bands - 1) / m_bands} : TileOrder{0, (n_tiles + n_bands - 1) / n_bands};
+}
+
 template <int BN, int STAGES, typename OutT, int ACT, bool ACCUM, bool ROPE = false, bool FP8 = false>
 cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorMap& to, const void* bias, int M, int N,
                    int K, int* status, cudaStream_t s, int static_w, const RopeSplitArgs& rs = RopeSplitArgs{},
@@ -551,7 +621,7 @@ cudaError_t launch(const CUtensorMap& tx, const CUtensorMap& tw, const CUtensorM
   const int avail = limited_sms(2 * max_pairs) / 2 > 0 ? limited_sms(2 * max_pairs) / 2 : 1;   // pairs within the SM budget
   const int pairs = tiles < avail ? tiles : avail;
   return launch_pdl(kern, dim3(2 * pairs), dim3(kThreads), smem_bytes, s, tx, tw, to, (const __nv_bfloat16*)bias, M, N, K,
-                    status, wait_limit_cycles(), static_w, rs, row_scale, col_scale);
+                    status, wait_limit_cycles(), static_w, choose_order(M, N, K, FP8 ? 1 : 2), rs, row_scale, col_scale);
 }
 
 template <int BN, int STAGES>
@@ -580,16 +650,39 @@ cudaError_t launch_bn(const CUtensorMap& tx, const CUtensorMap& tw, const CUtens
 
 }  // namespace
 
+// Launches linear_tc_pair() makes for a shape (see there).
+int linear_tc_pair_slices(int64_t N, int64_t K, int flags) {
+  int slices = 1;
+  if ((flags & EPD_LINEAR_ACCUMULATE) && !(flags & (EPD_LINEAR_GELU_TANH | EPD_LINEAR_GELU_ERF))) {
+    const double w_bytes = (double)N * K * 2;
+    while (slices < 4 && w_bytes / slices > 1.1 * kL2Resident) ++slices;
+  }
+  return slices;
+}
+
 // 256 x 256 tiles on CTA pairs.  Same argument contract as linear_tc().
+// A residual update (out += ...) whose weight matrix is too large for any band of it to stay in L2 (the 6B-class
+// fc2: 82 MB, 6.5 MB per tile row) is run as consecutive launches over slices of the contraction dimension, each
+// adding its part to `out`: a slice's share of w then fits (41 MB), x is read once per slice instead of once per
+// tile column.  The split depends on N and K only, so a row's result does not depend on the batch it is in.
 cudaError_t linear_tc_pair(const void* x, int64_t ldx, const void* w, int64_t ldw, const void* bias, void* out,
                            int64_t ldo, int64_t M, int64_t N, int64_t K, int flags, int* status, cudaStream_t s) {
   const bool out_f32 = flags & (EPD_LINEAR_ACCUMULATE | EPD_LINEAR_OUT_F32);
   constexpr int BN = 256;
-  CUtensorMap tx, tw, to;
-  if (!make_map(&tx, x, M, K, ldx, BM, 2) || !make_map(&tw, w, N, K, ldw, BN / 2, 2) ||
-      !make_map(&to, out, M, N, ldo, 32, out_f32 ? 4 : 2))
-    return cudaErrorInvalidValue;
-  return launch_bn<BN, 5>(tx, tw, to, bias, (int)M, (int)N, (int)K, flags, status, s);
+  const int slices = linear_tc_pair_slices(N, K, flags);
+  const int64_t k_slice = slices > 1 ? ((K + slices - 1) / slices + BK - 1) / BK * BK : K;
+  for (int64_t k0 = 0; k0 < K; k0 += k_slice) {
+    const int64_t kc = K - k0 < k_slice ? K - k0 : k_slice;
+    const char* xs = static_cast<const char*>(x) + k0 * 2;
+    const char* wsl = static_cast<const char*>(w) + k0 * 2;
+    CUtensorMap tx, tw, to;
+    if (!make_map(&tx, xs, M, kc, ldx, BM, 2) || !make_map(&tw, wsl, N, kc, ldw, BN / 2, 2) ||
+        !make_map(&to, out, M, N, ldo, 32, out_f32 ? 4 : 2))
+      return cudaErrorInvalidValue;
+    cudaError_t e = launch_bn<BN, 5>(tx, tw, to, k0 == 0 ? bias : nullptr, (int)M, (int)N, (int)kc, flags, status, s);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 // The same layer with 8-bit floating-point operands (E4M3): xq [M, K] and wq [N, K] hold byte codes, row_scale [M] and
