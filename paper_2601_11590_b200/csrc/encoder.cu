@@ -118,6 +118,7 @@ struct epd_encoder {
   bool profile = false;
   std::vector<cudaEvent_t> prof_events;
   std::vector<int> prof_class;
+  std::vector<int> prof_launches;   // kernel launches behind each event (a sliced linear layer makes several)
   size_t prof_used = 0;
   bool use_tc = false;
   bool fused_rope = false;         // QKV epilogue does rotary + split (batches of more than 128 tokens)
@@ -164,8 +165,12 @@ int mark(epd_encoder* enc, int cls, cudaStream_t s) {
     enc->prof_events.push_back(ev);
   }
   EPD_CUDA(cudaEventRecord(enc->prof_events[enc->prof_used], s));
-  if (enc->prof_class.size() <= enc->prof_used) enc->prof_class.resize(enc->prof_used + 1);
+  if (enc->prof_class.size() <= enc->prof_used) {
+    enc->prof_class.resize(enc->prof_used + 1);
+    enc->prof_launches.resize(enc->prof_used + 1);
+  }
   enc->prof_class[enc->prof_used] = cls;
+  enc->prof_launches[enc->prof_used] = 1;
   enc->prof_used++;
   return EPD_OK;
 }
@@ -185,7 +190,11 @@ int linear_dispatch(epd_encoder* enc, int dtype, const void* x, int64_t ldx, con
     if (forced_bn != 0 && forced_bn != 128 && forced_bn != 192 && forced_bn != 256) return EPD_EINVAL;
     EPD_CUDA(linear_tc(x, ldx, w, ldw, bias, out, ldo, M, N, K, enc ? (flags | kLinearStaticWeights) : flags, forced_bn,
                        status, s));
-    if (enc) enc->launches += linear_tc_launches(M, N, K, flags, forced_bn) - 1;   // the caller counted one
+    if (enc) {
+      const int extra = linear_tc_launches(M, N, K, flags, forced_bn) - 1;   // the caller counted one
+      enc->launches += extra;
+      if (enc->profile && enc->prof_used > 0) enc->prof_launches[enc->prof_used - 1] += extra;
+    }
     return EPD_OK;
   }
   EPD_CUDA(linear_fma(dtype, x, ldx, w, ldw, bias, out, ldo, M, N, K, flags, s));
@@ -970,7 +979,7 @@ int epd_debug_profile_read(epd_encoder_t* enc, float* ms, int64_t* launches) {
     float t = 0.0f;
     EPD_CUDA(cudaEventElapsedTime(&t, enc->prof_events[i], enc->prof_events[i + 1]));
     const int cls = enc->prof_class[i];
-    if (cls >= 0 && cls < KC_COUNT) { ms[cls] += t; launches[cls]++; }
+    if (cls >= 0 && cls < KC_COUNT) { ms[cls] += t; launches[cls] += enc->prof_launches[i]; }
   }
   return EPD_OK;
 }
