@@ -52,8 +52,8 @@ using namespace tc;
 
 constexpr int BQ = 128;          // query rows per tile; an item has two tiles
 constexpr int BKV = 64;          // keys per step
-constexpr int kThreads = 512;    // warps 0..7: loaders and issuing threads; warps 8..15: two softmax warpgroups
-constexpr int kRegsLow = 64, kRegsHigh = 192;   // 256 x 64 + 256 x 192 = 512 x 128
+constexpr int kThreads = 768;    // warps 0..7: loaders and issuing threads; warps 8..23: four softmax warpgroups
+constexpr int kRegsLow = 48, kRegsHigh = 96;    // 256 x 48 + 512 x 96 = 768 x 80
 constexpr int kMaxSegs = 128;    // segments one launch can describe
 constexpr float kRescaleThreshold = 8.0f;  // log2 of the largest P value tolerated before rescaling
 
@@ -85,78 +85,49 @@ __device__ __forceinline__ void umma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64
 #define EPD_R16(r, o) EPD_R8(r, o), EPD_R8(r, o + 8)
 #define EPD_W16(r, o) EPD_W8(r, o), EPD_W8(r, o + 8)
 #define EPD_R32(r, o) EPD_R16(r, o), EPD_R16(r, o + 16)
-#define EPD_W32(r, o) EPD_W16(r, o), EPD_W16(r, o + 16)
-#define EPD_R64(r, o) EPD_R32(r, o), EPD_R32(r, o + 32)
-#define EPD_W64(r, o) EPD_W32(r, o), EPD_W32(r, o + 32)
 
-// tcgen05.ld / tcgen05.st, shape 32x32b: thread i of the warp owns TMEM lane (base + i) and moves N
-// consecutive 32-bit columns.
-__device__ __forceinline__ void ld8(uint32_t taddr, uint32_t* r) {
-  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+// tcgen05.ld / tcgen05.st in the 16-lane fragment shapes.  A warp moves 16 TMEM lanes starting at the address's
+// lane (the first or second half of its lane quarter).  Shape 16x256b, per 8 columns: thread t holds rows
+// t / 4 and t / 4 + 8, columns 2 (t % 4) and 2 (t % 4) + 1; register 4 k + 2 a + b = row t / 4 + 8 a, column
+// 8 k + 2 (t % 4) + b.  Shape 16x128b, per 4 columns: register 2 k + a = row t / 4 + 8 a, column 4 k + t % 4.
+// A row is spread over the four threads of a quad; two bf16 packed from neighbouring columns of the first shape
+// land exactly on a column of the second.
+__device__ __forceinline__ void ld_frag_x2(uint32_t taddr, uint32_t* r) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                : EPD_R8(r, 0) : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void ld16(uint32_t taddr, uint32_t* r) {
+__device__ __forceinline__ void ld_frag_x4(uint32_t taddr, uint32_t* r) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : EPD_R16(r, 0) : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void ld32(uint32_t taddr, uint32_t* r) {
+__device__ __forceinline__ void ld_frag_x8(uint32_t taddr, uint32_t* r) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
       "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
       : EPD_R32(r, 0) : "r"(taddr) : "memory");
 }
-__device__ __forceinline__ void ld64(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x64.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
-      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
-      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];"
-      : EPD_R64(r, 0) : "r"(taddr) : "memory");
+// COLS columns (a multiple of 16) of 16 lanes: COLS / 2 registers.
+template <int COLS>
+__device__ __forceinline__ void ld_frag(uint32_t taddr, uint32_t* r) {
+  if constexpr (COLS >= 64) { ld_frag_x8(taddr, r); ld_frag<COLS - 64>(taddr + 64, r + 32); }
+  else if constexpr (COLS >= 32) { ld_frag_x4(taddr, r); ld_frag<COLS - 32>(taddr + 32, r + 16); }
+  else if constexpr (COLS >= 16) { ld_frag_x2(taddr, r); ld_frag<COLS - 16>(taddr + 16, r + 8); }
 }
-__device__ __forceinline__ void st8(uint32_t taddr, const uint32_t* r) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+__device__ __forceinline__ void st_frag16(uint32_t taddr, const uint32_t* r) {
+  asm volatile("tcgen05.st.sync.aligned.16x256b.x2.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
                ::"r"(taddr), EPD_W8(r, 0) : "memory");
 }
-__device__ __forceinline__ void st16(uint32_t taddr, const uint32_t* r) {
+// KEYS bf16 weights per row as KEYS / 2 packed columns, shape 16x128b: KEYS / 4 registers.
+template <int KEYS>
+__device__ __forceinline__ void st_pairs(uint32_t taddr, const uint32_t* r) {
+  static_assert(KEYS == 64, "one store of 32 columns");
   asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "tcgen05.st.sync.aligned.16x128b.x8.b32 [%0], "
       "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
       ::"r"(taddr), EPD_W16(r, 0) : "memory");
-}
-__device__ __forceinline__ void st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-      ::"r"(taddr), EPD_W32(r, 0) : "memory");
-}
-__device__ __forceinline__ void st64(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x64.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32, "
-      "%33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, %48, "
-      "%49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63, %64};"
-      ::"r"(taddr), EPD_W64(r, 0) : "memory");
-}
-// N columns (a multiple of 8) with as few instructions as possible.
-template <int N>
-__device__ __forceinline__ void ld_cols(uint32_t taddr, uint32_t* r) {
-  if constexpr (N >= 64) { ld64(taddr, r); ld_cols<N - 64>(taddr + 64, r + 64); }
-  else if constexpr (N >= 32) { ld32(taddr, r); ld_cols<N - 32>(taddr + 32, r + 32); }
-  else if constexpr (N >= 16) { ld16(taddr, r); ld_cols<N - 16>(taddr + 16, r + 16); }
-  else if constexpr (N >= 8) { ld8(taddr, r); ld_cols<N - 8>(taddr + 8, r + 8); }
-}
-template <int N>
-__device__ __forceinline__ void st_cols(uint32_t taddr, const uint32_t* r) {
-  if constexpr (N >= 64) { st64(taddr, r); st_cols<N - 64>(taddr + 64, r + 64); }
-  else if constexpr (N >= 32) { st32(taddr, r); st_cols<N - 32>(taddr + 32, r + 32); }
-  else if constexpr (N >= 16) { st16(taddr, r); st_cols<N - 16>(taddr + 16, r + 16); }
-  else if constexpr (N >= 8) { st8(taddr, r); st_cols<N - 8>(taddr + 8, r + 8); }
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -237,6 +208,7 @@ struct SegList {
   int n;
   int beg[kMaxSegs];
   int len[kMaxSegs];
+  int first[kMaxSegs];    // number of the segment's first item
 };
 
 struct Item {
@@ -246,22 +218,18 @@ struct Item {
 
 // Item i -> (segment, head, 256-row query block): segments in list order, then head, then query block, so
 // that neighbouring items (which run at the same time on different SMs) share K and V in L2.
-__device__ __forceinline__ Item decode_item(const SegList& segs, int heads, int i) {
-  Item it{0, 0, 0, 0, 0, false};
-  for (int s = 0; s < segs.n; ++s) {
-    const int qb = (segs.len[s] + 2 * BQ - 1) / (2 * BQ);
-    const int cnt = qb * heads;
-    if (i < cnt) {
-      it.head = i / qb;
-      it.seg_beg = segs.beg[s];
-      it.seg_len = segs.len[s];
-      it.q0 = it.seg_beg + (i - it.head * qb) * 2 * BQ;
-      it.n_kv = (it.seg_len + BKV - 1) / BKV;
-      it.two = it.q0 + BQ < it.seg_beg + it.seg_len;
-      return it;
-    }
-    i -= cnt;
-  }
+// A CTA's items come in ascending order: `seg` is the caller's cursor into the segment list (0 before its first item).
+__device__ __forceinline__ Item decode_item(const SegList& segs, int i, int& seg) {
+  while (seg + 1 < segs.n && i >= segs.first[seg + 1]) ++seg;
+  Item it;
+  it.seg_beg = segs.beg[seg];
+  it.seg_len = segs.len[seg];
+  const int qb = (it.seg_len + 2 * BQ - 1) / (2 * BQ);
+  i -= segs.first[seg];
+  it.head = i / qb;
+  it.q0 = it.seg_beg + (i - it.head * qb) * 2 * BQ;
+  it.n_kv = (it.seg_len + BKV - 1) / BKV;
+  it.two = it.q0 + BQ < it.seg_beg + it.seg_len;
   return it;
 }
 
@@ -285,10 +253,10 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
   uint64_t* v_full = k_empty + P::KS;         // [VS]
   uint64_t* v_empty = v_full + P::VS;         // [VS]  (2 arrivals)
   uint64_t* s_full = v_empty + P::VS;         // [2][2]  S_w[b] complete
-  uint64_t* p_full = s_full + 4;              // [2][2]  P written over S_w[b] (4 warp arrivals)
+  uint64_t* p_full = s_full + 4;              // [2][2]  P written over S_w[b] (8 warp arrivals)
   uint64_t* pv_done = p_full + 4;             // [2][2]  the P_w V product that read P from S_w[b] is complete
   uint64_t* o_done = pv_done + 4;             // [2]  the item's last P_w V is complete: O_w final
-  uint64_t* o_free = o_done + 2;              // [2]  O_w read out by its warpgroup (4 warp arrivals)
+  uint64_t* o_free = o_done + 2;              // [2]  O_w read out by its warps (8 warp arrivals)
   uint64_t* drain = o_free + 2;               // [4]  after an abort: the products of an issuing thread have completed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + P::kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -301,8 +269,8 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
     for (int i = 0; i < P::kNumBars; ++i) mbar_init(&bars[i], 1);
     for (int i = 0; i < P::KS; ++i) mbar_init(&k_empty[i], 2);
     for (int i = 0; i < P::VS; ++i) mbar_init(&v_empty[i], 2);
-    for (int i = 0; i < 4; ++i) mbar_init(&p_full[i], 4);
-    for (int w = 0; w < 2; ++w) mbar_init(&o_free[w], 4);
+    for (int i = 0; i < 4; ++i) mbar_init(&p_full[i], 8);
+    for (int w = 0; w < 2; ++w) mbar_init(&o_free[w], 8);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -323,8 +291,9 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
     if (lane == 0) {
       uint32_t kc = 0, n = 0;
       bool ok = true;
+      int seg_cur = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
-        const Item it = decode_item(segs, heads, item);
+        const Item it = decode_item(segs, item, seg_cur);
         const int row_base = it.head * T;
         const int qb = n % NQ;
         const uint32_t qphase = (n / NQ) & 1;
@@ -361,8 +330,9 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
     if (lane == 0) {
       uint32_t vc = 0;
       bool ok = true;
+      int seg_cur = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const Item it = decode_item(segs, heads, item);
+        const Item it = decode_item(segs, item, seg_cur);
         const int row_base = it.head * T;
         for (int j = 0; j < it.n_kv; ++j, ++vc) {
           const int row = row_base + it.seg_beg + j * BKV;
@@ -380,7 +350,9 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
     __syncwarp();
   } else if (warp == 1 || warp == 2) {
     // ---------------------------------------------------------------- P V products of query tile w
-    if (lane == 0) {
+    // The whole warp walks the loop (so that addresses and descriptors are warp-uniform values); one elected lane
+    // issues.
+    {
       const int w = warp - 1;
       uint32_t vc = 0;                 // V tiles seen (all of them, also in skipped items)
       uint32_t c = 0;                  // steps of this query tile so far: step c uses score buffer c & 1
@@ -389,27 +361,28 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
       constexpr uint32_t kVStep = P::kV32 ? 512 / 16 : 2048 / 16;   // 16 keys further down the V tile, 16-byte units
       const uint32_t tmem_o = tmem_base + (w ? P::kO1 : P::kO0);
       bool ok = true;
+      int seg_cur = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const Item it = decode_item(segs, heads, item);
+        const Item it = decode_item(segs, item, seg_cur);
         if (w == 1 && !it.two) {
           // nothing to compute for this query tile: hand every V slot back, each only once it has been filled
           // (so that an arrival can never be counted for a later use of the slot)
           for (int j = 0; j < it.n_kv; ++j, ++vc) {
-            if (!mbar_wait(&v_full[vc % P::VS], (vc / P::VS) & 1, wc)) { ok = false; break; }
-            mbar_arrive(&v_empty[vc % P::VS]);
+            if (!mbar_wait_warp(&v_full[vc % P::VS], (vc / P::VS) & 1, wc)) { ok = false; break; }
+            if (lane == 0) mbar_arrive(&v_empty[vc % P::VS]);
           }
           continue;
         }
         for (int t = 0; t < it.n_kv; ++t, ++vc, ++c) {
           const int vs = vc % P::VS;
-          if (!mbar_wait(&v_full[vs], (vc / P::VS) & 1, wc)) { ok = false; break; }
+          if (!mbar_wait_warp(&v_full[vs], (vc / P::VS) & 1, wc)) { ok = false; break; }
           if (t == 0) {
             // the accumulator of the query tile's previous item must have been read out
-            if (items_w > 0 && !mbar_wait(&o_free[w], (items_w - 1) & 1, wc)) { ok = false; break; }
+            if (items_w > 0 && !mbar_wait_warp(&o_free[w], (items_w - 1) & 1, wc)) { ok = false; break; }
             ++items_w;
           }
           // P of this step is in tensor memory
-          if (!mbar_wait(&p_full[2 * w + (c & 1)], (c >> 1) & 1, wc)) { ok = false; break; }
+          if (!mbar_wait_warp(&p_full[2 * w + (c & 1)], (c >> 1) & 1, wc)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sv = smem_u32(smem + P::kV + vs * P::kKTile);
           // MN-major V: boxes (16 or 64 columns wide) are kVBox apart, 8-row groups 256 / 1024 bytes apart
@@ -417,40 +390,44 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
           const uint32_t tmem_p = tmem_base + (2 * w + (c & 1)) * BKV;
           const int kv_valid = min(BKV, it.seg_len - t * BKV);
           const int steps = (kv_valid + 15) >> 4;
-          if (steps == BKV / 16) {
+          if (elect_one()) {
+            if (steps == BKV / 16) {
 #pragma unroll
-            for (int s = 0; s < BKV / 16; ++s)       // 16 bf16 of P = 8 columns
-              umma_ts(tmem_o, tmem_p + s * 8, dv + s * kVStep, idesc_pv, (t | s) != 0 ? 1u : 0u);
-          } else {
-            for (int s = 0; s < steps; ++s)
-              umma_ts(tmem_o, tmem_p + s * 8, dv + s * kVStep, idesc_pv, (t | s) != 0 ? 1u : 0u);
+              for (int s = 0; s < BKV / 16; ++s)       // 16 bf16 of P = 8 columns
+                umma_ts(tmem_o, tmem_p + s * 8, dv + s * kVStep, idesc_pv, (t | s) != 0 ? 1u : 0u);
+            } else {
+              for (int s = 0; s < steps; ++s)
+                umma_ts(tmem_o, tmem_p + s * 8, dv + s * kVStep, idesc_pv, (t | s) != 0 ? 1u : 0u);
+            }
+            umma_commit(&pv_done[2 * w + (c & 1)]);    // frees the score buffer, orders rescales
+            umma_commit(&v_empty[vs]);
+            if (t == it.n_kv - 1) umma_commit(&o_done[w]);
           }
-          umma_commit(&pv_done[2 * w + (c & 1)]);    // frees the score buffer, orders rescales
-          umma_commit(&v_empty[vs]);
-          if (t == it.n_kv - 1) umma_commit(&o_done[w]);
+          __syncwarp();
         }
       }
     }
     __syncwarp();
   } else if (warp == 4 || warp == 5) {
     // ---------------------------------------------------------------- score products of query tile w
-    if (lane == 0) {
+    {
       const int w = warp - 4;
       uint32_t kc = 0, n = 0;          // K tiles / items seen (all of them, also in skipped items)
       uint32_t g = 0;                  // score tiles of this query tile so far: tile g goes to buffer g & 1
       bool ok = true;
+      int seg_cur = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
-        const Item it = decode_item(segs, heads, item);
+        const Item it = decode_item(segs, item, seg_cur);
         const int qb = n % NQ;
         const uint32_t qphase = (n / NQ) & 1;
-        if (!mbar_wait(&q_full[w * NQ + qb], qphase, wc)) break;
+        if (!mbar_wait_warp(&q_full[w * NQ + qb], qphase, wc)) break;
         if (w == 1 && !it.two) {
           // nothing to compute for this query tile: hand the Q buffer and every K slot back, each only once it
           // has been filled
-          mbar_arrive(&q_empty[w * NQ + qb]);
+          if (lane == 0) mbar_arrive(&q_empty[w * NQ + qb]);
           for (int j = 0; j < it.n_kv; ++j, ++kc) {
-            if (!mbar_wait(&k_full[kc % P::KS], (kc / P::KS) & 1, wc)) { ok = false; break; }
-            mbar_arrive(&k_empty[kc % P::KS]);
+            if (!mbar_wait_warp(&k_full[kc % P::KS], (kc / P::KS) & 1, wc)) { ok = false; break; }
+            if (lane == 0) mbar_arrive(&k_empty[kc % P::KS]);
           }
           continue;
         }
@@ -459,11 +436,11 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
         const uint64_t dq_tail = smem_desc(sq + P::kMainBoxes * P::kQMain, 16, 256, 6);
         for (int t = 0; t < it.n_kv; ++t, ++kc, ++g) {
           const int ks = kc % P::KS;
-          if (!mbar_wait(&k_full[ks], (kc / P::KS) & 1, wc)) { ok = false; break; }
+          if (!mbar_wait_warp(&k_full[ks], (kc / P::KS) & 1, wc)) { ok = false; break; }
           // the buffer's previous content (P of the step two before) must have been consumed by its P V product.
           // One barrier per buffer: the buffer's next product cannot complete before these scores exist, so the
           // barrier is at most one phase past the one waited for and the parity is unambiguous.
-          if (g >= 2 && !mbar_wait(&pv_done[2 * w + (g & 1)], ((g >> 1) - 1) & 1, wc)) { ok = false; break; }
+          if (g >= 2 && !mbar_wait_warp(&pv_done[2 * w + (g & 1)], ((g >> 1) - 1) & 1, wc)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sk = smem_u32(smem + P::kK + ks * P::kKTile);
           const uint64_t dk_main = smem_desc(sk, 16, 1024, 2);
@@ -472,17 +449,20 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
           const int kv_valid = min(BKV, it.seg_len - t * BKV);
           const uint32_t idesc = kv_valid == BKV ? instr_desc(BKV, 0) : instr_desc((kv_valid + 15) & ~15, 0);
           // descriptor addresses count 16-byte units: one 16-element step inside a swizzled row is +2
+          if (elect_one()) {
 #pragma unroll
-          for (int b = 0; b < P::kMainBoxes; ++b) {
+            for (int b = 0; b < P::kMainBoxes; ++b) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_ss(tmem_s, dq_main + (b * P::kQMain / 16 + 2 * k), dk_main + (b * P::kKMain / 16 + 2 * k), idesc,
-                      (b | k) != 0);
+              for (int k = 0; k < 4; ++k)
+                umma_ss(tmem_s, dq_main + (b * P::kQMain / 16 + 2 * k), dk_main + (b * P::kKMain / 16 + 2 * k), idesc,
+                        (b | k) != 0);
+            }
+            if (P::kTail) umma_ss(tmem_s, dq_tail, dk_tail, idesc, 1);
+            umma_commit(&s_full[2 * w + (g & 1)]);
+            umma_commit(&k_empty[ks]);
+            if (t == it.n_kv - 1) umma_commit(&q_empty[w * NQ + qb]);   // the query tile's last score product
           }
-          if (P::kTail) umma_ss(tmem_s, dq_tail, dk_tail, idesc, 1);
-          umma_commit(&s_full[2 * w + (g & 1)]);
-          umma_commit(&k_empty[ks]);
-          if (t == it.n_kv - 1) umma_commit(&q_empty[w * NQ + qb]);   // the query tile's last score product
+          __syncwarp();
         }
       }
     }
@@ -490,99 +470,127 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
   } else if (warp >= 8) {
     // ---------------------------------------------------------------- softmax / rescale / epilogue
     regs_inc<kRegsHigh>();
-    const int w = (warp - 8) >> 2;                      // query tile of this warpgroup
+    const int grp = (warp - 8) >> 2;
+    const int w = grp >> 1;                             // query tile of this warp
+    const int hf = grp & 1;                             // which 16 rows of the warp's TMEM lane quarter
     const int qr = warp & 3;                            // TMEM lane quarter this warp may access
-    const int r = qr * 32 + lane;                       // query row inside the tile
-    const uint32_t lane_off = (uint32_t)(qr * 32) << 16;
+    const int quad = lane & 3;                          // the four threads of a quad share two rows
+    const int r0 = qr * 32 + hf * 16 + (lane >> 2);     // this thread's query rows inside the tile: r0 and r0 + 8
+    const uint32_t lane_off = (uint32_t)(qr * 32 + hf * 16) << 16;
     const uint32_t tmem_s0 = tmem_base + 2 * w * BKV + lane_off;   // S_w[0]; S_w[1] is BKV columns further
     const uint32_t tmem_o = tmem_base + (w ? P::kO1 : P::kO0) + lane_off;
-    uint32_t c = 0, oc = 0;                             // steps / items processed by this warpgroup
+    uint32_t c = 0, oc = 0;                             // steps / items processed by this warp
     bool ok = true;
+    int seg_cur = 0;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-      const Item it = decode_item(segs, heads, item);
+      const Item it = decode_item(segs, item, seg_cur);
       if (w == 1 && !it.two) continue;                  // no row of the segment in this query tile
-      float m = -INFINITY, l = 0.0f;
-      uint32_t s[BKV > DHP ? BKV : DHP];
+      float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.0f, 0.0f};
       for (int t = 0; t < it.n_kv; ++t, ++c) {
         const int kv_valid = min(BKV, it.seg_len - t * BKV);
         const uint32_t tmem_s = tmem_s0 + (c & 1) * BKV;   // P lives in the buffer's first BKV / 2 columns
         if (!mbar_wait_warp(&s_full[2 * w + (c & 1)], (c >> 1) & 1, wc)) { ok = false; break; }
         tc_fence_after();
-        if (kv_valid == BKV) {
-          ld_cols<BKV>(tmem_s, s);
-        } else {
-#pragma unroll
-          for (int q = 0; q < BKV / 16; ++q)
-            if (q * 16 < kv_valid) ld16(tmem_s + q * 16, s + q * 16);
-        }
+        // register 4 k + 2 a + b holds row r0 + 8 a, column 8 k + 2 quad + b
+        uint32_t s[BKV / 2];
+        ld_frag<BKV>(tmem_s, s);
         tmem_ld_wait();
 
-        float mx[4];
+        // P = exp2(S - m) as bf16 pairs, to be written over the first half of the score buffer: b32 column
+        // 4 k + quad of row r0 + 8 a is register 2 k + a.  Keys beyond the segment get weight zero (the products
+        // read P in whole groups of 16 keys).
+        uint32_t pk[BKV / 4];
+        float sum0 = 0.0f, sum1 = 0.0f;
+        auto weights = [&](float neg_m0, float neg_m1) {
+          sum0 = sum1 = 0.0f;
+          if (kv_valid == BKV) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) mx[i] = -INFINITY;
+            for (int k = 0; k < BKV / 8; ++k) {
+              const float p0 = ex2(__uint_as_float(s[4 * k]) + neg_m0);
+              const float p1 = ex2(__uint_as_float(s[4 * k + 1]) + neg_m0);
+              const float p2 = ex2(__uint_as_float(s[4 * k + 2]) + neg_m1);
+              const float p3 = ex2(__uint_as_float(s[4 * k + 3]) + neg_m1);
+              if (!ONES) { sum0 += p0 + p1; sum1 += p2 + p3; }
+              __nv_bfloat162 b0 = __floats2bfloat162_rn(p0, p1), b1 = __floats2bfloat162_rn(p2, p3);
+              pk[2 * k] = *reinterpret_cast<uint32_t*>(&b0);
+              pk[2 * k + 1] = *reinterpret_cast<uint32_t*>(&b1);
+            }
+          } else {
+#pragma unroll
+            for (int k = 0; k < BKV / 8; ++k) {
+              const int col = 8 * k + 2 * quad;
+              const float p0 = col < kv_valid ? ex2(__uint_as_float(s[4 * k]) + neg_m0) : 0.0f;
+              const float p1 = col + 1 < kv_valid ? ex2(__uint_as_float(s[4 * k + 1]) + neg_m0) : 0.0f;
+              const float p2 = col < kv_valid ? ex2(__uint_as_float(s[4 * k + 2]) + neg_m1) : 0.0f;
+              const float p3 = col + 1 < kv_valid ? ex2(__uint_as_float(s[4 * k + 3]) + neg_m1) : 0.0f;
+              if (!ONES) { sum0 += p0 + p1; sum1 += p2 + p3; }
+              __nv_bfloat162 b0 = __floats2bfloat162_rn(p0, p1), b1 = __floats2bfloat162_rn(p2, p3);
+              pk[2 * k] = *reinterpret_cast<uint32_t*>(&b0);
+              pk[2 * k + 1] = *reinterpret_cast<uint32_t*>(&b1);
+            }
+          }
+        };
+        // maximum over this thread's quarter of its two rows
+        float mx[2] = {-INFINITY, -INFINITY};
         if (kv_valid == BKV) {
+#pragma unroll
+          for (int k = 0; k < BKV / 8; ++k) {
+            mx[0] = max3(mx[0], __uint_as_float(s[4 * k]), __uint_as_float(s[4 * k + 1]));
+            mx[1] = max3(mx[1], __uint_as_float(s[4 * k + 2]), __uint_as_float(s[4 * k + 3]));
+          }
+        } else {
 #pragma unroll
           for (int i = 0; i < BKV / 2; ++i)
-            mx[i & 3] = max3(mx[i & 3], __uint_as_float(s[2 * i]), __uint_as_float(s[2 * i + 1]));
-        } else {
-#pragma unroll
-          for (int i = 0; i < BKV; ++i)
-            if (i < kv_valid) mx[i & 3] = fmaxf(mx[i & 3], __uint_as_float(s[i]));
+            if (8 * (i >> 2) + 2 * quad + (i & 1) < kv_valid) mx[(i >> 1) & 1] = fmaxf(mx[(i >> 1) & 1], __uint_as_float(s[i]));
         }
-        const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-        // advance the running max only when it would grow by more than the threshold
-        float scale = 1.0f;
-        bool grow = false;
-        if (t == 0) {
-          m = m_tile;
-        } else if (m_tile - m > kRescaleThreshold) {
-          scale = ex2(m - m_tile);
-          m = m_tile;
-          l *= scale;
-          grow = true;
+        // A row's running max only advances when it would grow by more than the threshold, so after an item's
+        // first step the weights are almost always taken against the running max as it stands: they are computed
+        // at once, alongside the maxima, and kept unless some thread of the warp finds its quarter of a row above
+        // the threshold (if none does, no row is, and the threads of a quad still share their rows' running max
+        // without having exchanged anything).  Otherwise, and in the first step, the quads exchange their
+        // maxima, take the same decision per row, rescale what has been accumulated and compute the weights
+        // against the new max.
+        bool exact = t == 0;
+        if (t != 0) {
+          weights(-m[0], -m[1]);
+          exact = __any_sync(0xffffffffu, mx[0] - m[0] > kRescaleThreshold || mx[1] - m[1] > kRescaleThreshold);
         }
-        if (__any_sync(0xffffffffu, grow)) {
-          // O_w must be quiescent: the product of step t-2 is complete (these scores were issued behind it); the
-          // product of step t-1 is the only one that may still be adding to it
-          if (!mbar_wait_warp(&pv_done[2 * w + ((c - 1) & 1)], ((c - 1) >> 1) & 1, wc)) { ok = false; break; }
-          tc_fence_after();
+        if (exact) {
+          float scale[2] = {1.0f, 1.0f};
 #pragma unroll
-          for (int q = 0; q < DHP / 16; ++q) {
-            uint32_t o[16];
-            ld16(tmem_o + q * 16, o);
+          for (int a = 0; a < 2; ++a) {
+            mx[a] = fmaxf(mx[a], __shfl_xor_sync(0xffffffffu, mx[a], 1));
+            mx[a] = fmaxf(mx[a], __shfl_xor_sync(0xffffffffu, mx[a], 2));
+            if (t == 0) {
+              m[a] = mx[a];
+            } else if (mx[a] - m[a] > kRescaleThreshold) {
+              scale[a] = ex2(m[a] - mx[a]);
+              m[a] = mx[a];
+              l[a] *= scale[a];
+            }
+          }
+          if (t != 0) {
+            // O_w must be quiescent: the product of step t-2 is complete (these scores were issued behind it); the
+            // product of step t-1 is the only one that may still be adding to it
+            if (!mbar_wait_warp(&pv_done[2 * w + ((c - 1) & 1)], ((c - 1) >> 1) & 1, wc)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int q = 0; q < DHP / 16; ++q) {
+              uint32_t o[8];
+              ld_frag<16>(tmem_o + q * 16, o);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 8; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * scale[(i >> 1) & 1]);
+              st_frag16(tmem_o + q * 16, o);
+            }
+            // the scores are still in their buffer
+            ld_frag<BKV>(tmem_s, s);
             tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * scale);
-            st16(tmem_o + q * 16, o);
           }
+          weights(-m[0], -m[1]);
         }
-        // P = exp2(S - m) as bf16 pairs, in place
-        const float neg_m = -m;
-        float sum[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        if (kv_valid == BKV) {
-#pragma unroll
-          for (int i = 0; i < BKV / 2; ++i) {
-            const float p0 = ex2(__uint_as_float(s[2 * i]) + neg_m);
-            const float p1 = ex2(__uint_as_float(s[2 * i + 1]) + neg_m);
-            if (!ONES) sum[i & 3] += p0 + p1;
-            __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-            s[i] = *reinterpret_cast<uint32_t*>(&b2);
-          }
-          st_cols<BKV / 2>(tmem_s, s);
-        } else {
-#pragma unroll
-          for (int i = 0; i < BKV / 2; ++i) {
-            const float p0 = 2 * i < kv_valid ? ex2(__uint_as_float(s[2 * i]) + neg_m) : 0.0f;
-            const float p1 = 2 * i + 1 < kv_valid ? ex2(__uint_as_float(s[2 * i + 1]) + neg_m) : 0.0f;
-            if (!ONES) sum[i & 3] += p0 + p1;
-            __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-            s[i] = *reinterpret_cast<uint32_t*>(&b2);
-          }
-#pragma unroll
-          for (int q = 0; q < BKV / 16; ++q)
-            if (q * 16 < kv_valid) st8(tmem_s + q * 8, s + q * 8);
-        }
-        if (!ONES) l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
+        st_pairs<BKV>(tmem_s, pk);
+        if (!ONES) { l[0] += sum0; l[1] += sum1; }
         tmem_st_wait();
         tc_fence_before();
         __syncwarp();
@@ -593,29 +601,39 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
       if (!mbar_wait_warp(&o_done[w], oc & 1, wc)) { ok = false; break; }
       ++oc;
       tc_fence_after();
-      const int token = it.q0 + w * BQ + r;
-      const bool row_ok = token < it.seg_beg + it.seg_len;
-      __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + it.head * dh;
-      // the whole accumulator row goes into the (dead) score registers, then the accumulator is handed back
-      ld_cols<DHP>(tmem_o, s);
+      // the accumulator rows go into registers (same fragment layout as the scores), then the accumulator is
+      // handed back
+      uint32_t o[DHP / 2];
+      ld_frag<DHP>(tmem_o, o);
       tmem_ld_wait();
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&o_free[w]);
-      if (ONES) l = __uint_as_float(s[DHP - 8]);       // head_dim = DHP - 8: the row sum sits in column head_dim
-      const float inv = 1.0f / l;
-      if (row_ok) {
+      if (ONES) {
+        // head_dim = DHP - 8: the row sums sit in column head_dim, held by the first thread of the quad
+        constexpr int kb = DHP / 8 - 1;
+        l[0] = __shfl_sync(0xffffffffu, __uint_as_float(o[4 * kb]), lane & ~3);
+        l[1] = __shfl_sync(0xffffffffu, __uint_as_float(o[4 * kb + 2]), lane & ~3);
+      } else {
 #pragma unroll
-        for (int g = 0; g < DHP / 8; ++g) {
-          if (g * 8 < dh) {                              // head_dim is a multiple of 8
-            uint32_t pk[4];
+        for (int a = 0; a < 2; ++a) {
+          l[a] += __shfl_xor_sync(0xffffffffu, l[a], 1);
+          l[a] += __shfl_xor_sync(0xffffffffu, l[a], 2);
+        }
+      }
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(s[8 * g + 2 * e]) * inv,
-                                                        __uint_as_float(s[8 * g + 2 * e + 1]) * inv);
-              pk[e] = *reinterpret_cast<uint32_t*>(&b2);
+      for (int a = 0; a < 2; ++a) {
+        const int token = it.q0 + w * BQ + r0 + 8 * a;
+        if (token < it.seg_beg + it.seg_len) {
+          const float inv = 1.0f / l[a];
+          __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + it.head * dh + 2 * quad;
+#pragma unroll
+          for (int k = 0; k < DHP / 8; ++k) {
+            if (k * 8 < dh) {                            // head_dim is a multiple of 8
+              __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[4 * k + 2 * a]) * inv,
+                                                        __uint_as_float(o[4 * k + 2 * a + 1]) * inv);
+              *reinterpret_cast<__nv_bfloat162*>(orow + k * 8) = b2;
             }
-            *reinterpret_cast<uint4*>(orow + g * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
       }
@@ -638,11 +656,15 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
         drain_ring(k_full, P::KS, kv_loads);
       }
       if (warp == 3) drain_ring(v_full, P::VS, kv_loads);
-      if (warp == 1 || warp == 2 || warp == 4 || warp == 5) {
+    }
+    if (warp == 1 || warp == 2 || warp == 4 || warp == 5) {
+      // the lane that issued the warp's products commits (a commit covers the products of its own thread)
+      if (elect_one()) {
         const int d = warp < 3 ? warp - 1 : warp - 2;
         umma_commit(&drain[d]);
         mbar_wait_drain(&drain[d], 0);
       }
+      __syncwarp();
     }
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
@@ -721,9 +743,10 @@ cudaError_t attention_pair(const void* q, const void* k, const void* v, const in
       const int sg = order[first + i];
       segs.beg[i] = host_cu_seqlens[sg];
       segs.len[i] = host_cu_seqlens[sg + 1] - host_cu_seqlens[sg];
+      segs.first[i] = n_items;
       n_items += (segs.len[i] + 2 * BQ - 1) / (2 * BQ) * heads;
     }
-    for (int i = segs.n; i < kMaxSegs; ++i) segs.beg[i] = segs.len[i] = 0;
+    for (int i = segs.n; i < kMaxSegs; ++i) segs.beg[i] = segs.len[i] = segs.first[i] = 0;
     cudaError_t e;
     switch (dhp) {
 #define EPD_ATT(D)                                                                                          \

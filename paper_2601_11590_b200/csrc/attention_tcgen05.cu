@@ -251,6 +251,7 @@ struct SegList {
   int n;
   int beg[kMaxSegs];
   int len[kMaxSegs];
+  int first[kMaxSegs];    // number of the segment's first item
 };
 
 struct Item {
@@ -259,22 +260,18 @@ struct Item {
 
 // Item i -> (segment, head, query tile): segments in list order, then head, then query tile, so
 // that neighbouring items (which run at the same time on different SMs) share K and V in L2.
+// A CTA's items come in ascending order: `seg` is the caller's cursor into the segment list (0 before its first item).
 template <int BKV>
-__device__ __forceinline__ Item decode_item(const SegList& segs, int heads, int i) {
-  Item it{0, 0, 0, 0, 0};
-  for (int s = 0; s < segs.n; ++s) {
-    const int qt = (segs.len[s] + BQ - 1) / BQ;
-    const int cnt = qt * heads;
-    if (i < cnt) {
-      it.head = i / qt;
-      it.seg_beg = segs.beg[s];
-      it.seg_len = segs.len[s];
-      it.q0 = it.seg_beg + (i - it.head * qt) * BQ;
-      it.n_kv = (it.seg_len + BKV - 1) / BKV;
-      return it;
-    }
-    i -= cnt;
-  }
+__device__ __forceinline__ Item decode_item(const SegList& segs, int i, int& seg) {
+  while (seg + 1 < segs.n && i >= segs.first[seg + 1]) ++seg;
+  Item it;
+  it.seg_beg = segs.beg[seg];
+  it.seg_len = segs.len[seg];
+  const int qt = (it.seg_len + BQ - 1) / BQ;
+  i -= segs.first[seg];
+  it.head = i / qt;
+  it.q0 = it.seg_beg + (i - it.head * qt) * BQ;
+  it.n_kv = (it.seg_len + BKV - 1) / BKV;
   return it;
 }
 
@@ -392,8 +389,9 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     if (lane == 0) {
       uint32_t kc = 0, n = 0;
       bool ok = true;
+      int seg_cur = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
-        const Item it = decode_item<BKV>(segs, heads, item);
+        const Item it = decode_item<BKV>(segs, item, seg_cur);
         const int row_base = it.head * T;
         const int qb = n & 1;
         if (!mbar_wait(&q_empty[qb], ((n >> 1) & 1) ^ 1, wc)) break;
@@ -426,8 +424,9 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     if (lane == 0) {
       uint32_t vc = 0;
       bool ok = true;
+      int seg_cur = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-        const Item it = decode_item<BKV>(segs, heads, item);
+        const Item it = decode_item<BKV>(segs, item, seg_cur);
         const int row_base = it.head * T;
         for (int j = 0; j < it.n_kv; ++j, ++vc) {
           const int row = row_base + it.seg_beg + j * BKV;
@@ -445,14 +444,16 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     __syncwarp();
   } else if (warp == 1) {
     // ---------------------------------------------------------------- Q K^T issuer:  S_w(j) = Q K_j^T
-    if (lane == 0) {
+    // The whole warp walks the loop and one elected lane issues (see elect_one()).
+    {
       uint32_t kc = 0, n = 0, sc0 = 0, sc1 = 0;        // sc_w: score tiles issued for warpgroup w
       int fw = 0;                                      // warpgroup that takes the item's first key tile
       bool ok = true;
+      int seg_cur = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
-        const Item it = decode_item<BKV>(segs, heads, item);
+        const Item it = decode_item<BKV>(segs, item, seg_cur);
         const int qb = n & 1;
-        if (!mbar_wait(&q_full[qb], (n >> 1) & 1, wc)) break;
+        if (!mbar_wait_warp(&q_full[qb], (n >> 1) & 1, wc)) break;
         const uint32_t sq = smem_u32(smem + P::kQ + qb * P::kQBytes);
         const uint64_t dq_main = smem_desc(sq, 16, 1024, 2);
         const uint64_t dq_tail = smem_desc(sq + P::kMainBoxes * P::kQMain, 16, 256, 6);
@@ -461,10 +462,10 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           const uint32_t kt = kc + j;                   // the tile's number in the K ring
           const int w = (j & 1) ^ fw;
           const int ks = kt % P::KS;
-          if (!mbar_wait(&k_full[ks], (kt / P::KS) & 1, wc)) { ok = false; break; }
+          if (!mbar_wait_warp(&k_full[ks], (kt / P::KS) & 1, wc)) { ok = false; break; }
           uint32_t& sc = w ? sc1 : sc0;
           // the warpgroup must have copied its previous score tile out of S_w
-          if (sc > 0 && !mbar_wait(&s_free[w], (sc - 1) & 1, wc)) { ok = false; break; }
+          if (sc > 0 && !mbar_wait_warp(&s_free[w], (sc - 1) & 1, wc)) { ok = false; break; }
           ++sc;
           tc_fence_after();
           const uint32_t sk = smem_u32(smem + P::kK + ks * P::kKStride);
@@ -474,17 +475,20 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           const int kv_valid = min(BKV, it.seg_len - j * BKV);
           const uint32_t idesc = kv_valid == BKV ? instr_desc(BKV, 0) : instr_desc((kv_valid + 15) & ~15, 0);
           // descriptor addresses count 16-byte units: one 16-element step inside a swizzled row is +2
+          if (elect_one()) {
 #pragma unroll
-          for (int b = 0; b < P::kMainBoxes; ++b) {
+            for (int b = 0; b < P::kMainBoxes; ++b) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_ss(tmem_s, dq_main + (b * P::kQMain / 16 + 2 * k), dk_main + (b * P::kKMain / 16 + 2 * k), idesc,
-                      (b | k) != 0);
+              for (int k = 0; k < 4; ++k)
+                umma_ss(tmem_s, dq_main + (b * P::kQMain / 16 + 2 * k), dk_main + (b * P::kKMain / 16 + 2 * k), idesc,
+                        (b | k) != 0);
+            }
+            if (P::kTail) umma_ss(tmem_s, dq_tail, dk_tail, idesc, 1);
+            umma_commit(&s_full[w]);
+            umma_commit(&k_empty[ks]);
+            if (i == it.n_kv - 1) umma_commit(&q_empty[qb]);
           }
-          if (P::kTail) umma_ss(tmem_s, dq_tail, dk_tail, idesc, 1);
-          umma_commit(&s_full[w]);
-          umma_commit(&k_empty[ks]);
-          if (i == it.n_kv - 1) umma_commit(&q_empty[qb]);
+          __syncwarp();
         }
         kc += it.n_kv;
         fw = next_first_warpgroup(fw, it.n_kv);
@@ -493,15 +497,17 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     __syncwarp();
   } else if (warp == 2) {
     // ---------------------------------------------------------------- P V issuer:  O_w += P_w(j) V_j
-    if (lane == 0) {
+    // The whole warp walks the loop and one elected lane issues.
+    {
       uint32_t vc = 0, n = 0, pc0 = 0, pc1 = 0;        // pc_w: P tiles consumed for warpgroup w
       uint32_t items0 = 0, items1 = 0;                 // items in which warpgroup 0 / 1 had key tiles
       int fw = 0;
       constexpr uint32_t idesc = instr_desc(DHP, 1);
       constexpr uint32_t kStep = P::kV32 ? 512 / 16 : 2048 / 16;   // 16 keys further down the V tile, 16-byte units
       bool ok = true;
+      int seg_cur = 0;
       for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
-        const Item it = decode_item<BKV>(segs, heads, item);
+        const Item it = decode_item<BKV>(segs, item, seg_cur);
         for (int i = 0; i < it.n_kv; ++i) {
           const int j = issue_order(i, it.n_kv, P::KS >= 4 && P::VS >= 4);
           const uint32_t vt = vc + j;                   // the tile's number in the V ring
@@ -509,13 +515,13 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           const int vs = vt % P::VS;
           uint32_t& pc = w ? pc1 : pc0;
           // V arrives long before P: take that wait first so that only P's is on the critical path
-          if (!mbar_wait(&v_full[vs], (vt / P::VS) & 1, wc)) { ok = false; break; }
-          if (!mbar_wait(&p_full[w], pc & 1, wc)) { ok = false; break; }
+          if (!mbar_wait_warp(&v_full[vs], (vt / P::VS) & 1, wc)) { ok = false; break; }
+          if (!mbar_wait_warp(&p_full[w], pc & 1, wc)) { ok = false; break; }
           ++pc;
           if (j < 2) {
             // the warpgroup's accumulator of its previous item must have been read out before it is overwritten
             uint32_t& items = w ? items1 : items0;
-            if (items > 0 && !mbar_wait(&o_free[w], (items - 1) & 1, wc)) { ok = false; break; }
+            if (items > 0 && !mbar_wait_warp(&o_free[w], (items - 1) & 1, wc)) { ok = false; break; }
             ++items;
           }
           tc_fence_after();
@@ -525,18 +531,21 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
           const uint32_t tmem_p = tmem_base + (w ? P::kP1 : P::kP0), tmem_o = tmem_base + (w ? P::kO1 : P::kO0);
           const uint32_t first = j >= 2 ? 1u : 0u;     // a warpgroup's first tile starts O_w afresh
           const int kv_valid = min(BKV, it.seg_len - j * BKV);
-          if (kv_valid == BKV) {
+          if (elect_one()) {
+            if (kv_valid == BKV) {
 #pragma unroll
-            for (int ks = 0; ks < BKV / 16; ++ks)       // 16 bf16 of P = 8 columns
-              umma_ts(tmem_o, tmem_p + ks * 8, dv + ks * kStep, idesc, ks == 0 ? first : 1u);
-          } else {
-            const int steps = (kv_valid + 15) >> 4;
-            for (int ks = 0; ks < steps; ++ks)
-              umma_ts(tmem_o, tmem_p + ks * 8, dv + ks * kStep, idesc, ks == 0 ? first : 1u);
+              for (int ks = 0; ks < BKV / 16; ++ks)       // 16 bf16 of P = 8 columns
+                umma_ts(tmem_o, tmem_p + ks * 8, dv + ks * kStep, idesc, ks == 0 ? first : 1u);
+            } else {
+              const int steps = (kv_valid + 15) >> 4;
+              for (int ks = 0; ks < steps; ++ks)
+                umma_ts(tmem_o, tmem_p + ks * 8, dv + ks * kStep, idesc, ks == 0 ? first : 1u);
+            }
+            umma_commit(&v_empty[vs]);
+            umma_commit(&p_free[w]);
+            if (j >= it.n_kv - 2) umma_commit(&o_done[w]);   // the warpgroup's last key tile of the item
           }
-          umma_commit(&v_empty[vs]);
-          umma_commit(&p_free[w]);
-          if (j >= it.n_kv - 2) umma_commit(&o_done[w]);   // the warpgroup's last key tile of the item
+          __syncwarp();
         }
         if (!ok) break;
         vc += it.n_kv;
@@ -558,8 +567,9 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     uint32_t pubs_me = 0, pubs_other = 0;               // (m, l) publications of this / the other warpgroup
     int fw = 0;                                         // warpgroup that takes the item's first key tile
     bool ok = true;
+    int seg_cur = 0;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
-      const Item it = decode_item<BKV>(segs, heads, item);
+      const Item it = decode_item<BKV>(segs, item, seg_cur);
       float m = -INFINITY, l = 0.0f;
       uint32_t s[BKV];
       // The loop is software-pipelined: the tcgen05.ld of the next score tile is issued right after
@@ -814,10 +824,10 @@ attention_tc_kernel(const __grid_constant__ Maps maps, const __grid_constant__ S
     if (lane == 0) {
       if (warp == 0) { drain_ring(q_full, 2, q_loads); drain_ring(k_full, P::KS, kv_loads); }
       if (warp == 3) drain_ring(v_full, P::VS, kv_loads);
-      if (warp == 1 || warp == 2) {
-        umma_commit(&drain[warp - 1]);
-        mbar_wait_drain(&drain[warp - 1], 0);
-      }
+    }
+    if ((warp == 1 || warp == 2) && elect_one()) {   // the lane that issued the products: a commit covers its own thread's
+      umma_commit(&drain[warp - 1]);
+      mbar_wait_drain(&drain[warp - 1], 0);
     }
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
@@ -893,9 +903,10 @@ cudaError_t attention_tc(const void* q, const void* k, const void* v, const int3
       const int sg = order[first + i];
       segs.beg[i] = host_cu_seqlens[sg];
       segs.len[i] = host_cu_seqlens[sg + 1] - host_cu_seqlens[sg];
+      segs.first[i] = n_items;
       n_items += (segs.len[i] + BQ - 1) / BQ * heads;
     }
-    for (int i = segs.n; i < kMaxSegs; ++i) segs.beg[i] = segs.len[i] = 0;
+    for (int i = segs.n; i < kMaxSegs; ++i) segs.beg[i] = segs.len[i] = segs.first[i] = 0;
     cudaError_t e;
     switch (dhp) {
 #define EPD_ATT(D)                                                                                          \

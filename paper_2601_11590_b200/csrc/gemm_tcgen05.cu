@@ -111,20 +111,26 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      prefetch_map(&tm_x);
-      prefetch_map(&tm_w);
+    // The whole warp walks the loop and one elected lane issues (see elect_one()).
+    {
+      if (lane == 0) {
+        prefetch_map(&tm_x);
+        prefetch_map(&tm_w);
+      }
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         const int m0 = (tile % m_tiles) * BM, n0 = (tile / m_tiles) * BN;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(&empty[stage], phase ^ 1, wc)) { ok = false; break; }
+          if (!mbar_wait_warp(&empty[stage], phase ^ 1, wc)) { ok = false; break; }
           uint8_t* sa = smem + stage * L::kStageBytes;
-          mbar_expect_tx(&full[stage], L::kStageBytes);
-          tma_load_2d(sa, &tm_x, kb * BK, m0, &full[stage]);
-          tma_load_2d(sa + L::kABytes, &tm_w, kb * BK, n0, &full[stage]);
+          if (elect_one()) {
+            mbar_expect_tx(&full[stage], L::kStageBytes);
+            tma_load_2d(sa, &tm_x, kb * BK, m0, &full[stage]);
+            tma_load_2d(sa + L::kABytes, &tm_w, kb * BK, n0, &full[stage]);
+          }
+          __syncwarp();
           ++loads_issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -133,7 +139,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // The whole warp walks the loop and one elected lane issues.
+    {
       constexpr uint32_t idesc = instr_desc_bf16(BN);
       int stage = 0;
       uint32_t phase = 0;
@@ -141,24 +148,28 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        if (!mbar_wait(&tmem_empty[acc], acc_phase ^ 1, wc)) break;
+        if (!mbar_wait_warp(&tmem_empty[acc], acc_phase ^ 1, wc)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kAccStride;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait(&full[stage], phase, wc)) { ok = false; break; }
+          if (!mbar_wait_warp(&full[stage], phase, wc)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint64_t da = smem_desc_k_sw128(sa), db = smem_desc_k_sw128(sa + L::kABytes);
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            // advancing 16 bf16 along K inside the swizzled row = 32 bytes = 2 descriptor units
-            umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+              // advancing 16 bf16 along K inside the swizzled row = 32 bytes = 2 descriptor units
+              umma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+            }
+            umma_commit(&empty[stage]);
           }
-          umma_commit(&empty[stage]);
+          __syncwarp();
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        umma_commit(&tmem_full[acc]);
+        if (elect_one()) umma_commit(&tmem_full[acc]);
+        __syncwarp();
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
@@ -256,7 +267,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant
     // stores; a fixed pause on top, then shared and tensor memory are released.
     if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, 0, kStatusTimeout);
     if (warp == 0 && lane == 0) drain_ring(full, STAGES, loads_issued);
-    if (warp == 1 && lane == 0) {
+    if (warp == 1 && elect_one()) {   // the lane that issued the products: a commit covers the products of its own thread
       umma_commit(drain_bar);
       mbar_wait_drain(drain_bar, 0);
     }

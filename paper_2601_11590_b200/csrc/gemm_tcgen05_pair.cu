@@ -251,27 +251,33 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
   // them before the wait below, so they arrive while the previous kernel is still finishing; the x tiles follow
   // after the wait, into the same stages, counted on the same barrier phase.
   int early = 0;
-  if (static_w && warp == 0 && lane == 0 && pair < num_tiles) {
-    prefetch_map(&tm_w);
+  if (static_w && warp == 0 && pair < num_tiles) {
     int mt, nt;
     tile_coords(pair, m_tiles, n_tiles, order, mt, nt);
     const int n0 = nt * BN + (int)rank * (BN / 2);
     const uint64_t pol_w = order.by_rows ? policy_evict_first() : policy_evict_last();
     early = k_blocks < STAGES ? k_blocks : STAGES;
-    for (int kb = 0; kb < early; ++kb) {
-      if (rank == 0) mbar_expect_tx(&full[kb], 2 * L::kStageBytes);
-      tma_load_2d_pair(smem + kb * L::kStageBytes + L::kABytes, &tm_w, kb * BKE, n0, map_to_rank(smem_u32(&full[kb]), 0),
-                       pol_w);
+    if (elect_one()) {
+      prefetch_map(&tm_w);
+      for (int kb = 0; kb < early; ++kb) {
+        if (rank == 0) mbar_expect_tx(&full[kb], 2 * L::kStageBytes);
+        tma_load_2d_pair(smem + kb * L::kStageBytes + L::kABytes, &tm_w, kb * BKE, n0,
+                         map_to_rank(smem_u32(&full[kb]), 0), pol_w);
+      }
     }
+    __syncwarp();
     loads_issued = early;     // for the drain after an abort: these stages have loads in flight
   }
   pdl_wait();   // nothing above touches global memory that an earlier kernel of the stream writes
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
-      prefetch_map(&tm_x);
-      prefetch_map(&tm_w);
+    // The whole warp walks the loop and one elected lane issues (see elect_one()).
+    {
+      if (lane == 0) {
+        prefetch_map(&tm_x);
+        prefetch_map(&tm_w);
+      }
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -285,17 +291,20 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
         const int m0 = mt * (2 * BM) + (int)rank * BM;        // this CTA's rows of x
         const int n0 = nt * BN + (int)rank * (BN / 2);       // this CTA's half of the w tile
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait<true>(&empty[stage], phase ^ 1, wc)) { ok = false; break; }
+          if (!mbar_wait_warp<true>(&empty[stage], phase ^ 1, wc)) { ok = false; break; }
           uint8_t* sa = smem + stage * L::kStageBytes;
           const uint32_t bar = map_to_rank(smem_u32(&full[stage]), 0);
-          if (early > 0) {
-            --early;                                  // this stage's bytes are expected and its w tile is on its way
-          } else {
-            // the leader's barrier counts the bytes of both CTAs
-            if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
-            tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BKE, n0, bar, pol_w);
+          const bool w_early = early > 0;             // this stage's bytes are expected and its w tile is on its way
+          if (w_early) --early;
+          if (elect_one()) {
+            if (!w_early) {
+              // the leader's barrier counts the bytes of both CTAs
+              if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
+              tma_load_2d_pair(sa + L::kABytes, &tm_w, kb * BKE, n0, bar, pol_w);
+            }
+            tma_load_2d_pair(sa, &tm_x, kb * BKE, m0, bar, pol_x);
           }
-          tma_load_2d_pair(sa, &tm_x, kb * BKE, m0, bar, pol_x);
+          __syncwarp();
           ++loads_issued;
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -304,7 +313,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (leader only)
-    if (lane == 0 && rank == 0) {
+    // The whole warp walks the loop and one elected lane issues (see elect_one()).
+    if (rank == 0) {
       constexpr uint32_t idesc = instr_desc_pair(BN, FP8);
       int stage = 0;
       uint32_t phase = 0;
@@ -312,22 +322,26 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
       uint32_t acc_phase = 0;
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += n_pairs) {
-        if (!mbar_wait<true>(&tmem_empty[acc], acc_phase ^ 1, wc)) break;
+        if (!mbar_wait_warp<true>(&tmem_empty[acc], acc_phase ^ 1, wc)) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * kAccStride;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!mbar_wait<true>(&full[stage], phase, wc)) { ok = false; break; }
+          if (!mbar_wait_warp<true>(&full[stage], phase, wc)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
           const uint64_t da = smem_desc_k_sw128(sa), db = smem_desc_k_sw128(sa + L::kABytes);
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)   // one MMA per 32 bytes along K inside the swizzled row = 2 descriptor units
-            umma_pair<FP8>(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
-          umma_commit_both(&empty[stage]);
+            for (int k = 0; k < BK / 16; ++k)   // one MMA per 32 bytes along K inside the swizzled row = 2 descriptor units
+              umma_pair<FP8>(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+            umma_commit_both(&empty[stage]);
+          }
+          __syncwarp();
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        umma_commit_both(&tmem_full[acc]);
+        if (elect_one()) umma_commit_both(&tmem_full[acc]);
+        __syncwarp();
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
@@ -535,9 +549,13 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_consta
     // which shared and tensor memory are released.
     if (threadIdx.x == 0 && status != nullptr) atomicCAS(status, 0, kStatusTimeout);
     if (warp == 0 && lane == 0 && rank == 0) drain_ring<true>(full, STAGES, loads_issued);
-    if (warp == 1 && lane == 0) {
-      if (rank == 0) umma_commit_both(drain_bar);
-      mbar_wait_drain<true>(drain_bar, 0);
+    if (warp == 1) {
+      // the lane that issued the products commits (a commit covers the products of its own thread)
+      if (elect_one()) {
+        if (rank == 0) umma_commit_both(drain_bar);
+        mbar_wait_drain<true>(drain_bar, 0);
+      }
+      __syncwarp();
     }
     for (int i = 0; i < 64; ++i) __nanosleep(1000);
     __syncthreads();
