@@ -135,6 +135,11 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
+// a_i for i in 0..3.
+__device__ __forceinline__ uint32_t sel4(int i, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3) {
+  const uint32_t lo = (i & 1) ? a1 : a0, hi = (i & 1) ? a3 : a2;
+  return (i & 2) ? hi : lo;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -621,21 +626,38 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
           l[a] += __shfl_xor_sync(0xffffffffu, l[a], 2);
         }
       }
+      // A thread holds two neighbouring columns of every 8-column block of its rows.  Four blocks at a time are
+      // transposed inside the quad (three exchanges), after which thread q of the quad holds all 8 columns of
+      // block 4 g + q and writes them as 16 bytes: a quad writes 64 contiguous bytes of a row.
+      constexpr int kBlocks = DHP / 8;
 #pragma unroll
       for (int a = 0; a < 2; ++a) {
         const int token = it.q0 + w * BQ + r0 + 8 * a;
-        if (token < it.seg_beg + it.seg_len) {
-          const float inv = 1.0f / l[a];
-          __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + it.head * dh + 2 * quad;
+        const bool row_ok = token < it.seg_beg + it.seg_len;
+        const float inv = 1.0f / l[a];
+        __nv_bfloat16* orow = out + (int64_t)token * (heads * dh) + it.head * dh;
+        auto word = [&](int k) {
+          __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[4 * k + 2 * a]) * inv,
+                                                    __uint_as_float(o[4 * k + 2 * a + 1]) * inv);
+          return *reinterpret_cast<uint32_t*>(&b2);
+        };
 #pragma unroll
-          for (int k = 0; k < DHP / 8; ++k) {
-            if (k * 8 < dh) {                            // head_dim is a multiple of 8
-              __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(o[4 * k + 2 * a]) * inv,
-                                                        __uint_as_float(o[4 * k + 2 * a + 1]) * inv);
-              *reinterpret_cast<__nv_bfloat162*>(orow + k * 8) = b2;
-            }
-          }
+        for (int g = 0; g < kBlocks / 4; ++g) {
+          const uint32_t w0 = word(4 * g), w1 = word(4 * g + 1), w2 = word(4 * g + 2), w3 = word(4 * g + 3);
+          // what lane q ^ r needs from this lane is this lane's word of block q ^ r
+          const uint32_t r0w = sel4(quad, w0, w1, w2, w3);
+          const uint32_t r1w = __shfl_xor_sync(0xffffffffu, sel4(quad ^ 1, w0, w1, w2, w3), 1);
+          const uint32_t r2w = __shfl_xor_sync(0xffffffffu, sel4(quad ^ 2, w0, w1, w2, w3), 2);
+          const uint32_t r3w = __shfl_xor_sync(0xffffffffu, sel4(quad ^ 3, w0, w1, w2, w3), 3);
+          // word j of the block comes from lane j of the quad, i.e. from the exchange with distance j ^ q
+          const uint4 v = make_uint4(sel4(quad, r0w, r1w, r2w, r3w), sel4(quad ^ 1, r0w, r1w, r2w, r3w),
+                                     sel4(quad ^ 2, r0w, r1w, r2w, r3w), sel4(quad ^ 3, r0w, r1w, r2w, r3w));
+          const int blk = 4 * g + quad;
+          if (row_ok && blk * 8 < dh) *reinterpret_cast<uint4*>(orow + blk * 8) = v;   // head_dim is a multiple of 8
         }
+#pragma unroll
+        for (int k = kBlocks / 4 * 4; k < kBlocks; ++k)
+          if (row_ok && k * 8 < dh) *reinterpret_cast<uint32_t*>(orow + k * 8 + 2 * quad) = word(k);
       }
     }
   }
