@@ -368,7 +368,8 @@ enum {
   EPD_ATTENTION_SPLIT_KEYS = 2,       /* force the tensor-core kernel that gives one query tile to both softmax
                                          warpgroups (alternate key tiles, merged at the end) */
   EPD_ATTENTION_TWO_QUERY_TILES = 4   /* force the tensor-core kernel with two query tiles per CTA sharing every
-                                         K / V tile; without either flag the faster one for the shape is chosen */
+                                         K / V tile; without either flag this kernel runs wherever it applies
+                                         (the choice depends on the head width only, never on the batch) */
 };
 
 /* Block-diagonal bidirectional attention.  q, k, v [heads, T, head_dim_padded] per dtype as written

@@ -929,12 +929,14 @@ cudaError_t attention_any(int dtype, const void* q, const void* k, const void* v
                           const int32_t* host_cu_seqlens, int n_seg, void* out, int64_t T, int heads, int head_dim,
                           int flags, int* status, cudaStream_t s) {
   if (dtype == EPD_DTYPE_BF16 && !(flags & EPD_ATTENTION_FORCE_FMA)) {
-    // Two tensor-core kernels.  Measured on B200 (TFLOP/s, two-query-tile kernel / split-keys kernel): head width
-    // 128, 16 x 1024 tokens 775 / 698; head width 72: 16 x 1024 tokens 543 / 396, one 16384-token segment 693 / 692,
-    // 8 x 784 tokens 297 / 331, mixed lengths 196..7056 608 / 632.  The choice depends on the head width only, never
-    // on what else is in the batch: an item's features must not change with the company it is encoded in.
+    // Two tensor-core kernels.  Measured on B200 in one run (TFLOP/s, two-query-tile kernel / split-keys kernel), head
+    // width 72: 16 x 1024 tokens 593 / 452, ten segments of 840..5208 tokens 686 / 633, a 16384-token segment plus
+    // 8 x 784 tokens 749 / 718, mixed lengths 196..7056 678 / 662, 8 x 784 tokens 336 / 356; head width 128, 16 x 1024
+    // tokens 953 / 700.  The two-query-tile kernel is the default wherever it applies.  The choice depends on the head
+    // width only, never on what else is in the batch: an item's features must not change with the company it is
+    // encoded in.
     const bool forced_pair = flags & EPD_ATTENTION_TWO_QUERY_TILES;
-    const bool prefer_pair = padded_head_dim(head_dim) == 128;
+    const bool prefer_pair = true;
     if ((forced_pair || (prefer_pair && !(flags & EPD_ATTENTION_SPLIT_KEYS))) &&
         attention_pair_supported(q, k, v, out, T, heads, head_dim))
       return attention_pair(q, k, v, host_cu_seqlens, n_seg, out, T, heads, head_dim, status, s);
