@@ -2,39 +2,45 @@
 //
 // Persistent kernel, one CTA per SM.  A work item is one (segment, head, 256 query rows): two tiles of 128
 // query rows that walk the segment's keys / values together, so every K and V tile brought into shared
-// memory serves both.  Each query tile w has its own softmax warpgroup (one thread per query row), its own
-// issuing thread, two score buffers S_w[0], S_w[1] and an output accumulator O_w in tensor memory, its own
-// running max and row sum; there is nothing to merge at the end of an item.  The keys are walked in steps of
-// 64; step t of query tile w uses score buffer t mod 2:
+// memory serves both.  Each query tile w has two score buffers S_w[0], S_w[1] and an output accumulator O_w in
+// tensor memory, its own running max and row sum, two issuing warps and eight softmax warps; there is nothing to
+// merge at the end of an item.  The keys are walked in steps of 64; step t of query tile w uses score buffer t mod 2:
 //   S_w[b] = Q_w K_t^T     tcgen05.mma, both operands K-major in shared memory, fp32 scores in TMEM
-//   online softmax         warpgroup w reads its S row into registers (tcgen05.ld), takes the row maximum,
+//   online softmax         the tile's softmax warps read S into registers (tcgen05.ld), take row maxima,
 //                          P = exp2(S - m) as bf16 pairs, written back over the first half of the same buffer
 //                          (tcgen05.st).  q arrives scaled by log2(e)/sqrt(head_dim): base-2 exponentials suffice
 //   O_w += P_w V_t         one tcgen05.mma per 16 keys with P as the TMEM operand, V read MN-major from shared
 //                          memory
-// Each query tile has two issuing threads: one issues  P_w V_t  as soon as P is written, the other issues
-// Q_w K_(t+2)^T  into the buffer P was read from as soon as that product is complete.  (Issuing a product, a
-// commit or a barrier wait each costs a thread 60 to 100 clocks, and a step needs nine products, four commits
-// and four waits per query tile: one thread per query tile was measured to take ~1600 clocks per step and was
-// the kernel's bound.)  While the softmax warpgroup works on one buffer, the score product for the other one is
-// already complete or under way: the tensor-pipe round trip is off the warpgroup's critical path, which is then
-// load - max - exponentials - store.  The unit that bounds the kernel at head width 72 is the exponential unit (16 results per clock per
-// SM: 1024 clocks for the 2 x 128 x 64 scores of a step against 810 clocks of products).
-// The running max only advances (and O_w is rescaled in TMEM) when it grows by more than 2^8; until then the
-// stale max serves P, the row sum and O_w alike, which leaves the result unchanged.  A rescale first waits for
-// the previous step's P V (the only product that may still be adding to O_w: the one before it is complete
-// once the scores of the current step are).  Where head_dim is below the padded width, column head_dim of V
-// holds 1.0 and column head_dim of O_w is the row sum of P, summed by the tensor core from the same bf16
-// values as the numerator.
+// Issuing: one warp issues  P_w V_t  as soon as P is written, another issues  Q_w K_(t+2)^T  into the buffer P was
+// read from as soon as that product is complete.  Each walks its loop as a whole warp and lets one elected lane
+// issue (a product then costs the thread 40 to 50 clocks; issued from inside a branch that only lane 0 takes it
+// cost ~130, and one thread per query tile was the kernel's bound).  While the softmax warps work on one buffer, the
+// score product for the other one is already complete or under way.
+// Softmax: a query tile's rows are spread over quads.  A warp reads 16 TMEM lanes in the 16x256b fragment shape:
+// thread t holds rows t/4 and t/4 + 8 and two neighbouring columns of every 8-column block, 32 scores per step;
+// the four softmax warps of an SM sub-partition are the two halves of a lane quarter for both query tiles.  The
+// running max only advances (and O_w is rescaled in TMEM) when it grows by more than 2^8; until then the stale max
+// serves P, the row sum and O_w alike, which leaves the result unchanged.  So after an item's first step the weights
+// are computed against the running max as it stands, alongside the maxima of the thread's own quarter of its rows,
+// and nothing is exchanged; only when some thread of the warp finds its quarter above the threshold do the quads
+// exchange maxima (two shuffles), rescale the accumulator (after waiting for the previous step's P V, the only
+// product that may still be adding to it) and compute the weights again from the scores, which are still in their
+// buffer.  Where head_dim is below the padded width, column head_dim of V holds 1.0 and column head_dim of O_w is
+// the row sum of P, summed by the tensor core from the same bf16 values as the numerator.  The bound at head width
+// 72 is the softmax warps' step (~1600 clocks, against 1024 of the exponential unit at 16 results per clock per SM
+// and 840 of products).
+// Epilogue: four 8-column blocks at a time are transposed inside the quad, so that a thread writes 16 bytes and a
+// quad 64 contiguous bytes of an output row.
 // A segment whose length is not a multiple of 256 ends with an item whose second query tile is partly or
 // wholly beyond the segment: rows beyond it are computed and not stored; a wholly empty second tile is
-// skipped (its issuing thread only hands the K / V slots back, its warpgroup idles for that item).
+// skipped (its issuing warps only hand the K / V slots back, its softmax warps idle for that item).
 // TMEM (512 columns): S_0[0] | S_0[1] | S_1[0] | S_1[1] | O_0 | O_1, 64 columns per score buffer and the
 // padded head width per accumulator.
 // Warp roles: warp 0 TMA producer of Q (per tile, NQ buffers) and the K ring, warp 3 TMA producer of the V
 // ring, warps 1 / 2 the P V products of query tile 0 / 1 (warp 1 also allocates tensor memory), warps 4 / 5
-// their score products, warps 6, 7 idle, warps 8..11 and 12..15 the softmax warpgroups of query tile 0 and 1
-// (also epilogue).  The softmax warps raise their register allowance at the expense of warps 0..7 (setmaxnreg).
+// their score products, warps 6, 7 idle, warps 8..23 softmax (and epilogue): warps 8..15 query tile 0, 16..23 query
+// tile 1, each half again split into the first and second 16 lanes of every TMEM lane quarter (warp & 3).  The
+// softmax warps raise their register allowance at the expense of warps 0..7 (setmaxnreg).
 // head_dim 72 is stored padded to 80.  Q and K tiles: columns 0..63 form a 128-byte-swizzled box, columns
 // 64..79 a 32-byte-swizzled box, each contraction step its own MMA.  V tiles: five 32-byte-swizzled boxes of 16
 // columns, so that one MMA covers all 80 output columns.
