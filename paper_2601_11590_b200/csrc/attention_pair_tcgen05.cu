@@ -61,8 +61,8 @@ constexpr int BKV = 64;          // keys per step
 constexpr int kThreads = 768;    // warps 0..7: loaders and issuing threads; warps 8..23: four softmax warpgroups
 // Registers move between the warps of one SM sub-partition only (warp index mod 4), and setmaxnreg.inc waits until
 // they are free: the plan must balance per sub-partition, where two warps of 0..7 and four softmax warps live:
-// 2 x 48 + 4 x 96 = 6 x 80, the count the kernel is launched with.
-constexpr int kRegsLow = 48, kRegsHigh = 96;
+// 2 x 64 + 4 x 88 = 6 x 80, the count the kernel is launched with.
+constexpr int kRegsLow = 64, kRegsHigh = 88;
 static_assert(2 * kRegsLow + 4 * kRegsHigh <= 6 * 80, "register plan does not balance per SM sub-partition");
 constexpr int kMaxSegs = 128;    // segments one launch can describe
 constexpr float kRescaleThreshold = 8.0f;  // log2 of the largest P value tolerated before rescaling
