@@ -77,3 +77,14 @@ def test_binding_has_no_cpu_path():
         pytest.skip("GPU present")
     with pytest.raises(RuntimeError, match="CUDA device"):
         epd.Encoder(synth.TINY_FP32, synth.make_weights(synth.TINY_FP32), 512)
+
+
+def test_bench_reads_the_recorded_dram_traffic():
+    """The roofline's `traffic` comes from the ncu summary under profiles/, which records the hash of the kernel
+    source it was captured from: a kernel edit without a new capture must show up here, not as a silent null in
+    the bench line."""
+    import bench
+    traffic = bench.linear_dram_traffic(bench.DEFAULT_WORKLOAD)
+    assert traffic is not None, "profiles/linear_dram_traffic_per_workload.txt is stale for the current kernel source"
+    assert 4e8 < traffic < 2e9          # bytes per launch: above the 510 MB of algorithmic bytes, far below the 3-5 GB of old
+    assert bench.linear_dram_traffic("no_such_workload") is None
