@@ -150,6 +150,18 @@ __device__ __forceinline__ uint32_t sel4(int i, uint32_t a0, uint32_t a1, uint32
   const uint32_t lo = (i & 1) ? a1 : a0, hi = (i & 1) ? a3 : a2;
   return (i & 2) ? hi : lo;
 }
+// 2^x for x below ~100 on the FMA and integer pipes: x is rounded to the nearest integer n by adding 1.5 * 2^23
+// (n lands in the low mantissa bits), 2^(x - n) is a cubic on [-0.5, 0.5] (relative error 7.5e-5, far inside the
+// bf16 rounding of the weights it is used for), and n goes into the exponent field by an integer add.
+__device__ __forceinline__ float ex2_fma(float x) {
+  x = fmaxf(x, -125.0f);
+  const float t = x + 12582912.0f;
+  const float f = x - (t - 12582912.0f);
+  float p = fmaf(0.05517167f, f, 0.24261113f);
+  p = fmaf(p, f, 0.69326097f);
+  p = fmaf(p, f, 0.99992806f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -524,7 +536,12 @@ attention_pair_kernel(const __grid_constant__ Maps maps, const __grid_constant__
               const float p0 = ex2(__uint_as_float(s[4 * k]) + neg_m0);
               const float p1 = ex2(__uint_as_float(s[4 * k + 1]) + neg_m0);
               const float p2 = ex2(__uint_as_float(s[4 * k + 2]) + neg_m1);
-              const float p3 = ex2(__uint_as_float(s[4 * k + 3]) + neg_m1);
+              // one exponential in eight is evaluated on the FMA pipe for head width 72 (padded to 80, row sums from
+              // the ones column), where the exponential unit is the busiest one and the FMA pipe has room: measured
+              // in one run +2.5 to +4 % there, -3 % at head width 128, -5 % at 64 and 80, where the row sums are added
+              // on the FMA pipe as well; one in four or one in sixteen were slower than none
+              const float p3 = (ONES && DHP == 80 && (k & 1)) ? ex2_fma(__uint_as_float(s[4 * k + 3]) + neg_m1)
+                                                              : ex2(__uint_as_float(s[4 * k + 3]) + neg_m1);
               if (!ONES) { sum0 += p0 + p1; sum1 += p2 + p3; }
               __nv_bfloat162 b0 = __floats2bfloat162_rn(p0, p1), b1 = __floats2bfloat162_rn(p2, p3);
               pk[2 * k] = *reinterpret_cast<uint32_t*>(&b0);
