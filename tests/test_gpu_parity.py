@@ -309,6 +309,18 @@ def test_attention_more_segments_than_one_launch_describes():
     assert_parity(got, fma, TOL_BF16_STEP)
 
 
+@pytest.mark.parametrize("dh", [64, 72, 80, 128])
+def test_attention_segment_lengths_around_the_tile_edges(dh):
+    """Segment lengths on both sides of every boundary the two-query-tile kernel has (the 16-key product group, the
+    64-key step, the 128-row query tile, the 256-row item with its empty or ragged second tile), packed into one
+    batch, against the oracle; both tensor-core kernels."""
+    seglens = [1, 2, 15, 16, 17, 63, 64, 65, 127, 128, 129, 191, 193, 255, 256, 257, 300, 383, 385, 511, 513]
+    for flags in (epd.ATTENTION_TWO_QUERY_TILES, epd.ATTENTION_SPLIT_KEYS):
+        got, ref = _attention_case(epd.DTYPE_BF16, 2, dh, seglens, 70 + dh, flags=flags)
+        assert np.isfinite(got).all()
+        assert_parity(got, ref, TOL_BF16_STEP, f"attention, head width {dh}, flags {flags}")
+
+
 @pytest.mark.parametrize("kernel", ["split_keys", "two_query_tiles"])
 def test_attention_rescale_path(kernel):
     """Keys ordered so that the running maximum keeps growing from tile to tile by far more than the
